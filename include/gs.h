@@ -1,0 +1,181 @@
+/* gs.h - C ABI of the B200 cached neighbour sampler (GraphSnapShot's GraphSDSampler hot path).
+ *
+ * The library keeps a per-node cache of fixed-width neighbour slots next to a CSR graph, and
+ * per mini-batch refreshes the cached rows of the frontier's nodes (all slots: Fully Cache
+ * Refresh; a fraction gamma of them: On-The-Fly), samples each hop's fan-out from the cache,
+ * relabels global ids to block-local ids, builds every hop's block CSR and gathers the input
+ * nodes' feature rows.  Every step runs in CUDA kernels built for sm_100a; there is no CPU
+ * fallback.
+ *
+ * General rules
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  All device buffers are
+ *     owned by the caller and must outlive the handle that borrows them.  The library allocates
+ *     no device memory; the two opaque handles are small host objects.
+ *   - Every call returns a gs_status; nothing throws, traps or aborts.  Host-side checks fail
+ *     before any kernel is launched.  Problems only the device can see (a seed id out of range,
+ *     a duplicate seed) set a status word that gs_batch_counts / gs_sync_status return; the
+ *     kernels of that batch then write nothing further.
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default stream)
+ *     and is asynchronous unless a call says it synchronises.
+ *   - Graph contract: CSR row v lists the in-neighbours of v in ascending order without
+ *     duplicates; num_nodes < 2^31; indptr is int64, ids are int32.
+ *   - Fan-outs are listed input-layer-first.  Sampling step k = 0..L-1 starts at the seeds and
+ *     uses layer l = L-1-k (the paper's loop "for l = L to 1", Algorithm 2 SampleBlocks).
+ *   - Randomness: every choice orders items by (key32(item), item) ascending where key32(i) is
+ *     word (i & 3) of Philox4x32-10(counter = (i >> 2, node, step, (purpose << 8) | tag),
+ *     key = (seed low word, seed high word)); purpose 1 = FILL over edge offsets of the node's
+ *     CSR row, 2 = EVICT over slot indices, 3 = PICK over slot indices; tag = layer, except
+ *     FILL/EVICT of a shared cache, which use 0xFF.  The result of a call is therefore unique.
+ */
+#ifndef GS_H
+#define GS_H
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gs_graph gs_graph; /* opaque host object */
+typedef struct gs_cache gs_cache; /* opaque host object */
+
+typedef enum {
+    GS_OK = 0,
+    GS_ERR_ARG = 1,       /* NULL pointer, size or parameter out of its documented range */
+    GS_ERR_ALIGN = 2,     /* a device pointer is not aligned as documented */
+    GS_ERR_RANGE = 3,     /* device-detected: a seed id outside [0, num_nodes) */
+    GS_ERR_WORKSPACE = 4, /* a caller-provided buffer is smaller than the *_bytes call reports */
+    GS_ERR_DUP_SEED = 5,  /* device-detected: the same seed id twice in one batch */
+    GS_ERR_CUDA = 6       /* a CUDA runtime call failed; see gs_last_error() */
+} gs_status;
+
+typedef enum { GS_MODE_FCR = 0, GS_MODE_OTF = 1 } gs_mode;
+typedef enum { GS_F32 = 0, GS_BF16 = 1 } gs_dtype;
+
+#define GS_MAX_HOPS 8
+#define GS_MAX_CACHE_WIDTH 32
+
+/* Graph "on disk" in the paper's terms (Section "System Components": the full graph G=(V,E) and
+ * the node embeddings H_v): a CSR adjacency and a row-major feature matrix, both resident in
+ * device memory and borrowed.
+ *   d_indptr   int64[num_nodes+1], 8-byte aligned     d_indices  int32[num_edges], 4-byte aligned
+ *   d_features [num_nodes][feat_ld] elements of `dtype` (feat_ld >= feat_dim, in elements);
+ *              may be NULL if gs_gather_features is never called.
+ * Validates sizes and alignment on the host only; launches nothing. */
+gs_status gs_graph_create(int64_t num_nodes, int64_t num_edges, const int64_t* d_indptr,
+                          const int32_t* d_indices, const void* d_features, gs_dtype dtype,
+                          int32_t feat_dim, int64_t feat_ld, gs_graph** out);
+void gs_graph_destroy(gs_graph*);
+
+/* Bytes of device memory the cache needs: a small state header, the relabel table (8 bytes per
+ * node) and the slot rows (num_hops caches, or one if shared != 0). */
+gs_status gs_cache_bytes(const gs_graph*, int32_t num_hops, int32_t cache_width, int32_t shared, size_t* bytes);
+
+/* Bytes of device scratch one gs_sample_batch call with at most max_seeds seeds needs.  The
+ * per-hop block arrays returned by gs_sample_batch live inside it. */
+gs_status gs_workspace_bytes(const gs_graph*, int32_t num_hops, const int32_t* fanouts, int32_t max_seeds, size_t* bytes);
+
+/* Static pre-sample (paper Algorithm 2, Initialize: "Pre-sample cache for each layer l"; Section
+ * "Static and Dynamic Sampling").  For every node and every layer (one row per node if shared):
+ * degree <= cache_width -> the row is the adjacency in CSR order, remaining slots -1; otherwise
+ * the row holds the cache_width neighbours first in FILL order at step 0, in that order.
+ *   fanouts          h_ int32[num_hops], each in [1, cache_width]
+ *   cache_width      in [1, GS_MAX_CACHE_WIDTH]
+ *   d_cache_storage  256-byte aligned, cache_bytes >= gs_cache_bytes(...); owned by the caller,
+ *                    initialised here, then read and written by every gs_sample_batch.
+ * Enqueues the kernels on `stream`; does not synchronise. */
+gs_status gs_cache_init(const gs_graph*, int32_t num_hops, const int32_t* fanouts, int32_t cache_width,
+                        uint64_t seed, int32_t shared, void* d_cache_storage, size_t cache_bytes,
+                        void* stream, gs_cache** out);
+void gs_cache_destroy(gs_cache*);
+
+/* One hop's message-flow graph ("blocks" of Algorithm 2/3), stored destination-major.  The
+ * destination nodes are the first *d_num_dst entries of the input-node list, the source nodes its
+ * first *d_num_src entries (so sources begin with the destinations).  Counts are device scalars;
+ * max_* are host-side upper bounds that size the arrays. */
+typedef struct {
+    int32_t max_dst, max_src, max_edges;
+    const int32_t* d_num_dst;   /* device scalar */
+    const int32_t* d_num_src;   /* device scalar */
+    const int32_t* d_num_edges; /* device scalar */
+    const int32_t* d_indptr;    /* [num_dst + 1] offsets into d_indices */
+    const int32_t* d_indices;   /* [num_edges] block-local source ids */
+} gs_block;
+
+/* One mini-batch (paper Algorithm 2 RefreshCache + SampleBlocks for GS_MODE_OTF, Algorithm 3
+ * CacheRefresh + SampleBlocks for GS_MODE_FCR; Section "Shared Cache Design" when the cache was
+ * created shared).  For step k = 0..L-1 with layer l = L-1-k:
+ *   refresh  every frontier node with degree > cache_width gets r of its slots replaced
+ *            (r = cache_width for FCR, floor(gamma*cache_width + 0.5) for OTF): the r slot indices
+ *            first in EVICT order are dropped, the others stay in place, and the dropped slots
+ *            (ascending) receive the neighbours first in FILL order among those not retained.
+ *            With a shared cache a node is refreshed only at the step it enters the frontier.
+ *   pick     all cached neighbours if there are at most f_l, else the f_l slots first in PICK
+ *            order, emitted in ascending slot index;
+ *   relabel  next frontier = frontier followed by unseen picked ids in row-major order.
+ * Arguments
+ *   d_seeds      int32[num_seeds], distinct ids in [0, num_nodes); 1 <= num_seeds <= the
+ *                max_seeds the workspace was sized for
+ *   gamma        in [0, 1] (ignored for FCR);  step >= 1 (step 0 is the pre-sample)
+ *   d_workspace  256-byte aligned, >= gs_workspace_bytes(..., num_seeds)
+ *   blocks       h_ array of num_hops entries, filled by layer (blocks[0] = input side)
+ *   d_input_nodes / d_num_input_nodes   receive device pointers to the global ids of the input
+ *                nodes (the last frontier) and to their count
+ * Block arrays and the input-node list stay valid until the next call on the same workspace.
+ * Asynchronous.  Calls on one cache must not overlap on the device. */
+gs_status gs_sample_batch(gs_cache*, const int32_t* d_seeds, int32_t num_seeds, gs_mode mode, double gamma,
+                          uint32_t step, void* d_workspace, size_t workspace_bytes, void* stream,
+                          gs_block* blocks, const int32_t** d_input_nodes, const int32_t** d_num_input_nodes);
+
+/* Same batch for a caller whose seeds are in HOST memory: copies h_seeds to the device, runs the
+ * batch, copies the counts back and synchronises `stream`.
+ *   h_num_nodes  int32[num_hops + 1]: n_0 (seeds) .. n_L (input nodes), by sampling step
+ *   h_num_edges  int32[num_hops]: edges per block, by layer
+ * Returns the device status of the batch. */
+gs_status gs_sample_batch_host(gs_cache*, const int32_t* h_seeds, int32_t num_seeds, gs_mode mode, double gamma,
+                               uint32_t step, void* d_workspace, size_t workspace_bytes, void* stream,
+                               gs_block* blocks, const int32_t** d_input_nodes,
+                               int32_t* h_num_nodes, int32_t* h_num_edges);
+
+/* Synchronises `stream` and returns the counts of the last batch on this cache (layout as in
+ * gs_sample_batch_host; either pointer may be NULL) and its device status. */
+gs_status gs_batch_counts(gs_cache*, void* stream, int32_t* h_num_nodes, int32_t* h_num_edges);
+
+/* Feature gather (the paper's "load embeddings", Section "System Components"):
+ * out[p, :] = features[ids[p], :] for p < count, a bitwise copy.
+ *   d_ids            int32 ids in [0, num_nodes)
+ *   d_count_or_null  device scalar with the row count, or NULL to use count_bound
+ *   count_bound      rows d_out has room for (and the count, when d_count_or_null is NULL)
+ *   d_out            [count_bound][out_ld] elements of the graph's dtype, out_ld >= feat_dim
+ * Uses 16-byte accesses when base pointers and both row pitches allow it, narrower otherwise. */
+gs_status gs_gather_features(const gs_graph*, const int32_t* d_ids, const int32_t* d_count_or_null,
+                             int32_t count_bound, void* d_out, int64_t out_ld, void* stream);
+
+/* Copy n logical cache rows (cache_width slots each, -1 = empty) of `layer` into d_out[n][cache_width]. */
+gs_status gs_cache_read_rows(const gs_cache*, int32_t layer, const int32_t* d_nodes, int32_t n,
+                             int32_t* d_out, void* stream);
+
+/* Checkpoint / resume: the slot rows as one opaque blob of gs_cache_export_bytes bytes. */
+gs_status gs_cache_export_bytes(const gs_cache*, size_t* bytes);
+gs_status gs_cache_export(const gs_cache*, void* d_dst, size_t bytes, void* stream);
+gs_status gs_cache_import(gs_cache*, const void* d_src, size_t bytes, void* stream);
+
+/* Synchronises `stream` and returns the device status of the last batch. */
+gs_status gs_sync_status(gs_cache*, void* stream);
+
+/* Selection tuning (never changes results, only which internal path finds them):
+ * expected number of candidate edges kept by the threshold scan for an OTF refill and for a full
+ * refill, and the degree above which a whole thread block scans one node.  Values <= 0 keep the
+ * defaults. */
+gs_status gs_cache_set_tuning(gs_cache*, double lambda_otf, double lambda_full, int32_t hub_degree);
+
+/* Number of kernels this library has launched in the calling process (monotonic). */
+int64_t gs_kernel_launches(void);
+
+/* Message of the last failing call in this thread ("" if none). */
+const char* gs_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,13 @@
+"""B200-native cached neighbour sampling (GraphSnapShot's GraphSDSampler hot path).
+
+Thin ctypes binding over the C-ABI CUDA library ``libgs.so`` (see ``include/gs.h``); every
+step of the path runs in that library's kernels.  There is no CPU fallback: if the library is
+missing or cannot be loaded, importing :mod:`paper_2406_17918_b200.binding` raises.
+"""
+from .binding import (  # noqa: F401
+    GS_MODE_FCR, GS_MODE_OTF, GS_F32, GS_BF16, GsError, Block, Graph, Cache,
+    gs_graph_create, gs_cache_bytes, gs_workspace_bytes, gs_cache_init, gs_sample_batch,
+    gs_sample_batch_host, gs_batch_counts, gs_gather_features, gs_cache_read_rows,
+    gs_cache_export, gs_cache_import, gs_sync_status, gs_cache_set_tuning, gs_kernel_launches,
+    gs_last_error, library_path, exported_symbols,
+)

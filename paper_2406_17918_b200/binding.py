@@ -1,0 +1,303 @@
+"""ctypes binding of ``libgs.so``: argument marshalling only.
+
+Functions keep the names and argument order of ``include/gs.h``.  Device buffers are torch CUDA
+tensors (torch is used for device memory and streams only); the binding passes their
+``data_ptr()`` and keeps them alive on the small Python handle objects.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import re
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libgs.so")
+_HEADER = os.path.join(os.path.dirname(_HERE), "include", "gs.h")
+
+GS_MODE_FCR, GS_MODE_OTF = 0, 1
+GS_F32, GS_BF16 = 0, 1
+GS_MAX_HOPS = 8
+
+_STATUS_NAMES = {0: "GS_OK", 1: "GS_ERR_ARG", 2: "GS_ERR_ALIGN", 3: "GS_ERR_RANGE", 4: "GS_ERR_WORKSPACE",
+                 5: "GS_ERR_DUP_SEED", 6: "GS_ERR_CUDA"}
+
+
+class GsError(RuntimeError):
+    def __init__(self, status, message):
+        super().__init__("%s: %s" % (_STATUS_NAMES.get(status, status), message))
+        self.status = status
+
+
+class _CBlock(ctypes.Structure):
+    _fields_ = [("max_dst", ctypes.c_int32), ("max_src", ctypes.c_int32), ("max_edges", ctypes.c_int32),
+                ("d_num_dst", ctypes.c_void_p), ("d_num_src", ctypes.c_void_p), ("d_num_edges", ctypes.c_void_p),
+                ("d_indptr", ctypes.c_void_p), ("d_indices", ctypes.c_void_p)]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def exported_symbols():
+    """Names of the functions ``include/gs.h`` declares."""
+    text = open(_HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(gs_[a-z_]+)\s*\(", text)))
+
+
+def _load():
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError("%s is missing: run `python -m paper_2406_17918_b200.build` "
+                          "(there is no CPU fallback)" % _LIB_PATH)
+    L = ctypes.CDLL(_LIB_PATH)
+    vp, i32, i64, u32, u64, dbl, sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32,
+                                       ctypes.c_uint64, ctypes.c_double, ctypes.c_size_t)
+    pvp = ctypes.POINTER(vp)
+    psz = ctypes.POINTER(sz)
+    sig = {
+        "gs_graph_create": [i64, i64, vp, vp, vp, ctypes.c_int, i32, i64, pvp],
+        "gs_cache_bytes": [vp, i32, i32, i32, psz],
+        "gs_workspace_bytes": [vp, i32, vp, i32, psz],
+        "gs_cache_init": [vp, i32, vp, i32, u64, i32, vp, sz, vp, pvp],
+        "gs_sample_batch": [vp, vp, i32, ctypes.c_int, dbl, u32, vp, sz, vp, vp, pvp, pvp],
+        "gs_sample_batch_host": [vp, vp, i32, ctypes.c_int, dbl, u32, vp, sz, vp, vp, pvp, vp, vp],
+        "gs_batch_counts": [vp, vp, vp, vp],
+        "gs_gather_features": [vp, vp, vp, i32, vp, i64, vp],
+        "gs_cache_read_rows": [vp, i32, vp, i32, vp, vp],
+        "gs_cache_export_bytes": [vp, psz],
+        "gs_cache_export": [vp, vp, sz, vp],
+        "gs_cache_import": [vp, vp, sz, vp],
+        "gs_sync_status": [vp, vp],
+        "gs_cache_set_tuning": [vp, dbl, dbl, i32],
+    }
+    for name, args in sig.items():
+        fn = getattr(L, name)
+        fn.argtypes = args
+        fn.restype = ctypes.c_int
+    L.gs_graph_destroy.argtypes = [vp]
+    L.gs_graph_destroy.restype = None
+    L.gs_cache_destroy.argtypes = [vp]
+    L.gs_cache_destroy.restype = None
+    L.gs_last_error.argtypes = []
+    L.gs_last_error.restype = ctypes.c_char_p
+    L.gs_kernel_launches.argtypes = []
+    L.gs_kernel_launches.restype = ctypes.c_int64
+    return L
+
+
+_L = _load()
+
+
+def gs_last_error() -> str:
+    return _L.gs_last_error().decode()
+
+
+def gs_kernel_launches() -> int:
+    return int(_L.gs_kernel_launches())
+
+
+def _check(status):
+    if status != 0:
+        raise GsError(status, gs_last_error())
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _i32_array(values):
+    return (ctypes.c_int32 * len(values))(*[int(v) for v in values])
+
+
+class Graph:
+    """Handle of gs_graph plus references that keep the borrowed tensors alive."""
+
+    def __init__(self, handle, indptr, indices, features, dtype, feat_dim):
+        self.handle, self.indptr, self.indices, self.features = handle, indptr, indices, features
+        self.dtype, self.feat_dim = dtype, feat_dim
+        self.num_nodes = indptr.numel() - 1
+
+    def close(self):
+        if self.handle:
+            _L.gs_graph_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Cache:
+    def __init__(self, handle, graph, storage, fanouts, cache_width, shared):
+        self.handle, self.graph, self.storage = handle, graph, storage
+        self.fanouts, self.cache_width, self.shared = list(fanouts), cache_width, bool(shared)
+        self.num_hops = len(self.fanouts)
+
+    def close(self):
+        if self.handle:
+            _L.gs_cache_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Block:
+    """Device view of one hop's block; tensors alias the workspace (no copies)."""
+
+    def __init__(self, cb: _CBlock, workspace: torch.Tensor, header: torch.Tensor):
+        self.max_dst, self.max_src, self.max_edges = cb.max_dst, cb.max_src, cb.max_edges
+        self._ws, self._hdr = workspace, header
+        self._indptr_off = cb.d_indptr - workspace.data_ptr()
+        self._indices_off = cb.d_indices - workspace.data_ptr()
+        hp = header.data_ptr()
+        self._cnt = ((cb.d_num_dst - hp) // 4, (cb.d_num_src - hp) // 4, (cb.d_num_edges - hp) // 4)
+
+    def counts_device(self):
+        """(num_dst, num_src, num_edges) as 0-d device tensors aliasing the cache's state header."""
+        h = self._hdr.view(torch.int32)
+        return tuple(h[i] for i in self._cnt)
+
+    def indptr(self, num_dst: int) -> torch.Tensor:
+        return self._ws[self._indptr_off:self._indptr_off + 4 * (num_dst + 1)].view(torch.int32)
+
+    def indices(self, num_edges: int) -> torch.Tensor:
+        return self._ws[self._indices_off:self._indices_off + 4 * num_edges].view(torch.int32)
+
+
+def gs_graph_create(indptr: torch.Tensor, indices: torch.Tensor, features, dtype=None) -> Graph:
+    if indptr.dtype != torch.int64 or indices.dtype != torch.int32:
+        raise TypeError("indptr must be int64 and indices int32")
+    if not (indptr.is_cuda and indices.is_cuda and indptr.is_contiguous() and indices.is_contiguous()):
+        raise ValueError("indptr/indices must be contiguous CUDA tensors")
+    feat_dim, feat_ld = 0, 0
+    if features is not None:
+        if not features.is_cuda or features.dim() != 2 or features.stride(1) != 1:
+            raise ValueError("features must be a row-major 2-D CUDA tensor")
+        dtype = {torch.float32: GS_F32, torch.bfloat16: GS_BF16}[features.dtype]
+        feat_dim, feat_ld = features.shape[1], features.stride(0)
+    elif dtype is None:
+        dtype = GS_F32
+    h = ctypes.c_void_p()
+    _check(_L.gs_graph_create(indptr.numel() - 1, indices.numel(), _ptr(indptr), _ptr(indices), _ptr(features),
+                              dtype, feat_dim, feat_ld, ctypes.byref(h)))
+    return Graph(h, indptr, indices, features, dtype, feat_dim)
+
+
+def gs_cache_bytes(graph: Graph, num_hops: int, cache_width: int, shared: bool) -> int:
+    out = ctypes.c_size_t()
+    _check(_L.gs_cache_bytes(graph.handle, num_hops, cache_width, int(shared), ctypes.byref(out)))
+    return out.value
+
+
+def gs_workspace_bytes(graph: Graph, fanouts, max_seeds: int) -> int:
+    out = ctypes.c_size_t()
+    _check(_L.gs_workspace_bytes(graph.handle, len(fanouts), _i32_array(fanouts), max_seeds, ctypes.byref(out)))
+    return out.value
+
+
+def gs_cache_init(graph: Graph, fanouts, cache_width: int, seed: int, shared: bool, storage: torch.Tensor = None,
+                  stream=None) -> Cache:
+    if storage is None:
+        storage = torch.empty(gs_cache_bytes(graph, len(fanouts), cache_width, shared), dtype=torch.uint8,
+                              device=graph.indptr.device)
+    h = ctypes.c_void_p()
+    _check(_L.gs_cache_init(graph.handle, len(fanouts), _i32_array(fanouts), cache_width, ctypes.c_uint64(seed),
+                            int(shared), _ptr(storage), storage.numel(), _stream(stream), ctypes.byref(h)))
+    return Cache(h, graph, storage, fanouts, cache_width, shared)
+
+
+def _blocks_out(cache: Cache, cblocks, workspace):
+    return [Block(cblocks[l], workspace, cache.storage) for l in range(cache.num_hops)]
+
+
+def gs_sample_batch(cache: Cache, seeds: torch.Tensor, mode: int, gamma: float, step: int, workspace: torch.Tensor,
+                    stream=None):
+    """Returns (blocks by layer, input_nodes tensor of capacity max_src, device count tensor)."""
+    if seeds.dtype != torch.int32 or not seeds.is_cuda or not seeds.is_contiguous():
+        raise TypeError("seeds must be a contiguous int32 CUDA tensor")
+    cblocks = (_CBlock * cache.num_hops)()
+    d_in, d_cnt = ctypes.c_void_p(), ctypes.c_void_p()
+    _check(_L.gs_sample_batch(cache.handle, _ptr(seeds), seeds.numel(), mode, float(gamma), step, _ptr(workspace),
+                              workspace.numel(), _stream(stream), cblocks, ctypes.byref(d_in), ctypes.byref(d_cnt)))
+    blocks = _blocks_out(cache, cblocks, workspace)
+    off = d_in.value - workspace.data_ptr()
+    input_nodes = workspace[off:off + 4 * blocks[0].max_src].view(torch.int32)
+    cnt_index = (d_cnt.value - cache.storage.data_ptr()) // 4
+    return blocks, input_nodes, cache.storage.view(torch.int32)[cnt_index]
+
+
+def gs_sample_batch_host(cache: Cache, seeds_host: torch.Tensor, mode: int, gamma: float, step: int,
+                         workspace: torch.Tensor, stream=None):
+    """Seeds in (pinned) host memory; synchronises.  Returns (blocks, input_nodes, n list, m list)."""
+    if seeds_host.dtype != torch.int32 or seeds_host.is_cuda or not seeds_host.is_contiguous():
+        raise TypeError("seeds_host must be a contiguous int32 CPU tensor")
+    cblocks = (_CBlock * cache.num_hops)()
+    d_in = ctypes.c_void_p()
+    n = (ctypes.c_int32 * (cache.num_hops + 1))()
+    m = (ctypes.c_int32 * cache.num_hops)()
+    _check(_L.gs_sample_batch_host(cache.handle, _ptr(seeds_host), seeds_host.numel(), mode, float(gamma), step,
+                                   _ptr(workspace), workspace.numel(), _stream(stream), cblocks, ctypes.byref(d_in),
+                                   n, m))
+    blocks = _blocks_out(cache, cblocks, workspace)
+    off = d_in.value - workspace.data_ptr()
+    input_nodes = workspace[off:off + 4 * blocks[0].max_src].view(torch.int32)
+    return blocks, input_nodes, list(n), list(m)
+
+
+def gs_batch_counts(cache: Cache, stream=None):
+    """Synchronises; returns ([n_0..n_L] by sampling step, [edges per block] by layer)."""
+    n = (ctypes.c_int32 * (cache.num_hops + 1))()
+    m = (ctypes.c_int32 * cache.num_hops)()
+    _check(_L.gs_batch_counts(cache.handle, _stream(stream), n, m))
+    return list(n), list(m)
+
+
+def gs_gather_features(graph: Graph, ids: torch.Tensor, count, out: torch.Tensor, stream=None):
+    """count: a 0-d int32 CUDA tensor (device scalar) or None to gather out.shape[0] rows."""
+    if ids.dtype != torch.int32 or not ids.is_cuda:
+        raise TypeError("ids must be an int32 CUDA tensor")
+    if out.dim() != 2 or out.stride(1) != 1 or out.dtype != graph.features.dtype:
+        raise TypeError("out must be a row-major 2-D tensor of the feature dtype")
+    bound = min(out.shape[0], ids.numel())
+    _check(_L.gs_gather_features(graph.handle, _ptr(ids), _ptr(count), bound, _ptr(out), out.stride(0),
+                                 _stream(stream)))
+    return out
+
+
+def gs_cache_read_rows(cache: Cache, layer: int, nodes: torch.Tensor, stream=None) -> torch.Tensor:
+    out = torch.empty((nodes.numel(), cache.cache_width), dtype=torch.int32, device=nodes.device)
+    _check(_L.gs_cache_read_rows(cache.handle, layer, _ptr(nodes), nodes.numel(), _ptr(out), _stream(stream)))
+    return out
+
+
+def gs_cache_export(cache: Cache, stream=None) -> torch.Tensor:
+    nbytes = ctypes.c_size_t()
+    _check(_L.gs_cache_export_bytes(cache.handle, ctypes.byref(nbytes)))
+    blob = torch.empty(nbytes.value, dtype=torch.uint8, device=cache.storage.device)
+    _check(_L.gs_cache_export(cache.handle, _ptr(blob), blob.numel(), _stream(stream)))
+    return blob
+
+
+def gs_cache_import(cache: Cache, blob: torch.Tensor, stream=None):
+    _check(_L.gs_cache_import(cache.handle, _ptr(blob), blob.numel(), _stream(stream)))
+
+
+def gs_sync_status(cache: Cache, stream=None):
+    _check(_L.gs_sync_status(cache.handle, _stream(stream)))
+
+
+def gs_cache_set_tuning(cache: Cache, lambda_otf=0.0, lambda_full=0.0, hub_degree=0):
+    _check(_L.gs_cache_set_tuning(cache.handle, float(lambda_otf), float(lambda_full), int(hub_degree)))

@@ -1,0 +1,445 @@
+// The C ABI: argument checks, device-state layout and the per-batch kernel sequence.
+#include <atomic>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "gs_internal.h"
+
+struct gs_graph {
+    int64_t num_nodes, num_edges;
+    const int64_t* d_indptr;
+    const int32_t* d_indices;
+    const void* d_features;
+    gs_dtype dtype;
+    int32_t feat_dim;
+    int64_t feat_ld;
+    int32_t elem_bytes;
+};
+
+struct gs_cache {
+    const gs_graph* graph;
+    int32_t L, W, pitch, shared, num_caches;
+    int32_t fanouts[GS_MAX_HOPS];
+    uint64_t seed;
+    char* d_storage;
+    int32_t* d_hdr;
+    unsigned long long* d_table;
+    int32_t* d_slots;
+    size_t slot_bytes;        // all caches
+    uint32_t serial;          // batches run; the relabel stamp is derived from it
+    float lambda_otf, lambda_full;
+    int32_t hub_degree;
+    int32_t* h_pinned;        // pinned staging for counts
+};
+
+namespace gs {
+
+static thread_local char g_err[512] = "";
+static std::atomic<long long> g_launches{0};
+
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static gs_status fail(gs_status code, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+static gs_status cuda_fail(cudaError_t e, const char* what) {
+    return fail(GS_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+#define GS_CUDA(call)                                          \
+    do {                                                       \
+        cudaError_t e__ = (call);                              \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #call);  \
+    } while (0)
+
+static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+static int32_t pitch_for(int32_t W) { return (W + 7) / 8 * 8; }
+
+static gs_status check_shape(const gs_graph* g, int32_t num_hops, int32_t cache_width) {
+    if (!g) return fail(GS_ERR_ARG, "graph is NULL");
+    if (num_hops < 1 || num_hops > GS_MAX_HOPS) return fail(GS_ERR_ARG, "num_hops %d outside [1, %d]", num_hops, GS_MAX_HOPS);
+    if (cache_width < 1 || cache_width > GS_MAX_CACHE_WIDTH)
+        return fail(GS_ERR_ARG, "cache_width %d outside [1, %d]", cache_width, GS_MAX_CACHE_WIDTH);
+    return GS_OK;
+}
+
+static size_t table_bytes(const gs_graph* g) { return align_up((size_t)g->num_nodes * 8, 256); }
+static size_t slots_bytes(const gs_graph* g, int32_t caches, int32_t W) {
+    return align_up((size_t)caches * (size_t)g->num_nodes * (size_t)pitch_for(W) * 4, 256);
+}
+
+static uint32_t key_word(uint32_t purpose, uint32_t tag) { return (purpose << 8) | tag; }
+
+static StepParams step_params(const gs_cache* c, int32_t layer, uint32_t step) {
+    StepParams P{};
+    const gs_graph* g = c->graph;
+    P.g = GraphView{g->d_indptr, g->d_indices, g->num_nodes};
+    const int32_t ci = c->shared ? 0 : layer;
+    P.slots = c->d_slots + (size_t)ci * (size_t)g->num_nodes * c->pitch;
+    P.pitch = c->pitch;
+    P.W = c->W;
+    P.f = c->fanouts[layer];
+    P.step = step;
+    P.key0 = (uint32_t)(c->seed & 0xFFFFFFFFu);
+    P.key1 = (uint32_t)(c->seed >> 32);
+    const uint32_t ctag = c->shared ? 0xFFu : (uint32_t)layer;
+    P.word_fill = key_word(1, ctag);
+    P.word_evict = key_word(2, ctag);
+    P.word_pick = key_word(3, (uint32_t)layer);
+    P.table = c->d_table;
+    P.status = c->d_hdr + HDR_STATUS;
+    P.lambda_otf = c->lambda_otf;
+    P.lambda_full = c->lambda_full;
+    P.hub_degree = c->hub_degree;
+    return P;
+}
+
+}  // namespace gs
+
+using namespace gs;
+
+extern "C" {
+
+const char* gs_last_error(void) { return g_err; }
+int64_t gs_kernel_launches(void) { return (int64_t)g_launches.load(); }
+
+gs_status gs_graph_create(int64_t num_nodes, int64_t num_edges, const int64_t* d_indptr, const int32_t* d_indices,
+                          const void* d_features, gs_dtype dtype, int32_t feat_dim, int64_t feat_ld, gs_graph** out) {
+    if (!out) return fail(GS_ERR_ARG, "out is NULL");
+    *out = nullptr;
+    if (num_nodes < 1 || num_nodes >= ((int64_t)1 << 31)) return fail(GS_ERR_ARG, "num_nodes %lld outside [1, 2^31)", (long long)num_nodes);
+    if (num_edges < 0) return fail(GS_ERR_ARG, "num_edges is negative");
+    if (!d_indptr) return fail(GS_ERR_ARG, "d_indptr is NULL");
+    if (!d_indices && num_edges > 0) return fail(GS_ERR_ARG, "d_indices is NULL");
+    if (!aligned(d_indptr, 8)) return fail(GS_ERR_ALIGN, "d_indptr must be 8-byte aligned");
+    if (!aligned(d_indices, 4)) return fail(GS_ERR_ALIGN, "d_indices must be 4-byte aligned");
+    if (dtype != GS_F32 && dtype != GS_BF16) return fail(GS_ERR_ARG, "unknown dtype %d", (int)dtype);
+    const int32_t eb = dtype == GS_F32 ? 4 : 2;
+    if (d_features) {
+        if (feat_dim < 1) return fail(GS_ERR_ARG, "feat_dim must be >= 1");
+        if (feat_ld < feat_dim) return fail(GS_ERR_ARG, "feat_ld %lld < feat_dim %d", (long long)feat_ld, feat_dim);
+        if (!aligned(d_features, (size_t)eb)) return fail(GS_ERR_ALIGN, "d_features must be aligned to its element size");
+    }
+    gs_graph* g = new (std::nothrow) gs_graph{num_nodes, num_edges, d_indptr, d_indices, d_features, dtype, feat_dim, feat_ld, eb};
+    if (!g) return fail(GS_ERR_ARG, "out of host memory");
+    *out = g;
+    return GS_OK;
+}
+
+void gs_graph_destroy(gs_graph* g) { delete g; }
+
+gs_status gs_cache_bytes(const gs_graph* g, int32_t num_hops, int32_t cache_width, int32_t shared, size_t* bytes) {
+    if (!bytes) return fail(GS_ERR_ARG, "bytes is NULL");
+    gs_status st = check_shape(g, num_hops, cache_width);
+    if (st != GS_OK) return st;
+    *bytes = HDR_BYTES + table_bytes(g) + slots_bytes(g, shared ? 1 : num_hops, cache_width);
+    return GS_OK;
+}
+
+static gs_status check_fanouts(int32_t num_hops, const int32_t* fanouts, int32_t limit) {
+    if (!fanouts) return fail(GS_ERR_ARG, "fanouts is NULL");
+    for (int l = 0; l < num_hops; ++l)
+        if (fanouts[l] < 1 || fanouts[l] > limit) return fail(GS_ERR_ARG, "fanouts[%d] = %d outside [1, %d]", l, fanouts[l], limit);
+    return GS_OK;
+}
+
+gs_status gs_workspace_bytes(const gs_graph* g, int32_t num_hops, const int32_t* fanouts, int32_t max_seeds, size_t* bytes) {
+    if (!bytes) return fail(GS_ERR_ARG, "bytes is NULL");
+    gs_status st = check_shape(g, num_hops, 1);
+    if (st != GS_OK) return st;
+    st = check_fanouts(num_hops, fanouts, GS_MAX_CACHE_WIDTH);
+    if (st != GS_OK) return st;
+    if (max_seeds < 1) return fail(GS_ERR_ARG, "max_seeds must be >= 1");
+    const Bounds b = make_bounds(g->num_nodes, num_hops, fanouts, max_seeds);
+    for (int k = 0; k < num_hops; ++k)
+        if (b.nb[k] + b.mb[k] >= ((int64_t)1 << 31)) return fail(GS_ERR_ARG, "batch too large: positions would exceed 2^31");
+    *bytes = make_layout(b).total;
+    return GS_OK;
+}
+
+gs_status gs_cache_init(const gs_graph* g, int32_t num_hops, const int32_t* fanouts, int32_t cache_width, uint64_t seed,
+                        int32_t shared, void* d_cache_storage, size_t cache_bytes, void* stream, gs_cache** out) {
+    if (!out) return fail(GS_ERR_ARG, "out is NULL");
+    *out = nullptr;
+    gs_status st = check_shape(g, num_hops, cache_width);
+    if (st != GS_OK) return st;
+    st = check_fanouts(num_hops, fanouts, cache_width);
+    if (st != GS_OK) return st;
+    if (!d_cache_storage) return fail(GS_ERR_ARG, "d_cache_storage is NULL");
+    if (!aligned(d_cache_storage, 256)) return fail(GS_ERR_ALIGN, "d_cache_storage must be 256-byte aligned");
+    size_t need = 0;
+    gs_cache_bytes(g, num_hops, cache_width, shared, &need);
+    if (cache_bytes < need) return fail(GS_ERR_WORKSPACE, "cache storage has %zu bytes, %zu needed", cache_bytes, need);
+
+    gs_cache* c = new (std::nothrow) gs_cache{};
+    if (!c) return fail(GS_ERR_ARG, "out of host memory");
+    c->graph = g;
+    c->L = num_hops;
+    c->W = cache_width;
+    c->pitch = pitch_for(cache_width);
+    c->shared = shared ? 1 : 0;
+    c->num_caches = shared ? 1 : num_hops;
+    memcpy(c->fanouts, fanouts, (size_t)num_hops * sizeof(int32_t));
+    c->seed = seed;
+    c->d_storage = (char*)d_cache_storage;
+    c->d_hdr = (int32_t*)c->d_storage;
+    c->d_table = (unsigned long long*)(c->d_storage + HDR_BYTES);
+    c->d_slots = (int32_t*)(c->d_storage + HDR_BYTES + table_bytes(g));
+    c->slot_bytes = (size_t)c->num_caches * (size_t)g->num_nodes * (size_t)c->pitch * 4;
+    c->serial = 0;
+    c->lambda_otf = 16.0f;
+    c->lambda_full = 72.0f;
+    c->hub_degree = 16384;
+    cudaError_t e = cudaMallocHost((void**)&c->h_pinned, 64 * sizeof(int32_t));
+    if (e != cudaSuccess) { delete c; return cuda_fail(e, "cudaMallocHost"); }
+
+    cudaStream_t s = (cudaStream_t)stream;
+    e = cudaMemsetAsync(c->d_hdr, 0, HDR_BYTES, s);
+    if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "cudaMemsetAsync"); }
+    // S0: a full refresh (r = W) of every node at step 0, rows with deg <= W copied verbatim.
+    // The relabel table is not in use yet and serves as the hub list of these launches.
+    for (int ci = 0; ci < c->num_caches; ++ci) {
+        StepParams P = step_params(c, ci, 0u);
+        P.r = c->W;
+        P.frontier = nullptr;
+        P.d_n = nullptr;
+        P.n_host = (int32_t)g->num_nodes;
+        P.d_refresh_from = nullptr;
+        P.do_pick = 0;
+        P.init_rows = 1;
+        P.hub_list = (int32_t*)c->d_table;
+        P.hub_count = c->d_hdr + HDR_HUBS + ci;
+        P.work_counter = c->d_hdr + HDR_WORK + ci;
+        e = launch_refresh_pick(P, g->num_nodes, s);
+        if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "pre-sample launch"); }
+    }
+    e = cudaMemsetAsync(c->d_table, 0xFF, (size_t)g->num_nodes * 8, s);
+    if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "cudaMemsetAsync"); }
+    *out = c;
+    return GS_OK;
+}
+
+void gs_cache_destroy(gs_cache* c) {
+    if (!c) return;
+    if (c->h_pinned) cudaFreeHost(c->h_pinned);
+    delete c;
+}
+
+gs_status gs_cache_set_tuning(gs_cache* c, double lambda_otf, double lambda_full, int32_t hub_degree) {
+    if (!c) return fail(GS_ERR_ARG, "cache is NULL");
+    if (lambda_otf > 0) c->lambda_otf = (float)lambda_otf;
+    if (lambda_full > 0) c->lambda_full = (float)lambda_full;
+    if (hub_degree > 0) c->hub_degree = hub_degree;
+    return GS_OK;
+}
+
+static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_seeds, gs_mode mode, double gamma,
+                             uint32_t step, void* d_workspace, size_t workspace_bytes, cudaStream_t s,
+                             gs_block* blocks, const int32_t** d_input_nodes, const int32_t** d_num_input_nodes) {
+    const gs_graph* g = c->graph;
+    const int L = c->L;
+    int32_t r;
+    if (mode == GS_MODE_FCR) {
+        r = c->W;
+    } else {
+        double rr = std::floor(gamma * (double)c->W + 0.5);
+        r = rr < 0 ? 0 : (rr > c->W ? c->W : (int32_t)rr);
+    }
+    const Bounds b = make_bounds(g->num_nodes, L, c->fanouts, num_seeds);
+    const WorkspaceLayout w = make_layout(b);
+    if (workspace_bytes < w.total) return fail(GS_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, w.total);
+    char* ws = (char*)d_workspace;
+    int32_t* frontier = (int32_t*)(ws + w.frontier);
+    int32_t* picked = (int32_t*)(ws + w.picked);
+    int32_t* aux = (int32_t*)(ws + w.aux);
+    int32_t* tiles_a = (int32_t*)(ws + w.tiles_a);
+    int32_t* tiles_e = (int32_t*)(ws + w.tiles_e);
+    int32_t* hub_list = (int32_t*)(ws + w.hub_list);
+
+    if (c->serial == 0xFFFFFFFEu) {  // stamp space used up: start over with a clean table
+        GS_CUDA(cudaMemsetAsync(c->d_table, 0xFF, (size_t)g->num_nodes * 8, s));
+        c->serial = 0;
+    }
+    c->serial += 1;
+    const uint32_t stamp = 0xFFFFFFFFu - c->serial;  // newer batches always win the atomicMin
+    GS_CUDA(cudaMemsetAsync(c->d_hdr, 0, HDR_BYTES, s));
+
+    for (int k = 0; k < L; ++k) {
+        const int layer = L - 1 - k;
+        int32_t* blk_indptr = (int32_t*)(ws + w.blk_indptr[k]);
+        int32_t* blk_indices = (int32_t*)(ws + w.blk_indices[k]);
+
+        CountParams C{};
+        C.g = GraphView{g->d_indptr, g->d_indices, g->num_nodes};
+        C.seeds = (k == 0) ? d_seeds : nullptr;
+        C.frontier = frontier;
+        C.hdr = c->d_hdr;
+        C.k = k;
+        C.f = c->fanouts[layer];
+        C.n_host = num_seeds;
+        C.blk_indptr = blk_indptr;
+        C.tile_sums = tiles_a;
+        C.table = c->d_table;
+        C.stamp = stamp;
+        GS_CUDA(launch_row_counts(C, b.nb[k], s));
+
+        StepParams P = step_params(c, layer, step);
+        P.r = r;
+        P.frontier = frontier;
+        P.d_n = c->d_hdr + HDR_N + k;
+        P.n_host = 0;
+        P.d_refresh_from = (c->shared && k > 0) ? c->d_hdr + HDR_N + (k - 1) : nullptr;
+        P.blk_indptr = blk_indptr;
+        P.picked = picked;
+        P.stamp = stamp;
+        P.hub_list = hub_list;
+        P.hub_count = c->d_hdr + HDR_HUBS + k;
+        P.work_counter = c->d_hdr + HDR_WORK + k;
+        P.do_pick = 1;
+        P.init_rows = 0;
+        GS_CUDA(launch_refresh_pick(P, b.nb[k], s));
+
+        RelabelParams R{};
+        R.hdr = c->d_hdr;
+        R.k = k;
+        R.picked = picked;
+        R.aux = aux;
+        R.tile_sums = tiles_e;
+        R.frontier = frontier;
+        R.local = blk_indices;
+        R.table = c->d_table;
+        R.stamp = stamp;
+        R.n_cap = b.nb[k + 1];
+        GS_CUDA(launch_relabel(R, b.mb[k], s));
+
+        gs_block& B = blocks[layer];
+        B.max_dst = (int32_t)b.nb[k];
+        B.max_src = (int32_t)b.nb[k + 1];
+        B.max_edges = (int32_t)b.mb[k];
+        B.d_num_dst = c->d_hdr + HDR_N + k;
+        B.d_num_src = c->d_hdr + HDR_N + k + 1;
+        B.d_num_edges = c->d_hdr + HDR_M + k;
+        B.d_indptr = blk_indptr;
+        B.d_indices = blk_indices;
+    }
+    if (d_input_nodes) *d_input_nodes = frontier;
+    if (d_num_input_nodes) *d_num_input_nodes = c->d_hdr + HDR_N + L;
+    return GS_OK;
+}
+
+static gs_status check_batch_args(gs_cache* c, const int32_t* seeds, int32_t num_seeds, gs_mode mode, double gamma,
+                                  uint32_t step, void* d_workspace, gs_block* blocks) {
+    if (!c) return fail(GS_ERR_ARG, "cache is NULL");
+    if (!seeds) return fail(GS_ERR_ARG, "seeds is NULL");
+    if (num_seeds < 1) return fail(GS_ERR_ARG, "num_seeds must be >= 1");
+    if ((int64_t)num_seeds > c->graph->num_nodes) return fail(GS_ERR_ARG, "more seeds than nodes");
+    if (mode != GS_MODE_FCR && mode != GS_MODE_OTF) return fail(GS_ERR_ARG, "unknown mode %d", (int)mode);
+    if (mode == GS_MODE_OTF && !(gamma >= 0.0 && gamma <= 1.0)) return fail(GS_ERR_ARG, "gamma outside [0, 1]");
+    if (step == 0) return fail(GS_ERR_ARG, "step 0 is reserved for the pre-sample");
+    if (!d_workspace) return fail(GS_ERR_ARG, "d_workspace is NULL");
+    if (!aligned(d_workspace, 256)) return fail(GS_ERR_ALIGN, "d_workspace must be 256-byte aligned");
+    if (!blocks) return fail(GS_ERR_ARG, "blocks is NULL");
+    return GS_OK;
+}
+
+gs_status gs_sample_batch(gs_cache* c, const int32_t* d_seeds, int32_t num_seeds, gs_mode mode, double gamma,
+                          uint32_t step, void* d_workspace, size_t workspace_bytes, void* stream, gs_block* blocks,
+                          const int32_t** d_input_nodes, const int32_t** d_num_input_nodes) {
+    gs_status st = check_batch_args(c, d_seeds, num_seeds, mode, gamma, step, d_workspace, blocks);
+    if (st != GS_OK) return st;
+    if (!aligned(d_seeds, 4)) return fail(GS_ERR_ALIGN, "d_seeds must be 4-byte aligned");
+    return sample_impl(c, d_seeds, num_seeds, mode, gamma, step, d_workspace, workspace_bytes, (cudaStream_t)stream,
+                       blocks, d_input_nodes, d_num_input_nodes);
+}
+
+gs_status gs_batch_counts(gs_cache* c, void* stream, int32_t* h_num_nodes, int32_t* h_num_edges) {
+    if (!c) return fail(GS_ERR_ARG, "cache is NULL");
+    cudaStream_t s = (cudaStream_t)stream;
+    GS_CUDA(cudaMemcpyAsync(c->h_pinned, c->d_hdr, (size_t)(HDR_M + GS_MAX_HOPS) * 4, cudaMemcpyDeviceToHost, s));
+    GS_CUDA(cudaStreamSynchronize(s));
+    const int status = c->h_pinned[HDR_STATUS];
+    if (h_num_nodes)
+        for (int k = 0; k <= c->L; ++k) h_num_nodes[k] = c->h_pinned[HDR_N + k];
+    if (h_num_edges)
+        for (int l = 0; l < c->L; ++l) h_num_edges[l] = c->h_pinned[HDR_M + (c->L - 1 - l)];
+    if (status == GS_ERR_RANGE) return fail(GS_ERR_RANGE, "a seed id is outside [0, num_nodes)");
+    if (status == GS_ERR_DUP_SEED) return fail(GS_ERR_DUP_SEED, "duplicate seed id in the batch");
+    if (status != 0) return fail(GS_ERR_CUDA, "unexpected device status %d", status);
+    return GS_OK;
+}
+
+gs_status gs_sync_status(gs_cache* c, void* stream) { return gs_batch_counts(c, stream, nullptr, nullptr); }
+
+gs_status gs_sample_batch_host(gs_cache* c, const int32_t* h_seeds, int32_t num_seeds, gs_mode mode, double gamma,
+                               uint32_t step, void* d_workspace, size_t workspace_bytes, void* stream, gs_block* blocks,
+                               const int32_t** d_input_nodes, int32_t* h_num_nodes, int32_t* h_num_edges) {
+    gs_status st = check_batch_args(c, h_seeds, num_seeds, mode, gamma, step, d_workspace, blocks);
+    if (st != GS_OK) return st;
+    // The seeds are staged in the relabel scratch array: its first writer (step 0's
+    // first-occurrence kernel) runs after the row-count kernel has copied the seeds out.
+    const Bounds b = make_bounds(c->graph->num_nodes, c->L, c->fanouts, num_seeds);
+    const WorkspaceLayout w = make_layout(b);
+    if (workspace_bytes < w.total) return fail(GS_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, w.total);
+    int32_t* d_stage = (int32_t*)((char*)d_workspace + w.aux);
+    cudaStream_t s = (cudaStream_t)stream;
+    GS_CUDA(cudaMemcpyAsync(d_stage, h_seeds, (size_t)num_seeds * 4, cudaMemcpyHostToDevice, s));
+    st = sample_impl(c, d_stage, num_seeds, mode, gamma, step, d_workspace, workspace_bytes, s, blocks, d_input_nodes, nullptr);
+    if (st != GS_OK) return st;
+    return gs_batch_counts(c, stream, h_num_nodes, h_num_edges);
+}
+
+gs_status gs_gather_features(const gs_graph* g, const int32_t* d_ids, const int32_t* d_count_or_null, int32_t count_bound,
+                             void* d_out, int64_t out_ld, void* stream) {
+    if (!g) return fail(GS_ERR_ARG, "graph is NULL");
+    if (!g->d_features) return fail(GS_ERR_ARG, "the graph was created without features");
+    if (count_bound < 0) return fail(GS_ERR_ARG, "count_bound is negative");
+    if (count_bound == 0) return GS_OK;  // nothing to copy; an empty output may have no address
+    if (!d_ids || !d_out) return fail(GS_ERR_ARG, "d_ids or d_out is NULL");
+    if (out_ld < g->feat_dim) return fail(GS_ERR_ARG, "out_ld %lld < feat_dim %d", (long long)out_ld, g->feat_dim);
+    if (!aligned(d_out, (size_t)g->elem_bytes)) return fail(GS_ERR_ALIGN, "d_out must be aligned to the element size");
+    if (!aligned(d_ids, 4)) return fail(GS_ERR_ALIGN, "d_ids must be 4-byte aligned");
+    GS_CUDA(launch_gather(g->d_features, g->feat_ld * g->elem_bytes, (int64_t)g->feat_dim * g->elem_bytes, d_ids,
+                          d_count_or_null, count_bound, d_out, out_ld * g->elem_bytes, (cudaStream_t)stream));
+    return GS_OK;
+}
+
+gs_status gs_cache_read_rows(const gs_cache* c, int32_t layer, const int32_t* d_nodes, int32_t n, int32_t* d_out, void* stream) {
+    if (!c) return fail(GS_ERR_ARG, "cache is NULL");
+    if (layer < 0 || layer >= c->L) return fail(GS_ERR_ARG, "layer %d outside [0, %d)", layer, c->L);
+    if (n < 0 || (n > 0 && (!d_nodes || !d_out))) return fail(GS_ERR_ARG, "bad node list");
+    const int32_t ci = c->shared ? 0 : layer;
+    const int32_t* slots = c->d_slots + (size_t)ci * (size_t)c->graph->num_nodes * c->pitch;
+    GS_CUDA(launch_read_rows(slots, c->pitch, c->W, d_nodes, n, d_out, (cudaStream_t)stream));
+    return GS_OK;
+}
+
+gs_status gs_cache_export_bytes(const gs_cache* c, size_t* bytes) {
+    if (!c || !bytes) return fail(GS_ERR_ARG, "NULL argument");
+    *bytes = c->slot_bytes;
+    return GS_OK;
+}
+
+gs_status gs_cache_export(const gs_cache* c, void* d_dst, size_t bytes, void* stream) {
+    if (!c || !d_dst) return fail(GS_ERR_ARG, "NULL argument");
+    if (bytes < c->slot_bytes) return fail(GS_ERR_WORKSPACE, "export buffer has %zu bytes, %zu needed", bytes, c->slot_bytes);
+    GS_CUDA(cudaMemcpyAsync(d_dst, c->d_slots, c->slot_bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    return GS_OK;
+}
+
+gs_status gs_cache_import(gs_cache* c, const void* d_src, size_t bytes, void* stream) {
+    if (!c || !d_src) return fail(GS_ERR_ARG, "NULL argument");
+    if (bytes != c->slot_bytes) return fail(GS_ERR_WORKSPACE, "import blob has %zu bytes, %zu expected", bytes, c->slot_bytes);
+    GS_CUDA(cudaMemcpyAsync(c->d_slots, d_src, c->slot_bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    return GS_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,99 @@
+// Device-side primitives: Philox4x32-10, warp selection, block scan.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gs {
+
+constexpr uint32_t FULL = 0xFFFFFFFFu;
+constexpr int CAND_CAP = 128;  // candidate buffer entries per node (4 per lane)
+
+enum Purpose : uint32_t { FILL = 1, EVICT = 2, PICK = 3 };
+
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and a key bump.
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               uint32_t k0, uint32_t k1) {
+#pragma unroll
+    for (int round = 0; round < 10; ++round) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        const uint32_t n0 = hi1 ^ c1 ^ k0;
+        const uint32_t n2 = hi0 ^ c3 ^ k1;
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+__device__ __forceinline__ uint32_t word_of(const uint4& o, uint32_t w) {
+    return w == 0 ? o.x : (w == 1 ? o.y : (w == 2 ? o.z : o.w));
+}
+
+__device__ __forceinline__ uint32_t lanemask_lt() {
+    uint32_t m;
+    asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+    return m;
+}
+
+// Lanes in `valid` hold (key, lane) pairs; returns the mask of the k pairs smallest in
+// (key, lane) order.  Runs min(k, n-k) rounds of a warp-wide min (or max) reduction.
+__device__ __forceinline__ uint32_t warp_smallest_k(uint32_t key, uint32_t valid, int k, int lane) {
+    const int n = __popc(valid);
+    if (k >= n) return valid;
+    if (k <= 0) return 0u;
+    const bool mine = (valid >> lane) & 1u;
+    if (k <= n - k) {
+        uint32_t sel = 0;
+        for (int t = 0; t < k; ++t) {
+            const bool live = mine && !((sel >> lane) & 1u);
+            const uint32_t x = live ? key : 0xFFFFFFFFu;
+            const uint32_t m = __reduce_min_sync(FULL, x);
+            const uint32_t b = __ballot_sync(FULL, live && x == m);
+            sel |= b & (0u - b);  // lowest lane among equal keys
+        }
+        return sel;
+    }
+    uint32_t rem = 0;
+    for (int t = 0; t < n - k; ++t) {
+        const bool live = mine && !((rem >> lane) & 1u);
+        const uint32_t x = live ? key : 0u;
+        const uint32_t m = __reduce_max_sync(FULL, x);
+        const uint32_t b = __ballot_sync(FULL, live && x == m);
+        rem |= 0x80000000u >> __clz(b);  // highest lane among equal keys is the largest pair
+    }
+    return valid & ~rem;
+}
+
+// Exclusive scan of one int per thread over a block of BT threads (BT a multiple of 32, <= 1024).
+// `warp_sums` is shared memory with at least 33 ints.  Returns the exclusive prefix; *total gets
+// the block sum.  Contains __syncthreads: every thread of the block must call it.
+template <int BT>
+__device__ __forceinline__ int block_exclusive_scan(int x, int* warp_sums, int* total) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    int incl = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int y = __shfl_up_sync(FULL, incl, d);
+        if (lane >= d) incl += y;
+    }
+    __syncthreads();  // protects warp_sums against a previous call's readers
+    if (lane == 31) warp_sums[wid] = incl;
+    __syncthreads();
+    if (wid == 0) {
+        int s = (lane < BT / 32) ? warp_sums[lane] : 0;
+        int si = s;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int y = __shfl_up_sync(FULL, si, d);
+            if (lane >= d) si += y;
+        }
+        if (lane < BT / 32) warp_sums[lane] = si - s;
+        if (lane == 31) warp_sums[32] = si;
+    }
+    __syncthreads();
+    *total = warp_sums[32];
+    return warp_sums[wid] + incl - x;
+}
+
+}  // namespace gs

@@ -1,0 +1,80 @@
+// S5 feature gather: out[p, :] = X[ids[p], :], a pure copy bound by HBM bandwidth.
+//
+// Rows are moved in the widest unit (16, 8, 4 or 2 bytes) that divides the row size, both row
+// pitches and both base addresses.  A block covers `rows_per_iter` rows at a time, a fixed group
+// of threads per row, and keeps four row groups in flight per thread.  Loads bypass L1 and are
+// marked streaming (no row is read twice: frontier ids are distinct), stores are streaming too.
+#include "gs_device.cuh"
+#include "gs_internal.h"
+
+namespace gs {
+
+constexpr int GT = 256;
+constexpr int G_UNROLL = 4;
+
+template <typename V> __device__ __forceinline__ V ld_stream(const V* p) { return __ldcs(p); }
+template <typename V> __device__ __forceinline__ void st_stream(V* p, V v) { __stcs(p, v); }
+
+template <typename V>
+__global__ void __launch_bounds__(GT) k_gather(const char* __restrict__ src, int64_t src_ld, int units,
+                                               const int32_t* __restrict__ ids, const int32_t* __restrict__ d_count,
+                                               int count_bound, char* __restrict__ dst, int64_t dst_ld) {
+    int n = d_count ? __ldg(d_count) : count_bound;
+    if (n > count_bound) n = count_bound;
+    // thread -> (row within group, first unit); tpr threads per row
+    const int tpr = units < GT ? units : GT;
+    const int rows_per_iter = GT / tpr;
+    const int r_in = threadIdx.x / tpr;
+    const int u0 = threadIdx.x - r_in * tpr;
+    if (r_in >= rows_per_iter) return;
+    const int64_t stride = (int64_t)gridDim.x * rows_per_iter;
+    for (int64_t row = (int64_t)blockIdx.x * rows_per_iter + r_in; row < n; row += stride * G_UNROLL) {
+        const V* s[G_UNROLL];
+        V* d[G_UNROLL];
+#pragma unroll
+        for (int j = 0; j < G_UNROLL; ++j) {
+            const int64_t rj = row + j * stride;
+            const int32_t id = rj < n ? __ldg(ids + rj) : -1;
+            s[j] = id >= 0 ? reinterpret_cast<const V*>(src + (int64_t)id * src_ld) : nullptr;
+            d[j] = reinterpret_cast<V*>(dst + rj * dst_ld);
+        }
+        for (int u = u0; u < units; u += tpr) {
+            V val[G_UNROLL];
+#pragma unroll
+            for (int j = 0; j < G_UNROLL; ++j)
+                if (s[j]) val[j] = ld_stream(s[j] + u);
+#pragma unroll
+            for (int j = 0; j < G_UNROLL; ++j)
+                if (s[j]) st_stream(d[j] + u, val[j]);
+        }
+    }
+}
+
+template <typename V>
+static void launch_t(const void* src, int64_t src_ld, int64_t row_bytes, const int32_t* ids, const int32_t* d_count,
+                     int32_t count_bound, void* dst, int64_t dst_ld, cudaStream_t s) {
+    const int units = (int)(row_bytes / (int64_t)sizeof(V));
+    const int tpr = units < GT ? units : GT;
+    const int rows_per_iter = GT / tpr;
+    int64_t blocks = ((int64_t)count_bound + (int64_t)rows_per_iter * G_UNROLL - 1) / ((int64_t)rows_per_iter * G_UNROLL);
+    const int64_t cap = 148 * 16;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    k_gather<V><<<(int)blocks, GT, 0, s>>>((const char*)src, src_ld, units, ids, d_count, count_bound, (char*)dst, dst_ld);
+}
+
+cudaError_t launch_gather(const void* src, int64_t src_ld_bytes, int64_t row_bytes, const int32_t* ids,
+                          const int32_t* d_count, int32_t count_bound, void* dst, int64_t dst_ld_bytes,
+                          cudaStream_t s) {
+    if (count_bound <= 0 || row_bytes <= 0) return cudaSuccess;
+    const uint64_t all = (uint64_t)(uintptr_t)src | (uint64_t)(uintptr_t)dst | (uint64_t)src_ld_bytes |
+                         (uint64_t)dst_ld_bytes | (uint64_t)row_bytes;
+    if ((all & 15) == 0) launch_t<uint4>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, s);
+    else if ((all & 7) == 0) launch_t<uint2>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, s);
+    else if ((all & 3) == 0) launch_t<uint32_t>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, s);
+    else launch_t<uint16_t>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, s);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+}  // namespace gs

@@ -1,0 +1,211 @@
+// Row counts + block CSR offsets (S4) and dedup / relabel (S3).
+//
+// Both are "tile-local scan, last block scans the tile sums" kernels: no block ever waits for
+// another one, so there is no spin anywhere.
+#include "gs_device.cuh"
+#include "gs_internal.h"
+
+namespace gs {
+
+__device__ __forceinline__ void raise_status(int32_t* status, int code) { atomicCAS(status, 0, code); }
+
+// In-place exclusive scan of tile_sums[0..T) by one block of 1024 threads; returns the total.
+__device__ int scan_tiles_in_place(int32_t* tile_sums, int T, int* warp_sums) {
+    int carry = 0;
+    for (int base = 0; base < T; base += 1024) {
+        const int i = base + (int)threadIdx.x;
+        const int x = (i < T) ? __ldcg(tile_sums + i) : 0;
+        int total;
+        const int excl = block_exclusive_scan<1024>(x, warp_sums, &total);
+        if (i < T) tile_sums[i] = carry + excl;
+        carry += total;
+    }
+    return carry;
+}
+
+// ---------------------------------------------------------------- row counts
+// Per frontier node p: count(p) = min(f, deg(frontier[p])) - the number of picks is known from the
+// degree alone, so the block CSR offsets exist before anything is sampled.  Step 0 also copies
+// the seeds into the frontier, validates them and preloads the relabel table with their positions.
+__global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
+    __shared__ int warp_sums[33];
+    __shared__ int is_last;
+    __shared__ int s_status;
+    int32_t* status = P.hdr + HDR_STATUS;
+    if (threadIdx.x == 0) s_status = __ldcg(status);
+    __syncthreads();
+    if (s_status != 0) return;  // block-uniform: the barriers below stay convergent
+    const int n = (P.k == 0) ? P.n_host : __ldcg(P.hdr + HDR_N + P.k);
+    const int p = blockIdx.x * SCAN_A_TILE + threadIdx.x;
+    int c = 0;
+    if (p < n) {
+        int v;
+        if (P.k == 0) {
+            v = P.seeds[p];
+            if (v < 0 || (int64_t)v >= P.g.num_nodes) {
+                raise_status(status, GS_ERR_RANGE);
+                v = -1;
+            } else {
+                P.frontier[p] = v;
+                const unsigned long long mine = ((unsigned long long)P.stamp << 32) | (unsigned)p;
+                const unsigned long long old = atomicMin(P.table + v, mine);
+                if ((uint32_t)(old >> 32) == P.stamp) raise_status(status, GS_ERR_DUP_SEED);
+            }
+        } else {
+            v = P.frontier[p];
+        }
+        if (v >= 0) {
+            const int64_t deg = P.g.indptr[v + 1] - P.g.indptr[v];
+            c = deg < (int64_t)P.f ? (int)deg : P.f;
+        }
+    }
+    int total;
+    const int excl = block_exclusive_scan<SCAN_A_TILE>(c, warp_sums, &total);
+    if (p < n) P.blk_indptr[p] = excl;
+    if (threadIdx.x == 0) {
+        P.tile_sums[blockIdx.x] = total;
+        __threadfence();
+        const int ticket = atomicAdd(P.hdr + HDR_TICKET_A + P.k, 1);
+        is_last = (ticket == (int)gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const int m = scan_tiles_in_place(P.tile_sums, (int)gridDim.x, warp_sums);
+    if (threadIdx.x == 0) {
+        P.hdr[HDR_M + P.k] = m;
+        if (P.k == 0) P.hdr[HDR_N] = n;
+    }
+}
+
+__global__ void __launch_bounds__(1024) k_row_offsets(CountParams P) {
+    if (__ldcg(P.hdr + HDR_STATUS) != 0) return;
+    const int n = (P.k == 0) ? P.n_host : __ldcg(P.hdr + HDR_N + P.k);
+    const int p = blockIdx.x * SCAN_A_TILE + threadIdx.x;
+    if (p < n) P.blk_indptr[p] += P.tile_sums[p / SCAN_A_TILE];
+    else if (p == n) P.blk_indptr[n] = __ldcg(P.hdr + HDR_M + P.k);
+}
+
+cudaError_t launch_row_counts(const CountParams& p, int64_t n_bound, cudaStream_t s) {
+    const int tiles = (int)((n_bound + SCAN_A_TILE - 1) / SCAN_A_TILE);
+    k_row_counts<<<tiles, SCAN_A_TILE, 0, s>>>(p);
+    k_row_offsets<<<(int)(n_bound / SCAN_A_TILE) + 1, SCAN_A_TILE, 0, s>>>(p);
+    count_launches(2);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- dedup + relabel
+// The picks were written with atomicMin(table[id], position) where the position of pick e in the
+// list "frontier ++ picked" is n + e; frontier members already sit in the table with positions
+// < n.  Pass 1 marks each id's first occurrence and scans the marks; pass 2 turns them into
+// block-local ids, appends the new ids to the frontier and stores their final position in the
+// table (which is exactly the preload the next step needs).
+//
+// aux[e] holds, for a first occurrence, -(tile-local rank)-1, otherwise the table position.
+__global__ void __launch_bounds__(1024) k_first_flags(RelabelParams P) {
+    __shared__ int warp_sums[33];
+    __shared__ int is_last;
+    __shared__ int s_status;
+    if (threadIdx.x == 0) s_status = __ldcg(P.hdr + HDR_STATUS);
+    __syncthreads();
+    if (s_status != 0) return;  // block-uniform
+    const int n = __ldcg(P.hdr + HDR_N + P.k);
+    const int m = __ldcg(P.hdr + HDR_M + P.k);
+    const int base = blockIdx.x * SCAN_E_TILE + threadIdx.x * 4;
+    int pos[4];
+    int flag[4];
+    int tsum = 0;
+    if (base < m) {
+        const int4 ids = *reinterpret_cast<const int4*>(P.picked + base);  // buffer is padded to 4
+        const int id[4] = {ids.x, ids.y, ids.z, ids.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            pos[j] = 0;
+            flag[j] = 0;
+            if (base + j < m) {
+                pos[j] = (int)(uint32_t)__ldcg(P.table + id[j]);
+                flag[j] = (pos[j] == n + base + j);
+                tsum += flag[j];
+            }
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { pos[j] = 0; flag[j] = 0; }
+    }
+    int total;
+    int run = block_exclusive_scan<1024>(tsum, warp_sums, &total);
+    if (base < m) {
+        int out[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            out[j] = flag[j] ? -run - 1 : pos[j];
+            run += flag[j];
+        }
+        *reinterpret_cast<int4*>(P.aux + base) = make_int4(out[0], out[1], out[2], out[3]);
+    }
+    if (threadIdx.x == 0) {
+        P.tile_sums[blockIdx.x] = total;
+        __threadfence();
+        const int ticket = atomicAdd(P.hdr + HDR_TICKET_E + P.k, 1);
+        is_last = (ticket == (int)gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const int fresh = scan_tiles_in_place(P.tile_sums, (int)gridDim.x, warp_sums);
+    if (threadIdx.x == 0) P.hdr[HDR_N + P.k + 1] = n + fresh;
+}
+
+__global__ void __launch_bounds__(256) k_relabel(RelabelParams P) {
+    if (__ldcg(P.hdr + HDR_STATUS) != 0) return;
+    const int n = __ldcg(P.hdr + HDR_N + P.k);
+    const int m = __ldcg(P.hdr + HDR_M + P.k);
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < m; e += gridDim.x * blockDim.x) {
+        const int val = P.aux[e];
+        int loc;
+        if (val < 0) {
+            loc = n + (-val - 1) + P.tile_sums[e / SCAN_E_TILE];
+            if ((int64_t)loc < P.n_cap) {
+                const int id = P.picked[e];
+                P.frontier[loc] = id;
+                P.table[id] = ((unsigned long long)P.stamp << 32) | (unsigned)loc;
+            }
+        } else if (val < n) {
+            loc = val;
+        } else {
+            const int e0 = val - n;
+            loc = n + (-P.aux[e0] - 1) + P.tile_sums[e0 / SCAN_E_TILE];
+        }
+        P.local[e] = loc;
+    }
+}
+
+cudaError_t launch_relabel(const RelabelParams& p, int64_t m_bound, cudaStream_t s) {
+    if (m_bound <= 0) m_bound = 1;
+    const int tiles = (int)((m_bound + SCAN_E_TILE - 1) / SCAN_E_TILE);
+    k_first_flags<<<tiles, 1024, 0, s>>>(p);
+    int64_t blocks = (m_bound + 255) / 256;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    k_relabel<<<(int)blocks, 256, 0, s>>>(p);
+    count_launches(2);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- logical cache rows (parity / debug)
+__global__ void k_read_rows(const int32_t* slots, int pitch, int W, const int32_t* nodes, int n, int32_t* out) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n * W) return;
+    const int row = i / W, j = i - row * W;
+    out[i] = slots[(int64_t)nodes[row] * pitch + j];
+}
+
+cudaError_t launch_read_rows(const int32_t* slots, int32_t pitch, int32_t W, const int32_t* nodes, int32_t n,
+                             int32_t* out, cudaStream_t s) {
+    if (n <= 0) return cudaSuccess;
+    const int64_t total = (int64_t)n * W;
+    k_read_rows<<<(int)((total + 255) / 256), 256, 0, s>>>(slots, pitch, W, nodes, n, out);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+}  // namespace gs

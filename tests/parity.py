@@ -1,0 +1,89 @@
+"""Runs the CUDA library and the CPU oracle on the same seeded inputs and compares every output
+bit for bit (tolerance 0: ids, offsets and copied feature bits are integers)."""
+import numpy as np
+import torch
+
+import oracle
+import paper_2406_17918_b200 as gs
+from workloads import batch_seeds, build_features, build_graph, seed_permutation
+
+MODES = {"fcr": (gs.GS_MODE_FCR, oracle.MODE_FCR), "otf": (gs.GS_MODE_OTF, oracle.MODE_OTF)}
+
+
+def bits(t: torch.Tensor) -> np.ndarray:
+    """Feature tensor -> integer bit patterns (numpy has no bfloat16)."""
+    t = t.detach().cpu().contiguous()
+    return t.view(torch.int32 if t.dtype == torch.float32 else torch.int16).numpy()
+
+
+class Pair:
+    """One graph resident on the GPU (library) and on the host (oracle), same bytes."""
+
+    def __init__(self, cfg, seed=0x1234ABCD5678EF01, gen_device="cuda", features=True):
+        self.cfg = cfg
+        g = build_graph(cfg, device=gen_device if cfg["kind"] == "rmat" else "cpu")
+        self.g_dev = g.to("cuda")
+        self.indptr = g.indptr.cpu().numpy()
+        self.indices = g.indices.cpu().numpy()
+        self.deg = self.indptr[1:] - self.indptr[:-1]
+        self.X = build_features(cfg, device="cuda" if cfg["feat_kind"] == "hash" else "cpu").to("cuda") if features else None
+        self.perm = seed_permutation(cfg)
+        self.L, self.W, self.shared = len(cfg["fanouts"]), cfg["cache_width"], cfg["shared"]
+        self.G = gs.gs_graph_create(self.g_dev.indptr, self.g_dev.indices, self.X)
+        self.seed = seed
+
+    def samplers(self, max_seeds, tuning=None):
+        C = gs.gs_cache_init(self.G, self.cfg["fanouts"], self.W, self.seed, self.shared)
+        if tuning:
+            gs.gs_cache_set_tuning(C, **tuning)
+        ws = torch.empty(gs.gs_workspace_bytes(self.G, self.cfg["fanouts"], max_seeds), dtype=torch.uint8, device="cuda")
+        O = oracle.Sampler(self.indptr, self.indices, self.cfg["fanouts"], self.W, self.seed, self.shared)
+        return C, ws, O
+
+    def check_rows(self, C, O, nodes):
+        nodes = np.asarray(nodes, dtype=np.int32)
+        for layer in range(1 if self.shared else self.L):
+            got = gs.gs_cache_read_rows(C, layer, torch.from_numpy(nodes).cuda()).cpu().numpy()
+            want = O.cache_rows(layer, nodes)
+            assert np.array_equal(got, want), "cache rows differ at layer %d" % layer
+
+    def check_batch(self, C, ws, O, seeds, mode, gamma, step, features=True, rows=True, host_api=False):
+        gm, om = MODES[mode]
+        if host_api:
+            blocks, input_nodes, n, m = gs.gs_sample_batch_host(C, seeds.cpu(), gm, gamma, step, ws)
+            cnt = None
+        else:
+            blocks, input_nodes, cnt = gs.gs_sample_batch(C, seeds.cuda(), gm, gamma, step, ws)
+            n, m = gs.gs_batch_counts(C)
+        frontier, n_o, blocks_o = O.sample_batch(seeds.cpu().numpy(), om, gamma, step)
+        assert n == n_o, (n, n_o)
+        got_frontier = input_nodes[: n[self.L]].cpu().numpy()
+        assert np.array_equal(got_frontier, frontier)
+        for layer in range(self.L):
+            k = self.L - 1 - layer
+            bo = blocks_o[layer]
+            assert m[layer] == bo.num_edges
+            assert blocks[layer].max_dst >= n[k] and blocks[layer].max_src >= n[k + 1] and blocks[layer].max_edges >= m[layer]
+            assert np.array_equal(blocks[layer].indptr(n[k]).cpu().numpy(), bo.indptr)
+            assert np.array_equal(blocks[layer].indices(m[layer]).cpu().numpy(), bo.indices)
+            d = [int(x) for x in blocks[layer].counts_device()]
+            assert d == [n[k], n[k + 1], m[layer]]
+        if rows:
+            self.check_rows(C, O, frontier)
+        if features and self.X is not None:
+            out = torch.full((n[self.L] + 3, self.X.shape[1]), 7, dtype=self.X.dtype, device="cuda")
+            gs.gs_gather_features(self.G, input_nodes, cnt, out)
+            Xh = bits(self.X)
+            assert np.array_equal(bits(out[: n[self.L]]), oracle.gather(Xh, frontier))
+            if cnt is not None:   # rows past the device count stay untouched
+                assert bool((out[n[self.L]:] == 7).all())
+        return n, m
+
+    def run(self, mode, gamma, batches, batch_size=None, tuning=None, first_step=1, **kw):
+        B = batch_size or self.cfg["batch"]
+        C, ws, O = self.samplers(B, tuning)
+        out = []
+        for b in range(batches):
+            seeds = batch_seeds(self.perm, b, B)
+            out.append(self.check_batch(C, ws, O, seeds, mode, gamma, first_step + b, **kw))
+        return C, ws, O, out

@@ -1,0 +1,145 @@
+"""CUDA library vs CPU oracle, element by element, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from workloads import batch_seeds, get_config
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    from parity import Pair
+    return Pair(get_config("tiny"))
+
+
+@pytest.fixture(scope="module")
+def mid():
+    from parity import Pair
+    return Pair(get_config("mid"))
+
+
+@pytest.fixture(scope="module")
+def shared_cfg():
+    from parity import Pair
+    return Pair(get_config("shared"))
+
+
+def test_presample_all_rows_tiny_mid(tiny, mid):
+    for pair in (tiny, mid):
+        C, ws, O = pair.samplers(8)
+        pair.check_rows(C, O, np.arange(pair.cfg["num_nodes"], dtype=np.int32))
+
+
+def test_tiny_otf_20_batches(tiny):
+    tiny.run("otf", 0.25, 20)
+
+
+def test_tiny_fcr_and_gamma_edges(tiny):
+    tiny.run("fcr", 0.0, 4)
+    tiny.run("otf", 0.0, 3)
+    tiny.run("otf", 1.0, 3)
+
+
+def test_tiny_host_seed_entry_point(tiny):
+    tiny.run("otf", 0.25, 3, host_api=True)
+
+
+@pytest.mark.parametrize("mode,gamma", [("fcr", 1.0), ("otf", 0.1), ("otf", 0.3), ("otf", 0.5)])
+def test_mid_runs(mid, mode, gamma):
+    mid.run(mode, gamma, 4)
+
+
+@pytest.mark.parametrize("tuning", [
+    dict(lambda_otf=0.5, lambda_full=1.0),          # thresholds too tight: retry and exact paths decide
+    dict(lambda_otf=1e6, lambda_full=1e6),          # thresholds too loose: buffer overflow -> exact path
+    dict(hub_degree=40),                            # almost every refreshed node takes the block kernel
+    dict(lambda_otf=0.5, lambda_full=1.0, hub_degree=40),
+    dict(lambda_otf=1e6, lambda_full=1e6, hub_degree=40),
+])
+def test_mid_internal_paths_agree(mid, tuning):
+    mid.run("otf", 0.3, 2, tuning=tuning)
+    mid.run("fcr", 1.0, 1, tuning=tuning)
+
+
+def test_shared_cache_mode(shared_cfg):
+    shared_cfg.run("otf", 0.3, 3)
+    shared_cfg.run("fcr", 0.0, 1)
+
+
+def test_shared_presample_sample(shared_cfg):
+    C, ws, O = shared_cfg.samplers(8)
+    rng = np.random.default_rng(1)
+    hubs = np.argsort(-shared_cfg.deg)[:200]
+    nodes = np.concatenate([hubs, rng.integers(0, shared_cfg.cfg["num_nodes"], 3000)]).astype(np.int32)
+    shared_cfg.check_rows(C, O, nodes)
+
+
+def test_ragged_batch_sizes(tiny):
+    for B in (1, 2, 31, 33, 1000):
+        tiny.run("otf", 0.25, 2, batch_size=B)
+
+
+def test_whole_graph_as_seeds(tiny):
+    # every node is a seed: later frontiers cannot grow, dedup sees only known ids
+    C, ws, O, out = tiny.run("otf", 0.25, 1, batch_size=tiny.cfg["num_nodes"])
+    n, m = out[0]
+    assert n[0] == n[-1] == tiny.cfg["num_nodes"]
+
+
+def test_resume_from_export(tiny):
+    import paper_2406_17918_b200 as gs
+    B = tiny.cfg["batch"]
+    C, ws, O = tiny.samplers(B)
+    for b in range(3):
+        tiny.check_batch(C, ws, O, batch_seeds(tiny.perm, b, B), "otf", 0.25, b + 1)
+    blob = gs.gs_cache_export(C)
+    C2, ws2, _ = tiny.samplers(B)
+    gs.gs_cache_import(C2, blob)
+    for b in range(3, 6):
+        tiny.check_batch(C2, ws2, O, batch_seeds(tiny.perm, b, B), "otf", 0.25, b + 1)
+
+
+def test_device_detected_errors(tiny):
+    import paper_2406_17918_b200 as gs
+    B = 16
+    C, ws, O = tiny.samplers(B)
+    good = batch_seeds(tiny.perm, 0, B)
+    bad = good.clone()
+    bad[5] = tiny.cfg["num_nodes"] + 3
+    gs.gs_sample_batch(C, bad.cuda(), gs.GS_MODE_OTF, 0.25, 1, ws)
+    with pytest.raises(gs.GsError) as e:
+        gs.gs_batch_counts(C)
+    assert e.value.status == 3
+    dup = good.clone()
+    dup[7] = dup[2]
+    gs.gs_sample_batch(C, dup.cuda(), gs.GS_MODE_OTF, 0.25, 1, ws)
+    with pytest.raises(gs.GsError) as e:
+        gs.gs_batch_counts(C)
+    assert e.value.status == 5
+    # the cache is untouched by the rejected batches and the handle still works
+    tiny.check_batch(C, ws, O, good, "otf", 0.25, 1)
+
+
+def test_gather_alignment_paths():
+    import paper_2406_17918_b200 as gs
+    from parity import bits
+    g = torch.Generator().manual_seed(0)
+    indptr = torch.zeros(101, dtype=torch.int64, device="cuda")
+    indices = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ids = torch.randint(0, 100, (257,), generator=g).to(torch.int32).cuda()
+    for dtype, d, ld in ((torch.float32, 100, 100), (torch.float32, 1433, 1433), (torch.bfloat16, 128, 128),
+                         (torch.bfloat16, 7, 7), (torch.float32, 6, 8), (torch.bfloat16, 130, 136), (torch.float32, 3, 3)):
+        base = torch.randn((100, ld), generator=g).to(dtype).cuda()
+        X = base[:, :d]
+        G = gs.gs_graph_create(indptr, indices, X)
+        for out_ld in (d, d + 3):
+            outb = torch.zeros((257, out_ld), dtype=dtype, device="cuda")
+            out = outb[:, :d]
+            gs.gs_gather_features(G, ids, None, out)
+            assert np.array_equal(bits(out), oracle.gather(bits(X), ids.cpu().numpy()))
+            assert bool((outb[:, d:] == 0).all())
+    out = torch.zeros((0, 3), dtype=torch.float32, device="cuda")
+    gs.gs_gather_features(G, ids, None, out)           # empty gather is a no-op
