@@ -1,0 +1,413 @@
+#!/usr/bin/env python
+"""Benchmark of the cached neighbour sampling hot path.
+
+One step = one mini-batch through the whole path: gs_sample_batch (refresh + pick + relabel +
+block CSR for every hop) followed by gs_gather_features for the input nodes, on fresh seeds and
+the next step number (the cache evolves as in training).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload scale|large|shared|mid|tiny]
+    python bench.py --impl reference ...        # times the CPU oracle on a bounded sample
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from workloads import batch_seeds, build_features, build_graph, get_config, seed_permutation  # noqa: E402
+
+METRIC = "sampled edges/s + feature GB/s per batch (OTF), fraction of HBM roofline"
+FALLBACK_HBM_GBS = 6650.0
+SAMPLER_SEED = 0x6A09E667F3BCC908
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.samples = []
+        self.proc = None
+        try:
+            uuid = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", uuid, "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float):
+        rows = [s for (t, s) in self.samples if t0 <= t <= t1] or [s for (_, s) in self.samples]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except Exception:
+                continue
+            for name, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- workload
+def run_spec(cfg):
+    """(mode, gamma) the metric is quoted on: the config's OTF run."""
+    for mode, gamma in cfg["runs"]:
+        if mode == "otf":
+            return mode, gamma
+    return cfg["runs"][0]
+
+
+def algorithmic_bytes(cfg, n, m_by_step, refreshed_by_step, r):
+    """Bytes the method itself must move for one batch (sector over-fetch excluded).
+
+    Per step k: two int64 row bounds and one cache row per frontier node, r neighbour ids read and
+    r slots written per refreshed node, picked ids written and re-read, one 8-byte relabel-table
+    entry per frontier node and per pick plus one written per new id, local ids and block offsets
+    written, new frontier ids written.  The key scan of a refreshed row moves no bytes: keys depend
+    on (node, offset, step), not on neighbour ids.  Features: id read, row read, row written."""
+    W = cfg["cache_width"]
+    L = len(cfg["fanouts"])
+    total = 0
+    for k in range(L):
+        nk, mk, uk = n[k], m_by_step[k], n[k + 1] - n[k]
+        total += 16 * nk + 4 * W * nk + 8 * r * refreshed_by_step[k]
+        total += 4 * mk + 8 * (nk + mk) + 8 * uk + 8 * mk + 4 * (nk + 1) + 4 * uk
+    s = 4 if cfg["feat_dtype"] == "f32" else 2
+    feat = n[L] * (4 + 2 * cfg["feat_dim"] * s)
+    return total + feat, feat
+
+
+def cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, budget_s=12.0, reps=1, first_seeds=None):
+    """Times the CPU oracle, as it stands, on the first `s` seeds of batch 0 (s grown until one
+    batch takes a few seconds).  Returns (edges/s, feature GB/s, description, seconds per batch)."""
+    import numpy as np
+
+    import oracle
+    from workloads import feature_rows
+
+    O = oracle.Sampler(indptr_h, indices_h, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED, cfg["shared"])
+    om = oracle.MODE_OTF if mode == "otf" else oracle.MODE_FCR
+    B = cfg["batch"]
+    s = first_seeds or max(1, min(B, 16))
+    step = 1
+    esize = 4 if cfg["feat_dtype"] == "f32" else 2
+    best = None
+    while True:
+        seeds = batch_seeds(perm, 0, B)[:s].numpy()
+        t0 = time.perf_counter()
+        frontier, n, blocks = O.sample_batch(seeds, om, gamma, step)
+        t_sample = time.perf_counter() - t0
+        # feature rows of the sampled nodes, re-evaluated or sliced on the host, then gathered row by row
+        ids = torch.from_numpy(frontier.astype("int64"))
+        if cfg["feat_kind"] == "hash":
+            Xs = feature_rows(cfg, ids)
+        else:
+            Xs = cpu_oracle_baseline.features[ids]
+        Xb = Xs.view(torch.int32 if esize == 4 else torch.int16).numpy()
+        t1 = time.perf_counter()
+        oracle.gather(Xb, np.arange(len(frontier), dtype=np.int32))
+        t_gather = time.perf_counter() - t1
+        dt = t_sample + t_gather
+        edges = sum(b.num_edges for b in blocks)
+        best = (edges / dt, len(frontier) * cfg["feat_dim"] * esize / dt / 1e9, s, dt)
+        step += 1
+        if dt >= budget_s / 4 or s >= B or first_seeds:
+            break
+        s = min(B, s * (4 if dt < budget_s / 16 else 2))
+    desc = ("oracle sample_batch + row-by-row gather, first %d of %d seeds of batch 0, %s gamma=%g, %.2f s"
+            % (best[2], B, mode, gamma, best[3]))
+    O.close()
+    return best[0], best[1], desc, best[3]
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="scale", choices=["tiny", "mid", "large", "shared", "scale"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    from paper_2406_17918_b200 import replicas
+
+    rank, local_rank, world = replicas.env_rank()
+    cfg = get_config(args.workload)
+    mode, gamma = run_spec(cfg)
+    L = len(cfg["fanouts"])
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        return reference_arm(args, cfg, mode, gamma)
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the sampler has no CPU fallback")
+    import paper_2406_17918_b200 as gs
+
+    device = torch.device("cuda", local_rank)
+    torch.cuda.set_device(device)
+    rank, local_rank, world = replicas.init("nccl", device)
+    if world != args.gpus:
+        print("warning: --gpus %d but WORLD_SIZE=%d" % (args.gpus, world), file=sys.stderr)
+
+    # ---- inputs, resident in HBM before anything is timed
+    t_setup = time.time()
+    g = build_graph(cfg, device=device)
+    X = build_features(cfg, device=device if cfg["feat_kind"] == "hash" else "cpu").to(device)
+    perm = seed_permutation(cfg, device=device)
+    torch.cuda.synchronize()
+    t_graph = time.time() - t_setup
+    G = gs.gs_graph_create(g.indptr, g.indices, X)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    C = gs.gs_cache_init(G, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED, cfg["shared"])
+    ev1.record()
+    torch.cuda.synchronize()
+    presample_ms = ev0.elapsed_time(ev1)
+    B = cfg["batch"]
+    ws = torch.empty(gs.gs_workspace_bytes(G, cfg["fanouts"], B), dtype=torch.uint8, device=device)
+    gm = gs.GS_MODE_OTF if mode == "otf" else gs.GS_MODE_FCR
+    r = int(gamma * cfg["cache_width"] + 0.5) if mode == "otf" else cfg["cache_width"]
+    hdr = C.storage[:256].view(torch.int32)
+
+    K, Wm = args.steps, args.warmup
+    seeds_all = [batch_seeds(perm, b, B, rank, world) for b in range(Wm + 2 * K)]
+    pinned_counts = torch.zeros((K, 64), dtype=torch.int32).pin_memory()
+    out = None
+
+    def one_step(b, step):
+        nonlocal out
+        blocks, input_nodes, cnt = gs.gs_sample_batch(C, seeds_all[b], gm, gamma, step, ws)
+        if out is None:
+            out = torch.empty((blocks[0].max_src, cfg["feat_dim"]), dtype=X.dtype, device=device)
+        return blocks, input_nodes, cnt
+
+    for b in range(Wm):
+        blocks, input_nodes, cnt = one_step(b, b + 1)
+        gs.gs_gather_features(G, input_nodes, cnt, out)
+    gs.gs_sync_status(C)
+
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(3 * K)]
+    clocks = ClockSampler(local_rank) if rank == 0 else None
+    time.sleep(0.3)
+    replicas.barrier()
+    torch.cuda.synchronize()
+    launches0 = gs.gs_kernel_launches()
+    wall0 = time.time()
+    for i in range(K):
+        b = Wm + i
+        events[3 * i].record()
+        blocks, input_nodes, cnt = one_step(b, b + 1)
+        events[3 * i + 1].record()
+        gs.gs_gather_features(G, input_nodes, cnt, out)
+        events[3 * i + 2].record()
+        pinned_counts[i].copy_(hdr, non_blocking=True)
+    end = torch.cuda.Event(enable_timing=True)
+    end.record()
+    torch.cuda.synchronize()
+    replicas.barrier()
+    wall1 = time.time()
+    launches = gs.gs_kernel_launches() - launches0
+    total_ms = events[0].elapsed_time(end)
+    gs.gs_sync_status(C)
+    if clocks:
+        time.sleep(0.1)
+        clocks.stop()
+
+    # word positions of the counts inside the cache's state header, by sampling step
+    n_words = [blocks[L - 1 - k].count_words()[0] for k in range(L)] + [blocks[0].count_words()[1]]
+    m_words = [blocks[L - 1 - k].count_words()[2] for k in range(L)]
+    counts = pinned_counts.numpy()
+    edges = 0
+    feat_rows = 0
+    sample_ms = sum(events[3 * i].elapsed_time(events[3 * i + 1]) for i in range(K))
+    gather_ms = sum(events[3 * i + 1].elapsed_time(events[3 * i + 2]) for i in range(K))
+    # refreshed nodes per step, from the last batch's frontier (outside the timed region)
+    deg = g.degrees()
+    n_last = [int(counts[K - 1][w]) for w in n_words]
+    fr = input_nodes[: n_last[L]].long()
+    over = (deg[fr] > cfg["cache_width"])
+    refreshed_frac = []
+    for k in range(L):
+        lo = n_last[k - 1] if (cfg["shared"] and k > 0) else 0
+        refreshed_frac.append(float(over[lo:n_last[k]].sum().item()) / max(1, n_last[k]))
+    alg_total, alg_feat = 0, 0
+    for i in range(K):
+        n = [int(counts[i][w]) for w in n_words]
+        m = [int(counts[i][w]) for w in m_words]
+        edges += sum(m)
+        feat_rows += n[L]
+        a, f = algorithmic_bytes(cfg, n, m, [refreshed_frac[k] * n[k] for k in range(L)], r)
+        alg_total += a
+        alg_feat += f
+
+    # ---- end-to-end: seeds in pinned host memory go in, the batch's counts come back, every step
+    e2e = None
+    if not args.no_e2e:
+        host_seeds = [seeds_all[Wm + K + i].cpu().pin_memory() for i in range(K)]
+        replicas.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e_edges = 0
+        e0.record()
+        for i in range(K):
+            step = Wm + K + i + 1
+            blocks, input_nodes, n, m = gs.gs_sample_batch_host(C, host_seeds[i], gm, gamma, step, ws)
+            gs.gs_gather_features(G, input_nodes, None, out[: n[L]])
+            e_edges += sum(m)
+        e1.record()
+        torch.cuda.synchronize()
+        replicas.barrier()
+        e_ms, (e_edges_all,) = replicas.aggregate(e0.elapsed_time(e1), [e_edges], device)
+        e2e = {"value": e_edges_all / (e_ms * 1e-3), "unit": "edges/s", "h2d_bytes_per_step": B * 4,
+               "d2h_bytes_per_step": gs.COUNTS_READBACK_BYTES,
+               "ms_per_step": e_ms / K}
+
+    t_ms, (edges_all, feat_rows_all, alg_all, alg_feat_all, gather_ms_max) = replicas.aggregate(
+        total_ms, [edges, feat_rows, alg_total, alg_feat, gather_ms], device)
+    if rank != 0:
+        replicas.shutdown()
+        return 0
+
+    esize = 4 if cfg["feat_dtype"] == "f32" else 2
+    peak, peak_kind = measured_peak()
+    secs = t_ms * 1e-3
+    gather_bytes_per_launch = alg_feat / K
+    gather_ms_per_launch = gather_ms / K
+    achieved = gather_bytes_per_launch / (gather_ms_per_launch * 1e-3) / 1e9
+    result = {
+        "metric": METRIC,
+        "value": edges_all / secs,
+        "unit": "edges/s",
+        "feature_gbs": feat_rows_all * cfg["feat_dim"] * esize / secs / 1e9,
+        "hbm_frac_batch": (alg_all / secs / 1e9) / peak / max(1, world),
+        "n_gpus": world,
+        "steps": K,
+        "warmup": Wm,
+        "ms_per_step": t_ms / K,
+        "higher_is_better": True,
+        "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": "int32 ids + %s feature copy" % cfg["feat_dtype"],
+        "data": "synthetic",
+        "config": {"workload": cfg["name"], "num_nodes": g.num_nodes, "num_edges": g.num_edges,
+                   "fanouts": cfg["fanouts"], "cache_width": cfg["cache_width"], "mode": mode, "gamma": gamma,
+                   "batch": B, "shared_cache": cfg["shared"], "feat_dim": cfg["feat_dim"],
+                   "parallelism": "replicas x%d" % world, "l2": "inputs_larger_than_L2",
+                   "sampled_edges_per_batch": edges / K, "input_nodes_per_batch": feat_rows / K},
+        "breakdown_ms_per_step": {"sample_batch": sample_ms / K, "gather_features": gather_ms / K},
+        "presample_ms": presample_ms,
+        "setup_s": {"graph_and_features": t_graph},
+        "roofline": {"kernel": "k_gather (feature rows)", "bound": "hbm", "achieved": achieved, "peak": peak,
+                     "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": None},
+        "algorithmic_bytes_per_batch": alg_total / K,
+        "gpu_launches": launches,
+        "clocks": clocks.summary(wall0, wall1) if clocks else None,
+    }
+    if e2e:
+        result["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        indptr_h, indices_h = g.indptr.cpu().numpy(), g.indices.cpu().numpy()
+        if cfg["feat_kind"] != "hash":
+            cpu_oracle_baseline.features = X.cpu()
+        v, fg, desc, _ = cpu_oracle_baseline(cfg, indptr_h, indices_h, perm.cpu(), mode, gamma)
+        result["cpu_baseline"] = {"value": v, "unit": "edges/s", "feature_gbs": fg, "cores": 1,
+                                  "host_cores": os.cpu_count(), "kind": "oracle", "sample": desc}
+    print(json.dumps(result))
+    replicas.shutdown()
+    return 0
+
+
+def reference_arm(args, cfg, mode, gamma):
+    """The CPU oracle, as it stands, on bounded samples of the same workload (one sample per step)."""
+    dev = "cuda" if (torch.cuda.is_available() and cfg["kind"] == "rmat") else "cpu"
+    g = build_graph(cfg, device=dev)
+    indptr_h, indices_h = g.indptr.cpu().numpy(), g.indices.cpu().numpy()
+    perm = seed_permutation(cfg)
+    if cfg["feat_kind"] != "hash":
+        cpu_oracle_baseline.features = build_features(cfg)
+    # size the per-step sample once, then time warm-up + K steps at that size
+    v, fg, desc, dt = cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, budget_s=8.0)
+    s = int(desc.split("first ")[1].split(" ")[0])
+    per_step_budget = max(1, min(args.steps, int(120.0 / max(dt, 1e-3))))
+    K = per_step_budget
+    tot_edges, tot_t, fgs = 0.0, 0.0, []
+    for i in range(min(args.warmup, 1) + K):
+        vv, ff, _, tt = cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, first_seeds=s)
+        if i >= min(args.warmup, 1):
+            tot_edges += vv * tt
+            tot_t += tt
+            fgs.append(ff)
+    value = tot_edges / tot_t
+    sample = "each step: " + desc.split(", %.2f" % dt)[0] + "; %d timed steps" % K
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "edges/s", "n_gpus": args.gpus,
+        "steps": K, "warmup": min(args.warmup, 1), "ms_per_step": tot_t / K * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int32 ids + %s feature copy" % cfg["feat_dtype"],
+        "data": "synthetic",
+        "config": {"workload": cfg["name"], "num_nodes": g.num_nodes, "num_edges": g.num_edges,
+                   "fanouts": cfg["fanouts"], "cache_width": cfg["cache_width"], "mode": mode, "gamma": gamma,
+                   "batch": cfg["batch"], "shared_cache": cfg["shared"], "feat_dim": cfg["feat_dim"]},
+        "cpu_baseline": {"value": value, "unit": "edges/s", "cores": 1, "host_cores": os.cpu_count(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "edges/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

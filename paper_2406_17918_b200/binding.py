@@ -19,6 +19,7 @@ _HEADER = os.path.join(os.path.dirname(_HERE), "include", "gs.h")
 GS_MODE_FCR, GS_MODE_OTF = 0, 1
 GS_F32, GS_BF16 = 0, 1
 GS_MAX_HOPS = 8
+COUNTS_READBACK_BYTES = 4 * (1 + (GS_MAX_HOPS + 1) + GS_MAX_HOPS)  # status + n_k + m_k, what gs_batch_counts copies
 
 _STATUS_NAMES = {0: "GS_OK", 1: "GS_ERR_ARG", 2: "GS_ERR_ALIGN", 3: "GS_ERR_RANGE", 4: "GS_ERR_WORKSPACE",
                  5: "GS_ERR_DUP_SEED", 6: "GS_ERR_CUDA"}
@@ -164,6 +165,10 @@ class Block:
         self._indices_off = cb.d_indices - workspace.data_ptr()
         hp = header.data_ptr()
         self._cnt = ((cb.d_num_dst - hp) // 4, (cb.d_num_src - hp) // 4, (cb.d_num_edges - hp) // 4)
+
+    def count_words(self):
+        """int32 word positions of (num_dst, num_src, num_edges) inside the cache storage."""
+        return self._cnt
 
     def counts_device(self):
         """(num_dst, num_src, num_edges) as 0-d device tensors aliasing the cache's state header."""
