@@ -162,7 +162,7 @@ gs_status gs_workspace_bytes(const gs_graph* g, int32_t num_hops, const int32_t*
     const Bounds b = make_bounds(g->num_nodes, num_hops, fanouts, max_seeds);
     for (int k = 0; k < num_hops; ++k)
         if (b.nb[k] + b.mb[k] >= ((int64_t)1 << 31)) return fail(GS_ERR_ARG, "batch too large: positions would exceed 2^31");
-    *bytes = make_layout(b).total;
+    *bytes = make_layout(b, g->num_edges).total;
     return GS_OK;
 }
 
@@ -198,7 +198,7 @@ gs_status gs_cache_init(const gs_graph* g, int32_t num_hops, const int32_t* fano
     c->serial = 0;
     c->lambda_otf = 16.0f;
     c->lambda_full = 72.0f;
-    c->hub_degree = 16384;
+    c->hub_degree = 8192;
     cudaError_t e = cudaMallocHost((void**)&c->h_pinned, 64 * sizeof(int32_t));
     if (e != cudaSuccess) { delete c; return cuda_fail(e, "cudaMallocHost"); }
 
@@ -206,7 +206,23 @@ gs_status gs_cache_init(const gs_graph* g, int32_t num_hops, const int32_t* fano
     e = cudaMemsetAsync(c->d_hdr, 0, HDR_BYTES, s);
     if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "cudaMemsetAsync"); }
     // S0: a full refresh (r = W) of every node at step 0, rows with deg <= W copied verbatim.
-    // The relabel table is not in use yet and serves as the hub list of these launches.
+    // The relabel table is not in use yet and serves as the hub storage of these launches; the
+    // hub degree is raised until the hubs it can produce fit there.
+    const size_t table_room = (size_t)g->num_nodes * 8;
+    int64_t hub_degree0 = c->hub_degree < HUB_MIN_DEGREE ? HUB_MIN_DEGREE : c->hub_degree;
+    int64_t cap0 = 0, items0 = 0;
+    size_t o_entry = 0, o_state = 0, o_items = 0, o_cand = 0;
+    for (int tries = 0; tries < 40; ++tries, hub_degree0 *= 2) {
+        cap0 = g->num_edges / hub_degree0 + 1;
+        if (cap0 > g->num_nodes) cap0 = g->num_nodes;
+        items0 = g->num_edges / (4 * (int64_t)HUB_CHUNK_QUADS) + cap0 + 1;
+        o_entry = 0;
+        o_state = align_up(o_entry + (size_t)cap0 * 8, 256);
+        o_items = align_up(o_state + (size_t)cap0 * 8, 256);
+        o_cand = align_up(o_items + (size_t)items0 * 4, 256);
+        if (o_cand + (size_t)cap0 * HUB_CAND_CAP * 8 <= table_room) break;
+        cap0 = 0;
+    }
     for (int ci = 0; ci < c->num_caches; ++ci) {
         StepParams P = step_params(c, ci, 0u);
         P.r = c->W;
@@ -216,9 +232,17 @@ gs_status gs_cache_init(const gs_graph* g, int32_t num_hops, const int32_t* fano
         P.d_refresh_from = nullptr;
         P.do_pick = 0;
         P.init_rows = 1;
-        P.hub_list = (int32_t*)c->d_table;
-        P.hub_count = c->d_hdr + HDR_HUBS + ci;
+        char* hub_base = (char*)c->d_table;
+        P.hub_entry = (int2*)(hub_base + o_entry);
+        P.hub_state = (int2*)(hub_base + o_state);
+        P.hub_items = (int32_t*)(hub_base + o_items);
+        P.hub_cand = (unsigned long long*)(hub_base + o_cand);
+        P.hub_counter = (unsigned long long*)(c->d_hdr + HDR_HUB64 + 2 * ci);
+        P.hub_cap = (int32_t)cap0;          // 0: the table is too small, every node is done by one warp
+        P.item_cap = (int32_t)items0;
+        P.hub_degree = cap0 > 0 ? (int32_t)(hub_degree0 > 0x7FFFFFFF ? 0x7FFFFFFF : hub_degree0) : 0x7FFFFFFF;
         P.work_counter = c->d_hdr + HDR_WORK + ci;
+        P.work_counter2 = c->d_hdr + HDR_WORK2 + ci;
         e = launch_refresh_pick(P, g->num_nodes, s);
         if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "pre-sample launch"); }
     }
@@ -255,7 +279,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         r = rr < 0 ? 0 : (rr > c->W ? c->W : (int32_t)rr);
     }
     const Bounds b = make_bounds(g->num_nodes, L, c->fanouts, num_seeds);
-    const WorkspaceLayout w = make_layout(b);
+    const WorkspaceLayout w = make_layout(b, g->num_edges);
     if (workspace_bytes < w.total) return fail(GS_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, w.total);
     char* ws = (char*)d_workspace;
     int32_t* frontier = (int32_t*)(ws + w.frontier);
@@ -263,7 +287,6 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
     int32_t* aux = (int32_t*)(ws + w.aux);
     int32_t* tiles_a = (int32_t*)(ws + w.tiles_a);
     int32_t* tiles_e = (int32_t*)(ws + w.tiles_e);
-    int32_t* hub_list = (int32_t*)(ws + w.hub_list);
 
     if (c->serial == 0xFFFFFFFEu) {  // stamp space used up: start over with a clean table
         GS_CUDA(cudaMemsetAsync(c->d_table, 0xFF, (size_t)g->num_nodes * 8, s));
@@ -290,6 +313,17 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         C.tile_sums = tiles_a;
         C.table = c->d_table;
         C.stamp = stamp;
+        // a partial refresh runs as scan + finish kernels; FCR (and r = 0) use the fused kernels
+        const bool split = (r > 0 && r < c->W);
+        C.split = split ? 1 : 0;
+        C.W = c->W;
+        C.r = r;
+        C.d_refresh_from = (c->shared && k > 0) ? c->d_hdr + HDR_N + (k - 1) : nullptr;
+        C.tile_sums2 = (int32_t*)(ws + w.tiles_a2);
+        C.item_start = (int32_t*)(ws + w.item_start);
+        C.items = (int32_t*)(ws + w.items);
+        C.cand_count = (int32_t*)(ws + w.cand_count);
+        C.scan_item_cap = w.scan_item_cap;
         GS_CUDA(launch_row_counts(C, b.nb[k], s));
 
         StepParams P = step_params(c, layer, step);
@@ -301,12 +335,28 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         P.blk_indptr = blk_indptr;
         P.picked = picked;
         P.stamp = stamp;
-        P.hub_list = hub_list;
-        P.hub_count = c->d_hdr + HDR_HUBS + k;
+        P.hub_entry = (int2*)(ws + w.hub_entry);
+        P.hub_state = (int2*)(ws + w.hub_state);
+        P.hub_items = (int32_t*)(ws + w.hub_items);
+        P.hub_cand = (unsigned long long*)(ws + w.hub_cand);
+        P.hub_counter = (unsigned long long*)(c->d_hdr + HDR_HUB64 + 2 * k);
+        P.hub_cap = (int32_t)w.hub_cap;
+        P.item_cap = (int32_t)w.item_cap;
         P.work_counter = c->d_hdr + HDR_WORK + k;
+        P.work_counter2 = c->d_hdr + HDR_WORK2 + k;
         P.do_pick = 1;
         P.init_rows = 0;
-        GS_CUDA(launch_refresh_pick(P, b.nb[k], s));
+        P.item_start = C.item_start;
+        P.items = C.items;
+        P.d_items_total = c->d_hdr + HDR_ITEMS + k;
+        P.cand_count = C.cand_count;
+        P.cand = (unsigned long long*)(ws + w.cand);
+        if (split) {
+            int64_t item_bound = b.nb[k] + g->num_edges / (4 * (int64_t)HUB_CHUNK_QUADS) + 1;
+            GS_CUDA(launch_scan_finish(P, b.nb[k], item_bound, s));
+        } else {
+            GS_CUDA(launch_refresh_pick(P, b.nb[k], s));
+        }
 
         RelabelParams R{};
         R.hdr = c->d_hdr;
@@ -387,7 +437,7 @@ gs_status gs_sample_batch_host(gs_cache* c, const int32_t* h_seeds, int32_t num_
     // The seeds are staged in the relabel scratch array: its first writer (step 0's
     // first-occurrence kernel) runs after the row-count kernel has copied the seeds out.
     const Bounds b = make_bounds(c->graph->num_nodes, c->L, c->fanouts, num_seeds);
-    const WorkspaceLayout w = make_layout(b);
+    const WorkspaceLayout w = make_layout(b, c->graph->num_edges);
     if (workspace_bytes < w.total) return fail(GS_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, w.total);
     int32_t* d_stage = (int32_t*)((char*)d_workspace + w.aux);
     cudaStream_t s = (cudaStream_t)stream;

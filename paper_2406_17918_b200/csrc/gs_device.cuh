@@ -37,32 +37,35 @@ __device__ __forceinline__ uint32_t lanemask_lt() {
 }
 
 // Lanes in `valid` hold (key, lane) pairs; returns the mask of the k pairs smallest in
-// (key, lane) order.  Runs min(k, n-k) rounds of a warp-wide min (or max) reduction.
+// (key, lane) order.  Keys are uniform 32-bit words, so the lanes with key <= k/n * 2^32 are
+// already close to the answer; the difference is repaired by a few rounds of a warp-wide max
+// (drop the largest selected pair) or min (add the smallest unselected pair).  Any guess gives
+// the exact result: every selected key is <= every unselected key.
 __device__ __forceinline__ uint32_t warp_smallest_k(uint32_t key, uint32_t valid, int k, int lane) {
     const int n = __popc(valid);
     if (k >= n) return valid;
     if (k <= 0) return 0u;
     const bool mine = (valid >> lane) & 1u;
-    if (k <= n - k) {
-        uint32_t sel = 0;
-        for (int t = 0; t < k; ++t) {
-            const bool live = mine && !((sel >> lane) & 1u);
-            const uint32_t x = live ? key : 0xFFFFFFFFu;
-            const uint32_t m = __reduce_min_sync(FULL, x);
-            const uint32_t b = __ballot_sync(FULL, live && x == m);
-            sel |= b & (0u - b);  // lowest lane among equal keys
-        }
-        return sel;
-    }
-    uint32_t rem = 0;
-    for (int t = 0; t < n - k; ++t) {
-        const bool live = mine && !((rem >> lane) & 1u);
+    const uint32_t guess = (uint32_t)(((unsigned long long)k << 32) / (unsigned)n) - 1u;
+    uint32_t sel = __ballot_sync(FULL, mine && key <= guess);
+    int c = __popc(sel);
+    while (c > k) {   // drop the largest selected pair: max key, highest lane among equals
+        const bool live = (sel >> lane) & 1u;
         const uint32_t x = live ? key : 0u;
         const uint32_t m = __reduce_max_sync(FULL, x);
         const uint32_t b = __ballot_sync(FULL, live && x == m);
-        rem |= 0x80000000u >> __clz(b);  // highest lane among equal keys is the largest pair
+        sel &= ~(0x80000000u >> __clz(b));
+        --c;
     }
-    return valid & ~rem;
+    while (c < k) {   // add the smallest unselected pair: min key, lowest lane among equals
+        const bool live = mine && !((sel >> lane) & 1u);
+        const uint32_t x = live ? key : 0xFFFFFFFFu;
+        const uint32_t m = __reduce_min_sync(FULL, x);
+        const uint32_t b = __ballot_sync(FULL, live && x == m);
+        sel |= b & (0u - b);
+        ++c;
+    }
+    return sel;
 }
 
 // Exclusive scan of one int per thread over a block of BT threads (BT a multiple of 32, <= 1024).

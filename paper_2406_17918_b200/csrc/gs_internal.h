@@ -16,9 +16,20 @@ constexpr int HDR_WORK = HDR_M + GS_MAX_HOPS;    // work-stealing counters  (GS_
 constexpr int HDR_HUBS = HDR_WORK + GS_MAX_HOPS; // hub list lengths
 constexpr int HDR_TICKET_A = HDR_HUBS + GS_MAX_HOPS;
 constexpr int HDR_TICKET_E = HDR_TICKET_A + GS_MAX_HOPS;
-constexpr int HDR_WORDS = HDR_TICKET_E + GS_MAX_HOPS;
+constexpr int HDR_WORK2 = HDR_TICKET_E + GS_MAX_HOPS;  // work counters of the hub-chunk kernel
+constexpr int HDR_ITEMS = HDR_WORK2 + GS_MAX_HOPS;     // scan work items per step (split OTF path)
+constexpr int HDR_WORDS = HDR_ITEMS + GS_MAX_HOPS;
+constexpr int HDR_HUB64 = 128;                   // 64-bit (hubs << 32 | chunks) counters, one per launch
 constexpr size_t HDR_BYTES = 1024;
-static_assert(HDR_WORDS * 4 <= HDR_BYTES, "header too small");
+static_assert(HDR_WORDS <= HDR_HUB64, "header words overlap the 64-bit counters");
+static_assert((HDR_HUB64 + 2 * GS_MAX_HOPS) * 4 <= HDR_BYTES, "header too small");
+
+constexpr int HUB_CHUNK_QUADS = 2048;   // one hub work item = 8192 edge offsets
+constexpr int HUB_MIN_DEGREE = 4096;    // lowest degree at which a node may be split over warps
+constexpr int HUB_CAND_CAP = 128;       // candidate entries per hub (same as a warp's buffer)
+
+constexpr int SPLIT_CAND_CAP = 32;      // candidates kept per node by the split OTF path (one per lane)
+constexpr int SMALL_DEGREE = 128;       // up to here a refresh needs no threshold scan: one Philox per lane covers the row
 
 constexpr int SCAN_A_TILE = 1024;  // frontier nodes per tile of the row-count scan
 constexpr int SCAN_E_TILE = 4096;  // picked edges per tile of the first-occurrence scan
@@ -47,11 +58,24 @@ struct WorkspaceLayout {
     size_t frontier;
     size_t blk_indptr[GS_MAX_HOPS];   // by sampling step
     size_t blk_indices[GS_MAX_HOPS];  // by sampling step
-    size_t picked, aux, tiles_a, tiles_e, hub_list;
+    size_t picked, aux, tiles_a, tiles_e;
+    size_t hub_entry, hub_state, hub_items, hub_cand;
+    int64_t hub_cap, item_cap;
+    size_t tiles_a2, item_start, items, cand_count, cand;   // split OTF path
+    int64_t scan_item_cap;
     size_t total;
 };
 
-inline WorkspaceLayout make_layout(const Bounds& b) {
+// Hubs are nodes with degree > HUB_MIN_DEGREE or more; their number among distinct frontier
+// nodes is bounded by num_edges / HUB_MIN_DEGREE, their chunks by num_edges / chunk + hubs.
+inline void hub_caps(int64_t num_edges, int64_t max_n, int64_t* hub_cap, int64_t* item_cap) {
+    int64_t h = num_edges / HUB_MIN_DEGREE + 1;
+    if (h > max_n) h = max_n;
+    *hub_cap = h;
+    *item_cap = num_edges / (4 * (int64_t)HUB_CHUNK_QUADS) + h + 1;
+}
+
+inline WorkspaceLayout make_layout(const Bounds& b, int64_t num_edges) {
     WorkspaceLayout w{};
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
@@ -67,7 +91,17 @@ inline WorkspaceLayout make_layout(const Bounds& b) {
     w.aux = take((size_t)max_m * 4 + 16);
     w.tiles_a = take(((size_t)max_n / SCAN_A_TILE + 2) * 4);
     w.tiles_e = take(((size_t)max_m / SCAN_E_TILE + 2) * 4);
-    w.hub_list = take((size_t)max_n * 4);
+    hub_caps(num_edges, max_n, &w.hub_cap, &w.item_cap);
+    w.hub_entry = take((size_t)w.hub_cap * 8);
+    w.hub_state = take((size_t)w.hub_cap * 8);
+    w.hub_items = take((size_t)w.item_cap * 4);
+    w.hub_cand = take((size_t)w.hub_cap * HUB_CAND_CAP * 8);
+    w.tiles_a2 = take(((size_t)max_n / SCAN_A_TILE + 2) * 4);
+    w.item_start = take(((size_t)max_n + 1) * 4);
+    w.scan_item_cap = max_n + num_edges / (4 * (int64_t)HUB_CHUNK_QUADS) + 1;
+    w.items = take((size_t)w.scan_item_cap * 4);
+    w.cand_count = take((size_t)max_n * 4);
+    w.cand = take((size_t)max_n * SPLIT_CAND_CAP * 8);
     w.total = off;
     return w;
 }
@@ -93,10 +127,22 @@ struct StepParams {
     int32_t* picked;             // global ids of the picks
     unsigned long long* table;   // relabel table, (stamp << 32) | position
     uint32_t stamp;
-    int32_t n_base_is_device;    // position of pick e in the concatenated list is *d_n + e
-    int32_t* hub_list;
-    int32_t* hub_count;
+    // hubs: nodes whose scan is split into chunks over many warps
+    int2* hub_entry;                 // (frontier position, first chunk)
+    int2* hub_state;                 // (candidates appended, chunks finished)
+    int32_t* hub_items;              // chunk -> hub entry
+    unsigned long long* hub_cand;    // [hub][HUB_CAND_CAP] (key << 32 | offset)
+    unsigned long long* hub_counter; // (entries << 32) | chunks
+    int32_t hub_cap, item_cap;
     int32_t* work_counter;
+    int32_t* work_counter2;
+    // split OTF path: scan work items (one per 8192-offset chunk of a refreshed node) and the
+    // per-node candidate lists they produce
+    const int32_t* item_start;       // [n+1] first item of each frontier position
+    const int32_t* items;            // item -> frontier position
+    const int32_t* d_items_total;
+    int32_t* cand_count;             // [n]
+    unsigned long long* cand;        // [n][SPLIT_CAND_CAP]
     int32_t* status;
     int32_t do_pick, init_rows;
     float lambda_otf, lambda_full;
@@ -115,6 +161,14 @@ struct CountParams {
     int32_t* tile_sums;
     unsigned long long* table;
     uint32_t stamp;
+    // split OTF path: also lays out the scan work items of the refreshed nodes
+    int32_t split, W, r;
+    const int32_t* d_refresh_from;
+    int32_t* tile_sums2;
+    int32_t* item_start;
+    int32_t* items;
+    int32_t* cand_count;
+    int64_t scan_item_cap;
 };
 
 struct RelabelParams {
@@ -134,6 +188,7 @@ void count_launches(int n);
 
 cudaError_t launch_row_counts(const CountParams& p, int64_t n_bound, cudaStream_t s);
 cudaError_t launch_refresh_pick(const StepParams& p, int64_t n_bound, cudaStream_t s);
+cudaError_t launch_scan_finish(const StepParams& p, int64_t n_bound, int64_t item_bound, cudaStream_t s);
 cudaError_t launch_relabel(const RelabelParams& p, int64_t m_bound, cudaStream_t s);
 cudaError_t launch_gather(const void* src, int64_t src_ld_bytes, int64_t row_bytes, const int32_t* ids,
                           const int32_t* d_count, int32_t count_bound, void* dst, int64_t dst_ld_bytes,

@@ -3,28 +3,31 @@
 // Every selection is "the k items first in (key, index) order" with Philox keys that depend on
 // (node, item index, step) only - not on the neighbour ids.  The scan over a node's deg edge
 // offsets therefore reads no CSR bytes: it evaluates one Philox block per four offsets, keeps the
-// offsets whose key is below a threshold chosen so that about lambda of them survive, and only
-// then reads the few neighbour ids it needs.  If the survivors turn out not to be enough (or
+// offsets whose key is at or below a threshold chosen so that about lambda of them survive, and
+// only then reads the few neighbour ids it needs.  If the survivors turn out not to be enough (or
 // too many for the buffer) the node is redone with a larger lambda and finally with an exact
-// running top-W, so the result never depends on the threshold.
+// running top-W, so the result never depends on the threshold.  The kernel is bound by integer
+// ALU throughput (Philox), not by memory.
 //
 // Refill rule used (it follows from the refresh definition): the r refill winners are the first r
 // entries, after removing retained neighbours, of the top-W list of ALL edge offsets in FILL
 // order, because at most W - r retained neighbours can precede the r-th winner.
+//
+// Two kernels per step:
+//   k_refresh_pick      one warp per frontier node, software-pipelined: while the neighbour ids
+//                       of node i are in flight the warp already scans node i+1.  Nodes above the
+//                       hub degree are only registered, as a list of 8192-offset chunks.
+//   k_refresh_pick_hub  one warp per chunk; candidates go to a per-hub buffer in global memory,
+//                       and the warp that finishes a hub's last chunk completes the node.  No
+//                       warp ever waits for another one.
 #include "gs_device.cuh"
 #include "gs_internal.h"
 
 namespace gs {
 
-constexpr int RP_THREADS = 256;         // warp-per-node kernel
+constexpr int RP_THREADS = 256;
 constexpr int RP_WARPS = RP_THREADS / 32;
-constexpr int HUB_THREADS = 512;        // block-per-node kernel
-
-struct NodeCtx {
-    int32_t v;
-    int64_t row_start;
-    uint32_t deg;
-};
+static_assert(CAND_CAP == HUB_CAND_CAP, "hub buffers are copied into a warp buffer");
 
 __device__ __forceinline__ uint32_t threshold_for(float lambda, uint32_t deg) {
     // inclusive key threshold: about lambda of deg uniform 32-bit keys fall at or below it
@@ -44,10 +47,13 @@ __device__ __forceinline__ int warp_collect(const StepParams& P, int32_t v, uint
         const uint32_t q = qb + lane;
         const uint4 o = philox4x32_10(q, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
         const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
+        const bool inq = q < q_end;
+        const bool any = inq && (min(min(kk[0], kk[1]), min(kk[2], kk[3])) <= tinc);
+        if (__ballot_sync(FULL, any) == 0) continue;   // the common case: nothing below the threshold
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
             const uint32_t off = 4u * q + w;
-            const bool hit = (q < q_end) && (off < deg) && (kk[w] <= tinc);
+            const bool hit = inq && (off < deg) && (kk[w] <= tinc);
             const uint32_t b = __ballot_sync(FULL, hit);
             if (b) {
                 if (hit) {
@@ -58,12 +64,14 @@ __device__ __forceinline__ int warp_collect(const StepParams& P, int32_t v, uint
             }
         }
     }
+    __syncwarp();
     return count;
 }
 
 // Exact fallback: one warp keeps the W smallest (key, offset) pairs in a sorted list, one per
 // lane, while scanning every offset.  Leaves them in buf[0..W) in order.
-__device__ void warp_exact_top(const StepParams& P, int32_t v, uint32_t deg, unsigned long long* buf, int lane) {
+__device__ __noinline__ void warp_exact_top(const StepParams& P, int32_t v, uint32_t deg, unsigned long long* buf,
+                                            int lane) {
     const int W = P.W;
     unsigned long long cur = ~0ull;
     const uint32_t nq = (deg + 3u) >> 2;
@@ -113,54 +121,121 @@ __device__ __forceinline__ unsigned long long warp_pop_min(unsigned long long (&
     return best;
 }
 
-// One warp: given c candidates in buf (all offsets with key <= threshold; `whole` = they are all
-// the offsets, or at least the exact top-W), fill the evicted slots.  Returns false if the
-// candidates cannot decide the refill (caller retries with more).
-__device__ bool warp_refill(const StepParams& P, const NodeCtx& nd, const unsigned long long* buf, int c,
-                            bool whole, uint32_t evict_mask, int32_t& slot, int lane) {
-    const int W = P.W;
-    const int r = __popc(evict_mask);
-    if (c > CAND_CAP) return false;
-    if (c < r) return false;
-    unsigned long long it[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) it[j] = (lane + 32 * j < c) ? buf[lane + 32 * j] : ~0ull;
-    const int limit = c < W ? c : W;          // never more than the top-W matter
-    const bool retained = (lane < W) && !((evict_mask >> lane) & 1u);
-    int taken = 0;
-    uint32_t valid = 0;
-    uint32_t my_off = 0;
-    int32_t my_nb = -1;
-    while (true) {
-        int g = r - __popc(valid);
-        if (g > limit - taken) g = limit - taken;
+// Refill of one node, split in two so that the neighbour-id loads issued by begin() can be in
+// flight while the warp works on something else.
+struct Refill {
+    unsigned long long it[4];  // candidates, four per lane
+    int c;                     // candidate count, -1 = unusable (too few / overflow)
+    int taken, g;              // extracted so far; size of the batch whose ids are in flight
+    bool whole;                // candidates are all offsets, or the exact top-W
+    uint32_t my_off;           // lane t holds the t-th candidate in FILL order ...
+    int32_t my_nb;             // ... and its neighbour id
+
+    __device__ __forceinline__ void extract(const StepParams& P, int64_t row_start, int lane) {
         for (int t = 0; t < g; ++t) {
             const unsigned long long best = warp_pop_min(it);
             if (lane == taken + t) my_off = (uint32_t)best;
         }
-        if (lane >= taken && lane < taken + g) my_nb = P.g.indices[nd.row_start + my_off];
-        for (int t = taken; t < taken + g; ++t) {
-            const int32_t x = __shfl_sync(FULL, my_nb, t);
-            const uint32_t hit = __ballot_sync(FULL, retained && slot == x);
-            if (hit == 0) valid |= 1u << t;
-        }
-        taken += g;
-        if (__popc(valid) >= r) break;
-        if (taken >= limit) {
-            // candidates exhausted: only conclusive if they covered the whole top-W
-            if (whole || c >= W) break;  // cannot happen with fewer than r valid (refill rule)
-            return false;
-        }
+        if (lane >= taken && lane < taken + g) my_nb = __ldg(P.g.indices + row_start + my_off);
     }
-    if (__popc(valid) < r) return false;
-    // t-th valid candidate -> t-th evicted slot (ascending slot index)
-    const bool ev = (evict_mask >> lane) & 1u;
-    const int e = __popc(evict_mask & lanemask_lt());
-    const int src = ev ? (int)__fns(valid, 0, e + 1) : 0;
-    const int32_t nv = __shfl_sync(FULL, my_nb, src & 31);
-    if (ev) slot = nv;
-    return true;
-}
+
+    __device__ __forceinline__ void begin(const StepParams& P, int64_t row_start, const unsigned long long* buf,
+                                          int count, bool all, int r, int lane) {
+        c = count;
+        whole = all;
+        taken = 0;
+        g = 0;
+        my_off = 0;
+        my_nb = -1;
+        if (count > CAND_CAP || count < r) { c = -1; return; }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) it[j] = (lane + 32 * j < c) ? buf[lane + 32 * j] : ~0ull;
+        const int limit = c < P.W ? c : P.W;
+        g = r < limit ? r : limit;
+        extract(P, row_start, lane);
+    }
+
+    // Completes the refill into `slot`.  Returns false if the candidates cannot decide it.
+    __device__ __forceinline__ bool finish(const StepParams& P, int64_t row_start, uint32_t evict_mask,
+                                           int32_t& slot, int lane) {
+        if (c < 0) return false;
+        const int W = P.W;
+        const int r = __popc(evict_mask);
+        const int limit = c < W ? c : W;  // never more than the top-W matter
+        const bool retained = (lane < W) && !((evict_mask >> lane) & 1u);
+        uint32_t valid = 0;
+        while (true) {
+            for (int t = taken; t < taken + g; ++t) {
+                const int32_t x = __shfl_sync(FULL, my_nb, t);
+                const uint32_t hit = __ballot_sync(FULL, retained && slot == x);
+                if (hit == 0) valid |= 1u << t;
+            }
+            taken += g;
+            if (__popc(valid) >= r) break;
+            if (taken >= limit) {
+                if (whole || c >= W) break;  // the whole top-W was examined (cannot lack winners)
+                return false;
+            }
+            g = r - __popc(valid);
+            if (g > limit - taken) g = limit - taken;
+            extract(P, row_start, lane);
+        }
+        if (__popc(valid) < r) return false;
+        // t-th valid candidate -> t-th evicted slot (ascending slot index)
+        const bool ev = (evict_mask >> lane) & 1u;
+        const int e = __popc(evict_mask & lanemask_lt());
+        const int src = ev ? (int)__fns(valid, 0, e + 1) : 0;
+        const int32_t nv = __shfl_sync(FULL, my_nb, src & 31);
+        if (ev) slot = nv;
+        return true;
+    }
+};
+
+// First attempt of a refill, split around the neighbour-id loads: issue() extracts the first
+// r (+1 spare) candidates in FILL order and starts loading their neighbour ids; settle() uses
+// them if they contain r neighbours that are not retained.  Anything else (too few candidates,
+// too many, more than one retained neighbour among them) is left to refill_slow().
+struct Quick {
+    int g;            // candidates whose ids are in flight (0 = attempt unusable)
+    uint32_t my_off;
+    int32_t my_nb;
+
+    __device__ __forceinline__ void issue(const StepParams& P, int64_t row_start, const unsigned long long* buf,
+                                          int count, int r, int lane) {
+        g = 0;
+        my_off = 0;
+        my_nb = -1;
+        if (count > CAND_CAP || count < r) return;
+        unsigned long long it[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) it[j] = (lane + 32 * j < count) ? buf[lane + 32 * j] : ~0ull;
+        const int limit = count < P.W ? count : P.W;
+        g = (r + 1 < limit) ? r + 1 : limit;
+        for (int t = 0; t < g; ++t) {
+            const unsigned long long best = warp_pop_min(it);
+            if (lane == t) my_off = (uint32_t)best;
+        }
+        if (lane < g) my_nb = __ldg(P.g.indices + row_start + my_off);
+    }
+
+    __device__ __forceinline__ bool settle(const StepParams& P, uint32_t evict_mask, int32_t& slot, int lane) {
+        if (g == 0) return false;
+        const int r = __popc(evict_mask);
+        const bool retained = (lane < P.W) && !((evict_mask >> lane) & 1u);
+        uint32_t valid = 0;
+        for (int t = 0; t < g; ++t) {
+            const int32_t x = __shfl_sync(FULL, my_nb, t);
+            if (__ballot_sync(FULL, retained && slot == x) == 0) valid |= 1u << t;
+        }
+        if (__popc(valid) < r) return false;
+        const bool ev = (evict_mask >> lane) & 1u;
+        const int e = __popc(evict_mask & lanemask_lt());
+        const int src = ev ? (int)__fns(valid, 0, e + 1) : 0;
+        const int32_t nv = __shfl_sync(FULL, my_nb, src & 31);
+        if (ev) slot = nv;
+        return true;
+    }
+};
 
 // Evicted slot mask for this node and step.
 __device__ __forceinline__ uint32_t evict_mask_for(const StepParams& P, int32_t v, int lane) {
@@ -171,45 +246,94 @@ __device__ __forceinline__ uint32_t evict_mask_for(const StepParams& P, int32_t 
 }
 
 // S2: choose and emit the picks of one node; registers their positions in the relabel table.
-__device__ __forceinline__ void warp_pick(const StepParams& P, const NodeCtx& nd, int p, int32_t slot, int lane) {
-    const int cnt = nd.deg < (uint32_t)P.W ? (int)nd.deg : P.W;
+__device__ __forceinline__ void warp_pick(const StepParams& P, int32_t v, uint32_t deg, int e_base, uint32_t n_base,
+                                          int32_t slot, int lane) {
+    const int cnt = deg < (uint32_t)P.W ? (int)deg : P.W;
     const uint32_t cmask = cnt >= 32 ? FULL : ((1u << cnt) - 1u);
     uint32_t pm = cmask;
     if (cnt > P.f) {
-        const uint4 o = philox4x32_10((uint32_t)lane >> 2, (uint32_t)nd.v, P.step, P.word_pick, P.key0, P.key1);
+        const uint4 o = philox4x32_10((uint32_t)lane >> 2, (uint32_t)v, P.step, P.word_pick, P.key0, P.key1);
         pm = warp_smallest_k(word_of(o, lane & 3), cmask, P.f, lane);
     }
     if ((pm >> lane) & 1u) {
-        const int e = P.blk_indptr[p] + __popc(pm & lanemask_lt());
+        const int e = e_base + __popc(pm & lanemask_lt());
         P.picked[e] = slot;
-        const uint32_t n = (uint32_t)__ldcg(P.d_n);
-        atomicMin(P.table + slot, ((unsigned long long)P.stamp << 32) | (n + (uint32_t)e));
+        atomicMin(P.table + slot, ((unsigned long long)P.stamp << 32) | (n_base + (uint32_t)e));
     }
 }
 
-__device__ __forceinline__ bool load_node(const StepParams& P, int p, NodeCtx& nd, int lane) {
-    int32_t v = P.frontier ? P.frontier[p] : p;
-    long long a = 0;
-    if (lane < 2) a = P.g.indptr[v + lane];
-    const long long rs = __shfl_sync(FULL, a, 0);
-    const long long re = __shfl_sync(FULL, a, 1);
-    nd.v = v;
-    nd.row_start = rs;
-    nd.deg = (uint32_t)(re - rs);
-    return true;
+// Retry ladder after a failed first attempt: a looser threshold, then the exact scan.
+__device__ __noinline__ void refill_slow(const StepParams& P, int32_t v, int64_t row_start, uint32_t deg,
+                                         uint32_t evict, unsigned long long* buf, int32_t& slot, int lane) {
+    Refill R;
+    const uint32_t nq = (deg + 3u) >> 2;
+    const int r = __popc(evict);
+    {
+        const uint32_t tinc = threshold_for(P.lambda_full, deg);
+        const int c = warp_collect(P, v, deg, 0, nq, tinc, buf, 0, lane);
+        R.begin(P, row_start, buf, c, tinc == 0xFFFFFFFFu, r, lane);
+        __syncwarp();
+        if (R.finish(P, row_start, evict, slot, lane)) return;
+    }
+    warp_exact_top(P, v, deg, buf, lane);
+    R.begin(P, row_start, buf, P.W, true, r, lane);
+    __syncwarp();
+    R.finish(P, row_start, evict, slot, lane);
+}
+
+__device__ __forceinline__ void store_row(const StepParams& P, int32_t* row, uint32_t evict, int32_t slot, int lane) {
+    if (P.init_rows) {
+        if (lane < P.pitch) row[lane] = (lane < P.W) ? slot : -1;
+    } else if ((evict >> lane) & 1u) {
+        row[lane] = slot;
+    }
+}
+
+// Registers a hub: reserves an entry and a contiguous range of chunk items with one atomicAdd.
+// Returns false if the hub storage is full; the caller then processes the node itself, and the
+// part of the reserved item range that exists is marked as holes for the chunk kernel to skip.
+// (With hub_degree >= HUB_MIN_DEGREE the storage cannot fill up: the frontier's nodes are
+// distinct, so their degrees sum to at most num_edges.)
+__device__ __forceinline__ bool hub_register(const StepParams& P, int p, uint32_t deg, int lane) {
+    const uint32_t nq = (deg + 3u) >> 2;
+    const uint32_t nch = (nq + HUB_CHUNK_QUADS - 1) / HUB_CHUNK_QUADS;
+    unsigned long long got = 0;
+    if (lane == 0) got = atomicAdd(P.hub_counter, (1ull << 32) | nch);
+    got = __shfl_sync(FULL, got, 0);
+    const long long h = (long long)(got >> 32);
+    const long long cb = (long long)(uint32_t)got;
+    const bool ok = h < P.hub_cap && cb + nch <= (long long)P.item_cap;
+    if (ok && lane == 0) {
+        P.hub_entry[h] = make_int2(p, (int)cb);
+        P.hub_state[h] = make_int2(0, 0);
+    }
+    for (long long c = cb + lane; c < cb + nch && c < (long long)P.item_cap; c += 32) P.hub_items[c] = ok ? (int)h : -1;
+    return ok;
 }
 
 // ---------------------------------------------------------------- warp-per-node kernel
-__global__ void __launch_bounds__(RP_THREADS) k_refresh_pick(StepParams P) {
+struct NodeState {
+    int32_t v;
+    int64_t row_start;
+    uint32_t deg;
+    int e_base;
+    int32_t slot;
+    uint32_t evict;
+    bool refresh, skip, tried_full;
+    Quick Q;
+};
+
+__global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick(const __grid_constant__ StepParams P) {
     __shared__ unsigned long long s_buf[RP_WARPS][CAND_CAP];
     if (__ldcg(P.status) != 0) return;   // set only by earlier kernels of the batch: uniform
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     unsigned long long* buf = s_buf[wid];
     const int n = P.d_n ? __ldcg(P.d_n) : P.n_host;
+    const uint32_t n_base = (uint32_t)n;
     const int refresh_from = P.d_refresh_from ? __ldcg(P.d_refresh_from) : 0;
     const int total_warps = gridDim.x * RP_WARPS;
-    int chunk = n / (total_warps * 8);
-    chunk = chunk < 1 ? 1 : (chunk > 64 ? 64 : chunk);
+    int chunk = n / (total_warps * 4);
+    chunk = chunk < 1 ? 1 : (chunk > 32 ? 32 : chunk);
     const int W = P.W;
 
     while (true) {
@@ -217,134 +341,420 @@ __global__ void __launch_bounds__(RP_THREADS) k_refresh_pick(StepParams P) {
         if (lane == 0) base = atomicAdd(P.work_counter, chunk);
         base = __shfl_sync(FULL, base, 0);
         if (base >= n) break;
-        const int end = base + chunk < n ? base + chunk : n;
-        for (int p = base; p < end; ++p) {
-            NodeCtx nd;
-            load_node(P, p, nd, lane);
-            int32_t* row = P.slots + (int64_t)nd.v * P.pitch;
-            int32_t slot = -1;
+        const int cnt = (base + chunk < n ? base + chunk : n) - base;
+        // the chunk's node ids, row bounds and pick offsets, one node per lane, all loads in flight together
+        int32_t v_l = 0;
+        long long lo_l = 0, hi_l = 0;
+        int eb_l = 0;
+        if (lane < cnt) {
+            v_l = P.frontier ? __ldg(P.frontier + base + lane) : base + lane;
+            lo_l = __ldg(P.g.indptr + v_l);
+            hi_l = __ldg(P.g.indptr + v_l + 1);
+            if (P.do_pick) eb_l = __ldg(P.blk_indptr + base + lane);
+        }
+        // first node's row (cache row, or the adjacency of a low-degree node when initialising)
+        auto fetch_row = [&](int i) -> int32_t {
+            const int32_t v = __shfl_sync(FULL, v_l, i);
+            const long long lo = __shfl_sync(FULL, lo_l, i);
+            const long long hi = __shfl_sync(FULL, hi_l, i);
+            int32_t x = -1;
             if (P.init_rows) {
-                if (nd.deg <= (uint32_t)W) {
-                    if (lane < (int)nd.deg) slot = P.g.indices[nd.row_start + lane];
-                    if (lane < P.pitch) row[lane] = slot;
-                }
+                if (hi - lo <= W && lane < (int)(hi - lo)) x = __ldg(P.g.indices + lo + lane);
             } else if (lane < W) {
-                slot = row[lane];
+                x = P.slots[(int64_t)v * P.pitch + lane];
             }
-            const bool refresh = nd.deg > (uint32_t)W && P.r > 0 && p >= refresh_from;
-            if (refresh) {
-                if (nd.deg > (uint32_t)P.hub_degree) {   // a whole block handles this one, pick included
-                    if (lane == 0) P.hub_list[atomicAdd(P.hub_count, 1)] = p;
-                    continue;
-                }
-                const uint32_t evict = evict_mask_for(P, nd.v, lane);
-                const uint32_t nq = (nd.deg + 3u) >> 2;
-                bool done = false;
-                if (P.r < W) {
-                    const uint32_t tinc = threshold_for(P.lambda_otf, nd.deg);
-                    const int c = warp_collect(P, nd.v, nd.deg, 0, nq, tinc, buf, 0, lane);
-                    __syncwarp();
-                    done = warp_refill(P, nd, buf, c, tinc == 0xFFFFFFFFu, evict, slot, lane);
-                    __syncwarp();
-                }
-                if (!done) {
-                    const uint32_t tinc = threshold_for(P.lambda_full, nd.deg);
-                    const int c = warp_collect(P, nd.v, nd.deg, 0, nq, tinc, buf, 0, lane);
-                    __syncwarp();
-                    done = warp_refill(P, nd, buf, c, tinc == 0xFFFFFFFFu, evict, slot, lane);
-                    __syncwarp();
-                }
-                if (!done) {
-                    warp_exact_top(P, nd.v, nd.deg, buf, lane);
-                    warp_refill(P, nd, buf, W, true, evict, slot, lane);
-                    __syncwarp();
-                }
-                if (P.init_rows) {
-                    if (lane < P.pitch) row[lane] = (lane < W) ? slot : -1;
-                } else if ((evict >> lane) & 1u) {
-                    row[lane] = slot;
+            return x;
+        };
+        int32_t row_next = fetch_row(0);
+        NodeState prev;
+        prev.skip = true;
+        bool have_prev = false;
+        for (int i = 0; i <= cnt; ++i) {
+            NodeState cur;
+            cur.skip = true;
+            if (i < cnt) {
+                // ---- phase A of node i: decide, scan, issue the neighbour-id loads
+                cur.v = __shfl_sync(FULL, v_l, i);
+                cur.row_start = __shfl_sync(FULL, lo_l, i);
+                cur.deg = (uint32_t)(__shfl_sync(FULL, hi_l, i) - cur.row_start);
+                cur.e_base = __shfl_sync(FULL, eb_l, i);
+                cur.slot = row_next;
+                if (i + 1 < cnt) row_next = fetch_row(i + 1);
+                cur.skip = false;
+                cur.evict = 0;
+                cur.tried_full = false;
+                cur.Q.g = 0;
+                cur.refresh = cur.deg > (uint32_t)W && P.r > 0 && base + i >= refresh_from;
+                if (cur.refresh && cur.deg > (uint32_t)P.hub_degree && hub_register(P, base + i, cur.deg, lane)) {
+                    cur.skip = true;   // the hub kernel does everything for this node, pick included
+                } else if (cur.refresh) {
+                    cur.evict = evict_mask_for(P, cur.v, lane);
+                    cur.tried_full = !(P.r < W);
+                    const uint32_t tinc = threshold_for(cur.tried_full ? P.lambda_full : P.lambda_otf, cur.deg);
+                    const int c = warp_collect(P, cur.v, cur.deg, 0, (cur.deg + 3u) >> 2, tinc, buf, 0, lane);
+                    cur.Q.issue(P, cur.row_start, buf, c, __popc(cur.evict), lane);
+                    __syncwarp();   // buf may be reused from here on: the first candidates live in registers
                 }
             }
-            if (P.do_pick) warp_pick(P, nd, p, slot, lane);
+            if (have_prev && !prev.skip) {
+                // ---- phase B of node i-1: its neighbour ids have had a whole scan to arrive
+                if (prev.refresh) {
+                    if (!prev.Q.settle(P, prev.evict, prev.slot, lane))
+                        refill_slow(P, prev.v, prev.row_start, prev.deg, prev.evict, buf, prev.slot, lane);
+                    __syncwarp();
+                }
+                if (prev.refresh || (P.init_rows && prev.deg <= (uint32_t)W))
+                    store_row(P, P.slots + (int64_t)prev.v * P.pitch, prev.evict, prev.slot, lane);
+                if (P.do_pick) warp_pick(P, prev.v, prev.deg, prev.e_base, n_base, prev.slot, lane);
+            }
+            prev = cur;
+            have_prev = true;
         }
     }
 }
 
-// ---------------------------------------------------------------- block-per-node kernel (hubs)
-__global__ void __launch_bounds__(HUB_THREADS) k_refresh_pick_hub(StepParams P) {
-    __shared__ unsigned long long s_buf[CAND_CAP];
-    __shared__ int s_count;
-    __shared__ int s_done;
+// ---------------------------------------------------------------- warp-per-chunk kernel (hubs)
+__global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick_hub(const __grid_constant__ StepParams P) {
+    __shared__ unsigned long long s_buf[RP_WARPS][CAND_CAP];
     if (__ldcg(P.status) != 0) return;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    const int nwarps = HUB_THREADS / 32;
-    const int nh = __ldcg(P.hub_count);
+    unsigned long long* buf = s_buf[wid];
+    const unsigned long long packed = __ldcg(P.hub_counter);
+    int total = (int)(uint32_t)packed;
+    if (total > P.item_cap) total = P.item_cap;
+    if (total == 0) return;
+    const uint32_t n_base = (uint32_t)(P.d_n ? __ldcg(P.d_n) : P.n_host);
     const int W = P.W;
-    for (int h = blockIdx.x; h < nh; h += gridDim.x) {
-        const int p = __ldcg(P.hub_list + h);
-        NodeCtx nd;
-        load_node(P, p, nd, lane);
-        int32_t* row = P.slots + (int64_t)nd.v * P.pitch;
-        int32_t slot = -1;
-        uint32_t evict = 0;
-        if (wid == 0) {
-            if (!P.init_rows && lane < W) slot = row[lane];
-            evict = evict_mask_for(P, nd.v, lane);
-        }
-        const uint32_t nq = (nd.deg + 3u) >> 2;
-        for (int attempt = (P.r < W ? 0 : 1); attempt < 3; ++attempt) {
-            __syncthreads();
-            if (threadIdx.x == 0) { s_count = 0; s_done = 0; }
-            __syncthreads();
-            uint32_t tinc = 0xFFFFFFFFu;
-            if (attempt < 2) {
-                tinc = threshold_for(attempt == 0 ? P.lambda_otf : P.lambda_full, nd.deg);
-                // each warp scans a contiguous slice of quads into a private count, then appends
-                const uint32_t per = (nq + nwarps - 1) / nwarps;
-                const uint32_t qa = wid * per < nq ? wid * per : nq;
-                const uint32_t qe = qa + per < nq ? qa + per : nq;
-                const uint32_t lt = lanemask_lt();
-                for (uint32_t qb = qa; qb < qe; qb += 32) {
-                    const uint32_t q = qb + lane;
-                    const uint4 o = philox4x32_10(q, (uint32_t)nd.v, P.step, P.word_fill, P.key0, P.key1);
-                    const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
+    const uint32_t lt = lanemask_lt();
+    // a hub's candidates must never run short: its retry would be a serial scan of the whole row
+    const float lam = P.r < W ? fmaxf(P.lambda_otf, 32.0f) : P.lambda_full;
+
+    while (true) {
+        int w = 0;
+        if (lane == 0) w = atomicAdd(P.work_counter2, 1);
+        w = __shfl_sync(FULL, w, 0);
+        if (w >= total) break;
+        const int h = __ldcg(P.hub_items + w);
+        if (h < 0) continue;   // a hole left by a hub that did not fit
+        const int2 ent = __ldcg(P.hub_entry + h);
+        const int p = ent.x;
+        const int32_t v = P.frontier ? __ldg(P.frontier + p) : p;
+        const long long rs = __ldg(P.g.indptr + v);
+        const uint32_t deg = (uint32_t)(__ldg(P.g.indptr + v + 1) - rs);
+        const uint32_t nq = (deg + 3u) >> 2;
+        const uint32_t nch = (nq + HUB_CHUNK_QUADS - 1) / HUB_CHUNK_QUADS;
+        const uint32_t qa = (uint32_t)(w - ent.y) * HUB_CHUNK_QUADS;
+        const uint32_t qe = qa + HUB_CHUNK_QUADS < nq ? qa + HUB_CHUNK_QUADS : nq;
+        const uint32_t tinc = threshold_for(lam, deg);
+        unsigned long long* cand = P.hub_cand + (size_t)h * HUB_CAND_CAP;
+        int* cand_count = &P.hub_state[h].x;
+        for (uint32_t qb = qa; qb < qe; qb += 32) {
+            const uint32_t q = qb + lane;
+            const uint4 o = philox4x32_10(q, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
+            const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
+            const bool inq = q < qe;
+            const bool any = inq && (min(min(kk[0], kk[1]), min(kk[2], kk[3])) <= tinc);
+            if (__ballot_sync(FULL, any) == 0) continue;
 #pragma unroll
-                    for (int w = 0; w < 4; ++w) {
-                        const uint32_t off = 4u * q + w;
-                        const bool hit = (q < qe) && (off < nd.deg) && (kk[w] <= tinc);
-                        const uint32_t b = __ballot_sync(FULL, hit);
-                        if (b) {
-                            int basepos = 0;
-                            if (lane == 0) basepos = atomicAdd(&s_count, __popc(b));
-                            basepos = __shfl_sync(FULL, basepos, 0);
-                            if (hit) {
-                                const int pos = basepos + __popc(b & lt);
-                                if (pos < CAND_CAP) s_buf[pos] = ((unsigned long long)kk[w] << 32) | off;
-                            }
-                        }
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t off = 4u * q + j;
+                const bool hit = inq && (off < deg) && (kk[j] <= tinc);
+                const uint32_t b = __ballot_sync(FULL, hit);
+                if (b) {
+                    int basepos = 0;
+                    if (lane == 0) basepos = atomicAdd(cand_count, __popc(b));
+                    basepos = __shfl_sync(FULL, basepos, 0);
+                    if (hit) {
+                        const int pos = basepos + __popc(b & lt);
+                        if (pos < HUB_CAND_CAP) cand[pos] = ((unsigned long long)kk[j] << 32) | off;
                     }
                 }
-            } else if (wid == 0) {
-                warp_exact_top(P, nd.v, nd.deg, s_buf, lane);
-                if (lane == 0) s_count = W;
             }
-            __syncthreads();
-            if (wid == 0) {
-                const bool ok = warp_refill(P, nd, s_buf, s_count, attempt == 2 || tinc == 0xFFFFFFFFu, evict, slot, lane);
-                if (lane == 0) s_done = ok ? 1 : 0;
-            }
-            __syncthreads();
-            if (s_done) break;
         }
-        if (wid == 0) {
-            if (P.init_rows) {
-                if (lane < P.pitch) row[lane] = (lane < W) ? slot : -1;
-            } else if ((evict >> lane) & 1u) {
-                row[lane] = slot;
+        // the warp that finishes the hub's last chunk completes the node
+        __threadfence();
+        int ticket = 0;
+        if (lane == 0) ticket = atomicAdd(&P.hub_state[h].y, 1);
+        ticket = __shfl_sync(FULL, ticket, 0);
+        if (ticket != (int)nch - 1) continue;
+        __threadfence();
+        const int c = __ldcg(cand_count);
+        for (int j = lane; j < CAND_CAP; j += 32)
+            if (j < c) buf[j] = __ldcg(cand + j);
+        __syncwarp();
+        int32_t* row = P.slots + (int64_t)v * P.pitch;
+        int32_t slot = (!P.init_rows && lane < W) ? row[lane] : -1;
+        const uint32_t evict = evict_mask_for(P, v, lane);
+        Quick Q;
+        Q.issue(P, rs, buf, c, __popc(evict), lane);
+        __syncwarp();
+        if (!Q.settle(P, evict, slot, lane)) refill_slow(P, v, rs, deg, evict, buf, slot, lane);
+        __syncwarp();
+        store_row(P, row, evict, slot, lane);
+        if (P.do_pick) warp_pick(P, v, deg, __ldg(P.blk_indptr + p), n_base, slot, lane);
+    }
+}
+
+// ================================================================ split OTF path
+// For a partial refresh (0 < r < W) the work is split in two kernels:
+//   k_scan    one warp per work item (an 8192-offset chunk of one refreshed node): nothing but
+//             Philox blocks and a threshold compare, at full occupancy; the few offsets below the
+//             threshold go to the node's candidate list in global memory (at most 32, one per lane).
+//   k_finish  one warp per frontier node: eviction, refill from the candidate list, row update
+//             and the pick.  Rows of up to SMALL_DEGREE neighbours skip the scan: one Philox block
+//             per lane covers the whole row, and the refill is decided in registers.
+// Nodes whose candidate list cannot decide the refill (too few, too many, or several retained
+// neighbours among the first ones) take the retry ladder of the fused path.
+
+__global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ StepParams P) {
+    if (__ldcg(P.status) != 0) return;
+    const int lane = threadIdx.x & 31;
+    const int total = __ldcg(P.d_items_total);
+    const int total_warps = gridDim.x * RP_WARPS;
+    int batch = total / (total_warps * 4);
+    batch = batch < 1 ? 1 : (batch > 32 ? 32 : batch);
+    const uint32_t lt = lanemask_lt();
+    while (true) {
+        int base = 0;
+        if (lane == 0) base = atomicAdd(P.work_counter2, batch);
+        base = __shfl_sync(FULL, base, 0);
+        if (base >= total) break;
+        const int cnt = (base + batch < total ? base + batch : total) - base;
+        int p_l = 0, chunk_l = 0;
+        int32_t v_l = 0;
+        long long lo_l = 0, hi_l = 0;
+        if (lane < cnt) {
+            p_l = __ldg(P.items + base + lane);
+            chunk_l = base + lane - __ldg(P.item_start + p_l);
+            v_l = __ldg(P.frontier + p_l);
+            lo_l = __ldg(P.g.indptr + v_l);
+            hi_l = __ldg(P.g.indptr + v_l + 1);
+        }
+        for (int i = 0; i < cnt; ++i) {
+            const int p = __shfl_sync(FULL, p_l, i);
+            const int chunk = __shfl_sync(FULL, chunk_l, i);
+            const int32_t v = __shfl_sync(FULL, v_l, i);
+            const uint32_t deg = (uint32_t)(__shfl_sync(FULL, hi_l, i) - __shfl_sync(FULL, lo_l, i));
+            const uint32_t nq = (deg + 3u) >> 2;
+            const bool single = nq <= (uint32_t)HUB_CHUNK_QUADS;
+            const uint32_t qa = (uint32_t)chunk * HUB_CHUNK_QUADS;
+            const uint32_t qe = qa + HUB_CHUNK_QUADS < nq ? qa + HUB_CHUNK_QUADS : nq;
+            const uint32_t tinc = threshold_for(P.lambda_otf, deg);
+            unsigned long long* cand = P.cand + (size_t)p * SPLIT_CAND_CAP;
+            int count = 0;
+            for (uint32_t qb = qa; qb < qe; qb += 32) {
+                const uint32_t q = qb + lane;
+                const uint4 o = philox4x32_10(q, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
+                const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
+                const bool inq = q < qe;
+                const bool any = inq && (min(min(kk[0], kk[1]), min(kk[2], kk[3])) <= tinc);
+                if (__ballot_sync(FULL, any) == 0) continue;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t off = 4u * q + j;
+                    const bool hit = inq && (off < deg) && (kk[j] <= tinc);
+                    const uint32_t b = __ballot_sync(FULL, hit);
+                    if (b) {
+                        int basepos = count;
+                        if (!single) {   // several warps share this node's list
+                            if (lane == 0) basepos = atomicAdd(P.cand_count + p, __popc(b));
+                            basepos = __shfl_sync(FULL, basepos, 0);
+                        }
+                        if (hit) {
+                            const int pos = basepos + __popc(b & lt);
+                            if (pos < SPLIT_CAND_CAP) cand[pos] = ((unsigned long long)kk[j] << 32) | off;
+                        }
+                        count += __popc(b);
+                    }
+                }
             }
-            if (P.do_pick) warp_pick(P, nd, p, slot, lane);
+            if (single && lane == 0) P.cand_count[p] = count;
         }
     }
+}
+
+// EVICT keys (lanes 0-7 compute the eight slot quads) and PICK keys (lanes 8-15) from one Philox call.
+__device__ __forceinline__ void evict_pick_keys(const StepParams& P, int32_t v, int lane, uint32_t& ekey,
+                                                uint32_t& pkey) {
+    const bool second = (lane >> 3) & 1;
+    const uint4 o = philox4x32_10((uint32_t)lane & 7u, (uint32_t)v, P.step, second ? P.word_pick : P.word_evict,
+                                  P.key0, P.key1);
+    const int src = lane >> 2, w = lane & 3;
+    const uint32_t e0 = __shfl_sync(FULL, o.x, src), e1 = __shfl_sync(FULL, o.y, src);
+    const uint32_t e2 = __shfl_sync(FULL, o.z, src), e3 = __shfl_sync(FULL, o.w, src);
+    const uint32_t p0 = __shfl_sync(FULL, o.x, src + 8), p1 = __shfl_sync(FULL, o.y, src + 8);
+    const uint32_t p2 = __shfl_sync(FULL, o.z, src + 8), p3 = __shfl_sync(FULL, o.w, src + 8);
+    ekey = w == 0 ? e0 : (w == 1 ? e1 : (w == 2 ? e2 : e3));
+    pkey = w == 0 ? p0 : (w == 1 ? p1 : (w == 2 ? p2 : p3));
+}
+
+// Refill of a row with at most SMALL_DEGREE neighbours, decided in registers: lane l holds offsets
+// 4l..4l+3 with their keys and neighbour ids; offsets whose neighbour is retained are struck out
+// and the r smallest remaining (key, offset) pairs go to the evicted slots in ascending order.
+__device__ __forceinline__ void small_refill(const StepParams& P, int32_t v, int64_t row_start, uint32_t deg,
+                                             uint32_t evict, int32_t& slot, int lane) {
+    const uint4 o = philox4x32_10((uint32_t)lane, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
+    const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
+    int32_t nb[4];
+    bool ok[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint32_t off = 4u * lane + j;
+        ok[j] = off < deg;
+        nb[j] = ok[j] ? __ldg(P.g.indices + row_start + off) : -1;
+    }
+    const uint32_t wmask = P.W >= 32 ? FULL : ((1u << P.W) - 1u);
+    uint32_t rm = wmask & ~evict;
+    while (rm) {
+        const int t = __ffs(rm) - 1;
+        rm &= rm - 1;
+        const int32_t s = __shfl_sync(FULL, slot, t);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) ok[j] = ok[j] && nb[j] != s;
+    }
+    unsigned long long it[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) it[j] = ok[j] ? (((unsigned long long)kk[j] << 32) | (4u * lane + j)) : ~0ull;
+    uint32_t em = evict;
+    while (em) {
+        const int dst = __ffs(em) - 1;
+        em &= em - 1;
+        unsigned long long before[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) before[j] = it[j];
+        const unsigned long long best = warp_pop_min(it);
+        int32_t mine = -1;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (before[j] == best) mine = nb[j];
+        const uint32_t owner = __ballot_sync(FULL, mine >= 0);
+        const int32_t nv = __shfl_sync(FULL, mine, __ffs(owner) - 1);
+        if (lane == dst) slot = nv;
+    }
+}
+
+__global__ void __launch_bounds__(RP_THREADS, 4) k_finish(const __grid_constant__ StepParams P) {
+    __shared__ unsigned long long s_buf[RP_WARPS][CAND_CAP];
+    if (__ldcg(P.status) != 0) return;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    unsigned long long* buf = s_buf[wid];
+    const int n = __ldcg(P.d_n);
+    const uint32_t n_base = (uint32_t)n;
+    const int refresh_from = P.d_refresh_from ? __ldcg(P.d_refresh_from) : 0;
+    const int total_warps = gridDim.x * RP_WARPS;
+    int chunk = n / (total_warps * 2);
+    chunk = chunk < 1 ? 1 : (chunk > 32 ? 32 : chunk);
+    const int W = P.W;
+    const uint32_t wmask = W >= 32 ? FULL : ((1u << W) - 1u);
+
+    while (true) {
+        int base = 0;
+        if (lane == 0) base = atomicAdd(P.work_counter, chunk);
+        base = __shfl_sync(FULL, base, 0);
+        if (base >= n) break;
+        const int cnt = (base + chunk < n ? base + chunk : n) - base;
+        int32_t v_l = 0;
+        long long lo_l = 0, hi_l = 0;
+        int eb_l = 0, cc_l = 0;
+        if (lane < cnt) {
+            v_l = __ldg(P.frontier + base + lane);
+            lo_l = __ldg(P.g.indptr + v_l);
+            hi_l = __ldg(P.g.indptr + v_l + 1);
+            eb_l = __ldg(P.blk_indptr + base + lane);
+            cc_l = __ldcg(P.cand_count + base + lane);
+        }
+        // one node ahead: its cache row and its candidate list are in flight while this one is decided
+        int32_t row_next = -1;
+        unsigned long long cand_next = ~0ull;
+        auto prefetch = [&](int i) {
+            const int32_t v = __shfl_sync(FULL, v_l, i);
+            const int cc = __shfl_sync(FULL, cc_l, i);
+            row_next = lane < W ? P.slots[(int64_t)v * P.pitch + lane] : -1;
+            cand_next = (lane < cc && lane < SPLIT_CAND_CAP) ? __ldcg(P.cand + (size_t)(base + i) * SPLIT_CAND_CAP + lane) : ~0ull;
+        };
+        prefetch(0);
+        for (int i = 0; i < cnt; ++i) {
+            const int p = base + i;
+            const int32_t v = __shfl_sync(FULL, v_l, i);
+            const int64_t rs = __shfl_sync(FULL, lo_l, i);
+            const uint32_t deg = (uint32_t)(__shfl_sync(FULL, hi_l, i) - rs);
+            const int e_base = __shfl_sync(FULL, eb_l, i);
+            const int cc = __shfl_sync(FULL, cc_l, i);
+            int32_t slot = row_next;
+            unsigned long long cand = cand_next;
+            if (i + 1 < cnt) prefetch(i + 1);
+            const bool refresh = deg > (uint32_t)W && p >= refresh_from;
+            const int ncached = deg < (uint32_t)W ? (int)deg : W;
+            uint32_t ekey = 0, pkey = 0;
+            if (refresh || ncached > P.f) evict_pick_keys(P, v, lane, ekey, pkey);
+            if (refresh) {
+                const uint32_t evict = warp_smallest_k(ekey, wmask, P.r, lane);
+                if (deg <= (uint32_t)SMALL_DEGREE) {
+                    small_refill(P, v, rs, deg, evict, slot, lane);
+                } else {
+                    bool done = false;
+                    if (cc >= P.r && cc <= SPLIT_CAND_CAP) {
+                        // first r (+ spares) candidates in FILL order, one candidate per lane
+                        const int limit = cc < W ? cc : W;
+                        int g = P.r + (deg < 1024u ? 4 : 1);
+                        g = g < limit ? g : limit;
+                        uint32_t my_off = 0;
+                        for (int t = 0; t < g; ++t) {
+                            const uint32_t hi = (uint32_t)(cand >> 32);
+                            const uint32_t mhi = __reduce_min_sync(FULL, hi);
+                            const uint32_t lo = (hi == mhi) ? (uint32_t)cand : 0xFFFFFFFFu;
+                            const uint32_t mlo = __reduce_min_sync(FULL, lo);
+                            if (cand == (((unsigned long long)mhi << 32) | mlo)) cand = ~0ull;
+                            if (lane == t) my_off = mlo;
+                        }
+                        const int32_t my_nb = lane < g ? __ldg(P.g.indices + rs + my_off) : -1;
+                        const bool retained = (lane < W) && !((evict >> lane) & 1u);
+                        uint32_t valid = 0;
+                        for (int t = 0; t < g; ++t) {
+                            const int32_t x = __shfl_sync(FULL, my_nb, t);
+                            if (__ballot_sync(FULL, retained && slot == x) == 0) valid |= 1u << t;
+                        }
+                        if (__popc(valid) >= P.r) {
+                            // t-th valid candidate -> t-th evicted slot, through shared memory
+                            const int vr = __popc(valid & lanemask_lt());
+                            int32_t* stage = reinterpret_cast<int32_t*>(buf);
+                            if (((valid >> lane) & 1u) && vr < P.r) stage[vr] = my_nb;
+                            __syncwarp();
+                            if ((evict >> lane) & 1u) slot = stage[__popc(evict & lanemask_lt())];
+                            __syncwarp();
+                            done = true;
+                        }
+                    }
+                    if (!done) {
+                        refill_slow(P, v, rs, deg, evict, buf, slot, lane);
+                        __syncwarp();
+                    }
+                }
+                if ((evict >> lane) & 1u) P.slots[(int64_t)v * P.pitch + lane] = slot;
+            }
+            // S2 pick
+            const uint32_t cmask = ncached >= 32 ? FULL : ((1u << ncached) - 1u);
+            uint32_t pm = cmask;
+            if (ncached > P.f) pm = warp_smallest_k(pkey, cmask, P.f, lane);
+            if ((pm >> lane) & 1u) {
+                const int e = e_base + __popc(pm & lanemask_lt());
+                P.picked[e] = slot;
+                atomicMin(P.table + slot, ((unsigned long long)P.stamp << 32) | (n_base + (uint32_t)e));
+            }
+        }
+    }
+}
+
+cudaError_t launch_scan_finish(const StepParams& p, int64_t n_bound, int64_t item_bound, cudaStream_t s) {
+    const int64_t cap = 148 * 8;
+    int64_t sb = (item_bound + RP_WARPS - 1) / RP_WARPS;
+    sb = sb > cap ? cap : (sb < 1 ? 1 : sb);
+    k_scan<<<(int)sb, RP_THREADS, 0, s>>>(p);
+    int64_t fb = (n_bound + RP_WARPS - 1) / RP_WARPS;
+    fb = fb > cap ? cap : (fb < 1 ? 1 : fb);
+    k_finish<<<(int)fb, RP_THREADS, 0, s>>>(p);
+    count_launches(2);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_refresh_pick(const StepParams& p, int64_t n_bound, cudaStream_t s) {
@@ -353,10 +763,12 @@ cudaError_t launch_refresh_pick(const StepParams& p, int64_t n_bound, cudaStream
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     k_refresh_pick<<<(int)blocks, RP_THREADS, 0, s>>>(p);
-    int64_t hub_blocks = n_bound < 148 * 4 ? n_bound : 148 * 4;
-    if (hub_blocks < 1) hub_blocks = 1;
-    k_refresh_pick_hub<<<(int)hub_blocks, HUB_THREADS, 0, s>>>(p);
-    count_launches(2);
+    int launched = 1;
+    if (p.hub_cap > 0) {
+        k_refresh_pick_hub<<<(int)cap, RP_THREADS, 0, s>>>(p);
+        launched = 2;
+    }
+    count_launches(launched);
     return cudaGetLastError();
 }
 

@@ -38,6 +38,8 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
     const int n = (P.k == 0) ? P.n_host : __ldcg(P.hdr + HDR_N + P.k);
     const int p = blockIdx.x * SCAN_A_TILE + threadIdx.x;
     int c = 0;
+    int nch = 0;   // scan work items of this node (split path only)
+    const int refresh_from = (P.split && P.d_refresh_from) ? __ldcg(P.d_refresh_from) : 0;
     if (p < n) {
         int v;
         if (P.k == 0) {
@@ -57,12 +59,22 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
         if (v >= 0) {
             const int64_t deg = P.g.indptr[v + 1] - P.g.indptr[v];
             c = deg < (int64_t)P.f ? (int)deg : P.f;
+            if (P.split && deg > (int64_t)SMALL_DEGREE && deg > (int64_t)P.W && p >= refresh_from) {
+                const int64_t nq = (deg + 3) >> 2;
+                nch = (int)((nq + HUB_CHUNK_QUADS - 1) / HUB_CHUNK_QUADS);
+            }
         }
     }
     int total;
     const int excl = block_exclusive_scan<SCAN_A_TILE>(c, warp_sums, &total);
     if (p < n) P.blk_indptr[p] = excl;
+    int total2 = 0;
+    if (P.split) {
+        const int excl2 = block_exclusive_scan<SCAN_A_TILE>(nch, warp_sums, &total2);
+        if (p < n) P.item_start[p] = excl2;
+    }
     if (threadIdx.x == 0) {
+        if (P.split) P.tile_sums2[blockIdx.x] = total2;
         P.tile_sums[blockIdx.x] = total;
         __threadfence();
         const int ticket = atomicAdd(P.hdr + HDR_TICKET_A + P.k, 1);
@@ -72,8 +84,11 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
     if (!is_last) return;
     __threadfence();
     const int m = scan_tiles_in_place(P.tile_sums, (int)gridDim.x, warp_sums);
+    int items = 0;
+    if (P.split) items = scan_tiles_in_place(P.tile_sums2, (int)gridDim.x, warp_sums);
     if (threadIdx.x == 0) {
         P.hdr[HDR_M + P.k] = m;
+        P.hdr[HDR_ITEMS + P.k] = items;
         if (P.k == 0) P.hdr[HDR_N] = n;
     }
 }
@@ -84,6 +99,24 @@ __global__ void __launch_bounds__(1024) k_row_offsets(CountParams P) {
     const int p = blockIdx.x * SCAN_A_TILE + threadIdx.x;
     if (p < n) P.blk_indptr[p] += P.tile_sums[p / SCAN_A_TILE];
     else if (p == n) P.blk_indptr[n] = __ldcg(P.hdr + HDR_M + P.k);
+    if (!P.split) return;
+    // scan work items: node p owns items [item_start[p], item_start[p+1]), one per chunk of its row
+    int first = 0, next = 0;
+    if (p < n) {
+        const int tile = p / SCAN_A_TILE;
+        first = P.item_start[p] + P.tile_sums2[tile];
+        if (p + 1 >= n) next = __ldcg(P.hdr + HDR_ITEMS + P.k);
+        else if ((p + 1) % SCAN_A_TILE == 0) next = P.tile_sums2[tile + 1];   // first node of the next tile
+        else next = P.item_start[p + 1] + P.tile_sums2[tile];
+    }
+    __syncthreads();   // tile-local values are all read before any is overwritten below
+    if (p < n) {
+        P.item_start[p] = first;
+        P.cand_count[p] = 0;
+        for (int w = first; w < next && (int64_t)w < P.scan_item_cap; ++w) P.items[w] = p;
+    } else if (p == n) {
+        P.item_start[n] = __ldcg(P.hdr + HDR_ITEMS + P.k);
+    }
 }
 
 cudaError_t launch_row_counts(const CountParams& p, int64_t n_bound, cudaStream_t s) {
