@@ -160,6 +160,11 @@ gs_status gs_cache_export_bytes(const gs_cache*, size_t* bytes);
 gs_status gs_cache_export(const gs_cache*, void* d_dst, size_t bytes, void* stream);
 gs_status gs_cache_import(gs_cache*, const void* d_src, size_t bytes, void* stream);
 
+/* Synchronises `stream` and copies three counters of the last batch (or of the pre-sample, if no
+ * batch ran yet) into h_stats: [0] nodes whose refill had to be redone by a full rescan on one
+ * warp, [1] nodes handed to the chunked multi-warp scan, [2] reserved (0).  Diagnostics only. */
+gs_status gs_batch_stats(gs_cache*, void* stream, int64_t* h_stats);
+
 /* Synchronises `stream` and returns the device status of the last batch. */
 gs_status gs_sync_status(gs_cache*, void* stream);
 

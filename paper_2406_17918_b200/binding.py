@@ -71,6 +71,7 @@ def _load():
         "gs_cache_export": [vp, vp, sz, vp],
         "gs_cache_import": [vp, vp, sz, vp],
         "gs_sync_status": [vp, vp],
+        "gs_batch_stats": [vp, vp, vp],
         "gs_cache_set_tuning": [vp, dbl, dbl, i32],
     }
     for name, args in sig.items():
@@ -298,6 +299,13 @@ def gs_cache_export(cache: Cache, stream=None) -> torch.Tensor:
 
 def gs_cache_import(cache: Cache, blob: torch.Tensor, stream=None):
     _check(_L.gs_cache_import(cache.handle, _ptr(blob), blob.numel(), _stream(stream)))
+
+
+def gs_batch_stats(cache: Cache, stream=None):
+    """Synchronises; {'slow_refills': ..., 'queued_rescans': ...} of the last batch."""
+    out = (ctypes.c_int64 * 3)()
+    _check(_L.gs_batch_stats(cache.handle, _stream(stream), out))
+    return {"slow_refills": int(out[0]), "queued_rescans": int(out[1])}
 
 
 def gs_sync_status(cache: Cache, stream=None):

@@ -97,6 +97,7 @@ static StepParams step_params(const gs_cache* c, int32_t layer, uint32_t step) {
     P.word_pick = key_word(3, (uint32_t)layer);
     P.table = c->d_table;
     P.status = c->d_hdr + HDR_STATUS;
+    P.stats = c->d_hdr + HDR_STAT_SLOW;
     P.lambda_otf = c->lambda_otf;
     P.lambda_full = c->lambda_full;
     P.hub_degree = c->hub_degree;
@@ -344,6 +345,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         P.item_cap = (int32_t)w.item_cap;
         P.work_counter = c->d_hdr + HDR_WORK + k;
         P.work_counter2 = c->d_hdr + HDR_WORK2 + k;
+        P.work_counter_scan = c->d_hdr + HDR_WORK3 + k;
         P.do_pick = 1;
         P.init_rows = 0;
         P.item_start = C.item_start;
@@ -424,6 +426,15 @@ gs_status gs_batch_counts(gs_cache* c, void* stream, int32_t* h_num_nodes, int32
     if (status == GS_ERR_RANGE) return fail(GS_ERR_RANGE, "a seed id is outside [0, num_nodes)");
     if (status == GS_ERR_DUP_SEED) return fail(GS_ERR_DUP_SEED, "duplicate seed id in the batch");
     if (status != 0) return fail(GS_ERR_CUDA, "unexpected device status %d", status);
+    return GS_OK;
+}
+
+gs_status gs_batch_stats(gs_cache* c, void* stream, int64_t* h_stats) {
+    if (!c || !h_stats) return fail(GS_ERR_ARG, "NULL argument");
+    cudaStream_t s = (cudaStream_t)stream;
+    GS_CUDA(cudaMemcpyAsync(c->h_pinned, c->d_hdr + HDR_STAT_SLOW, 3 * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    GS_CUDA(cudaStreamSynchronize(s));
+    for (int i = 0; i < 3; ++i) h_stats[i] = c->h_pinned[i];
     return GS_OK;
 }
 

@@ -46,7 +46,7 @@ __device__ __forceinline__ uint32_t warp_smallest_k(uint32_t key, uint32_t valid
     if (k >= n) return valid;
     if (k <= 0) return 0u;
     const bool mine = (valid >> lane) & 1u;
-    const uint32_t guess = (uint32_t)(((unsigned long long)k << 32) / (unsigned)n) - 1u;
+    const uint32_t guess = __float2uint_rz(__fdividef((float)k, (float)n) * 4294967040.0f);  // k < n <= 32
     uint32_t sel = __ballot_sync(FULL, mine && key <= guess);
     int c = __popc(sel);
     while (c > k) {   // drop the largest selected pair: max key, highest lane among equals

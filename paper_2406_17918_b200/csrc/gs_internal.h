@@ -18,13 +18,17 @@ constexpr int HDR_TICKET_A = HDR_HUBS + GS_MAX_HOPS;
 constexpr int HDR_TICKET_E = HDR_TICKET_A + GS_MAX_HOPS;
 constexpr int HDR_WORK2 = HDR_TICKET_E + GS_MAX_HOPS;  // work counters of the hub-chunk kernel
 constexpr int HDR_ITEMS = HDR_WORK2 + GS_MAX_HOPS;     // scan work items per step (split OTF path)
-constexpr int HDR_WORDS = HDR_ITEMS + GS_MAX_HOPS;
+constexpr int HDR_WORK3 = HDR_ITEMS + GS_MAX_HOPS;     // work counters of the scan kernel
+constexpr int HDR_STAT_SLOW = HDR_WORK3 + GS_MAX_HOPS;    // nodes whose refill was retried by one warp (whole batch)
+constexpr int HDR_STAT_QUEUED = HDR_STAT_SLOW + 1;        // nodes handed to the chunked hub kernel
+constexpr int HDR_STAT_REFRESHED = HDR_STAT_QUEUED + 1;   // nodes refreshed
+constexpr int HDR_WORDS = HDR_STAT_REFRESHED + 1;
 constexpr int HDR_HUB64 = 128;                   // 64-bit (hubs << 32 | chunks) counters, one per launch
 constexpr size_t HDR_BYTES = 1024;
 static_assert(HDR_WORDS <= HDR_HUB64, "header words overlap the 64-bit counters");
 static_assert((HDR_HUB64 + 2 * GS_MAX_HOPS) * 4 <= HDR_BYTES, "header too small");
 
-constexpr int HUB_CHUNK_QUADS = 2048;   // one hub work item = 8192 edge offsets
+constexpr int HUB_CHUNK_QUADS = 1024;   // one scan work item = 4096 edge offsets
 constexpr int HUB_MIN_DEGREE = 4096;    // lowest degree at which a node may be split over warps
 constexpr int HUB_CAND_CAP = 128;       // candidate entries per hub (same as a warp's buffer)
 
@@ -136,7 +140,8 @@ struct StepParams {
     int32_t hub_cap, item_cap;
     int32_t* work_counter;
     int32_t* work_counter2;
-    // split OTF path: scan work items (one per 8192-offset chunk of a refreshed node) and the
+    int32_t* work_counter_scan;
+    // split OTF path: scan work items (one per 4096-offset chunk of a refreshed node) and the
     // per-node candidate lists they produce
     const int32_t* item_start;       // [n+1] first item of each frontier position
     const int32_t* items;            // item -> frontier position
@@ -144,6 +149,7 @@ struct StepParams {
     int32_t* cand_count;             // [n]
     unsigned long long* cand;        // [n][SPLIT_CAND_CAP]
     int32_t* status;
+    int32_t* stats;                  // header words HDR_STAT_*: rare-event counters
     int32_t do_pick, init_rows;
     float lambda_otf, lambda_full;
     int32_t hub_degree;

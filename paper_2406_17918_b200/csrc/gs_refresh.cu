@@ -16,7 +16,7 @@
 // Two kernels per step:
 //   k_refresh_pick      one warp per frontier node, software-pipelined: while the neighbour ids
 //                       of node i are in flight the warp already scans node i+1.  Nodes above the
-//                       hub degree are only registered, as a list of 8192-offset chunks.
+//                       hub degree are only registered, as a list of 4096-offset chunks.
 //   k_refresh_pick_hub  one warp per chunk; candidates go to a per-hub buffer in global memory,
 //                       and the warp that finishes a hub's last chunk completes the node.  No
 //                       warp ever waits for another one.
@@ -27,6 +27,7 @@ namespace gs {
 
 constexpr int RP_THREADS = 256;
 constexpr int RP_WARPS = RP_THREADS / 32;
+constexpr int RETRY_QUEUE_DEGREE = 2048;  // split path: longer rows that need a rescan go to the hub kernel
 static_assert(CAND_CAP == HUB_CAND_CAP, "hub buffers are copied into a warp buffer");
 
 __device__ __forceinline__ uint32_t threshold_for(float lambda, uint32_t deg) {
@@ -268,6 +269,7 @@ __device__ __noinline__ void refill_slow(const StepParams& P, int32_t v, int64_t
     Refill R;
     const uint32_t nq = (deg + 3u) >> 2;
     const int r = __popc(evict);
+    if (lane == 0) atomicAdd(P.stats + 0, 1);
     {
         const uint32_t tinc = threshold_for(P.lambda_full, deg);
         const int c = warp_collect(P, v, deg, 0, nq, tinc, buf, 0, lane);
@@ -304,6 +306,7 @@ __device__ __forceinline__ bool hub_register(const StepParams& P, int p, uint32_
     const long long cb = (long long)(uint32_t)got;
     const bool ok = h < P.hub_cap && cb + nch <= (long long)P.item_cap;
     if (ok && lane == 0) {
+        atomicAdd(P.stats + 1, 1);
         P.hub_entry[h] = make_int2(p, (int)cb);
         P.hub_state[h] = make_int2(0, 0);
     }
@@ -497,7 +500,7 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick_hub(const __grid
 
 // ================================================================ split OTF path
 // For a partial refresh (0 < r < W) the work is split in two kernels:
-//   k_scan    one warp per work item (an 8192-offset chunk of one refreshed node): nothing but
+//   k_scan    one warp per work item (a 4096-offset chunk of one refreshed node): nothing but
 //             Philox blocks and a threshold compare, at full occupancy; the few offsets below the
 //             threshold go to the node's candidate list in global memory (at most 32, one per lane).
 //   k_finish  one warp per frontier node: eviction, refill from the candidate list, row update
@@ -516,7 +519,7 @@ __global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ Ste
     const uint32_t lt = lanemask_lt();
     while (true) {
         int base = 0;
-        if (lane == 0) base = atomicAdd(P.work_counter2, batch);
+        if (lane == 0) base = atomicAdd(P.work_counter_scan, batch);
         base = __shfl_sync(FULL, base, 0);
         if (base >= total) break;
         const int cnt = (base + batch < total ? base + batch : total) - base;
@@ -542,17 +545,21 @@ __global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ Ste
             const uint32_t tinc = threshold_for(P.lambda_otf, deg);
             unsigned long long* cand = P.cand + (size_t)p * SPLIT_CAND_CAP;
             int count = 0;
-            for (uint32_t qb = qa; qb < qe; qb += 32) {
-                const uint32_t q = qb + lane;
-                const uint4 o = philox4x32_10(q, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
-                const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
-                const bool inq = q < qe;
-                const bool any = inq && (min(min(kk[0], kk[1]), min(kk[2], kk[3])) <= tinc);
+            // two independent Philox blocks per lane and iteration (256 offsets per warp iteration):
+            // a lone warp at the tail of the launch is bound by the latency of the dependent rounds
+            for (uint32_t qb = qa; qb < qe; qb += 64) {
+                const uint32_t q0 = qb + lane, q1 = qb + 32 + lane;
+                const uint4 o0 = philox4x32_10(q0, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
+                const uint4 o1 = philox4x32_10(q1, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
+                const uint32_t kk[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
+                const bool in0 = q0 < qe, in1 = q1 < qe;
+                const bool any = (in0 && (min(min(kk[0], kk[1]), min(kk[2], kk[3])) <= tinc)) ||
+                                 (in1 && (min(min(kk[4], kk[5]), min(kk[6], kk[7])) <= tinc));
                 if (__ballot_sync(FULL, any) == 0) continue;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t off = 4u * q + j;
-                    const bool hit = inq && (off < deg) && (kk[j] <= tinc);
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t off = 4u * (j < 4 ? q0 : q1) + (j & 3);
+                    const bool hit = (j < 4 ? in0 : in1) && (off < deg) && (kk[j] <= tinc);
                     const uint32_t b = __ballot_sync(FULL, hit);
                     if (b) {
                         int basepos = count;
@@ -726,6 +733,9 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_finish(const __grid_constant_
                         }
                     }
                     if (!done) {
+                        // A long row is not rescanned by this one warp: it is queued for the chunked
+                        // hub kernel, which redoes the node (pick included) with all warps.
+                        if (deg > (uint32_t)RETRY_QUEUE_DEGREE && hub_register(P, p, deg, lane)) continue;
                         refill_slow(P, v, rs, deg, evict, buf, slot, lane);
                         __syncwarp();
                     }
@@ -753,7 +763,12 @@ cudaError_t launch_scan_finish(const StepParams& p, int64_t n_bound, int64_t ite
     int64_t fb = (n_bound + RP_WARPS - 1) / RP_WARPS;
     fb = fb > cap ? cap : (fb < 1 ? 1 : fb);
     k_finish<<<(int)fb, RP_THREADS, 0, s>>>(p);
-    count_launches(2);
+    int launched = 2;
+    if (p.hub_cap > 0) {   // rows queued for a rescan (rare); exits at once when there are none
+        k_refresh_pick_hub<<<(int)cap, RP_THREADS, 0, s>>>(p);
+        launched = 3;
+    }
+    count_launches(launched);
     return cudaGetLastError();
 }
 
