@@ -510,8 +510,10 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick_hub(const __grid
 // neighbours among the first ones) take the retry ladder of the fused path.
 
 __global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ StepParams P) {
+    __shared__ unsigned long long s_stage[RP_WARPS][SPLIT_CAND_CAP];
     if (__ldcg(P.status) != 0) return;
     const int lane = threadIdx.x & 31;
+    unsigned long long* stage = s_stage[threadIdx.x >> 5];
     const int total = __ldcg(P.d_items_total);
     const int total_warps = gridDim.x * RP_WARPS;
     int batch = total / (total_warps * 4);
@@ -543,8 +545,7 @@ __global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ Ste
             const uint32_t qa = (uint32_t)chunk * HUB_CHUNK_QUADS;
             const uint32_t qe = qa + HUB_CHUNK_QUADS < nq ? qa + HUB_CHUNK_QUADS : nq;
             const uint32_t tinc = threshold_for(P.lambda_otf, deg);
-            unsigned long long* cand = P.cand + (size_t)p * SPLIT_CAND_CAP;
-            int count = 0;
+            int count = 0;   // hits of this item, staged in shared memory (those beyond the cap are only counted)
             // two independent Philox blocks per lane and iteration (256 offsets per warp iteration):
             // a lone warp at the tail of the launch is bound by the latency of the dependent rounds
             for (uint32_t qb = qa; qb < qe; qb += 64) {
@@ -562,20 +563,27 @@ __global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ Ste
                     const bool hit = (j < 4 ? in0 : in1) && (off < deg) && (kk[j] <= tinc);
                     const uint32_t b = __ballot_sync(FULL, hit);
                     if (b) {
-                        int basepos = count;
-                        if (!single) {   // several warps share this node's list
-                            if (lane == 0) basepos = atomicAdd(P.cand_count + p, __popc(b));
-                            basepos = __shfl_sync(FULL, basepos, 0);
-                        }
                         if (hit) {
-                            const int pos = basepos + __popc(b & lt);
-                            if (pos < SPLIT_CAND_CAP) cand[pos] = ((unsigned long long)kk[j] << 32) | off;
+                            const int pos = count + __popc(b & lt);
+                            if (pos < SPLIT_CAND_CAP) stage[pos] = ((unsigned long long)kk[j] << 32) | off;
                         }
                         count += __popc(b);
                     }
                 }
             }
-            if (single && lane == 0) P.cand_count[p] = count;
+            __syncwarp();
+            // publish: the only warp of a short row owns the list; the chunks of a long row reserve
+            // their range with one atomic per chunk, so no warp waits on an atomic inside the scan
+            int dst = 0;
+            if (single) {
+                if (lane == 0) P.cand_count[p] = count;
+            } else if (count > 0) {
+                if (lane == 0) dst = atomicAdd(P.cand_count + p, count);
+                dst = __shfl_sync(FULL, dst, 0);
+            }
+            if (lane < count && dst + lane < SPLIT_CAND_CAP)
+                P.cand[(size_t)p * SPLIT_CAND_CAP + dst + lane] = stage[lane];
+            __syncwarp();
         }
     }
 }

@@ -9,14 +9,15 @@ namespace gs {
 
 __device__ __forceinline__ void raise_status(int32_t* status, int code) { atomicCAS(status, 0, code); }
 
-// In-place exclusive scan of tile_sums[0..T) by one block of 1024 threads; returns the total.
+// In-place exclusive scan of tile_sums[0..T) by one block of BT threads; returns the total.
+template <int BT>
 __device__ int scan_tiles_in_place(int32_t* tile_sums, int T, int* warp_sums) {
     int carry = 0;
-    for (int base = 0; base < T; base += 1024) {
+    for (int base = 0; base < T; base += BT) {
         const int i = base + (int)threadIdx.x;
         const int x = (i < T) ? __ldcg(tile_sums + i) : 0;
         int total;
-        const int excl = block_exclusive_scan<1024>(x, warp_sums, &total);
+        const int excl = block_exclusive_scan<BT>(x, warp_sums, &total);
         if (i < T) tile_sums[i] = carry + excl;
         carry += total;
     }
@@ -83,9 +84,9 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    const int m = scan_tiles_in_place(P.tile_sums, (int)gridDim.x, warp_sums);
+    const int m = scan_tiles_in_place<SCAN_A_TILE>(P.tile_sums, (int)gridDim.x, warp_sums);
     int items = 0;
-    if (P.split) items = scan_tiles_in_place(P.tile_sums2, (int)gridDim.x, warp_sums);
+    if (P.split) items = scan_tiles_in_place<SCAN_A_TILE>(P.tile_sums2, (int)gridDim.x, warp_sums);
     if (threadIdx.x == 0) {
         P.hdr[HDR_M + P.k] = m;
         P.hdr[HDR_ITEMS + P.k] = items;
@@ -135,46 +136,79 @@ cudaError_t launch_row_counts(const CountParams& p, int64_t n_bound, cudaStream_
 // table (which is exactly the preload the next step needs).
 //
 // aux[e] holds, for a first occurrence, -(tile-local rank)-1, otherwise the table position.
-__global__ void __launch_bounds__(1024) k_first_flags(RelabelParams P) {
+constexpr int FF_THREADS = 256;                 // 8 warps, each owns 512 consecutive picks of the tile
+static_assert(SCAN_E_TILE == FF_THREADS * 16, "tile = 16 picks per thread");
+
+__global__ void __launch_bounds__(FF_THREADS) k_first_flags(RelabelParams P) {
     __shared__ int warp_sums[33];
+    __shared__ int s_wtot[FF_THREADS / 32];
     __shared__ int is_last;
     __shared__ int s_status;
     if (threadIdx.x == 0) s_status = __ldcg(P.hdr + HDR_STATUS);
     __syncthreads();
     if (s_status != 0) return;  // block-uniform
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int n = __ldcg(P.hdr + HDR_N + P.k);
     const int m = __ldcg(P.hdr + HDR_M + P.k);
-    const int base = blockIdx.x * SCAN_E_TILE + threadIdx.x * 4;
-    int pos[4];
-    int flag[4];
-    int tsum = 0;
-    if (base < m) {
-        const int4 ids = *reinterpret_cast<const int4*>(P.picked + base);  // buffer is padded to 4
-        const int id[4] = {ids.x, ids.y, ids.z, ids.w};
+    const int wbase = blockIdx.x * SCAN_E_TILE + wid * 512;
+    // 16 independent table probes per thread are in flight before anything is consumed
+    int id[4][4];
+    int pos[4][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            pos[j] = 0;
-            flag[j] = 0;
-            if (base + j < m) {
-                pos[j] = (int)(uint32_t)__ldcg(P.table + id[j]);
-                flag[j] = (pos[j] == n + base + j);
-                tsum += flag[j];
-            }
-        }
-    } else {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) { pos[j] = 0; flag[j] = 0; }
+    for (int j = 0; j < 4; ++j) {
+        const int e0 = wbase + j * 128 + lane * 4;
+        int4 v = make_int4(0, 0, 0, 0);
+        if (e0 < m) v = *reinterpret_cast<const int4*>(P.picked + e0);  // buffer is padded to 4
+        id[j][0] = v.x; id[j][1] = v.y; id[j][2] = v.z; id[j][3] = v.w;
     }
-    int total;
-    int run = block_exclusive_scan<1024>(tsum, warp_sums, &total);
-    if (base < m) {
-        int out[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            out[j] = flag[j] ? -run - 1 : pos[j];
-            run += flag[j];
+    for (int j = 0; j < 4; ++j) {
+        const int e0 = wbase + j * 128 + lane * 4;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) pos[j][i] = (e0 + i < m) ? (int)(uint32_t)__ldcg(P.table + id[j][i]) : -1;
+    }
+    int cnt[4], incl[4], before[4];
+    int wtotal = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int e0 = wbase + j * 128 + lane * 4;
+        int c = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) c += (e0 + i < m && pos[j][i] == n + e0 + i) ? 1 : 0;
+        cnt[j] = c;
+        int x = c;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int y = __shfl_up_sync(FULL, x, d);
+            if (lane >= d) x += y;
         }
-        *reinterpret_cast<int4*>(P.aux + base) = make_int4(out[0], out[1], out[2], out[3]);
+        incl[j] = x;
+        before[j] = wtotal;
+        wtotal += __shfl_sync(FULL, x, 31);
+    }
+    if (lane == 0) s_wtot[wid] = wtotal;
+    __syncthreads();
+    int woff = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < FF_THREADS / 32; ++w) {
+        const int t = s_wtot[w];
+        if (w < wid) woff += t;
+        total += t;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int e0 = wbase + j * 128 + lane * 4;
+        if (e0 < m) {
+            int run = woff + before[j] + incl[j] - cnt[j];
+            int out[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const bool first = (e0 + i < m) && pos[j][i] == n + e0 + i;
+                out[i] = first ? -run - 1 : pos[j][i];
+                run += first ? 1 : 0;
+            }
+            *reinterpret_cast<int4*>(P.aux + e0) = make_int4(out[0], out[1], out[2], out[3]);
+        }
     }
     if (threadIdx.x == 0) {
         P.tile_sums[blockIdx.x] = total;
@@ -185,39 +219,59 @@ __global__ void __launch_bounds__(1024) k_first_flags(RelabelParams P) {
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    const int fresh = scan_tiles_in_place(P.tile_sums, (int)gridDim.x, warp_sums);
+    const int fresh = scan_tiles_in_place<FF_THREADS>(P.tile_sums, (int)gridDim.x, warp_sums);
     if (threadIdx.x == 0) P.hdr[HDR_N + P.k + 1] = n + fresh;
 }
 
+// Four consecutive picks per thread, so that the dependent probes of four items overlap.
 __global__ void __launch_bounds__(256) k_relabel(RelabelParams P) {
     if (__ldcg(P.hdr + HDR_STATUS) != 0) return;
     const int n = __ldcg(P.hdr + HDR_N + P.k);
     const int m = __ldcg(P.hdr + HDR_M + P.k);
-    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < m; e += gridDim.x * blockDim.x) {
-        const int val = P.aux[e];
-        int loc;
-        if (val < 0) {
-            loc = n + (-val - 1) + P.tile_sums[e / SCAN_E_TILE];
-            if ((int64_t)loc < P.n_cap) {
-                const int id = P.picked[e];
-                P.frontier[loc] = id;
-                P.table[id] = ((unsigned long long)P.stamp << 32) | (unsigned)loc;
+    for (int e0 = 4 * (blockIdx.x * blockDim.x + threadIdx.x); e0 < m; e0 += 4 * gridDim.x * blockDim.x) {
+        const int4 a = *reinterpret_cast<const int4*>(P.aux + e0);   // padded to 4
+        const int val[4] = {a.x, a.y, a.z, a.w};
+        int ref[4], tile[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            // first occurrence: own mark; later occurrence of a new id: the mark of its first occurrence
+            const int src = (val[i] < 0) ? e0 + i : (val[i] >= n ? val[i] - n : -1);
+            ref[i] = val[i];
+            tile[i] = 0;
+            if (e0 + i < m && src >= 0) {
+                if (val[i] >= 0) ref[i] = P.aux[src];
+                tile[i] = P.tile_sums[src / SCAN_E_TILE];
             }
-        } else if (val < n) {
-            loc = val;
-        } else {
-            const int e0 = val - n;
-            loc = n + (-P.aux[e0] - 1) + P.tile_sums[e0 / SCAN_E_TILE];
         }
-        P.local[e] = loc;
+        int out[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            int loc = val[i];
+            if (e0 + i < m && (val[i] < 0 || val[i] >= n)) {
+                loc = n + (-ref[i] - 1) + tile[i];
+                if (val[i] < 0 && (int64_t)loc < P.n_cap) {
+                    const int id = P.picked[e0 + i];
+                    P.frontier[loc] = id;
+                    P.table[id] = ((unsigned long long)P.stamp << 32) | (unsigned)loc;
+                }
+            }
+            out[i] = loc;
+        }
+        if (e0 + 3 < m) {
+            *reinterpret_cast<int4*>(P.local + e0) = make_int4(out[0], out[1], out[2], out[3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (e0 + i < m) P.local[e0 + i] = out[i];
+        }
     }
 }
 
 cudaError_t launch_relabel(const RelabelParams& p, int64_t m_bound, cudaStream_t s) {
     if (m_bound <= 0) m_bound = 1;
     const int tiles = (int)((m_bound + SCAN_E_TILE - 1) / SCAN_E_TILE);
-    k_first_flags<<<tiles, 1024, 0, s>>>(p);
-    int64_t blocks = (m_bound + 255) / 256;
+    k_first_flags<<<tiles, FF_THREADS, 0, s>>>(p);
+    int64_t blocks = (m_bound + 1023) / 1024;
     if (blocks > 148 * 32) blocks = 148 * 32;
     k_relabel<<<(int)blocks, 256, 0, s>>>(p);
     count_launches(2);

@@ -8,6 +8,16 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+def pytest_sessionstart(session):
+    """Make sure the in-tree CUDA library and the C oracle exist (nvcc cross-compiles without a GPU)."""
+    import importlib.util
+
+    spec = importlib.util.spec_from_file_location("_gs_build", os.path.join(ROOT, "paper_2406_17918_b200", "build.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    mod.build()
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); run with -m gpu")
 
