@@ -160,10 +160,21 @@ gs_status gs_cache_export_bytes(const gs_cache*, size_t* bytes);
 gs_status gs_cache_export(const gs_cache*, void* d_dst, size_t bytes, void* stream);
 gs_status gs_cache_import(gs_cache*, const void* d_src, size_t bytes, void* stream);
 
-/* Synchronises `stream` and copies three counters of the last batch (or of the pre-sample, if no
- * batch ran yet) into h_stats: [0] nodes whose refill had to be redone by a full rescan on one
- * warp, [1] nodes handed to the chunked multi-warp scan, [2] reserved (0).  Diagnostics only. */
+/* Synchronises `stream` and copies four counters of the last batch into h_stats[4]:
+ * [0] nodes whose refill had to be redone by a full rescan on one warp, [1] nodes handed to the
+ * chunked multi-warp rescan, and, for a partial refresh (0 < r < cache_width) only,
+ * [2] nodes refreshed, [3] Philox blocks (4 edge offsets each) the threshold scan evaluates.
+ * Diagnostics only. */
 gs_status gs_batch_stats(gs_cache*, void* stream, int64_t* h_stats);
+
+/* Optional device-side timing of the kernels of gs_sample_batch.  Between _begin and _end every
+ * batch (up to max_batches, in [1, 4096]) records CUDA events on its own stream around four
+ * kernel groups of each sampling step: row counts / block offsets, threshold scan, finish (or
+ * the fused refresh + pick kernels), dedup + relabel.  _end synchronises `stream`, writes the
+ * summed milliseconds of the four groups to h_ms[4] and the number of batches timed to
+ * *h_batches, and releases the events.  Events are host objects; no device memory is used. */
+gs_status gs_cache_profile_begin(gs_cache*, int32_t max_batches);
+gs_status gs_cache_profile_end(gs_cache*, void* stream, double* h_ms, int64_t* h_batches);
 
 /* Synchronises `stream` and returns the device status of the last batch. */
 gs_status gs_sync_status(gs_cache*, void* stream);

@@ -72,6 +72,8 @@ def _load():
         "gs_cache_import": [vp, vp, sz, vp],
         "gs_sync_status": [vp, vp],
         "gs_batch_stats": [vp, vp, vp],
+        "gs_cache_profile_begin": [vp, i32],
+        "gs_cache_profile_end": [vp, vp, vp, vp],
         "gs_cache_set_tuning": [vp, dbl, dbl, i32],
     }
     for name, args in sig.items():
@@ -303,9 +305,22 @@ def gs_cache_import(cache: Cache, blob: torch.Tensor, stream=None):
 
 def gs_batch_stats(cache: Cache, stream=None):
     """Synchronises; {'slow_refills': ..., 'queued_rescans': ...} of the last batch."""
-    out = (ctypes.c_int64 * 3)()
+    out = (ctypes.c_int64 * 4)()
     _check(_L.gs_batch_stats(cache.handle, _stream(stream), out))
-    return {"slow_refills": int(out[0]), "queued_rescans": int(out[1])}
+    return {"slow_refills": int(out[0]), "queued_rescans": int(out[1]), "refreshed_nodes": int(out[2]),
+            "philox_blocks": int(out[3])}
+
+
+def gs_cache_profile_begin(cache: Cache, max_batches: int):
+    _check(_L.gs_cache_profile_begin(cache.handle, int(max_batches)))
+
+
+def gs_cache_profile_end(cache: Cache, stream=None):
+    """Synchronises; ({'row_counts': ms, 'scan': ms, 'finish': ms, 'relabel': ms}, batches timed)."""
+    ms = (ctypes.c_double * 4)()
+    nb = ctypes.c_int64()
+    _check(_L.gs_cache_profile_end(cache.handle, _stream(stream), ms, ctypes.byref(nb)))
+    return dict(zip(("row_counts", "scan", "finish", "relabel"), [float(x) for x in ms])), int(nb.value)
 
 
 def gs_sync_status(cache: Cache, stream=None):

@@ -33,7 +33,13 @@ struct gs_cache {
     float lambda_otf, lambda_full;
     int32_t hub_degree;
     int32_t* h_pinned;        // pinned staging for counts
+    // optional device timing of the kernel groups (gs_cache_profile_begin / _end)
+    cudaEvent_t* prof_events;
+    int32_t prof_cap, prof_used;   // in batches
 };
+
+constexpr int PROF_GROUPS = 4;               // row counts | scan | finish or fused refresh+pick | relabel
+constexpr int PROF_EVENTS_PER_STEP = PROF_GROUPS + 1;
 
 namespace gs {
 
@@ -256,7 +262,54 @@ gs_status gs_cache_init(const gs_graph* g, int32_t num_hops, const int32_t* fano
 void gs_cache_destroy(gs_cache* c) {
     if (!c) return;
     if (c->h_pinned) cudaFreeHost(c->h_pinned);
+    if (c->prof_events) {
+        for (int i = 0; i < c->prof_cap * c->L * PROF_EVENTS_PER_STEP; ++i) cudaEventDestroy(c->prof_events[i]);
+        delete[] c->prof_events;
+    }
     delete c;
+}
+
+gs_status gs_cache_profile_begin(gs_cache* c, int32_t max_batches) {
+    if (!c) return fail(GS_ERR_ARG, "cache is NULL");
+    if (max_batches < 1 || max_batches > 4096) return fail(GS_ERR_ARG, "max_batches outside [1, 4096]");
+    if (c->prof_events) return fail(GS_ERR_ARG, "profiling is already on");
+    const int n = max_batches * c->L * PROF_EVENTS_PER_STEP;
+    c->prof_events = new (std::nothrow) cudaEvent_t[n];
+    if (!c->prof_events) return fail(GS_ERR_ARG, "out of host memory");
+    for (int i = 0; i < n; ++i) {
+        cudaError_t e = cudaEventCreate(&c->prof_events[i]);
+        if (e != cudaSuccess) {
+            for (int j = 0; j < i; ++j) cudaEventDestroy(c->prof_events[j]);
+            delete[] c->prof_events;
+            c->prof_events = nullptr;
+            return cuda_fail(e, "cudaEventCreate");
+        }
+    }
+    c->prof_cap = max_batches;
+    c->prof_used = 0;
+    return GS_OK;
+}
+
+gs_status gs_cache_profile_end(gs_cache* c, void* stream, double* h_ms, int64_t* h_batches) {
+    if (!c || !h_ms || !h_batches) return fail(GS_ERR_ARG, "NULL argument");
+    if (!c->prof_events) return fail(GS_ERR_ARG, "profiling is not on");
+    GS_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    for (int gI = 0; gI < PROF_GROUPS; ++gI) h_ms[gI] = 0.0;
+    for (int b = 0; b < c->prof_used; ++b)
+        for (int k = 0; k < c->L; ++k) {
+            cudaEvent_t* ev = c->prof_events + ((size_t)b * c->L + k) * PROF_EVENTS_PER_STEP;
+            for (int gI = 0; gI < PROF_GROUPS; ++gI) {
+                float ms = 0.f;
+                GS_CUDA(cudaEventElapsedTime(&ms, ev[gI], ev[gI + 1]));
+                h_ms[gI] += ms;
+            }
+        }
+    *h_batches = c->prof_used;
+    for (int i = 0; i < c->prof_cap * c->L * PROF_EVENTS_PER_STEP; ++i) cudaEventDestroy(c->prof_events[i]);
+    delete[] c->prof_events;
+    c->prof_events = nullptr;
+    c->prof_cap = c->prof_used = 0;
+    return GS_OK;
 }
 
 gs_status gs_cache_set_tuning(gs_cache* c, double lambda_otf, double lambda_full, int32_t hub_degree) {
@@ -297,8 +350,11 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
     const uint32_t stamp = 0xFFFFFFFFu - c->serial;  // newer batches always win the atomicMin
     GS_CUDA(cudaMemsetAsync(c->d_hdr, 0, HDR_BYTES, s));
 
+    const bool prof = c->prof_events && c->prof_used < c->prof_cap;
     for (int k = 0; k < L; ++k) {
         const int layer = L - 1 - k;
+        cudaEvent_t* ev = prof ? c->prof_events + ((size_t)c->prof_used * L + k) * PROF_EVENTS_PER_STEP : nullptr;
+        if (ev) GS_CUDA(cudaEventRecord(ev[0], s));
         int32_t* blk_indptr = (int32_t*)(ws + w.blk_indptr[k]);
         int32_t* blk_indices = (int32_t*)(ws + w.blk_indices[k]);
 
@@ -326,6 +382,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         C.cand_count = (int32_t*)(ws + w.cand_count);
         C.scan_item_cap = w.scan_item_cap;
         GS_CUDA(launch_row_counts(C, b.nb[k], s));
+        if (ev) GS_CUDA(cudaEventRecord(ev[1], s));
 
         StepParams P = step_params(c, layer, step);
         P.r = r;
@@ -355,10 +412,14 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         P.cand = (unsigned long long*)(ws + w.cand);
         if (split) {
             int64_t item_bound = b.nb[k] + g->num_edges / (4 * (int64_t)HUB_CHUNK_QUADS) + 1;
-            GS_CUDA(launch_scan_finish(P, b.nb[k], item_bound, s));
+            GS_CUDA(launch_scan(P, item_bound, s));
+            if (ev) GS_CUDA(cudaEventRecord(ev[2], s));
+            GS_CUDA(launch_finish(P, b.nb[k], s));
         } else {
+            if (ev) GS_CUDA(cudaEventRecord(ev[2], s));
             GS_CUDA(launch_refresh_pick(P, b.nb[k], s));
         }
+        if (ev) GS_CUDA(cudaEventRecord(ev[3], s));
 
         RelabelParams R{};
         R.hdr = c->d_hdr;
@@ -372,6 +433,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         R.stamp = stamp;
         R.n_cap = b.nb[k + 1];
         GS_CUDA(launch_relabel(R, b.mb[k], s));
+        if (ev) GS_CUDA(cudaEventRecord(ev[4], s));
 
         gs_block& B = blocks[layer];
         B.max_dst = (int32_t)b.nb[k];
@@ -383,6 +445,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         B.d_indptr = blk_indptr;
         B.d_indices = blk_indices;
     }
+    if (prof) c->prof_used += 1;
     if (d_input_nodes) *d_input_nodes = frontier;
     if (d_num_input_nodes) *d_num_input_nodes = c->d_hdr + HDR_N + L;
     return GS_OK;
@@ -432,9 +495,9 @@ gs_status gs_batch_counts(gs_cache* c, void* stream, int32_t* h_num_nodes, int32
 gs_status gs_batch_stats(gs_cache* c, void* stream, int64_t* h_stats) {
     if (!c || !h_stats) return fail(GS_ERR_ARG, "NULL argument");
     cudaStream_t s = (cudaStream_t)stream;
-    GS_CUDA(cudaMemcpyAsync(c->h_pinned, c->d_hdr + HDR_STAT_SLOW, 3 * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    GS_CUDA(cudaMemcpyAsync(c->h_pinned, c->d_hdr + HDR_STAT_SLOW, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
     GS_CUDA(cudaStreamSynchronize(s));
-    for (int i = 0; i < 3; ++i) h_stats[i] = c->h_pinned[i];
+    for (int i = 0; i < 4; ++i) h_stats[i] = (int64_t)(uint32_t)c->h_pinned[i];
     return GS_OK;
 }
 

@@ -22,7 +22,8 @@ constexpr int HDR_WORK3 = HDR_ITEMS + GS_MAX_HOPS;     // work counters of the s
 constexpr int HDR_STAT_SLOW = HDR_WORK3 + GS_MAX_HOPS;    // nodes whose refill was retried by one warp (whole batch)
 constexpr int HDR_STAT_QUEUED = HDR_STAT_SLOW + 1;        // nodes handed to the chunked hub kernel
 constexpr int HDR_STAT_REFRESHED = HDR_STAT_QUEUED + 1;   // nodes refreshed
-constexpr int HDR_WORDS = HDR_STAT_REFRESHED + 1;
+constexpr int HDR_STAT_QUADS = HDR_STAT_REFRESHED + 1;    // Philox blocks the scan kernel has to evaluate
+constexpr int HDR_WORDS = HDR_STAT_QUADS + 1;
 constexpr int HDR_HUB64 = 128;                   // 64-bit (hubs << 32 | chunks) counters, one per launch
 constexpr size_t HDR_BYTES = 1024;
 static_assert(HDR_WORDS <= HDR_HUB64, "header words overlap the 64-bit counters");
@@ -194,7 +195,8 @@ void count_launches(int n);
 
 cudaError_t launch_row_counts(const CountParams& p, int64_t n_bound, cudaStream_t s);
 cudaError_t launch_refresh_pick(const StepParams& p, int64_t n_bound, cudaStream_t s);
-cudaError_t launch_scan_finish(const StepParams& p, int64_t n_bound, int64_t item_bound, cudaStream_t s);
+cudaError_t launch_scan(const StepParams& p, int64_t item_bound, cudaStream_t s);
+cudaError_t launch_finish(const StepParams& p, int64_t n_bound, cudaStream_t s);
 cudaError_t launch_relabel(const RelabelParams& p, int64_t m_bound, cudaStream_t s);
 cudaError_t launch_gather(const void* src, int64_t src_ld_bytes, int64_t row_bytes, const int32_t* ids,
                           const int32_t* d_count, int32_t count_bound, void* dst, int64_t dst_ld_bytes,

@@ -763,18 +763,24 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_finish(const __grid_constant_
     }
 }
 
-cudaError_t launch_scan_finish(const StepParams& p, int64_t n_bound, int64_t item_bound, cudaStream_t s) {
+cudaError_t launch_scan(const StepParams& p, int64_t item_bound, cudaStream_t s) {
     const int64_t cap = 148 * 8;
     int64_t sb = (item_bound + RP_WARPS - 1) / RP_WARPS;
     sb = sb > cap ? cap : (sb < 1 ? 1 : sb);
     k_scan<<<(int)sb, RP_THREADS, 0, s>>>(p);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_finish(const StepParams& p, int64_t n_bound, cudaStream_t s) {
+    const int64_t cap = 148 * 8;
     int64_t fb = (n_bound + RP_WARPS - 1) / RP_WARPS;
     fb = fb > cap ? cap : (fb < 1 ? 1 : fb);
     k_finish<<<(int)fb, RP_THREADS, 0, s>>>(p);
-    int launched = 2;
+    int launched = 1;
     if (p.hub_cap > 0) {   // rows queued for a rescan (rare); exits at once when there are none
         k_refresh_pick_hub<<<(int)cap, RP_THREADS, 0, s>>>(p);
-        launched = 3;
+        launched = 2;
     }
     count_launches(launched);
     return cudaGetLastError();

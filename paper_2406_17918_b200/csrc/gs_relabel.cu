@@ -40,6 +40,7 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
     const int p = blockIdx.x * SCAN_A_TILE + threadIdx.x;
     int c = 0;
     int nch = 0;   // scan work items of this node (split path only)
+    unsigned quads = 0, refreshed = 0;
     const int refresh_from = (P.split && P.d_refresh_from) ? __ldcg(P.d_refresh_from) : 0;
     if (p < n) {
         int v;
@@ -63,7 +64,9 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
             if (P.split && deg > (int64_t)SMALL_DEGREE && deg > (int64_t)P.W && p >= refresh_from) {
                 const int64_t nq = (deg + 3) >> 2;
                 nch = (int)((nq + HUB_CHUNK_QUADS - 1) / HUB_CHUNK_QUADS);
+                quads = (unsigned)nq;
             }
+            if (P.split && deg > (int64_t)P.W && p >= refresh_from) refreshed = 1;
         }
     }
     int total;
@@ -71,6 +74,11 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
     if (p < n) P.blk_indptr[p] = excl;
     int total2 = 0;
     if (P.split) {
+        const unsigned wq = __reduce_add_sync(FULL, quads), wr = __reduce_add_sync(FULL, refreshed);
+        if ((threadIdx.x & 31) == 0 && wr) {
+            atomicAdd((unsigned*)(P.hdr + HDR_STAT_QUADS), wq);
+            atomicAdd((unsigned*)(P.hdr + HDR_STAT_REFRESHED), wr);
+        }
         const int excl2 = block_exclusive_scan<SCAN_A_TILE>(nch, warp_sums, &total2);
         if (p < n) P.item_start[p] = excl2;
     }
