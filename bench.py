@@ -30,6 +30,10 @@ from workloads import batch_seeds, build_features, build_graph, get_config, seed
 
 METRIC = "sampled edges/s + feature GB/s per batch (OTF), fraction of HBM roofline"
 FALLBACK_HBM_GBS = 6650.0
+# INT32 ALU peak of one B200: 148 SMs x 128 lanes x 1.965 GHz lane-ops/s.  One Philox4x32-10 block needs
+# ten rounds of two 32x32->64 multiplies (two lane-ops each on this GPU) and two 3-input xors: 60 lane-ops.
+ALU_LANE_OPS = 148 * 128 * 1.965e9
+PHILOX_LANE_OPS = 60.0
 SAMPLER_SEED = 0x6A09E667F3BCC908
 
 
@@ -220,11 +224,12 @@ def main():
     ws = torch.empty(gs.gs_workspace_bytes(G, cfg["fanouts"], B), dtype=torch.uint8, device=device)
     gm = gs.GS_MODE_OTF if mode == "otf" else gs.GS_MODE_FCR
     r = int(gamma * cfg["cache_width"] + 0.5) if mode == "otf" else cfg["cache_width"]
-    hdr = C.storage[:256].view(torch.int32)
+    hdr = C.storage[:512].view(torch.int32)
+    stat0 = gs.gs_stats_word_offset()
 
     K, Wm = args.steps, args.warmup
     seeds_all = [batch_seeds(perm, b, B, rank, world) for b in range(Wm + 2 * K)]
-    pinned_counts = torch.zeros((K, 64), dtype=torch.int32).pin_memory()
+    pinned_counts = torch.zeros((K, 128), dtype=torch.int32).pin_memory()
     out = None
 
     def one_step(b, step):
@@ -245,6 +250,7 @@ def main():
     replicas.barrier()
     torch.cuda.synchronize()
     launches0 = gs.gs_kernel_launches()
+    gs.gs_cache_profile_begin(C, K)     # CUDA events around the batch's kernel groups, on the launching stream
     wall0 = time.time()
     for i in range(K):
         b = Wm + i
@@ -261,6 +267,7 @@ def main():
     wall1 = time.time()
     launches = gs.gs_kernel_launches() - launches0
     total_ms = events[0].elapsed_time(end)
+    group_ms, _ = gs.gs_cache_profile_end(C)
     gs.gs_sync_status(C)
     if clocks:
         time.sleep(0.1)
@@ -284,6 +291,8 @@ def main():
         lo = n_last[k - 1] if (cfg["shared"] and k > 0) else 0
         refreshed_frac.append(float(over[lo:n_last[k]].sum().item()) / max(1, n_last[k]))
     alg_total, alg_feat = 0, 0
+    philox_blocks = sum(int(counts[i][stat0 + 3]) & 0xFFFFFFFF for i in range(K))
+    slow_refills = sum(int(counts[i][stat0]) for i in range(K))
     for i in range(K):
         n = [int(counts[i][w]) for w in n_words]
         m = [int(counts[i][w]) for w in m_words]
@@ -315,8 +324,8 @@ def main():
                "d2h_bytes_per_step": gs.COUNTS_READBACK_BYTES,
                "ms_per_step": e_ms / K}
 
-    t_ms, (edges_all, feat_rows_all, alg_all, alg_feat_all, gather_ms_max) = replicas.aggregate(
-        total_ms, [edges, feat_rows, alg_total, alg_feat, gather_ms], device)
+    t_ms, (edges_all, feat_rows_all, alg_all, alg_feat_all, gather_ms_max, philox_all) = replicas.aggregate(
+        total_ms, [edges, feat_rows, alg_total, alg_feat, gather_ms, philox_blocks], device)
     if rank != 0:
         replicas.shutdown()
         return 0
@@ -327,12 +336,29 @@ def main():
     gather_bytes_per_launch = alg_feat / K
     gather_ms_per_launch = gather_ms / K
     achieved = gather_bytes_per_launch / (gather_ms_per_launch * 1e-3) / 1e9
+    roof_gather = {"kernel": "k_gather (feature rows), 1 launch per step", "bound": "hbm", "achieved": achieved,
+                   "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                   "ms_per_launch": gather_ms_per_launch, "traffic": None}
+    # the threshold scan (k_scan, one launch per sampling step) is bound by integer ALU work: Philox blocks
+    scan_launches = K * L
+    roof_scan = None
+    if group_ms["scan"] > 0 and philox_blocks > 0:
+        a_scan = philox_blocks / (group_ms["scan"] * 1e-3) / 1e9
+        p_scan = ALU_LANE_OPS / PHILOX_LANE_OPS / 1e9
+        roof_scan = {"kernel": "k_scan (Philox threshold scan), %d launches per step" % L, "bound": "alu",
+                     "achieved": a_scan, "peak": p_scan, "peak_kind": "derived: 148 SMs x 128 lanes x 1.965 GHz / 60 lane-ops per block",
+                     "unit": "G Philox4x32-10 blocks/s", "frac": a_scan / p_scan,
+                     "ms_per_launch": group_ms["scan"] / scan_launches, "traffic": None}
+    groups = dict(group_ms)
+    groups["gather"] = gather_ms
+    dominant = max(groups, key=groups.get)
     result = {
         "metric": METRIC,
         "value": edges_all / secs,
         "unit": "edges/s",
         "feature_gbs": feat_rows_all * cfg["feat_dim"] * esize / secs / 1e9,
         "hbm_frac_batch": (alg_all / secs / 1e9) / peak / max(1, world),
+        "hbm_frac_batch_incl_scanned_csr": ((alg_all + 16.0 * philox_all) / secs / 1e9) / peak / max(1, world),
         "n_gpus": world,
         "steps": K,
         "warmup": Wm,
@@ -347,11 +373,14 @@ def main():
                    "batch": B, "shared_cache": cfg["shared"], "feat_dim": cfg["feat_dim"],
                    "parallelism": "replicas x%d" % world, "l2": "inputs_larger_than_L2",
                    "sampled_edges_per_batch": edges / K, "input_nodes_per_batch": feat_rows / K},
-        "breakdown_ms_per_step": {"sample_batch": sample_ms / K, "gather_features": gather_ms / K},
+        "breakdown_ms_per_step": {"sample_batch": sample_ms / K, "gather_features": gather_ms / K,
+                                  "kernel_groups": {k: v / K for k, v in groups.items()}, "dominant": dominant},
+        "philox_blocks_per_batch": philox_blocks / K,
+        "slow_refills_per_batch": slow_refills / K,
         "presample_ms": presample_ms,
         "setup_s": {"graph_and_features": t_graph},
-        "roofline": {"kernel": "k_gather (feature rows)", "bound": "hbm", "achieved": achieved, "peak": peak,
-                     "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": None},
+        "roofline": roof_scan if (dominant == "scan" and roof_scan) else roof_gather,
+        "roofline_gather": roof_gather,
         "algorithmic_bytes_per_batch": alg_total / K,
         "gpu_launches": launches,
         "clocks": clocks.summary(wall0, wall1) if clocks else None,

@@ -167,6 +167,10 @@ gs_status gs_cache_import(gs_cache*, const void* d_src, size_t bytes, void* stre
  * Diagnostics only. */
 gs_status gs_batch_stats(gs_cache*, void* stream, int64_t* h_stats);
 
+/* Index (in int32 words from the start of the cache storage) of the four gs_batch_stats counters,
+ * for callers that copy the state header asynchronously instead of synchronising per batch. */
+int32_t gs_stats_word_offset(void);
+
 /* Optional device-side timing of the kernels of gs_sample_batch.  Between _begin and _end every
  * batch (up to max_batches, in [1, 4096]) records CUDA events on its own stream around four
  * kernel groups of each sampling step: row counts / block offsets, threshold scan, finish (or

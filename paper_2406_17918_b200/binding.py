@@ -86,12 +86,18 @@ def _load():
     L.gs_cache_destroy.restype = None
     L.gs_last_error.argtypes = []
     L.gs_last_error.restype = ctypes.c_char_p
+    L.gs_stats_word_offset.argtypes = []
+    L.gs_stats_word_offset.restype = ctypes.c_int32
     L.gs_kernel_launches.argtypes = []
     L.gs_kernel_launches.restype = ctypes.c_int64
     return L
 
 
 _L = _load()
+
+
+def gs_stats_word_offset() -> int:
+    return int(_L.gs_stats_word_offset())
 
 
 def gs_last_error() -> str:

@@ -117,6 +117,7 @@ using namespace gs;
 extern "C" {
 
 const char* gs_last_error(void) { return g_err; }
+int32_t gs_stats_word_offset(void) { return HDR_STAT_SLOW; }
 int64_t gs_kernel_launches(void) { return (int64_t)g_launches.load(); }
 
 gs_status gs_graph_create(int64_t num_nodes, int64_t num_edges, const int64_t* d_indptr, const int32_t* d_indices,
