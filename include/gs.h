@@ -127,6 +127,48 @@ gs_status gs_sample_batch(gs_cache*, const int32_t* d_seeds, int32_t num_seeds, 
                           uint32_t step, void* d_workspace, size_t workspace_bytes, void* stream,
                           gs_block* blocks, const int32_t** d_input_nodes, const int32_t** d_num_input_nodes);
 
+/* Caller-owned output arrays of one hop for gs_sample_batch_noalloc (capacities in int32 entries). */
+typedef struct {
+    int32_t* d_indptr;
+    int64_t indptr_capacity;
+    int32_t* d_indices;
+    int64_t indices_capacity;
+} gs_block_buffers;
+
+/* Bytes of the scratch array built into the library for gs_sample_batch_noalloc.  Every GPU that
+ * loads the library holds this much device memory from load until the process exits. */
+#define GS_NOALLOC_SCRATCH_BYTES (64u << 20)
+
+/* The same mini-batch as gs_sample_batch, for callers that cannot provide a scratch workspace
+ * because they are not allowed to allocate device memory (a memory pool owns the whole device, a
+ * host application hands out fixed buffers, a start-up memory budget is enforced).  The paper
+ * has no counterpart to this call; it exists only for such deployments.  It allocates nothing
+ * (no cudaMalloc / cudaFree, no allocating library routine): the scratch is a fixed array of
+ * GS_NOALLOC_SCRATCH_BYTES inside the library, and the results go to buffers the caller passes:
+ *   d_input_nodes   int32[input_nodes_capacity] receives the input-node list (the last frontier)
+ *   h_buffers       h_ array of num_hops entries, by layer: where each block's offsets and
+ *                   block-local source ids go.  With n_0 = num_seeds, m_k = n_k * fanout of step k
+ *                   and n_{k+1} = min(num_nodes, n_k + m_k), the block of step k needs n_k + 1
+ *                   offsets and m_k indices, and the input-node list needs n_L ids.
+ *   blocks          filled as by gs_sample_batch, pointing into the caller's buffers
+ *   d_num_input_nodes  receives a device pointer to the count (may be NULL)
+ * Everything else (seeds, mode, gamma, step, results, status reporting through gs_batch_counts) is
+ * as for gs_sample_batch, and the results are bit-identical.
+ * Limits and rules
+ *   - A batch needs as much scratch as gs_workspace_bytes reports for it; if that exceeds
+ *     GS_NOALLOC_SCRATCH_BYTES the call returns GS_ERR_WORKSPACE (message with both sizes) and
+ *     launches nothing.  Too-small output buffers are rejected the same way.
+ *   - The first call on each device looks up the device address of the built-in array (with that
+ *     device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents; the
+ *     kernels initialise every part of it they read, so nothing has to be cleared between calls.
+ *     Two calls whose kernels overlap on the GPU (different streams, different caches) race on
+ *     the array: run them one after the other. */
+gs_status gs_sample_batch_noalloc(gs_cache*, const int32_t* d_seeds, int32_t num_seeds, gs_mode mode, double gamma,
+                                  uint32_t step, int32_t* d_input_nodes, int64_t input_nodes_capacity,
+                                  const gs_block_buffers* h_buffers, void* stream, gs_block* blocks,
+                                  const int32_t** d_num_input_nodes);
+
 /* Same batch for a caller whose seeds are in HOST memory: copies h_seeds to the device, runs the
  * batch, copies the counts back and synchronises `stream`.
  *   h_num_nodes  int32[num_hops + 1]: n_0 (seeds) .. n_L (input nodes), by sampling step

@@ -37,6 +37,14 @@ class _CBlock(ctypes.Structure):
                 ("d_indptr", ctypes.c_void_p), ("d_indices", ctypes.c_void_p)]
 
 
+class _CBlockBuffers(ctypes.Structure):
+    _fields_ = [("d_indptr", ctypes.c_void_p), ("indptr_capacity", ctypes.c_int64),
+                ("d_indices", ctypes.c_void_p), ("indices_capacity", ctypes.c_int64)]
+
+
+NOALLOC_SCRATCH_BYTES = 64 << 20
+
+
 def library_path() -> str:
     return _LIB_PATH
 
@@ -64,6 +72,7 @@ def _load():
         "gs_cache_init": [vp, i32, vp, i32, u64, i32, vp, sz, vp, pvp],
         "gs_sample_batch": [vp, vp, i32, ctypes.c_int, dbl, u32, vp, sz, vp, vp, pvp, pvp],
         "gs_sample_batch_host": [vp, vp, i32, ctypes.c_int, dbl, u32, vp, sz, vp, vp, pvp, vp, vp],
+        "gs_sample_batch_noalloc": [vp, vp, i32, ctypes.c_int, dbl, u32, vp, i64, vp, vp, vp, pvp],
         "gs_batch_counts": [vp, vp, vp, vp],
         "gs_gather_features": [vp, vp, vp, i32, vp, i64, vp],
         "gs_cache_read_rows": [vp, i32, vp, i32, vp, vp],
@@ -269,6 +278,43 @@ def gs_sample_batch_host(cache: Cache, seeds_host: torch.Tensor, mode: int, gamm
     off = d_in.value - workspace.data_ptr()
     input_nodes = workspace[off:off + 4 * blocks[0].max_src].view(torch.int32)
     return blocks, input_nodes, list(n), list(m)
+
+
+class OutBlock:
+    """One hop's block as written by gs_sample_batch_noalloc into the caller's tensors."""
+
+    def __init__(self, cb, indptr, indices):
+        self.max_dst, self.max_src, self.max_edges = cb.max_dst, cb.max_src, cb.max_edges
+        self._indptr, self._indices = indptr, indices
+
+    def indptr(self, num_dst: int) -> torch.Tensor:
+        return self._indptr[: num_dst + 1]
+
+    def indices(self, num_edges: int) -> torch.Tensor:
+        return self._indices[:num_edges]
+
+
+def gs_sample_batch_noalloc(cache: Cache, seeds: torch.Tensor, mode: int, gamma: float, step: int,
+                            input_nodes: torch.Tensor, indptr_bufs, indices_bufs, stream=None):
+    """The batch call for callers that may not allocate device memory: scratch is the library's
+    built-in array, results land in the int32 CUDA tensors passed here (`indptr_bufs[l]`,
+    `indices_bufs[l]` by layer, and `input_nodes`).  Nothing is allocated by this function either.
+    Returns the blocks (views of the caller's tensors), by layer."""
+    if seeds.dtype != torch.int32 or not seeds.is_cuda or not seeds.is_contiguous():
+        raise TypeError("seeds must be a contiguous int32 CUDA tensor")
+    bufs = (_CBlockBuffers * cache.num_hops)()
+    for l in range(cache.num_hops):
+        for t in (indptr_bufs[l], indices_bufs[l]):
+            if t.dtype != torch.int32 or not t.is_cuda or not t.is_contiguous():
+                raise TypeError("block buffers must be contiguous int32 CUDA tensors")
+        bufs[l].d_indptr, bufs[l].indptr_capacity = indptr_bufs[l].data_ptr(), indptr_bufs[l].numel()
+        bufs[l].d_indices, bufs[l].indices_capacity = indices_bufs[l].data_ptr(), indices_bufs[l].numel()
+    cblocks = (_CBlock * cache.num_hops)()
+    d_cnt = ctypes.c_void_p()
+    _check(_L.gs_sample_batch_noalloc(cache.handle, _ptr(seeds), seeds.numel(), mode, float(gamma), step,
+                                      _ptr(input_nodes), input_nodes.numel(), bufs, _stream(stream), cblocks,
+                                      ctypes.byref(d_cnt)))
+    return [OutBlock(cblocks[l], indptr_bufs[l], indices_bufs[l]) for l in range(cache.num_hops)]
 
 
 def gs_batch_counts(cache: Cache, stream=None):

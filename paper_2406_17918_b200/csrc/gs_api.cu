@@ -56,6 +56,14 @@ static gs_status fail(gs_status code, const char* fmt, ...) {
     return code;
 }
 
+gs_status set_error(gs_status code, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
 static gs_status cuda_fail(cudaError_t e, const char* what) {
     return fail(GS_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
 }
@@ -323,7 +331,8 @@ gs_status gs_cache_set_tuning(gs_cache* c, double lambda_otf, double lambda_full
 
 static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_seeds, gs_mode mode, double gamma,
                              uint32_t step, void* d_workspace, size_t workspace_bytes, cudaStream_t s,
-                             gs_block* blocks, const int32_t** d_input_nodes, const int32_t** d_num_input_nodes) {
+                             gs_block* blocks, const int32_t** d_input_nodes, const int32_t** d_num_input_nodes,
+                             const OutputBuffers* out = nullptr) {
     const gs_graph* g = c->graph;
     const int L = c->L;
     int32_t r;
@@ -342,6 +351,18 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
     int32_t* aux = (int32_t*)(ws + w.aux);
     int32_t* tiles_a = (int32_t*)(ws + w.tiles_a);
     int32_t* tiles_e = (int32_t*)(ws + w.tiles_e);
+    if (out) {   // outputs go to the caller's buffers; only the scratch regions of `ws` are used
+        if (!out->input_nodes || out->input_nodes_capacity < b.nb[L])
+            return fail(GS_ERR_WORKSPACE, "input-node buffer holds %lld ids, %lld needed", (long long)out->input_nodes_capacity, (long long)b.nb[L]);
+        for (int k = 0; k < L; ++k) {
+            const int layer = L - 1 - k;
+            if (!out->indptr[layer] || !out->indices[layer]) return fail(GS_ERR_ARG, "block buffers of layer %d are NULL", layer);
+            if (out->indptr_capacity[layer] < b.nb[k] + 1 || out->indices_capacity[layer] < b.mb[k])
+                return fail(GS_ERR_WORKSPACE, "block buffers of layer %d are too small: need %lld offsets and %lld indices",
+                            layer, (long long)b.nb[k] + 1, (long long)b.mb[k]);
+        }
+        frontier = out->input_nodes;
+    }
 
     if (c->serial == 0xFFFFFFFEu) {  // stamp space used up: start over with a clean table
         GS_CUDA(cudaMemsetAsync(c->d_table, 0xFF, (size_t)g->num_nodes * 8, s));
@@ -356,8 +377,8 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         const int layer = L - 1 - k;
         cudaEvent_t* ev = prof ? c->prof_events + ((size_t)c->prof_used * L + k) * PROF_EVENTS_PER_STEP : nullptr;
         if (ev) GS_CUDA(cudaEventRecord(ev[0], s));
-        int32_t* blk_indptr = (int32_t*)(ws + w.blk_indptr[k]);
-        int32_t* blk_indices = (int32_t*)(ws + w.blk_indices[k]);
+        int32_t* blk_indptr = out ? out->indptr[layer] : (int32_t*)(ws + w.blk_indptr[k]);
+        int32_t* blk_indices = out ? out->indices[layer] : (int32_t*)(ws + w.blk_indices[k]);
 
         CountParams C{};
         C.g = GraphView{g->d_indptr, g->d_indices, g->num_nodes};
@@ -466,6 +487,25 @@ static gs_status check_batch_args(gs_cache* c, const int32_t* seeds, int32_t num
     if (!blocks) return fail(GS_ERR_ARG, "blocks is NULL");
     return GS_OK;
 }
+
+}  // extern "C"
+
+namespace gs {
+int32_t cache_num_hops(const gs_cache* c) { return c ? c->L : 0; }
+
+gs_status sample_batch_checked(gs_cache* c, const int32_t* d_seeds, int32_t num_seeds, gs_mode mode, double gamma,
+                               uint32_t step, void* d_workspace, size_t workspace_bytes, cudaStream_t s,
+                               gs_block* blocks, const int32_t** d_input_nodes, const int32_t** d_num_input_nodes,
+                               const OutputBuffers* out) {
+    gs_status st = check_batch_args(c, d_seeds, num_seeds, mode, gamma, step, d_workspace, blocks);
+    if (st != GS_OK) return st;
+    if (!aligned(d_seeds, 4)) return fail(GS_ERR_ALIGN, "d_seeds must be 4-byte aligned");
+    return sample_impl(c, d_seeds, num_seeds, mode, gamma, step, d_workspace, workspace_bytes, s, blocks, d_input_nodes,
+                       d_num_input_nodes, out);
+}
+}  // namespace gs
+
+extern "C" {
 
 gs_status gs_sample_batch(gs_cache* c, const int32_t* d_seeds, int32_t num_seeds, gs_mode mode, double gamma,
                           uint32_t step, void* d_workspace, size_t workspace_bytes, void* stream, gs_block* blocks,

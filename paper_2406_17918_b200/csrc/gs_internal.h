@@ -193,6 +193,25 @@ struct RelabelParams {
 
 void count_launches(int n);
 
+// Caller-owned output buffers that replace the output regions of the workspace (used by the
+// entry point whose scratch is a static device array).  Arrays are indexed by layer.
+struct OutputBuffers {
+    int32_t* input_nodes;
+    int64_t input_nodes_capacity;
+    int32_t* indptr[GS_MAX_HOPS];
+    int64_t indptr_capacity[GS_MAX_HOPS];
+    int32_t* indices[GS_MAX_HOPS];
+    int64_t indices_capacity[GS_MAX_HOPS];
+};
+
+// Argument checks + one batch; `out` may be NULL (outputs then live in the workspace).
+gs_status sample_batch_checked(gs_cache* c, const int32_t* d_seeds, int32_t num_seeds, gs_mode mode, double gamma,
+                               uint32_t step, void* d_workspace, size_t workspace_bytes, cudaStream_t s,
+                               gs_block* blocks, const int32_t** d_input_nodes, const int32_t** d_num_input_nodes,
+                               const OutputBuffers* out);
+gs_status set_error(gs_status code, const char* fmt, ...);
+int32_t cache_num_hops(const gs_cache* c);
+
 cudaError_t launch_row_counts(const CountParams& p, int64_t n_bound, cudaStream_t s);
 cudaError_t launch_refresh_pick(const StepParams& p, int64_t n_bound, cudaStream_t s);
 cudaError_t launch_scan(const StepParams& p, int64_t item_bound, cudaStream_t s);
