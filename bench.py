@@ -128,7 +128,7 @@ def algorithmic_bytes(cfg, n, m_by_step, refreshed_by_step, r):
     return total + feat, feat
 
 
-def cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, budget_s=12.0, reps=1, first_seeds=None):
+def cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, budget_s=32.0, reps=1, first_seeds=None):
     """Times the CPU oracle, as it stands, on the first `s` seeds of batch 0 (s grown until one
     batch takes a few seconds).  Returns (edges/s, feature GB/s, description, seconds per batch)."""
     import numpy as np
@@ -174,7 +174,7 @@ def cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, budget_s=12
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="scale", choices=["tiny", "mid", "large", "shared", "scale"])
