@@ -68,8 +68,11 @@ class Pair:
             assert np.array_equal(blocks[layer].indices(m[layer]).cpu().numpy(), bo.indices)
             d = [int(x) for x in blocks[layer].counts_device()]
             assert d == [n[k], n[k + 1], m[layer]]
-        if rows:
+        if rows is True:
             self.check_rows(C, O, frontier)
+        elif rows:   # an int: that many sampled frontier nodes
+            pickrng = np.random.default_rng(step)
+            self.check_rows(C, O, frontier[pickrng.choice(len(frontier), min(int(rows), len(frontier)), replace=False)])
         if features and self.X is not None:
             out = torch.full((n[self.L] + 3, self.X.shape[1]), 7, dtype=self.X.dtype, device="cuda")
             gs.gs_gather_features(self.G, input_nodes, cnt, out)
