@@ -212,7 +212,7 @@ gs_status gs_cache_init(const gs_graph* g, int32_t num_hops, const int32_t* fano
     c->d_slots = (int32_t*)(c->d_storage + HDR_BYTES + table_bytes(g));
     c->slot_bytes = (size_t)c->num_caches * (size_t)g->num_nodes * (size_t)c->pitch * 4;
     c->serial = 0;
-    c->lambda_otf = 16.0f;
+    c->lambda_otf = 18.0f;
     c->lambda_full = 72.0f;
     c->hub_degree = 8192;
     cudaError_t e = cudaMallocHost((void**)&c->h_pinned, 64 * sizeof(int32_t));
@@ -239,6 +239,9 @@ gs_status gs_cache_init(const gs_graph* g, int32_t num_hops, const int32_t* fano
         if (o_cand + (size_t)cap0 * HUB_CAND_CAP * 8 <= table_room) break;
         cap0 = 0;
     }
+    e = launch_init_low_rows(GraphView{g->d_indptr, g->d_indices, g->num_nodes}, c->d_slots, c->pitch, c->W,
+                             c->num_caches, s);
+    if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "pre-sample launch"); }
     for (int ci = 0; ci < c->num_caches; ++ci) {
         StepParams P = step_params(c, ci, 0u);
         P.r = c->W;

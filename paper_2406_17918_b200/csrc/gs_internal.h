@@ -33,7 +33,7 @@ constexpr int HUB_CHUNK_QUADS = 1024;   // one scan work item = 4096 edge offset
 constexpr int HUB_MIN_DEGREE = 4096;    // lowest degree at which a node may be split over warps
 constexpr int HUB_CAND_CAP = 128;       // candidate entries per hub (same as a warp's buffer)
 
-constexpr int SPLIT_CAND_CAP = 32;      // candidates kept per node by the split OTF path (one per lane)
+constexpr int SPLIT_CAND_CAP = 64;      // candidates kept per node by the split OTF path (two per lane)
 constexpr int SMALL_DEGREE = 128;       // up to here a refresh needs no threshold scan: one Philox per lane covers the row
 
 constexpr int SCAN_A_TILE = 1024;  // frontier nodes per tile of the row-count scan
@@ -214,6 +214,8 @@ int32_t cache_num_hops(const gs_cache* c);
 
 cudaError_t launch_row_counts(const CountParams& p, int64_t n_bound, cudaStream_t s);
 cudaError_t launch_refresh_pick(const StepParams& p, int64_t n_bound, cudaStream_t s);
+cudaError_t launch_init_low_rows(const GraphView& g, int32_t* slots, int32_t pitch, int32_t W, int32_t caches,
+                                 cudaStream_t s);
 cudaError_t launch_scan(const StepParams& p, int64_t item_bound, cudaStream_t s);
 cudaError_t launch_finish(const StepParams& p, int64_t n_bound, cudaStream_t s);
 cudaError_t launch_relabel(const RelabelParams& p, int64_t m_bound, cudaStream_t s);

@@ -355,34 +355,38 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick(const __grid_con
             hi_l = __ldg(P.g.indptr + v_l + 1);
             if (P.do_pick) eb_l = __ldg(P.blk_indptr + base + lane);
         }
-        // first node's row (cache row, or the adjacency of a low-degree node when initialising)
+        // the current cache row of a node (nothing to read when the rows are being initialised)
         auto fetch_row = [&](int i) -> int32_t {
             const int32_t v = __shfl_sync(FULL, v_l, i);
-            const long long lo = __shfl_sync(FULL, lo_l, i);
-            const long long hi = __shfl_sync(FULL, hi_l, i);
-            int32_t x = -1;
-            if (P.init_rows) {
-                if (hi - lo <= W && lane < (int)(hi - lo)) x = __ldg(P.g.indices + lo + lane);
-            } else if (lane < W) {
-                x = P.slots[(int64_t)v * P.pitch + lane];
-            }
-            return x;
+            return (!P.init_rows && lane < W) ? P.slots[(int64_t)v * P.pitch + lane] : -1;
         };
-        int32_t row_next = fetch_row(0);
+        // nodes of the chunk this kernel has work for: all of them when picking; when initialising only
+        // the rows that need a selection (rows that hold their whole adjacency are written by k_init_low_rows)
+        uint32_t todo = __ballot_sync(FULL, lane < cnt && (!P.init_rows || hi_l - lo_l > (long long)W));
+        auto next_node = [&]() -> int {
+            if (!todo) return -1;
+            const int b = __ffs(todo) - 1;
+            todo &= todo - 1;
+            return b;
+        };
+        int i = next_node();
+        int32_t row_next = i >= 0 ? fetch_row(i) : -1;
         NodeState prev;
         prev.skip = true;
         bool have_prev = false;
-        for (int i = 0; i <= cnt; ++i) {
+        while (true) {
             NodeState cur;
             cur.skip = true;
-            if (i < cnt) {
+            const bool ran = i >= 0;
+            if (ran) {
+                const int i_next = next_node();
                 // ---- phase A of node i: decide, scan, issue the neighbour-id loads
                 cur.v = __shfl_sync(FULL, v_l, i);
                 cur.row_start = __shfl_sync(FULL, lo_l, i);
                 cur.deg = (uint32_t)(__shfl_sync(FULL, hi_l, i) - cur.row_start);
                 cur.e_base = __shfl_sync(FULL, eb_l, i);
                 cur.slot = row_next;
-                if (i + 1 < cnt) row_next = fetch_row(i + 1);
+                if (i_next >= 0) row_next = fetch_row(i_next);
                 cur.skip = false;
                 cur.evict = 0;
                 cur.tried_full = false;
@@ -398,6 +402,7 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick(const __grid_con
                     cur.Q.issue(P, cur.row_start, buf, c, __popc(cur.evict), lane);
                     __syncwarp();   // buf may be reused from here on: the first candidates live in registers
                 }
+                i = i_next;
             }
             if (have_prev && !prev.skip) {
                 // ---- phase B of node i-1: its neighbour ids have had a whole scan to arrive
@@ -406,12 +411,12 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick(const __grid_con
                         refill_slow(P, prev.v, prev.row_start, prev.deg, prev.evict, buf, prev.slot, lane);
                     __syncwarp();
                 }
-                if (prev.refresh || (P.init_rows && prev.deg <= (uint32_t)W))
-                    store_row(P, P.slots + (int64_t)prev.v * P.pitch, prev.evict, prev.slot, lane);
+                if (prev.refresh) store_row(P, P.slots + (int64_t)prev.v * P.pitch, prev.evict, prev.slot, lane);
                 if (P.do_pick) warp_pick(P, prev.v, prev.deg, prev.e_base, n_base, prev.slot, lane);
             }
             prev = cur;
             have_prev = true;
+            if (!ran) break;
         }
     }
 }
@@ -502,7 +507,7 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick_hub(const __grid
 // For a partial refresh (0 < r < W) the work is split in two kernels:
 //   k_scan    one warp per work item (a 4096-offset chunk of one refreshed node): nothing but
 //             Philox blocks and a threshold compare, at full occupancy; the few offsets below the
-//             threshold go to the node's candidate list in global memory (at most 32, one per lane).
+//             threshold go to the node's candidate list in global memory (at most 64, two per lane).
 //   k_finish  one warp per frontier node: eviction, refill from the candidate list, row update
 //             and the pick.  Rows of up to SMALL_DEGREE neighbours skip the scan: one Philox block
 //             per lane covers the whole row, and the refill is decided in registers.
@@ -581,8 +586,8 @@ __global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ Ste
                 if (lane == 0) dst = atomicAdd(P.cand_count + p, count);
                 dst = __shfl_sync(FULL, dst, 0);
             }
-            if (lane < count && dst + lane < SPLIT_CAND_CAP)
-                P.cand[(size_t)p * SPLIT_CAND_CAP + dst + lane] = stage[lane];
+            for (int t = lane; t < count && t < SPLIT_CAND_CAP; t += 32)
+                if (dst + t < SPLIT_CAND_CAP) P.cand[(size_t)p * SPLIT_CAND_CAP + dst + t] = stage[t];
             __syncwarp();
         }
     }
@@ -680,12 +685,14 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_finish(const __grid_constant_
         }
         // one node ahead: its cache row and its candidate list are in flight while this one is decided
         int32_t row_next = -1;
-        unsigned long long cand_next = ~0ull;
+        unsigned long long cand_next = ~0ull, cand_next2 = ~0ull;
         auto prefetch = [&](int i) {
             const int32_t v = __shfl_sync(FULL, v_l, i);
             const int cc = __shfl_sync(FULL, cc_l, i);
             row_next = lane < W ? P.slots[(int64_t)v * P.pitch + lane] : -1;
-            cand_next = (lane < cc && lane < SPLIT_CAND_CAP) ? __ldcg(P.cand + (size_t)(base + i) * SPLIT_CAND_CAP + lane) : ~0ull;
+            const unsigned long long* cl = P.cand + (size_t)(base + i) * SPLIT_CAND_CAP;
+            cand_next = (lane < cc) ? __ldcg(cl + lane) : ~0ull;
+            cand_next2 = (lane + 32 < cc && lane + 32 < SPLIT_CAND_CAP) ? __ldcg(cl + lane + 32) : ~0ull;
         };
         prefetch(0);
         for (int i = 0; i < cnt; ++i) {
@@ -696,7 +703,7 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_finish(const __grid_constant_
             const int e_base = __shfl_sync(FULL, eb_l, i);
             const int cc = __shfl_sync(FULL, cc_l, i);
             int32_t slot = row_next;
-            unsigned long long cand = cand_next;
+            unsigned long long cand = cand_next, cand2 = cand_next2;
             if (i + 1 < cnt) prefetch(i + 1);
             const bool refresh = deg > (uint32_t)W && p >= refresh_from;
             const int ncached = deg < (uint32_t)W ? (int)deg : W;
@@ -709,26 +716,39 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_finish(const __grid_constant_
                 } else {
                     bool done = false;
                     if (cc >= P.r && cc <= SPLIT_CAND_CAP) {
-                        // first r (+ spares) candidates in FILL order, one candidate per lane
+                        // Candidates are taken in FILL order, a few at a time, until r of them are not
+                        // retained neighbours; lane t keeps the t-th candidate.  Never more than the
+                        // first W matter (refill rule), so W lanes are enough.
                         const int limit = cc < W ? cc : W;
-                        int g = P.r + (deg < 1024u ? 4 : 1);
-                        g = g < limit ? g : limit;
-                        uint32_t my_off = 0;
-                        for (int t = 0; t < g; ++t) {
-                            const uint32_t hi = (uint32_t)(cand >> 32);
-                            const uint32_t mhi = __reduce_min_sync(FULL, hi);
-                            const uint32_t lo = (hi == mhi) ? (uint32_t)cand : 0xFFFFFFFFu;
-                            const uint32_t mlo = __reduce_min_sync(FULL, lo);
-                            if (cand == (((unsigned long long)mhi << 32) | mlo)) cand = ~0ull;
-                            if (lane == t) my_off = mlo;
-                        }
-                        const int32_t my_nb = lane < g ? __ldg(P.g.indices + rs + my_off) : -1;
                         const bool retained = (lane < W) && !((evict >> lane) & 1u);
-                        uint32_t valid = 0;
-                        for (int t = 0; t < g; ++t) {
-                            const int32_t x = __shfl_sync(FULL, my_nb, t);
-                            if (__ballot_sync(FULL, retained && slot == x) == 0) valid |= 1u << t;
+                        int taken = 0;
+                        int g = P.r + (deg < 1024u ? 4 : 1);
+                        uint32_t my_off = 0, valid = 0;
+                        int32_t my_nb = -1;
+                        while (true) {
+                            g = g < limit - taken ? g : limit - taken;
+                            for (int t = taken; t < taken + g; ++t) {
+                                const unsigned long long loc = cand < cand2 ? cand : cand2;
+                                const uint32_t hi = (uint32_t)(loc >> 32);
+                                const uint32_t mhi = __reduce_min_sync(FULL, hi);
+                                const uint32_t lo = (hi == mhi) ? (uint32_t)loc : 0xFFFFFFFFu;
+                                const uint32_t mlo = __reduce_min_sync(FULL, lo);
+                                const unsigned long long best = ((unsigned long long)mhi << 32) | mlo;
+                                if (cand == best) cand = ~0ull;
+                                if (cand2 == best) cand2 = ~0ull;
+                                if (lane == t) my_off = mlo;
+                            }
+                            if (lane >= taken && lane < taken + g) my_nb = __ldg(P.g.indices + rs + my_off);
+                            for (int t = taken; t < taken + g; ++t) {
+                                const int32_t x = __shfl_sync(FULL, my_nb, t);
+                                if (__ballot_sync(FULL, retained && slot == x) == 0) valid |= 1u << t;
+                            }
+                            taken += g;
+                            if (__popc(valid) >= P.r || taken >= limit) break;
+                            g = P.r - __popc(valid) + 1;
                         }
+                        // enough winners, or the whole top-W was examined (which cannot lack winners);
+                        // a list shorter than W that ran dry decides nothing and the row is rescanned
                         if (__popc(valid) >= P.r) {
                             // t-th valid candidate -> t-th evicted slot, through shared memory
                             const int vr = __popc(valid & lanemask_lt());
@@ -783,6 +803,29 @@ cudaError_t launch_finish(const StepParams& p, int64_t n_bound, cudaStream_t s) 
         launched = 2;
     }
     count_launches(launched);
+    return cudaGetLastError();
+}
+
+// S0 for rows that hold their whole adjacency (deg <= W): slot j = j-th neighbour in CSR order, -1
+// beyond; the same row goes to every cache.  One thread per slot, fully coalesced stores.
+__global__ void __launch_bounds__(256) k_init_low_rows(GraphView g, int32_t* slots, int pitch, int W, int caches) {
+    const int64_t total = g.num_nodes * (int64_t)pitch;
+    const int64_t cache_stride = total;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t v = idx / pitch;
+        const int j = (int)(idx - v * pitch);
+        const long long rs = __ldg(g.indptr + v);
+        const long long deg = __ldg(g.indptr + v + 1) - rs;
+        if (deg > (long long)W) continue;
+        const int32_t val = (j < (int)deg) ? __ldg(g.indices + rs + j) : -1;
+        for (int c = 0; c < caches; ++c) __stcs(slots + c * cache_stride + idx, val);
+    }
+}
+
+cudaError_t launch_init_low_rows(const GraphView& g, int32_t* slots, int32_t pitch, int32_t W, int32_t caches,
+                                 cudaStream_t s) {
+    k_init_low_rows<<<148 * 16, 256, 0, s>>>(g, slots, pitch, W, caches);
+    count_launches(1);
     return cudaGetLastError();
 }
 
