@@ -105,6 +105,10 @@ static StepParams step_params(const gs_cache* c, int32_t layer, uint32_t step) {
     P.step = step;
     P.key0 = (uint32_t)(c->seed & 0xFFFFFFFFu);
     P.key1 = (uint32_t)(c->seed >> 32);
+    for (int i = 0; i < 10; ++i) {
+        P.rk[2 * i] = P.key0 + (uint32_t)i * 0x9E3779B9u;
+        P.rk[2 * i + 1] = P.key1 + (uint32_t)i * 0xBB67AE85u;
+    }
     const uint32_t ctag = c->shared ? 0xFFu : (uint32_t)layer;
     P.word_fill = key_word(1, ctag);
     P.word_evict = key_word(2, ctag);

@@ -26,6 +26,21 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
     return make_uint4(c0, c1, c2, c3);
 }
 
+// Same function with the ten round keys precomputed (k0 + i*0x9E3779B9, k1 + i*0xBB67AE85): when
+// `rk` lives in kernel-parameter space the keys become constant-bank operands of the xors.
+__device__ __forceinline__ uint4 philox4x32_10_rk(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                  const uint32_t (&rk)[20]) {
+#pragma unroll
+    for (int round = 0; round < 10; ++round) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        const uint32_t n0 = hi1 ^ c1 ^ rk[2 * round];
+        const uint32_t n2 = hi0 ^ c3 ^ rk[2 * round + 1];
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
 __device__ __forceinline__ uint32_t word_of(const uint4& o, uint32_t w) {
     return w == 0 ? o.x : (w == 1 ? o.y : (w == 2 ? o.z : o.w));
 }

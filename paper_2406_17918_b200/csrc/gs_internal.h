@@ -29,7 +29,10 @@ constexpr size_t HDR_BYTES = 1024;
 static_assert(HDR_WORDS <= HDR_HUB64, "header words overlap the 64-bit counters");
 static_assert((HDR_HUB64 + 2 * GS_MAX_HOPS) * 4 <= HDR_BYTES, "header too small");
 
-constexpr int HUB_CHUNK_QUADS = 1024;   // one scan work item = 4096 edge offsets
+#ifndef GS_SCAN_CHUNK_QUADS
+#define GS_SCAN_CHUNK_QUADS 1024
+#endif
+constexpr int HUB_CHUNK_QUADS = GS_SCAN_CHUNK_QUADS;   // one scan work item = 4 x this many edge offsets
 constexpr int HUB_MIN_DEGREE = 4096;    // lowest degree at which a node may be split over warps
 constexpr int HUB_CAND_CAP = 128;       // candidate entries per hub (same as a warp's buffer)
 
@@ -123,6 +126,7 @@ struct StepParams {
     int32_t* slots;        // this step's cache: [num_nodes][pitch]
     int32_t pitch, W, f, r;
     uint32_t step, key0, key1;
+    uint32_t rk[20];       // Philox round keys derived from (key0, key1)
     uint32_t word_fill, word_evict, word_pick;  // (purpose << 8) | tag
     const int32_t* frontier;     // NULL: identity (node id = position)
     const int32_t* d_n;          // device count of frontier nodes, or NULL -> n_host

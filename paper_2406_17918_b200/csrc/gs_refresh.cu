@@ -25,6 +25,12 @@
 
 namespace gs {
 
+#ifndef GS_SCAN_BATCH_DIV
+#define GS_SCAN_BATCH_DIV 4
+#endif
+#ifndef GS_SCAN_GRID_PER_SM
+#define GS_SCAN_GRID_PER_SM 8
+#endif
 constexpr int RP_THREADS = 256;
 constexpr int RP_WARPS = RP_THREADS / 32;
 constexpr int RETRY_QUEUE_DEGREE = 2048;  // split path: longer rows that need a rescan go to the hub kernel
@@ -521,7 +527,7 @@ __global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ Ste
     unsigned long long* stage = s_stage[threadIdx.x >> 5];
     const int total = __ldcg(P.d_items_total);
     const int total_warps = gridDim.x * RP_WARPS;
-    int batch = total / (total_warps * 4);
+    int batch = total / (total_warps * GS_SCAN_BATCH_DIV);
     batch = batch < 1 ? 1 : (batch > 32 ? 32 : batch);
     const uint32_t lt = lanemask_lt();
     while (true) {
@@ -551,21 +557,13 @@ __global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ Ste
             const uint32_t qe = qa + HUB_CHUNK_QUADS < nq ? qa + HUB_CHUNK_QUADS : nq;
             const uint32_t tinc = threshold_for(P.lambda_otf, deg);
             int count = 0;   // hits of this item, staged in shared memory (those beyond the cap are only counted)
-            // two independent Philox blocks per lane and iteration (256 offsets per warp iteration):
-            // a lone warp at the tail of the launch is bound by the latency of the dependent rounds
-            for (uint32_t qb = qa; qb < qe; qb += 64) {
-                const uint32_t q0 = qb + lane, q1 = qb + 32 + lane;
-                const uint4 o0 = philox4x32_10(q0, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
-                const uint4 o1 = philox4x32_10(q1, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
-                const uint32_t kk[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
-                const bool in0 = q0 < qe, in1 = q1 < qe;
-                const bool any = (in0 && (min(min(kk[0], kk[1]), min(kk[2], kk[3])) <= tinc)) ||
-                                 (in1 && (min(min(kk[4], kk[5]), min(kk[6], kk[7])) <= tinc));
-                if (__ballot_sync(FULL, any) == 0) continue;
+            // Appends the offsets of one lane-quad whose key is at or below the threshold.
+            auto take_hits = [&](uint32_t q, const uint4& o, bool inq) {
+                const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const uint32_t off = 4u * (j < 4 ? q0 : q1) + (j & 3);
-                    const bool hit = (j < 4 ? in0 : in1) && (off < deg) && (kk[j] <= tinc);
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t off = 4u * q + j;
+                    const bool hit = inq && (off < deg) && (kk[j] <= tinc);
                     const uint32_t b = __ballot_sync(FULL, hit);
                     if (b) {
                         if (hit) {
@@ -575,6 +573,32 @@ __global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ Ste
                         count += __popc(b);
                     }
                 }
+            };
+            // Main loop: four independent Philox blocks per lane and iteration (512 offsets per warp
+            // iteration), all quads in range, one vote per iteration.  The ragged end goes quad by quad.
+            uint32_t qb = qa;
+            for (; qb + 128 <= qe; qb += 128) {
+                const uint32_t q = qb + lane;
+                const uint4 o0 = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
+                const uint4 o1 = philox4x32_10_rk(q + 32, (uint32_t)v, P.step, P.word_fill, P.rk);
+                const uint4 o2 = philox4x32_10_rk(q + 64, (uint32_t)v, P.step, P.word_fill, P.rk);
+                const uint4 o3 = philox4x32_10_rk(q + 96, (uint32_t)v, P.step, P.word_fill, P.rk);
+                const uint32_t m0 = min(min(o0.x, o0.y), min(o0.z, o0.w));
+                const uint32_t m1 = min(min(o1.x, o1.y), min(o1.z, o1.w));
+                const uint32_t m2 = min(min(o2.x, o2.y), min(o2.z, o2.w));
+                const uint32_t m3 = min(min(o3.x, o3.y), min(o3.z, o3.w));
+                if (__ballot_sync(FULL, min(min(m0, m1), min(m2, m3)) <= tinc) == 0) continue;
+                take_hits(q, o0, true);
+                take_hits(q + 32, o1, true);
+                take_hits(q + 64, o2, true);
+                take_hits(q + 96, o3, true);
+            }
+            for (; qb < qe; qb += 32) {
+                const uint32_t q = qb + lane;
+                const uint4 o = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
+                const bool inq = q < qe;
+                if (__ballot_sync(FULL, inq && min(min(o.x, o.y), min(o.z, o.w)) <= tinc) == 0) continue;
+                take_hits(q, o, inq);
             }
             __syncwarp();
             // publish: the only warp of a short row owns the list; the chunks of a long row reserve
@@ -784,7 +808,7 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_finish(const __grid_constant_
 }
 
 cudaError_t launch_scan(const StepParams& p, int64_t item_bound, cudaStream_t s) {
-    const int64_t cap = 148 * 8;
+    const int64_t cap = 148 * GS_SCAN_GRID_PER_SM;
     int64_t sb = (item_bound + RP_WARPS - 1) / RP_WARPS;
     sb = sb > cap ? cap : (sb < 1 ? 1 : sb);
     k_scan<<<(int)sb, RP_THREADS, 0, s>>>(p);
