@@ -527,13 +527,22 @@ __global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ Ste
     unsigned long long* stage = s_stage[threadIdx.x >> 5];
     const int total = __ldcg(P.d_items_total);
     const int total_warps = gridDim.x * RP_WARPS;
+    // Work is handed out in batches of 1..32 items; every warp owns one batch up front, the rest
+    // goes through the shared counter.
     int batch = total / (total_warps * GS_SCAN_BATCH_DIV);
     batch = batch < 1 ? 1 : (batch > 32 ? 32 : batch);
     const uint32_t lt = lanemask_lt();
+    const int warp_gid = blockIdx.x * RP_WARPS + (threadIdx.x >> 5);
+    bool first_grab = true;
     while (true) {
         int base = 0;
-        if (lane == 0) base = atomicAdd(P.work_counter_scan, batch);
-        base = __shfl_sync(FULL, base, 0);
+        if (first_grab) {
+            base = warp_gid * batch;
+            first_grab = false;
+        } else {
+            if (lane == 0) base = atomicAdd(P.work_counter_scan, batch) + total_warps * batch;
+            base = __shfl_sync(FULL, base, 0);
+        }
         if (base >= total) break;
         const int cnt = (base + batch < total ? base + batch : total) - base;
         int p_l = 0, chunk_l = 0;
@@ -687,14 +696,21 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_finish(const __grid_constant_
     const int refresh_from = P.d_refresh_from ? __ldcg(P.d_refresh_from) : 0;
     const int total_warps = gridDim.x * RP_WARPS;
     int chunk = n / (total_warps * 2);
-    chunk = chunk < 1 ? 1 : (chunk > 32 ? 32 : chunk);
+    chunk = chunk < 4 ? 4 : (chunk > 32 ? 32 : chunk);
     const int W = P.W;
     const uint32_t wmask = W >= 32 ? FULL : ((1u << W) - 1u);
+    const int warp_gid = blockIdx.x * RP_WARPS + wid;
+    bool first_grab = true;   // one chunk per warp is assigned statically, the rest through the counter
 
     while (true) {
         int base = 0;
-        if (lane == 0) base = atomicAdd(P.work_counter, chunk);
-        base = __shfl_sync(FULL, base, 0);
+        if (first_grab) {
+            base = warp_gid * chunk;
+            first_grab = false;
+        } else {
+            if (lane == 0) base = atomicAdd(P.work_counter, chunk) + total_warps * chunk;
+            base = __shfl_sync(FULL, base, 0);
+        }
         if (base >= n) break;
         const int cnt = (base + chunk < n ? base + chunk : n) - base;
         int32_t v_l = 0;
