@@ -16,8 +16,8 @@ _SRC = os.path.join(_HERE, "gso.c")
 _HDR = os.path.join(_HERE, "gso.h")
 _LIB = os.path.join(_HERE, "libgso.so")
 
-MODE_FCR, MODE_OTF = 0, 1
-FILL, EVICT, PICK = 1, 2, 3
+MODE_FCR, MODE_OTF, MODE_FBL = 0, 1, 2
+FILL, EVICT, PICK, FETCH = 1, 2, 3, 4
 
 KEY_FN = ctypes.CFUNCTYPE(ctypes.c_uint32, ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32,
                           ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32)
@@ -57,6 +57,7 @@ def lib():
         L.gso_refresh_node.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_uint32, ctypes.c_int32]
         L.gso_pick_node.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_uint32,
                                     ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32)]
+        L.gso_fbl_node.argtypes = L.gso_pick_node.argtypes
         L.gso_sample_batch.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int,
                                        ctypes.c_double, ctypes.c_uint32]
         for name in ("gso_num_nodes", "gso_num_edges"):
@@ -164,6 +165,13 @@ class Sampler:
         out = np.empty(self.W, dtype=np.int32)
         cnt = ctypes.c_int32(0)
         if lib().gso_pick_node(self._h, layer, int(v), step, out.ctypes.data, ctypes.byref(cnt)):
+            raise ValueError("bad arguments")
+        return out[: cnt.value].copy()
+
+    def fbl_node(self, layer, v, step):
+        out = np.empty(max(self.fanouts), dtype=np.int32)
+        cnt = ctypes.c_int32(0)
+        if lib().gso_fbl_node(self._h, layer, int(v), step, out.ctypes.data, ctypes.byref(cnt)):
             raise ValueError("bad arguments")
         return out[: cnt.value].copy()
 

@@ -182,6 +182,27 @@ static int32_t pick_row(gso_sampler* s, int32_t layer, int32_t v, uint32_t step,
     return f;
 }
 
+/* Full Batch Load for one node (paper Section "Full Batch Load (FBL)": the neighbourhood is
+ * re-sampled from the graph for every batch, no cache): all neighbours if there are at most f,
+ * else the f edge offsets first in FETCH order at this step, emitted in ascending offset. */
+static int32_t fbl_row(gso_sampler* s, int32_t layer, int32_t v, uint32_t step, int32_t* out) {
+    int64_t deg = degree(s, v);
+    int32_t f = s->fanouts[layer];
+    if (deg <= f) {
+        for (int64_t j = 0; j < deg; ++j) out[j] = nbr(s, v, (uint32_t)j);
+        return (int32_t)deg;
+    }
+    item_t* it = (item_t*)malloc((size_t)deg * sizeof(item_t));
+    for (int64_t i = 0; i < deg; ++i) it[i].idx = (uint32_t)i;
+    order_items(s, it, deg, GSO_FETCH, (uint32_t)layer, (uint32_t)v, step);
+    int32_t chosen[64];
+    for (int32_t t = 0; t < f; ++t) chosen[t] = (int32_t)it[t].idx;
+    free(it);
+    qsort(chosen, (size_t)f, sizeof(int32_t), i32_cmp);
+    for (int32_t t = 0; t < f; ++t) out[t] = nbr(s, v, (uint32_t)chosen[t]);
+    return f;
+}
+
 /* ------------------------------------------------------------------ lifetime */
 gso_sampler* gso_create(int64_t num_nodes, const int64_t* indptr, const int32_t* indices,
                         int32_t num_hops, const int32_t* fanouts, int32_t cache_width,
@@ -244,6 +265,12 @@ int gso_refresh_node(gso_sampler* s, int32_t layer, int32_t v, uint32_t step, in
     return 0;
 }
 
+int gso_fbl_node(gso_sampler* s, int32_t layer, int32_t v, uint32_t step, int32_t* out, int32_t* count) {
+    if (bad_node(s, layer, v) || !out || !count) return 1;
+    *count = fbl_row(s, layer, v, step, out);
+    return 0;
+}
+
 int gso_pick_node(gso_sampler* s, int32_t layer, int32_t v, uint32_t step, int32_t* out, int32_t* count) {
     if (bad_node(s, layer, v) || !out || !count) return 1;
     *count = pick_row(s, layer, v, step, out);
@@ -256,7 +283,7 @@ int gso_pick_node(gso_sampler* s, int32_t layer, int32_t v, uint32_t step, int32
  * relabel: frontier_{k+1} = frontier_k followed by the unseen picked ids in row-major order. */
 int gso_sample_batch(gso_sampler* s, const int32_t* seeds, int32_t num_seeds, int mode, double gamma, uint32_t step) {
     if (!s || !seeds || num_seeds < 1 || step == 0) return 1;
-    if (mode != GSO_MODE_FCR && mode != GSO_MODE_OTF) return 2;
+    if (mode != GSO_MODE_FCR && mode != GSO_MODE_OTF && mode != GSO_MODE_FBL) return 2;
     if (mode == GSO_MODE_OTF && !(gamma >= 0.0 && gamma <= 1.0)) return 1;
     for (int32_t p = 0; p < num_seeds; ++p)
         if (seeds[p] < 0 || seeds[p] >= s->N) return 3;
@@ -297,8 +324,12 @@ int gso_sample_batch(gso_sampler* s, const int32_t* seeds, int32_t num_seeds, in
         int32_t m = 0;
         for (int32_t p = 0; p < nk; ++p) {
             int32_t v = s->frontier[p];
-            if (p >= refresh_from) refresh_row(s, l, v, step, r);
             indptr[p] = m;
+            if (mode == GSO_MODE_FBL) {
+                m += fbl_row(s, l, v, step, picked + m);
+                continue;
+            }
+            if (p >= refresh_from) refresh_row(s, l, v, step, r);
             m += pick_row(s, l, v, step, picked + m);
         }
         indptr[nk] = m;

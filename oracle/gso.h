@@ -62,9 +62,12 @@ int gso_cache_set_row(gso_sampler*, int32_t layer, int32_t v, const int32_t* row
 /* One node's refresh (r slots) and pick at a given layer/step; exposed for sampled checks. */
 int gso_refresh_node(gso_sampler*, int32_t layer, int32_t v, uint32_t step, int32_t r);
 int gso_pick_node(gso_sampler*, int32_t layer, int32_t v, uint32_t step, int32_t* out, int32_t* count);
+/* Full Batch Load pick of one node (no cache involved); out has room for fanout entries. */
+int gso_fbl_node(gso_sampler*, int32_t layer, int32_t v, uint32_t step, int32_t* out, int32_t* count);
 
-/* One batch.  mode/gamma as in the paper (gamma ignored for FCR and FBL); for
- * GSO_MODE_OTF_FETCH `gamma` carries the fetch rate delta.  step >= 1.  Seeds must be distinct.
+/* One batch.  mode/gamma as in the paper (gamma ignored for FCR and FBL).  GSO_MODE_FBL samples
+ * every hop straight from the graph and leaves the cache untouched; GSO_MODE_OTF_FETCH is
+ * reserved (not implemented).  step >= 1.  Seeds must be distinct.
  * Returns 0, or nonzero on bad arguments. Results stay valid until the next call. */
 int gso_sample_batch(gso_sampler*, const int32_t* seeds, int32_t num_seeds, int mode, double gamma, uint32_t step);
 
