@@ -137,7 +137,7 @@ def cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, budget_s=32
     from workloads import feature_rows
 
     O = oracle.Sampler(indptr_h, indices_h, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED, cfg["shared"])
-    om = oracle.MODE_OTF if mode == "otf" else oracle.MODE_FCR
+    om = {"otf": oracle.MODE_OTF, "fcr": oracle.MODE_FCR, "fbl": oracle.MODE_FBL}[mode]
     B = cfg["batch"]
     s = first_seeds or max(1, min(B, 16))
     step = 1
@@ -178,6 +178,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="scale", choices=["tiny", "mid", "large", "shared", "scale"])
+    ap.add_argument("--mode", default=None, choices=["otf", "fcr", "fbl"],
+                    help="sampling mode (default: the config's OTF run); fbl = no cache, the paper's baseline sampler")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -189,6 +191,8 @@ def main():
     rank, local_rank, world = replicas.env_rank()
     cfg = get_config(args.workload)
     mode, gamma = run_spec(cfg)
+    if args.mode and args.mode != mode:
+        mode, gamma = args.mode, (1.0 if args.mode == "fcr" else 0.0)
     L = len(cfg["fanouts"])
 
     if args.impl == "reference":
@@ -222,7 +226,7 @@ def main():
     presample_ms = ev0.elapsed_time(ev1)
     B = cfg["batch"]
     ws = torch.empty(gs.gs_workspace_bytes(G, cfg["fanouts"], B), dtype=torch.uint8, device=device)
-    gm = gs.GS_MODE_OTF if mode == "otf" else gs.GS_MODE_FCR
+    gm = {"otf": gs.GS_MODE_OTF, "fcr": gs.GS_MODE_FCR, "fbl": gs.GS_MODE_FBL}[mode]
     r = int(gamma * cfg["cache_width"] + 0.5) if mode == "otf" else cfg["cache_width"]
     hdr = C.storage[:512].view(torch.int32)
     stat0 = gs.gs_stats_word_offset()

@@ -49,7 +49,7 @@ typedef enum {
     GS_ERR_CUDA = 6       /* a CUDA runtime call failed; see gs_last_error() */
 } gs_status;
 
-typedef enum { GS_MODE_FCR = 0, GS_MODE_OTF = 1 } gs_mode;
+typedef enum { GS_MODE_FCR = 0, GS_MODE_OTF = 1, GS_MODE_FBL = 2 } gs_mode;
 typedef enum { GS_F32 = 0, GS_BF16 = 1 } gs_dtype;
 
 #define GS_MAX_HOPS 8
@@ -113,6 +113,11 @@ typedef struct {
  *   pick     all cached neighbours if there are at most f_l, else the f_l slots first in PICK
  *            order, emitted in ascending slot index;
  *   relabel  next frontier = frontier followed by unseen picked ids in row-major order.
+ * GS_MODE_FBL (the paper's Full Batch Load, Section "Full Batch Load (FBL)": no cache, every
+ * neighbourhood is re-sampled from the graph) skips refresh and cache altogether: a node with at
+ * most f_l neighbours takes them all, otherwise the f_l edge offsets first in FETCH order
+ * (purpose 4, tag = layer, this step) are taken and emitted in ascending offset.  The cache is
+ * neither read nor written; gamma is ignored.
  * Arguments
  *   d_seeds      int32[num_seeds], distinct ids in [0, num_nodes); 1 <= num_seeds <= the
  *                max_seeds the workspace was sized for

@@ -343,7 +343,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
     const gs_graph* g = c->graph;
     const int L = c->L;
     int32_t r;
-    if (mode == GS_MODE_FCR) {
+    if (mode == GS_MODE_FCR || mode == GS_MODE_FBL) {
         r = c->W;
     } else {
         double rr = std::floor(gamma * (double)c->W + 0.5);
@@ -400,7 +400,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         C.table = c->d_table;
         C.stamp = stamp;
         // a partial refresh runs as scan + finish kernels; FCR (and r = 0) use the fused kernels
-        const bool split = (r > 0 && r < c->W);
+        const bool split = (r > 0 && r < c->W) && mode != GS_MODE_FBL;
         C.split = split ? 1 : 0;
         C.W = c->W;
         C.r = r;
@@ -434,6 +434,12 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         P.work_counter_scan = c->d_hdr + HDR_WORK3 + k;
         P.do_pick = 1;
         P.init_rows = 0;
+        if (mode == GS_MODE_FBL) {   // the fused kernels with W = r = f and FETCH keys; no cache row is touched
+            P.fbl = 1;
+            P.W = P.r = P.f;
+            P.word_fill = key_word(4, (uint32_t)layer);
+            P.d_refresh_from = nullptr;
+        }
         P.item_start = C.item_start;
         P.items = C.items;
         P.d_items_total = c->d_hdr + HDR_ITEMS + k;
@@ -486,7 +492,7 @@ static gs_status check_batch_args(gs_cache* c, const int32_t* seeds, int32_t num
     if (!seeds) return fail(GS_ERR_ARG, "seeds is NULL");
     if (num_seeds < 1) return fail(GS_ERR_ARG, "num_seeds must be >= 1");
     if ((int64_t)num_seeds > c->graph->num_nodes) return fail(GS_ERR_ARG, "more seeds than nodes");
-    if (mode != GS_MODE_FCR && mode != GS_MODE_OTF) return fail(GS_ERR_ARG, "unknown mode %d", (int)mode);
+    if (mode != GS_MODE_FCR && mode != GS_MODE_OTF && mode != GS_MODE_FBL) return fail(GS_ERR_ARG, "unknown mode %d", (int)mode);
     if (mode == GS_MODE_OTF && !(gamma >= 0.0 && gamma <= 1.0)) return fail(GS_ERR_ARG, "gamma outside [0, 1]");
     if (step == 0) return fail(GS_ERR_ARG, "step 0 is reserved for the pre-sample");
     if (!d_workspace) return fail(GS_ERR_ARG, "d_workspace is NULL");

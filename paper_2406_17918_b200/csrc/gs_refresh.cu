@@ -269,6 +269,22 @@ __device__ __forceinline__ void warp_pick(const StepParams& P, int32_t v, uint32
     }
 }
 
+// Full Batch Load emission: lanes < cnt hold the chosen neighbour ids; they go out in ascending
+// edge offset, which for a sorted CSR row is ascending id.
+__device__ __forceinline__ void warp_emit_sorted(const StepParams& P, int cnt, int e_base, uint32_t n_base,
+                                                 int32_t id, int lane) {
+    int rank = 0;
+    for (int t = 0; t < cnt; ++t) {
+        const int32_t x = __shfl_sync(FULL, id, t);
+        rank += (x < id) ? 1 : 0;
+    }
+    if (lane < cnt) {
+        const int e = e_base + rank;
+        P.picked[e] = id;
+        atomicMin(P.table + id, ((unsigned long long)P.stamp << 32) | (n_base + (uint32_t)e));
+    }
+}
+
 // Retry ladder after a failed first attempt: a looser threshold, then the exact scan.
 __device__ __noinline__ void refill_slow(const StepParams& P, int32_t v, int64_t row_start, uint32_t deg,
                                          uint32_t evict, unsigned long long* buf, int32_t& slot, int lane) {
@@ -364,7 +380,7 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick(const __grid_con
         // the current cache row of a node (nothing to read when the rows are being initialised)
         auto fetch_row = [&](int i) -> int32_t {
             const int32_t v = __shfl_sync(FULL, v_l, i);
-            return (!P.init_rows && lane < W) ? P.slots[(int64_t)v * P.pitch + lane] : -1;
+            return (!P.init_rows && !P.fbl && lane < W) ? P.slots[(int64_t)v * P.pitch + lane] : -1;
         };
         // nodes of the chunk this kernel has work for: all of them when picking; when initialising only
         // the rows that need a selection (rows that hold their whole adjacency are written by k_init_low_rows)
@@ -398,6 +414,8 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick(const __grid_con
                 cur.tried_full = false;
                 cur.Q.g = 0;
                 cur.refresh = cur.deg > (uint32_t)W && P.r > 0 && base + i >= refresh_from;
+                if (P.fbl && !cur.refresh && lane < (int)cur.deg)   // few neighbours: take them all
+                    cur.slot = __ldg(P.g.indices + cur.row_start + lane);
                 if (cur.refresh && cur.deg > (uint32_t)P.hub_degree && hub_register(P, base + i, cur.deg, lane)) {
                     cur.skip = true;   // the hub kernel does everything for this node, pick included
                 } else if (cur.refresh) {
@@ -417,8 +435,12 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick(const __grid_con
                         refill_slow(P, prev.v, prev.row_start, prev.deg, prev.evict, buf, prev.slot, lane);
                     __syncwarp();
                 }
-                if (prev.refresh) store_row(P, P.slots + (int64_t)prev.v * P.pitch, prev.evict, prev.slot, lane);
-                if (P.do_pick) warp_pick(P, prev.v, prev.deg, prev.e_base, n_base, prev.slot, lane);
+                if (P.fbl) {
+                    warp_emit_sorted(P, prev.deg < (uint32_t)W ? (int)prev.deg : W, prev.e_base, n_base, prev.slot, lane);
+                } else {
+                    if (prev.refresh) store_row(P, P.slots + (int64_t)prev.v * P.pitch, prev.evict, prev.slot, lane);
+                    if (P.do_pick) warp_pick(P, prev.v, prev.deg, prev.e_base, n_base, prev.slot, lane);
+                }
             }
             prev = cur;
             have_prev = true;
@@ -497,15 +519,19 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick_hub(const __grid
             if (j < c) buf[j] = __ldcg(cand + j);
         __syncwarp();
         int32_t* row = P.slots + (int64_t)v * P.pitch;
-        int32_t slot = (!P.init_rows && lane < W) ? row[lane] : -1;
+        int32_t slot = (!P.init_rows && !P.fbl && lane < W) ? row[lane] : -1;
         const uint32_t evict = evict_mask_for(P, v, lane);
         Quick Q;
         Q.issue(P, rs, buf, c, __popc(evict), lane);
         __syncwarp();
         if (!Q.settle(P, evict, slot, lane)) refill_slow(P, v, rs, deg, evict, buf, slot, lane);
         __syncwarp();
-        store_row(P, row, evict, slot, lane);
-        if (P.do_pick) warp_pick(P, v, deg, __ldg(P.blk_indptr + p), n_base, slot, lane);
+        if (P.fbl) {
+            warp_emit_sorted(P, W, __ldg(P.blk_indptr + p), n_base, slot, lane);
+        } else {
+            store_row(P, row, evict, slot, lane);
+            if (P.do_pick) warp_pick(P, v, deg, __ldg(P.blk_indptr + p), n_base, slot, lane);
+        }
     }
 }
 

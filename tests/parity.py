@@ -7,7 +7,8 @@ import oracle
 import paper_2406_17918_b200 as gs
 from workloads import batch_seeds, build_features, build_graph, seed_permutation
 
-MODES = {"fcr": (gs.GS_MODE_FCR, oracle.MODE_FCR), "otf": (gs.GS_MODE_OTF, oracle.MODE_OTF)}
+MODES = {"fcr": (gs.GS_MODE_FCR, oracle.MODE_FCR), "otf": (gs.GS_MODE_OTF, oracle.MODE_OTF),
+         "fbl": (gs.GS_MODE_FBL, oracle.MODE_FBL)}
 
 
 def bits(t: torch.Tensor) -> np.ndarray:

@@ -64,6 +64,15 @@ def test_mid_internal_paths_agree(mid, tuning):
     mid.run("fcr", 1.0, 1, tuning=tuning)
 
 
+def test_full_batch_load_mode(tiny, mid, shared_cfg):
+    # no cache: every hop samples the CSR rows directly; cache rows must stay as pre-sampled
+    tiny.run("fbl", 0.0, 5)
+    mid.run("fbl", 0.0, 2)
+    mid.run("fbl", 0.0, 1, tuning=dict(hub_degree=40))
+    mid.run("fbl", 0.0, 1, tuning=dict(lambda_full=1.0))
+    shared_cfg.run("fbl", 0.0, 1)
+
+
 def test_shared_cache_mode(shared_cfg):
     shared_cfg.run("otf", 0.3, 3)
     shared_cfg.run("fcr", 0.0, 1)
