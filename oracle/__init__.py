@@ -16,7 +16,7 @@ _SRC = os.path.join(_HERE, "gso.c")
 _HDR = os.path.join(_HERE, "gso.h")
 _LIB = os.path.join(_HERE, "libgso.so")
 
-MODE_FCR, MODE_OTF, MODE_FBL = 0, 1, 2
+MODE_FCR, MODE_OTF, MODE_FBL, MODE_OTF_FETCH = 0, 1, 2, 3
 FILL, EVICT, PICK, FETCH = 1, 2, 3, 4
 
 KEY_FN = ctypes.CFUNCTYPE(ctypes.c_uint32, ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32,
@@ -58,6 +58,10 @@ def lib():
         L.gso_pick_node.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_uint32,
                                     ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32)]
         L.gso_fbl_node.argtypes = L.gso_pick_node.argtypes
+        L.gso_fetch_node.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_uint32, ctypes.c_int32,
+                                     ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32)]
+        L.gso_fetch_count.argtypes = [ctypes.c_double, ctypes.c_int32]
+        L.gso_fetch_count.restype = ctypes.c_int32
         L.gso_sample_batch.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int,
                                        ctypes.c_double, ctypes.c_uint32]
         for name in ("gso_num_nodes", "gso_num_edges"):
@@ -84,6 +88,10 @@ def philox4x32_10(ctr, key):
     o = (ctypes.c_uint32 * 4)()
     lib().gso_philox4x32_10(c, k, o)
     return [int(x) for x in o]
+
+
+def fetch_count(delta: float, f: int) -> int:
+    return int(lib().gso_fetch_count(delta, f))
 
 
 def refresh_count(mode: int, gamma: float, W: int) -> int:
@@ -165,6 +173,13 @@ class Sampler:
         out = np.empty(self.W, dtype=np.int32)
         cnt = ctypes.c_int32(0)
         if lib().gso_pick_node(self._h, layer, int(v), step, out.ctypes.data, ctypes.byref(cnt)):
+            raise ValueError("bad arguments")
+        return out[: cnt.value].copy()
+
+    def fetch_node(self, layer, v, step, n_fetch):
+        out = np.empty(max(self.fanouts), dtype=np.int32)
+        cnt = ctypes.c_int32(0)
+        if lib().gso_fetch_node(self._h, layer, int(v), step, int(n_fetch), out.ctypes.data, ctypes.byref(cnt)):
             raise ValueError("bad arguments")
         return out[: cnt.value].copy()
 

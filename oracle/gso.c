@@ -91,6 +91,13 @@ int32_t gso_refresh_count(int mode, double gamma, int32_t W) {
     return (int32_t)r;
 }
 
+int32_t gso_fetch_count(double delta, int32_t f) {
+    double n = floor(delta * (double)f + 0.5);
+    if (n < 0) n = 0;
+    if (n > f) n = f;
+    return (int32_t)n;
+}
+
 static int64_t degree(const gso_sampler* s, int32_t v) { return s->indptr[v + 1] - s->indptr[v]; }
 static int32_t nbr(const gso_sampler* s, int32_t v, uint32_t i) { return s->indices[s->indptr[v] + (int64_t)i]; }
 static int32_t cache_of(const gso_sampler* s, int32_t layer) { return s->shared ? 0 : layer; }
@@ -203,6 +210,41 @@ static int32_t fbl_row(gso_sampler* s, int32_t layer, int32_t v, uint32_t step, 
     return f;
 }
 
+/* OTF Fetch for one node (paper Section "OTF Fetch": the sample is part cache, part graph, with
+ * fetch rate delta; the cache is not modified).  A row that holds its whole adjacency is sampled
+ * like any cached row.  Otherwise n_fetch = floor(delta*f + 0.5) neighbours come from the graph and
+ * f - n_fetch from the cache: the cache part is the f - n_fetch slots first in PICK order, emitted
+ * in ascending slot index; the fetched part is the n_fetch edge offsets first in FETCH order among
+ * those whose neighbour is not one of the cache picks, emitted in that order after the cache part. */
+static int32_t fetch_row(gso_sampler* s, int32_t layer, int32_t v, uint32_t step, int32_t n_fetch, int32_t* out) {
+    int64_t deg = degree(s, v);
+    int32_t W = s->W, f = s->fanouts[layer];
+    if (deg <= W || n_fetch <= 0) return pick_row(s, layer, v, step, out);
+    if (n_fetch > f) n_fetch = f;
+    int32_t n_cache = f - n_fetch;
+    const int32_t* row = row_of(s, layer, v);
+    item_t slots[64];
+    for (int32_t j = 0; j < W; ++j) slots[j].idx = (uint32_t)j;
+    order_items(s, slots, W, GSO_PICK, (uint32_t)layer, (uint32_t)v, step);
+    int32_t chosen[64];
+    for (int32_t t = 0; t < n_cache; ++t) chosen[t] = (int32_t)slots[t].idx;
+    qsort(chosen, (size_t)n_cache, sizeof(int32_t), i32_cmp);
+    for (int32_t t = 0; t < n_cache; ++t) out[t] = row[chosen[t]];
+    item_t* cand = (item_t*)malloc((size_t)deg * sizeof(item_t));
+    int64_t nc = 0;
+    for (int64_t i = 0; i < deg; ++i) {
+        int32_t u = nbr(s, v, (uint32_t)i);
+        int taken = 0;
+        for (int32_t t = 0; t < n_cache; ++t)
+            if (out[t] == u) taken = 1;
+        if (!taken) cand[nc++].idx = (uint32_t)i;
+    }
+    order_items(s, cand, nc, GSO_FETCH, (uint32_t)layer, (uint32_t)v, step);
+    for (int32_t t = 0; t < n_fetch; ++t) out[n_cache + t] = nbr(s, v, cand[t].idx);
+    free(cand);
+    return f;
+}
+
 /* ------------------------------------------------------------------ lifetime */
 gso_sampler* gso_create(int64_t num_nodes, const int64_t* indptr, const int32_t* indices,
                         int32_t num_hops, const int32_t* fanouts, int32_t cache_width,
@@ -271,6 +313,13 @@ int gso_fbl_node(gso_sampler* s, int32_t layer, int32_t v, uint32_t step, int32_
     return 0;
 }
 
+int gso_fetch_node(gso_sampler* s, int32_t layer, int32_t v, uint32_t step, int32_t n_fetch, int32_t* out,
+                   int32_t* count) {
+    if (bad_node(s, layer, v) || !out || !count || n_fetch < 0) return 1;
+    *count = fetch_row(s, layer, v, step, n_fetch, out);
+    return 0;
+}
+
 int gso_pick_node(gso_sampler* s, int32_t layer, int32_t v, uint32_t step, int32_t* out, int32_t* count) {
     if (bad_node(s, layer, v) || !out || !count) return 1;
     *count = pick_row(s, layer, v, step, out);
@@ -283,8 +332,8 @@ int gso_pick_node(gso_sampler* s, int32_t layer, int32_t v, uint32_t step, int32
  * relabel: frontier_{k+1} = frontier_k followed by the unseen picked ids in row-major order. */
 int gso_sample_batch(gso_sampler* s, const int32_t* seeds, int32_t num_seeds, int mode, double gamma, uint32_t step) {
     if (!s || !seeds || num_seeds < 1 || step == 0) return 1;
-    if (mode != GSO_MODE_FCR && mode != GSO_MODE_OTF && mode != GSO_MODE_FBL) return 2;
-    if (mode == GSO_MODE_OTF && !(gamma >= 0.0 && gamma <= 1.0)) return 1;
+    if (mode != GSO_MODE_FCR && mode != GSO_MODE_OTF && mode != GSO_MODE_FBL && mode != GSO_MODE_OTF_FETCH) return 2;
+    if ((mode == GSO_MODE_OTF || mode == GSO_MODE_OTF_FETCH) && !(gamma >= 0.0 && gamma <= 1.0)) return 1;
     for (int32_t p = 0; p < num_seeds; ++p)
         if (seeds[p] < 0 || seeds[p] >= s->N) return 3;
     int32_t r = gso_refresh_count(mode, gamma, s->W);
@@ -327,6 +376,10 @@ int gso_sample_batch(gso_sampler* s, const int32_t* seeds, int32_t num_seeds, in
             indptr[p] = m;
             if (mode == GSO_MODE_FBL) {
                 m += fbl_row(s, l, v, step, picked + m);
+                continue;
+            }
+            if (mode == GSO_MODE_OTF_FETCH) {
+                m += fetch_row(s, l, v, step, gso_fetch_count(gamma, f), picked + m);
                 continue;
             }
             if (p >= refresh_from) refresh_row(s, l, v, step, r);

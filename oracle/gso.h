@@ -62,12 +62,17 @@ int gso_cache_set_row(gso_sampler*, int32_t layer, int32_t v, const int32_t* row
 /* One node's refresh (r slots) and pick at a given layer/step; exposed for sampled checks. */
 int gso_refresh_node(gso_sampler*, int32_t layer, int32_t v, uint32_t step, int32_t r);
 int gso_pick_node(gso_sampler*, int32_t layer, int32_t v, uint32_t step, int32_t* out, int32_t* count);
+/* OTF Fetch pick of one node with n_fetch neighbours taken from the graph; cache not modified. */
+int gso_fetch_node(gso_sampler*, int32_t layer, int32_t v, uint32_t step, int32_t n_fetch, int32_t* out,
+                   int32_t* count);
+/* Neighbours fetched from the graph per node in OTF Fetch: floor(delta*f + 0.5). */
+int32_t gso_fetch_count(double delta, int32_t f);
 /* Full Batch Load pick of one node (no cache involved); out has room for fanout entries. */
 int gso_fbl_node(gso_sampler*, int32_t layer, int32_t v, uint32_t step, int32_t* out, int32_t* count);
 
 /* One batch.  mode/gamma as in the paper (gamma ignored for FCR and FBL).  GSO_MODE_FBL samples
- * every hop straight from the graph and leaves the cache untouched; GSO_MODE_OTF_FETCH is
- * reserved (not implemented).  step >= 1.  Seeds must be distinct.
+ * every hop straight from the graph and leaves the cache untouched; for GSO_MODE_OTF_FETCH
+ * `gamma` carries the fetch rate delta, and the cache is not modified either.  step >= 1.  Seeds must be distinct.
  * Returns 0, or nonzero on bad arguments. Results stay valid until the next call. */
 int gso_sample_batch(gso_sampler*, const int32_t* seeds, int32_t num_seeds, int mode, double gamma, uint32_t step);
 
