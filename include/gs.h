@@ -49,7 +49,7 @@ typedef enum {
     GS_ERR_CUDA = 6       /* a CUDA runtime call failed; see gs_last_error() */
 } gs_status;
 
-typedef enum { GS_MODE_FCR = 0, GS_MODE_OTF = 1, GS_MODE_FBL = 2 } gs_mode;
+typedef enum { GS_MODE_FCR = 0, GS_MODE_OTF = 1, GS_MODE_FBL = 2, GS_MODE_OTF_FETCH = 3 } gs_mode;
 typedef enum { GS_F32 = 0, GS_BF16 = 1 } gs_dtype;
 
 #define GS_MAX_HOPS 8
@@ -118,6 +118,12 @@ typedef struct {
  * most f_l neighbours takes them all, otherwise the f_l edge offsets first in FETCH order
  * (purpose 4, tag = layer, this step) are taken and emitted in ascending offset.  The cache is
  * neither read nor written; gamma is ignored.
+ * GS_MODE_OTF_FETCH (the paper's second OTF mode, Section "OTF Fetch": the sample is
+ * delta * FetchFromDisk + (1 - delta) * SampleFromCache) takes `gamma` as the fetch rate delta and
+ * never modifies the cache.  A row that holds its whole adjacency is sampled as in `pick`.
+ * Otherwise n = floor(delta*f_l + 0.5) neighbours are fetched from the graph and f_l - n come from
+ * the cache: first the f_l - n slots first in PICK order (ascending slot index), then the n edge
+ * offsets first in FETCH order among those whose neighbour is not one of these cache picks.
  * Arguments
  *   d_seeds      int32[num_seeds], distinct ids in [0, num_nodes); 1 <= num_seeds <= the
  *                max_seeds the workspace was sized for

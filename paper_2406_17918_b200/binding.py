@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libgs.so")
 _HEADER = os.path.join(os.path.dirname(_HERE), "include", "gs.h")
 
-GS_MODE_FCR, GS_MODE_OTF, GS_MODE_FBL = 0, 1, 2
+GS_MODE_FCR, GS_MODE_OTF, GS_MODE_FBL, GS_MODE_OTF_FETCH = 0, 1, 2, 3
 GS_F32, GS_BF16 = 0, 1
 GS_MAX_HOPS = 8
 COUNTS_READBACK_BYTES = 4 * (1 + (GS_MAX_HOPS + 1) + GS_MAX_HOPS)  # status + n_k + m_k, what gs_batch_counts copies

@@ -345,6 +345,8 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
     int32_t r;
     if (mode == GS_MODE_FCR || mode == GS_MODE_FBL) {
         r = c->W;
+    } else if (mode == GS_MODE_OTF_FETCH) {
+        r = 0;   // nothing is ever evicted; the per-layer fetch count is derived below
     } else {
         double rr = std::floor(gamma * (double)c->W + 0.5);
         r = rr < 0 ? 0 : (rr > c->W ? c->W : (int32_t)rr);
@@ -400,11 +402,16 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         C.table = c->d_table;
         C.stamp = stamp;
         // a partial refresh runs as scan + finish kernels; FCR (and r = 0) use the fused kernels
-        const bool split = (r > 0 && r < c->W) && mode != GS_MODE_FBL;
+        int32_t n_fetch = 0;
+        if (mode == GS_MODE_OTF_FETCH) {
+            double nf = std::floor(gamma * (double)c->fanouts[layer] + 0.5);
+            n_fetch = nf < 0 ? 0 : (nf > c->fanouts[layer] ? c->fanouts[layer] : (int32_t)nf);
+        }
+        const bool split = ((r > 0 && r < c->W) && mode != GS_MODE_FBL) || n_fetch > 0;
         C.split = split ? 1 : 0;
         C.W = c->W;
-        C.r = r;
-        C.d_refresh_from = (c->shared && k > 0) ? c->d_hdr + HDR_N + (k - 1) : nullptr;
+        C.r = n_fetch > 0 ? n_fetch : r;
+        C.d_refresh_from = (c->shared && k > 0 && mode != GS_MODE_OTF_FETCH) ? c->d_hdr + HDR_N + (k - 1) : nullptr;
         C.tile_sums2 = (int32_t*)(ws + w.tiles_a2);
         C.item_start = (int32_t*)(ws + w.item_start);
         C.items = (int32_t*)(ws + w.items);
@@ -434,6 +441,12 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         P.work_counter_scan = c->d_hdr + HDR_WORK3 + k;
         P.do_pick = 1;
         P.init_rows = 0;
+        if (n_fetch > 0) {           // scan + finish with FETCH keys; the finish kernel emits cache part + fetched part
+            P.fetch = 1;
+            P.r = n_fetch;
+            P.word_fill = key_word(4, (uint32_t)layer);
+            P.d_refresh_from = nullptr;
+        }
         if (mode == GS_MODE_FBL) {   // the fused kernels with W = r = f and FETCH keys; no cache row is touched
             P.fbl = 1;
             P.W = P.r = P.f;
@@ -492,8 +505,10 @@ static gs_status check_batch_args(gs_cache* c, const int32_t* seeds, int32_t num
     if (!seeds) return fail(GS_ERR_ARG, "seeds is NULL");
     if (num_seeds < 1) return fail(GS_ERR_ARG, "num_seeds must be >= 1");
     if ((int64_t)num_seeds > c->graph->num_nodes) return fail(GS_ERR_ARG, "more seeds than nodes");
-    if (mode != GS_MODE_FCR && mode != GS_MODE_OTF && mode != GS_MODE_FBL) return fail(GS_ERR_ARG, "unknown mode %d", (int)mode);
-    if (mode == GS_MODE_OTF && !(gamma >= 0.0 && gamma <= 1.0)) return fail(GS_ERR_ARG, "gamma outside [0, 1]");
+    if (mode != GS_MODE_FCR && mode != GS_MODE_OTF && mode != GS_MODE_FBL && mode != GS_MODE_OTF_FETCH)
+        return fail(GS_ERR_ARG, "unknown mode %d", (int)mode);
+    if ((mode == GS_MODE_OTF || mode == GS_MODE_OTF_FETCH) && !(gamma >= 0.0 && gamma <= 1.0))
+        return fail(GS_ERR_ARG, "gamma outside [0, 1]");
     if (step == 0) return fail(GS_ERR_ARG, "step 0 is reserved for the pre-sample");
     if (!d_workspace) return fail(GS_ERR_ARG, "d_workspace is NULL");
     if (!aligned(d_workspace, 256)) return fail(GS_ERR_ALIGN, "d_workspace must be 256-byte aligned");

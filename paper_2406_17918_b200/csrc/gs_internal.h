@@ -156,6 +156,7 @@ struct StepParams {
     int32_t* status;
     int32_t* stats;                  // header words HDR_STAT_*: rare-event counters
     int32_t do_pick, init_rows;
+    int32_t fetch;                   // OTF Fetch: r neighbours come from the graph, f - r from the cache; no row is written
     int32_t fbl;                     // Full Batch Load: W = r = f, no cache row is read or written
     float lambda_otf, lambda_full;
     int32_t hub_degree;

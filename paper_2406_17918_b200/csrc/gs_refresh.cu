@@ -775,8 +775,21 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_finish(const __grid_constant_
             const int ncached = deg < (uint32_t)W ? (int)deg : W;
             uint32_t ekey = 0, pkey = 0;
             if (refresh || ncached > P.f) evict_pick_keys(P, v, lane, ekey, pkey);
+            uint32_t cache_part = 0;   // OTF Fetch: lanes of the cache slots that are part of the sample
             if (refresh) {
-                const uint32_t evict = warp_smallest_k(ekey, wmask, P.r, lane);
+                uint32_t evict;
+                if (P.fetch) {
+                    // The f - r cache picks play the part of the retained slots, the r fetched
+                    // neighbours land in the r lowest other lanes; the other slots are blanked so that
+                    // only the cache picks exclude candidates.  The row itself is not modified.
+                    cache_part = warp_smallest_k(pkey, wmask, P.f - P.r, lane);
+                    const uint32_t rest = wmask & ~cache_part;
+                    const bool mine = ((rest >> lane) & 1u) && __popc(rest & lanemask_lt()) < P.r;
+                    evict = __ballot_sync(FULL, mine);
+                    if (!((cache_part >> lane) & 1u)) slot = -1;
+                } else {
+                    evict = warp_smallest_k(ekey, wmask, P.r, lane);
+                }
                 if (deg <= (uint32_t)SMALL_DEGREE) {
                     small_refill(P, v, rs, deg, evict, slot, lane);
                 } else {
@@ -829,10 +842,22 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_finish(const __grid_constant_
                     if (!done) {
                         // A long row is not rescanned by this one warp: it is queued for the chunked
                         // hub kernel, which redoes the node (pick included) with all warps.
-                        if (deg > (uint32_t)RETRY_QUEUE_DEGREE && hub_register(P, p, deg, lane)) continue;
+                        if (!P.fetch && deg > (uint32_t)RETRY_QUEUE_DEGREE && hub_register(P, p, deg, lane)) continue;
                         refill_slow(P, v, rs, deg, evict, buf, slot, lane);
                         __syncwarp();
                     }
+                }
+                if (P.fetch) {
+                    // emit the cache part in ascending slot index, then the fetched part in FETCH order
+                    const uint32_t lt = lanemask_lt();
+                    int e = -1;
+                    if ((cache_part >> lane) & 1u) e = e_base + __popc(cache_part & lt);
+                    else if ((evict >> lane) & 1u) e = e_base + (P.f - P.r) + __popc(evict & lt);
+                    if (e >= 0) {
+                        P.picked[e] = slot;
+                        atomicMin(P.table + slot, ((unsigned long long)P.stamp << 32) | (n_base + (uint32_t)e));
+                    }
+                    continue;
                 }
                 if ((evict >> lane) & 1u) P.slots[(int64_t)v * P.pitch + lane] = slot;
             }

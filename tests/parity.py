@@ -8,7 +8,7 @@ import paper_2406_17918_b200 as gs
 from workloads import batch_seeds, build_features, build_graph, seed_permutation
 
 MODES = {"fcr": (gs.GS_MODE_FCR, oracle.MODE_FCR), "otf": (gs.GS_MODE_OTF, oracle.MODE_OTF),
-         "fbl": (gs.GS_MODE_FBL, oracle.MODE_FBL)}
+         "fbl": (gs.GS_MODE_FBL, oracle.MODE_FBL), "fetch": (gs.GS_MODE_OTF_FETCH, oracle.MODE_OTF_FETCH)}
 
 
 def bits(t: torch.Tensor) -> np.ndarray:

@@ -73,6 +73,23 @@ def test_full_batch_load_mode(tiny, mid, shared_cfg):
     shared_cfg.run("fbl", 0.0, 1)
 
 
+@pytest.mark.parametrize("delta", [0.0, 0.04, 0.3, 0.5, 1.0])
+def test_otf_fetch_mode(tiny, mid, delta):
+    # part of every sample comes straight from the graph; the cache rows must stay as pre-sampled
+    tiny.run("fetch", delta, 3)
+    mid.run("fetch", delta, 2)
+
+
+def test_otf_fetch_mode_internal_paths_and_shared(mid, shared_cfg):
+    mid.run("fetch", 0.4, 1, tuning=dict(lambda_otf=0.5, lambda_full=1.0))
+    mid.run("fetch", 0.4, 1, tuning=dict(lambda_otf=1e6, lambda_full=1e6))
+    shared_cfg.run("fetch", 0.3, 2)
+    # modes can be mixed on one cache from batch to batch
+    C, ws, O = mid.samplers(mid.cfg["batch"])
+    for b, (mode, rate) in enumerate([("otf", 0.3), ("fetch", 0.5), ("fbl", 0.0), ("fcr", 0.0), ("fetch", 0.2), ("otf", 0.1)]):
+        mid.check_batch(C, ws, O, batch_seeds(mid.perm, b, mid.cfg["batch"]), mode, rate, b + 1)
+
+
 def test_shared_cache_mode(shared_cfg):
     shared_cfg.run("otf", 0.3, 3)
     shared_cfg.run("fcr", 0.0, 1)
