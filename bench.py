@@ -137,7 +137,7 @@ def cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, budget_s=32
     from workloads import feature_rows
 
     O = oracle.Sampler(indptr_h, indices_h, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED, cfg["shared"])
-    om = {"otf": oracle.MODE_OTF, "fcr": oracle.MODE_FCR, "fbl": oracle.MODE_FBL}[mode]
+    om = {"otf": oracle.MODE_OTF, "fcr": oracle.MODE_FCR, "fbl": oracle.MODE_FBL, "fetch": oracle.MODE_OTF_FETCH}[mode]
     B = cfg["batch"]
     s = first_seeds or max(1, min(B, 16))
     step = 1
@@ -178,8 +178,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="scale", choices=["tiny", "mid", "large", "shared", "scale"])
-    ap.add_argument("--mode", default=None, choices=["otf", "fcr", "fbl"],
-                    help="sampling mode (default: the config's OTF run); fbl = no cache, the paper's baseline sampler")
+    ap.add_argument("--mode", default=None, choices=["otf", "fcr", "fbl", "fetch"],
+                    help="sampling mode (default: the config's OTF run); fbl = no cache, the paper's baseline "
+                         "sampler; fetch = OTF Fetch")
+    ap.add_argument("--rate", type=float, default=None, help="gamma (otf) or delta (fetch); default: the config's")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -192,7 +194,9 @@ def main():
     cfg = get_config(args.workload)
     mode, gamma = run_spec(cfg)
     if args.mode and args.mode != mode:
-        mode, gamma = args.mode, (1.0 if args.mode == "fcr" else 0.0)
+        mode, gamma = args.mode, {"fcr": 1.0, "fbl": 0.0, "fetch": 0.5, "otf": gamma}[args.mode]
+    if args.rate is not None:
+        gamma = args.rate
     L = len(cfg["fanouts"])
 
     if args.impl == "reference":
@@ -226,8 +230,8 @@ def main():
     presample_ms = ev0.elapsed_time(ev1)
     B = cfg["batch"]
     ws = torch.empty(gs.gs_workspace_bytes(G, cfg["fanouts"], B), dtype=torch.uint8, device=device)
-    gm = {"otf": gs.GS_MODE_OTF, "fcr": gs.GS_MODE_FCR, "fbl": gs.GS_MODE_FBL}[mode]
-    r = int(gamma * cfg["cache_width"] + 0.5) if mode == "otf" else cfg["cache_width"]
+    gm = {"otf": gs.GS_MODE_OTF, "fcr": gs.GS_MODE_FCR, "fbl": gs.GS_MODE_FBL, "fetch": gs.GS_MODE_OTF_FETCH}[mode]
+    r = {"otf": int(gamma * cfg["cache_width"] + 0.5), "fcr": cfg["cache_width"], "fbl": 0, "fetch": 0}[mode]
     hdr = C.storage[:512].view(torch.int32)
     stat0 = gs.gs_stats_word_offset()
 
