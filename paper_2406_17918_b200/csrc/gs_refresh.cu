@@ -28,6 +28,9 @@ namespace gs {
 #ifndef GS_SCAN_BATCH_DIV
 #define GS_SCAN_BATCH_DIV 4
 #endif
+#ifndef GS_FINISH_MIN_BLOCKS
+#define GS_FINISH_MIN_BLOCKS 4
+#endif
 #ifndef GS_SCAN_GRID_PER_SM
 #define GS_SCAN_GRID_PER_SM 8
 #endif
@@ -712,7 +715,7 @@ __device__ __forceinline__ void small_refill(const StepParams& P, int32_t v, int
     }
 }
 
-__global__ void __launch_bounds__(RP_THREADS, 4) k_finish(const __grid_constant__ StepParams P) {
+__global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(const __grid_constant__ StepParams P) {
     __shared__ unsigned long long s_buf[RP_WARPS][CAND_CAP];
     if (__ldcg(P.status) != 0) return;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;

@@ -103,6 +103,29 @@ def test_shared_presample_sample(shared_cfg):
     shared_cfg.check_rows(C, O, nodes)
 
 
+def test_batch_stats_and_event_profile(mid):
+    """The diagnostics counters agree with the oracle's own count of refreshed rows, and the optional
+    event timing returns one positive figure per kernel group."""
+    import paper_2406_17918_b200 as gs
+    B = mid.cfg["batch"]
+    C, ws, O = mid.samplers(B)
+    gs.gs_cache_profile_begin(C, 2)
+    for b in range(3):                                  # the third batch is beyond max_batches: not timed
+        seeds = batch_seeds(mid.perm, b, B)
+        n, m = mid.check_batch(C, ws, O, seeds, "otf", 0.3, b + 1, features=False, rows=False)
+        st = gs.gs_batch_stats(C)
+        refreshed, scanned = O.stats()
+        assert st["refreshed_nodes"] == refreshed
+        assert 0 <= st["slow_refills"] <= refreshed and st["queued_rescans"] <= st["slow_refills"]
+        assert 0 < st["philox_blocks"] <= (scanned + 3 * refreshed) // 4 + refreshed
+    ms, batches = gs.gs_cache_profile_end(C)
+    assert batches == 2 and set(ms) == {"row_counts", "scan", "finish", "relabel"}
+    assert all(v > 0 for v in ms.values())
+    with pytest.raises(gs.GsError):
+        gs.gs_cache_profile_end(C)                      # not on any more
+    assert gs.gs_stats_word_offset() > 0
+
+
 def test_ragged_batch_sizes(tiny):
     for B in (1, 2, 31, 33, 1000):
         tiny.run("otf", 0.25, 2, batch_size=B)
