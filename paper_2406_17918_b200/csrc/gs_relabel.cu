@@ -37,6 +37,9 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
     __syncthreads();
     if (s_status != 0) return;  // block-uniform: the barriers below stay convergent
     const int n = (P.k == 0) ? P.n_host : __ldcg(P.hdr + HDR_N + P.k);
+    // the grid is sized for the worst case; only the tiles that hold frontier nodes take part
+    const int tiles = (n + SCAN_A_TILE - 1) / SCAN_A_TILE;
+    if ((int)blockIdx.x >= tiles) return;
     const int p = blockIdx.x * SCAN_A_TILE + threadIdx.x;
     int c = 0;
     int nch = 0;   // scan work items of this node (split path only)
@@ -87,14 +90,14 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
         P.tile_sums[blockIdx.x] = total;
         __threadfence();
         const int ticket = atomicAdd(P.hdr + HDR_TICKET_A + P.k, 1);
-        is_last = (ticket == (int)gridDim.x - 1);
+        is_last = (ticket == tiles - 1);
     }
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    const int m = scan_tiles_in_place<SCAN_A_TILE>(P.tile_sums, (int)gridDim.x, warp_sums);
+    const int m = scan_tiles_in_place<SCAN_A_TILE>(P.tile_sums, tiles, warp_sums);
     int items = 0;
-    if (P.split) items = scan_tiles_in_place<SCAN_A_TILE>(P.tile_sums2, (int)gridDim.x, warp_sums);
+    if (P.split) items = scan_tiles_in_place<SCAN_A_TILE>(P.tile_sums2, tiles, warp_sums);
     if (threadIdx.x == 0) {
         P.hdr[HDR_M + P.k] = m;
         P.hdr[HDR_ITEMS + P.k] = items;
@@ -158,6 +161,9 @@ __global__ void __launch_bounds__(FF_THREADS) k_first_flags(RelabelParams P) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int n = __ldcg(P.hdr + HDR_N + P.k);
     const int m = __ldcg(P.hdr + HDR_M + P.k);
+    // worst-case grid: tiles beyond the picks leave at once (at least one tile stays, to publish n_{k+1})
+    const int tiles = m > 0 ? (m + SCAN_E_TILE - 1) / SCAN_E_TILE : 1;
+    if ((int)blockIdx.x >= tiles) return;
     const int wbase = blockIdx.x * SCAN_E_TILE + wid * 512;
     // 16 independent table probes per thread are in flight before anything is consumed
     int id[4][4];
@@ -222,12 +228,12 @@ __global__ void __launch_bounds__(FF_THREADS) k_first_flags(RelabelParams P) {
         P.tile_sums[blockIdx.x] = total;
         __threadfence();
         const int ticket = atomicAdd(P.hdr + HDR_TICKET_E + P.k, 1);
-        is_last = (ticket == (int)gridDim.x - 1);
+        is_last = (ticket == tiles - 1);
     }
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    const int fresh = scan_tiles_in_place<FF_THREADS>(P.tile_sums, (int)gridDim.x, warp_sums);
+    const int fresh = scan_tiles_in_place<FF_THREADS>(P.tile_sums, tiles, warp_sums);
     if (threadIdx.x == 0) P.hdr[HDR_N + P.k + 1] = n + fresh;
 }
 
