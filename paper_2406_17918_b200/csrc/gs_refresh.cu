@@ -551,9 +551,11 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick_hub(const __grid
 
 __global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ StepParams P) {
     __shared__ unsigned long long s_stage[RP_WARPS][SPLIT_CAND_CAP];
+    __shared__ int s_hits[RP_WARPS];
     if (__ldcg(P.status) != 0) return;
     const int lane = threadIdx.x & 31;
     unsigned long long* stage = s_stage[threadIdx.x >> 5];
+    int* hits = &s_hits[threadIdx.x >> 5];
     const int total = __ldcg(P.d_items_total);
     const int total_warps = gridDim.x * RP_WARPS;
     // Work is handed out in batches of 1..32 items; every warp owns one batch up front, the rest
@@ -594,26 +596,27 @@ __global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ Ste
             const uint32_t qa = (uint32_t)chunk * HUB_CHUNK_QUADS;
             const uint32_t qe = qa + HUB_CHUNK_QUADS < nq ? qa + HUB_CHUNK_QUADS : nq;
             const uint32_t tinc = threshold_for(P.lambda_otf, deg);
-            int count = 0;   // hits of this item, staged in shared memory (those beyond the cap are only counted)
-            // Appends the offsets of one lane-quad whose key is at or below the threshold.
+            // Hits of this item are staged in shared memory; each hitting lane reserves its place with a
+            // shared-memory atomic (hits are rare, the order inside the list does not matter), so an
+            // iteration with hits costs a few instructions, not a vote per key.  Hits beyond the cap
+            // are only counted.
+            if (lane == 0) *hits = 0;
+            __syncwarp();
             auto take_hits = [&](uint32_t q, const uint4& o, bool inq) {
                 const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
+                if (!inq || min(min(kk[0], kk[1]), min(kk[2], kk[3])) > tinc) return;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const uint32_t off = 4u * q + j;
-                    const bool hit = inq && (off < deg) && (kk[j] <= tinc);
-                    const uint32_t b = __ballot_sync(FULL, hit);
-                    if (b) {
-                        if (hit) {
-                            const int pos = count + __popc(b & lt);
-                            if (pos < SPLIT_CAND_CAP) stage[pos] = ((unsigned long long)kk[j] << 32) | off;
-                        }
-                        count += __popc(b);
+                    if (off < deg && kk[j] <= tinc) {
+                        const int pos = atomicAdd(hits, 1);
+                        if (pos < SPLIT_CAND_CAP) stage[pos] = ((unsigned long long)kk[j] << 32) | off;
                     }
                 }
             };
             // Main loop: four independent Philox blocks per lane and iteration (512 offsets per warp
-            // iteration), all quads in range, one vote per iteration.  The ragged end goes quad by quad.
+            // iteration), all quads in range, one vote per iteration.  The ragged end takes up to four
+            // masked blocks at once as well.
             uint32_t qb = qa;
             for (; qb + 128 <= qe; qb += 128) {
                 const uint32_t q = qb + lane;
@@ -631,13 +634,27 @@ __global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ Ste
                 take_hits(q + 64, o2, true);
                 take_hits(q + 96, o3, true);
             }
-            for (; qb < qe; qb += 32) {
+            if (qb < qe) {
                 const uint32_t q = qb + lane;
-                const uint4 o = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
-                const bool inq = q < qe;
-                if (__ballot_sync(FULL, inq && min(min(o.x, o.y), min(o.z, o.w)) <= tinc) == 0) continue;
-                take_hits(q, o, inq);
+                const int groups = (int)((qe - qb + 31u) >> 5);   // 1..4 groups of 32 quads remain
+                if (groups > 2) {
+                    const uint4 o0 = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
+                    const uint4 o1 = philox4x32_10_rk(q + 32, (uint32_t)v, P.step, P.word_fill, P.rk);
+                    const uint4 o2 = philox4x32_10_rk(q + 64, (uint32_t)v, P.step, P.word_fill, P.rk);
+                    const uint4 o3 = philox4x32_10_rk(q + 96, (uint32_t)v, P.step, P.word_fill, P.rk);
+                    take_hits(q, o0, q < qe);
+                    take_hits(q + 32, o1, q + 32 < qe);
+                    take_hits(q + 64, o2, q + 64 < qe);
+                    take_hits(q + 96, o3, q + 96 < qe);
+                } else {
+                    const uint4 o0 = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
+                    const uint4 o1 = philox4x32_10_rk(q + 32, (uint32_t)v, P.step, P.word_fill, P.rk);
+                    take_hits(q, o0, q < qe);
+                    take_hits(q + 32, o1, q + 32 < qe);
+                }
             }
+            __syncwarp();
+            const int count = *hits;
             __syncwarp();
             // publish: the only warp of a short row owns the list; the chunks of a long row reserve
             // their range with one atomic per chunk, so no warp waits on an atomic inside the scan
