@@ -28,6 +28,9 @@ namespace gs {
 #ifndef GS_SCAN_BATCH_DIV
 #define GS_SCAN_BATCH_DIV 4
 #endif
+#ifndef GS_SCAN_MIN_BLOCKS
+#define GS_SCAN_MIN_BLOCKS 1
+#endif
 #ifndef GS_FINISH_MIN_BLOCKS
 #define GS_FINISH_MIN_BLOCKS 4
 #endif
@@ -201,6 +204,88 @@ struct Refill {
     }
 };
 
+// Removes and returns the largest of the candidates a warp holds four-per-lane, looking only at
+// those whose flag bit is set; clears that flag.
+__device__ __forceinline__ void warp_drop_max(const unsigned long long (&it)[4], uint32_t& flags) {
+    unsigned long long loc = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        if (((flags >> j) & 1u) && it[j] >= loc) loc = it[j];
+    const bool have = flags != 0;
+    const uint32_t hi = have ? (uint32_t)(loc >> 32) : 0u;
+    const uint32_t mhi = __reduce_max_sync(FULL, hi);
+    const uint32_t lo = (have && hi == mhi) ? (uint32_t)loc : 0u;
+    const uint32_t mlo = __reduce_max_sync(FULL, lo);
+    const unsigned long long worst = ((unsigned long long)mhi << 32) | mlo;
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        if (((flags >> j) & 1u) && it[j] == worst) flags &= ~(1u << j);
+}
+
+// The W smallest of `count` candidates (W <= count <= CAND_CAP) in ascending order, one per lane:
+// a threshold guess selects about W of them (keys are uniform below the scan threshold), a few
+// max/min reductions repair the count, the survivors are compacted through `buf` and sorted with
+// a 32-lane bitonic network.  Lanes >= W return ~0.
+__device__ __forceinline__ unsigned long long warp_top_sorted(unsigned long long* buf, int count, int W,
+                                                              uint32_t tinc, int lane) {
+    unsigned long long it[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) it[j] = (lane + 32 * j < count) ? buf[lane + 32 * j] : ~0ull;
+    __syncwarp();
+    const uint32_t guess = (uint32_t)(((unsigned long long)tinc * (unsigned)W) / (unsigned)count);
+    uint32_t flags = 0;
+    int cnt = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const bool s = it[j] != ~0ull && (uint32_t)(it[j] >> 32) <= guess;
+        if (s) flags |= 1u << j;
+        cnt += __popc(__ballot_sync(FULL, s));
+    }
+    while (cnt > W) {
+        warp_drop_max(it, flags);
+        --cnt;
+    }
+    while (cnt < W) {   // add the smallest candidate that is not selected yet
+        unsigned long long loc = ~0ull;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (!((flags >> j) & 1u) && it[j] < loc) loc = it[j];
+        const uint32_t hi = (uint32_t)(loc >> 32);
+        const uint32_t mhi = __reduce_min_sync(FULL, hi);
+        const uint32_t lo = (hi == mhi) ? (uint32_t)loc : 0xFFFFFFFFu;
+        const uint32_t mlo = __reduce_min_sync(FULL, lo);
+        const unsigned long long best = ((unsigned long long)mhi << 32) | mlo;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (!((flags >> j) & 1u) && it[j] == best) flags |= 1u << j;
+        ++cnt;
+    }
+    // compact the W survivors into buf[0..W)
+    int base = 0;
+    const uint32_t lt = lanemask_lt();
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const bool s = (flags >> j) & 1u;
+        const uint32_t b = __ballot_sync(FULL, s);
+        if (s) buf[base + __popc(b & lt)] = it[j];
+        base += __popc(b);
+    }
+    __syncwarp();
+    unsigned long long x = lane < W ? buf[lane] : ~0ull;
+    __syncwarp();
+#pragma unroll
+    for (int k = 2; k <= 32; k <<= 1) {
+#pragma unroll
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            const unsigned long long other = __shfl_xor_sync(FULL, x, j);
+            const bool up = (lane & k) == 0, lower = (lane & j) == 0;
+            const bool take_min = (lower == up);
+            x = take_min ? (other < x ? other : x) : (other > x ? other : x);
+        }
+    }
+    return x;
+}
+
 // First attempt of a refill, split around the neighbour-id loads: issue() extracts the first
 // r (+1 spare) candidates in FILL order and starts loading their neighbour ids; settle() uses
 // them if they contain r neighbours that are not retained.  Anything else (too few candidates,
@@ -210,12 +295,18 @@ struct Quick {
     uint32_t my_off;
     int32_t my_nb;
 
-    __device__ __forceinline__ void issue(const StepParams& P, int64_t row_start, const unsigned long long* buf,
-                                          int count, int r, int lane) {
+    __device__ __forceinline__ void issue(const StepParams& P, int64_t row_start, unsigned long long* buf,
+                                          int count, int r, uint32_t tinc, int lane) {
         g = 0;
         my_off = 0;
         my_nb = -1;
         if (count > CAND_CAP || count < r) return;
+        if (r >= P.W) {   // full refill: the whole top-W in order, nothing is retained
+            g = P.W;
+            my_off = (uint32_t)warp_top_sorted(buf, count, P.W, tinc, lane);
+            if (lane < g) my_nb = __ldg(P.g.indices + row_start + my_off);
+            return;
+        }
         unsigned long long it[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) it[j] = (lane + 32 * j < count) ? buf[lane + 32 * j] : ~0ull;
@@ -231,6 +322,10 @@ struct Quick {
     __device__ __forceinline__ bool settle(const StepParams& P, uint32_t evict_mask, int32_t& slot, int lane) {
         if (g == 0) return false;
         const int r = __popc(evict_mask);
+        if (r >= P.W) {   // full refill: candidate t is slot t
+            if (lane < P.W) slot = my_nb;
+            return true;
+        }
         const bool retained = (lane < P.W) && !((evict_mask >> lane) & 1u);
         uint32_t valid = 0;
         for (int t = 0; t < g; ++t) {
@@ -426,7 +521,7 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick(const __grid_con
                     cur.tried_full = !(P.r < W);
                     const uint32_t tinc = threshold_for(cur.tried_full ? P.lambda_full : P.lambda_otf, cur.deg);
                     const int c = warp_collect(P, cur.v, cur.deg, 0, (cur.deg + 3u) >> 2, tinc, buf, 0, lane);
-                    cur.Q.issue(P, cur.row_start, buf, c, __popc(cur.evict), lane);
+                    cur.Q.issue(P, cur.row_start, buf, c, __popc(cur.evict), tinc, lane);
                     __syncwarp();   // buf may be reused from here on: the first candidates live in registers
                 }
                 i = i_next;
@@ -525,7 +620,7 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick_hub(const __grid
         int32_t slot = (!P.init_rows && !P.fbl && lane < W) ? row[lane] : -1;
         const uint32_t evict = evict_mask_for(P, v, lane);
         Quick Q;
-        Q.issue(P, rs, buf, c, __popc(evict), lane);
+        Q.issue(P, rs, buf, c, __popc(evict), tinc, lane);
         __syncwarp();
         if (!Q.settle(P, evict, slot, lane)) refill_slow(P, v, rs, deg, evict, buf, slot, lane);
         __syncwarp();
@@ -549,7 +644,7 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick_hub(const __grid
 // Nodes whose candidate list cannot decide the refill (too few, too many, or several retained
 // neighbours among the first ones) take the retry ladder of the fused path.
 
-__global__ void __launch_bounds__(RP_THREADS) k_scan(const __grid_constant__ StepParams P) {
+__global__ void __launch_bounds__(RP_THREADS, GS_SCAN_MIN_BLOCKS) k_scan(const __grid_constant__ StepParams P) {
     __shared__ unsigned long long s_stage[RP_WARPS][SPLIT_CAND_CAP];
     __shared__ int s_hits[RP_WARPS];
     if (__ldcg(P.status) != 0) return;
