@@ -407,11 +407,14 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
             double nf = std::floor(gamma * (double)c->fanouts[layer] + 0.5);
             n_fetch = nf < 0 ? 0 : (nf > c->fanouts[layer] ? c->fanouts[layer] : (int32_t)nf);
         }
-        const bool split = ((r > 0 && r < c->W) && mode != GS_MODE_FBL) || n_fetch > 0;
+        // every mode that scans rows runs as scan + finish kernels; only a batch that refreshes
+        // nothing (OTF with r = 0, OTF Fetch with no fetch at this layer) needs the pick alone
+        const bool fbl = (mode == GS_MODE_FBL);
+        const bool split = fbl || r > 0 || n_fetch > 0;
         C.split = split ? 1 : 0;
-        C.W = c->W;
-        C.r = n_fetch > 0 ? n_fetch : r;
-        C.d_refresh_from = (c->shared && k > 0 && mode != GS_MODE_OTF_FETCH) ? c->d_hdr + HDR_N + (k - 1) : nullptr;
+        C.W = fbl ? c->fanouts[layer] : c->W;
+        C.r = n_fetch > 0 ? n_fetch : (fbl ? c->fanouts[layer] : r);
+        C.d_refresh_from = (c->shared && k > 0 && mode != GS_MODE_OTF_FETCH && !fbl) ? c->d_hdr + HDR_N + (k - 1) : nullptr;
         C.tile_sums2 = (int32_t*)(ws + w.tiles_a2);
         C.item_start = (int32_t*)(ws + w.item_start);
         C.items = (int32_t*)(ws + w.items);
@@ -447,11 +450,16 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
             P.word_fill = key_word(4, (uint32_t)layer);
             P.d_refresh_from = nullptr;
         }
-        if (mode == GS_MODE_FBL) {   // the fused kernels with W = r = f and FETCH keys; no cache row is touched
+        if (fbl) {   // W = r = f and FETCH keys; no cache row is touched
             P.fbl = 1;
             P.W = P.r = P.f;
             P.word_fill = key_word(4, (uint32_t)layer);
             P.d_refresh_from = nullptr;
+        }
+        if (P.r >= P.W) {
+            // a full refill needs the whole top-W in the 64-entry candidate list: aim at the middle
+            // of [W, 64] (for W = 32 about 1 % of the rows miss on either side and are rescanned)
+            P.lambda_otf = c->lambda_full * (float)(P.W + SPLIT_CAND_CAP) / 144.0f;
         }
         P.item_start = C.item_start;
         P.items = C.items;

@@ -870,7 +870,7 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
         auto prefetch = [&](int i) {
             const int32_t v = __shfl_sync(FULL, v_l, i);
             const int cc = __shfl_sync(FULL, cc_l, i);
-            row_next = lane < W ? P.slots[(int64_t)v * P.pitch + lane] : -1;
+            row_next = (!P.fbl && lane < W) ? P.slots[(int64_t)v * P.pitch + lane] : -1;
             const unsigned long long* cl = P.cand + (size_t)(base + i) * SPLIT_CAND_CAP;
             cand_next = (lane < cc) ? __ldcg(cl + lane) : ~0ull;
             cand_next2 = (lane + 32 < cc && lane + 32 < SPLIT_CAND_CAP) ? __ldcg(cl + lane + 32) : ~0ull;
@@ -888,10 +888,54 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
             if (i + 1 < cnt) prefetch(i + 1);
             const bool refresh = deg > (uint32_t)W && p >= refresh_from;
             const int ncached = deg < (uint32_t)W ? (int)deg : W;
+            if (P.fbl && !refresh) {
+                // Full Batch Load of a short row: the whole adjacency, already in ascending offset
+                if (lane < (int)deg) {
+                    const int32_t id = __ldg(P.g.indices + rs + lane);
+                    const int e = e_base + lane;
+                    P.picked[e] = id;
+                    atomicMin(P.table + id, ((unsigned long long)P.stamp << 32) | (n_base + (uint32_t)e));
+                }
+                continue;
+            }
             uint32_t ekey = 0, pkey = 0;
-            if (refresh || ncached > P.f) evict_pick_keys(P, v, lane, ekey, pkey);
+            if (!P.fbl && (refresh || ncached > P.f)) evict_pick_keys(P, v, lane, ekey, pkey);
             uint32_t cache_part = 0;   // OTF Fetch: lanes of the cache slots that are part of the sample
-            if (refresh) {
+            if (refresh && P.r >= W) {
+                // Full refill (FCR, and Full Batch Load with W = f): the W offsets first in key order,
+                // in that order.  Short rows take every offset as a candidate, longer ones the list
+                // the scan kernel left; a list that cannot hold the top-W sends the row to a rescan.
+                int c = -1;
+                uint32_t tinc = 0xFFFFFFFFu;
+                if (deg <= (uint32_t)SMALL_DEGREE) {
+                    const uint4 o = philox4x32_10((uint32_t)lane, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
+                    const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (4u * lane + j < deg) buf[4 * lane + j] = ((unsigned long long)kk[j] << 32) | (4u * lane + j);
+                    c = (int)deg;
+                } else if (cc >= W && cc <= SPLIT_CAND_CAP) {
+                    if (lane < cc) buf[lane] = cand;
+                    if (lane + 32 < cc) buf[lane + 32] = cand2;
+                    c = cc;
+                    tinc = threshold_for(P.lambda_otf, deg);
+                }
+                __syncwarp();
+                if (c >= W) {
+                    const unsigned long long x = warp_top_sorted(buf, c, W, tinc, lane);
+                    slot = lane < W ? __ldg(P.g.indices + rs + (uint32_t)x) : -1;
+                    __syncwarp();
+                } else {
+                    if (deg > (uint32_t)RETRY_QUEUE_DEGREE && hub_register(P, p, deg, lane)) continue;
+                    refill_slow(P, v, rs, deg, wmask, buf, slot, lane);
+                    __syncwarp();
+                }
+                if (P.fbl) {
+                    warp_emit_sorted(P, W, e_base, n_base, slot, lane);
+                    continue;
+                }
+                if (lane < W) P.slots[(int64_t)v * P.pitch + lane] = slot;
+            } else if (refresh) {
                 uint32_t evict;
                 if (P.fetch) {
                     // The f - r cache picks play the part of the retained slots, the r fetched
