@@ -52,6 +52,8 @@ def lib():
         L.gso_destroy.restype = None
         L.gso_set_key_fn.argtypes = [ctypes.c_void_p, KEY_FN, ctypes.c_void_p]
         L.gso_set_key_fn.restype = None
+        L.gso_set_theta.argtypes = [ctypes.c_void_p, ctypes.c_int64]
+        L.gso_set_theta.restype = None
         L.gso_cache_row.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]
         L.gso_cache_set_row.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]
         L.gso_refresh_node.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_uint32, ctypes.c_int32]
@@ -141,6 +143,10 @@ class Sampler:
             self.close()
         except Exception:
             pass
+
+    def set_theta(self, theta):
+        """Dense/sparse split: nodes with degree <= theta are sampled straight from the graph."""
+        lib().gso_set_theta(self._h, int(theta))
 
     def set_key_fn(self, fn):
         """fn(purpose, tag, v, step, i) -> uint32 replaces the Philox keys (None restores them)."""

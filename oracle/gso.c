@@ -13,6 +13,7 @@ struct gso_sampler {
     const int64_t* indptr;
     const int32_t* indices;
     int32_t L, W, shared;
+    int64_t theta;   /* dense/sparse split: rows with degree <= theta are never cached (-1: no split) */
     int32_t fanouts[GSO_MAX_HOPS];
     uint64_t seed;
     gso_key_fn key_fn;
@@ -256,6 +257,7 @@ gso_sampler* gso_create(int64_t num_nodes, const int64_t* indptr, const int32_t*
     gso_sampler* s = (gso_sampler*)calloc(1, sizeof(gso_sampler));
     s->N = num_nodes; s->indptr = indptr; s->indices = indices;
     s->L = num_hops; s->W = cache_width; s->seed = seed; s->shared = shared ? 1 : 0;
+    s->theta = -1;
     memcpy(s->fanouts, fanouts, (size_t)num_hops * sizeof(int32_t));
     s->num_caches = s->shared ? 1 : num_hops;
     for (int32_t c = 0; c < s->num_caches; ++c) s->rows[c] = (int32_t**)calloc((size_t)num_nodes, sizeof(int32_t*));
@@ -284,6 +286,7 @@ void gso_destroy(gso_sampler* s) {
 }
 
 void gso_set_key_fn(gso_sampler* s, gso_key_fn fn, void* ctx) { s->key_fn = fn; s->key_ctx = ctx; }
+void gso_set_theta(gso_sampler* s, int64_t theta) { s->theta = theta < 0 ? -1 : theta; }
 
 static int bad_node(const gso_sampler* s, int32_t layer, int32_t v) {
     return !s || layer < 0 || layer >= s->L || v < 0 || v >= s->N;
@@ -374,7 +377,10 @@ int gso_sample_batch(gso_sampler* s, const int32_t* seeds, int32_t num_seeds, in
         for (int32_t p = 0; p < nk; ++p) {
             int32_t v = s->frontier[p];
             indptr[p] = m;
-            if (mode == GSO_MODE_FBL) {
+            /* Dense/sparse split (paper Section "Graph Splitting and Sampling Strategies"): nodes with
+             * degree <= theta form the sparse part and are sampled straight from the graph (FBL)
+             * in every mode; only the dense part is cached, refreshed and sampled from the cache. */
+            if (mode == GSO_MODE_FBL || degree(s, v) <= s->theta) {
                 m += fbl_row(s, l, v, step, picked + m);
                 continue;
             }

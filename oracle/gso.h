@@ -53,6 +53,10 @@ gso_sampler* gso_create(int64_t num_nodes, const int64_t* indptr, const int32_t*
                         uint64_t seed, int32_t shared);
 void gso_destroy(gso_sampler*);
 void gso_set_key_fn(gso_sampler*, gso_key_fn fn, void* ctx);
+/* Dense/sparse split by degree threshold theta (paper Section "Graph Splitting and Sampling
+ * Strategies"): nodes with degree <= theta are sampled by the FBL rule in every mode and never
+ * touch the cache; theta < 0 switches the split off (the default). */
+void gso_set_theta(gso_sampler*, int64_t theta);
 
 /* Current cache row of node v (layer ignored in shared mode); untouched rows are the static
  * pre-sample.  out has cache_width entries, -1 = empty slot. */
