@@ -89,6 +89,25 @@ gs_status gs_cache_init(const gs_graph*, int32_t num_hops, const int32_t* fanout
                         void* stream, gs_cache** out);
 void gs_cache_destroy(gs_cache*);
 
+/* Dense / sparse split (paper Section "Graph Splitting and Sampling Strategies": nodes with
+ * degree > theta form the dense part, which is cached and refreshed by FCR / OTF; the remaining,
+ * sparse part is loaded from the graph for every batch).  A split cache stores rows only for the
+ * dense part, plus a 4-byte row index per node, instead of one row per node.
+ *   theta        in [cache_width, 128]
+ *   dense_rows   the number of nodes with degree > theta, counted by the caller (the storage is
+ *                sized from it); gs_cache_init_split verifies it on the device and returns
+ *                GS_ERR_ARG if it is wrong
+ * Sampling with a split cache: a node of the sparse part is sampled by the Full Batch Load rule in
+ * every mode (all neighbours if there are at most f_l, else the f_l edge offsets first in FETCH
+ * order, emitted in ascending offset) and is never refreshed; the dense part behaves exactly as
+ * with gs_cache_init.  gs_cache_read_rows returns -1 slots for sparse nodes.
+ * gs_cache_init_split synchronises `stream` once (to verify dense_rows). */
+gs_status gs_cache_bytes_split(const gs_graph*, int32_t num_hops, int32_t cache_width, int32_t shared,
+                               int64_t dense_rows, size_t* bytes);
+gs_status gs_cache_init_split(const gs_graph*, int32_t num_hops, const int32_t* fanouts, int32_t cache_width,
+                              uint64_t seed, int32_t shared, int32_t theta, int64_t dense_rows,
+                              void* d_cache_storage, size_t cache_bytes, void* stream, gs_cache** out);
+
 /* One hop's message-flow graph ("blocks" of Algorithm 2/3), stored destination-major.  The
  * destination nodes are the first *d_num_dst entries of the input-node list, the source nodes its
  * first *d_num_src entries (so sources begin with the destinations).  Counts are device scalars;

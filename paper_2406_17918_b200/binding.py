@@ -70,6 +70,8 @@ def _load():
         "gs_cache_bytes": [vp, i32, i32, i32, psz],
         "gs_workspace_bytes": [vp, i32, vp, i32, psz],
         "gs_cache_init": [vp, i32, vp, i32, u64, i32, vp, sz, vp, pvp],
+        "gs_cache_bytes_split": [vp, i32, i32, i32, i64, psz],
+        "gs_cache_init_split": [vp, i32, vp, i32, u64, i32, i32, i64, vp, sz, vp, pvp],
         "gs_sample_batch": [vp, vp, i32, ctypes.c_int, dbl, u32, vp, sz, vp, vp, pvp, pvp],
         "gs_sample_batch_host": [vp, vp, i32, ctypes.c_int, dbl, u32, vp, sz, vp, vp, pvp, vp, vp],
         "gs_sample_batch_noalloc": [vp, vp, i32, ctypes.c_int, dbl, u32, vp, i64, vp, vp, vp, pvp],
@@ -239,6 +241,28 @@ def gs_cache_init(graph: Graph, fanouts, cache_width: int, seed: int, shared: bo
     h = ctypes.c_void_p()
     _check(_L.gs_cache_init(graph.handle, len(fanouts), _i32_array(fanouts), cache_width, ctypes.c_uint64(seed),
                             int(shared), _ptr(storage), storage.numel(), _stream(stream), ctypes.byref(h)))
+    return Cache(h, graph, storage, fanouts, cache_width, shared)
+
+
+def gs_cache_bytes_split(graph: Graph, num_hops: int, cache_width: int, shared: bool, dense_rows: int) -> int:
+    out = ctypes.c_size_t()
+    _check(_L.gs_cache_bytes_split(graph.handle, num_hops, cache_width, int(shared), dense_rows, ctypes.byref(out)))
+    return out.value
+
+
+def gs_cache_init_split(graph: Graph, fanouts, cache_width: int, seed: int, shared: bool, theta: int,
+                        dense_rows: int = None, storage: torch.Tensor = None, stream=None) -> Cache:
+    """Cache rows only for nodes with degree > theta; the others are sampled from the graph."""
+    if dense_rows is None:
+        deg = graph.indptr[1:] - graph.indptr[:-1]
+        dense_rows = int((deg > theta).sum().item())
+    if storage is None:
+        storage = torch.empty(gs_cache_bytes_split(graph, len(fanouts), cache_width, shared, dense_rows),
+                              dtype=torch.uint8, device=graph.indptr.device)
+    h = ctypes.c_void_p()
+    _check(_L.gs_cache_init_split(graph.handle, len(fanouts), _i32_array(fanouts), cache_width, ctypes.c_uint64(seed),
+                                  int(shared), int(theta), int(dense_rows), _ptr(storage), storage.numel(),
+                                  _stream(stream), ctypes.byref(h)))
     return Cache(h, graph, storage, fanouts, cache_width, shared)
 
 

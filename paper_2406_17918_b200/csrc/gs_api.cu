@@ -32,6 +32,9 @@ struct gs_cache {
     uint32_t serial;          // batches run; the relabel stamp is derived from it
     float lambda_otf, lambda_full;
     int32_t hub_degree;
+    int32_t theta;            // split cache: nodes with degree <= theta have no row (-1: every node has one)
+    int64_t rows;             // cache rows per cache (num_nodes, or the dense nodes of a split cache)
+    int32_t* d_row_index;     // split cache only
     int32_t* h_pinned;        // pinned staging for counts
     // optional device timing of the kernel groups (gs_cache_profile_begin / _end)
     cudaEvent_t* prof_events;
@@ -98,7 +101,10 @@ static StepParams step_params(const gs_cache* c, int32_t layer, uint32_t step) {
     const gs_graph* g = c->graph;
     P.g = GraphView{g->d_indptr, g->d_indices, g->num_nodes};
     const int32_t ci = c->shared ? 0 : layer;
-    P.slots = c->d_slots + (size_t)ci * (size_t)g->num_nodes * c->pitch;
+    P.slots = c->d_slots + (size_t)ci * (size_t)c->rows * c->pitch;
+    P.row_index = c->d_row_index;
+    P.theta = c->theta;
+    P.word_fetch = key_word(4, (uint32_t)layer);
     P.pitch = c->pitch;
     P.W = c->W;
     P.f = c->fanouts[layer];
@@ -186,8 +192,23 @@ gs_status gs_workspace_bytes(const gs_graph* g, int32_t num_hops, const int32_t*
     return GS_OK;
 }
 
-gs_status gs_cache_init(const gs_graph* g, int32_t num_hops, const int32_t* fanouts, int32_t cache_width, uint64_t seed,
-                        int32_t shared, void* d_cache_storage, size_t cache_bytes, void* stream, gs_cache** out) {
+static size_t row_index_bytes(const gs_graph* g) { return align_up((size_t)g->num_nodes * 4, 256); }
+
+gs_status gs_cache_bytes_split(const gs_graph* g, int32_t num_hops, int32_t cache_width, int32_t shared,
+                               int64_t dense_rows, size_t* bytes) {
+    if (!bytes) return fail(GS_ERR_ARG, "bytes is NULL");
+    gs_status st = check_shape(g, num_hops, cache_width);
+    if (st != GS_OK) return st;
+    if (dense_rows < 0 || dense_rows > g->num_nodes) return fail(GS_ERR_ARG, "dense_rows outside [0, num_nodes]");
+    const size_t rows = (size_t)(dense_rows > 0 ? dense_rows : 1);
+    *bytes = HDR_BYTES + table_bytes(g) + row_index_bytes(g) +
+             align_up((size_t)(shared ? 1 : num_hops) * rows * (size_t)pitch_for(cache_width) * 4, 256);
+    return GS_OK;
+}
+
+static gs_status cache_init_impl(const gs_graph* g, int32_t num_hops, const int32_t* fanouts, int32_t cache_width,
+                                 uint64_t seed, int32_t shared, int32_t theta, int64_t dense_rows,
+                                 void* d_cache_storage, size_t cache_bytes, void* stream, gs_cache** out) {
     if (!out) return fail(GS_ERR_ARG, "out is NULL");
     *out = nullptr;
     gs_status st = check_shape(g, num_hops, cache_width);
@@ -196,8 +217,13 @@ gs_status gs_cache_init(const gs_graph* g, int32_t num_hops, const int32_t* fano
     if (st != GS_OK) return st;
     if (!d_cache_storage) return fail(GS_ERR_ARG, "d_cache_storage is NULL");
     if (!aligned(d_cache_storage, 256)) return fail(GS_ERR_ALIGN, "d_cache_storage must be 256-byte aligned");
+    const bool split_cache = theta >= 0;
+    if (split_cache && (theta < cache_width || theta > SMALL_DEGREE))
+        return fail(GS_ERR_ARG, "theta %d outside [cache_width, %d]", theta, SMALL_DEGREE);
     size_t need = 0;
-    gs_cache_bytes(g, num_hops, cache_width, shared, &need);
+    if (split_cache) st = gs_cache_bytes_split(g, num_hops, cache_width, shared, dense_rows, &need);
+    else st = gs_cache_bytes(g, num_hops, cache_width, shared, &need);
+    if (st != GS_OK) return st;
     if (cache_bytes < need) return fail(GS_ERR_WORKSPACE, "cache storage has %zu bytes, %zu needed", cache_bytes, need);
 
     gs_cache* c = new (std::nothrow) gs_cache{};
@@ -213,8 +239,11 @@ gs_status gs_cache_init(const gs_graph* g, int32_t num_hops, const int32_t* fano
     c->d_storage = (char*)d_cache_storage;
     c->d_hdr = (int32_t*)c->d_storage;
     c->d_table = (unsigned long long*)(c->d_storage + HDR_BYTES);
-    c->d_slots = (int32_t*)(c->d_storage + HDR_BYTES + table_bytes(g));
-    c->slot_bytes = (size_t)c->num_caches * (size_t)g->num_nodes * (size_t)c->pitch * 4;
+    c->theta = split_cache ? theta : -1;
+    c->rows = split_cache ? (dense_rows > 0 ? dense_rows : 1) : g->num_nodes;
+    c->d_row_index = split_cache ? (int32_t*)(c->d_storage + HDR_BYTES + table_bytes(g)) : nullptr;
+    c->d_slots = (int32_t*)(c->d_storage + HDR_BYTES + table_bytes(g) + (split_cache ? row_index_bytes(g) : 0));
+    c->slot_bytes = (size_t)c->num_caches * (size_t)c->rows * (size_t)c->pitch * 4;
     c->serial = 0;
     c->lambda_otf = 18.0f;
     c->lambda_full = 72.0f;
@@ -243,9 +272,26 @@ gs_status gs_cache_init(const gs_graph* g, int32_t num_hops, const int32_t* fano
         if (o_cand + (size_t)cap0 * HUB_CAND_CAP * 8 <= table_room) break;
         cap0 = 0;
     }
-    e = launch_init_low_rows(GraphView{g->d_indptr, g->d_indices, g->num_nodes}, c->d_slots, c->pitch, c->W,
-                             c->num_caches, s);
-    if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "pre-sample launch"); }
+    if (split_cache) {
+        // Row index of the dense part (tile sums live in the not yet used relabel table); the number
+        // of dense nodes the caller sized the storage for must be the graph's.
+        int32_t* d_cnt = c->d_hdr + HDR_WORDS;
+        e = launch_build_row_index(GraphView{g->d_indptr, g->d_indices, g->num_nodes}, theta, c->d_row_index,
+                                   (int32_t*)c->d_table, d_cnt, s);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(c->h_pinned, d_cnt, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "row index"); }
+        if ((int64_t)c->h_pinned[1] != dense_rows) {
+            const long long got = c->h_pinned[1];
+            cudaFreeHost(c->h_pinned);
+            delete c;
+            return fail(GS_ERR_ARG, "dense_rows = %lld, but %lld nodes have a degree above theta", (long long)dense_rows, got);
+        }
+    } else {
+        e = launch_init_low_rows(GraphView{g->d_indptr, g->d_indices, g->num_nodes}, c->d_slots, c->pitch, c->W,
+                                 c->num_caches, s);
+        if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "pre-sample launch"); }
+    }
     for (int ci = 0; ci < c->num_caches; ++ci) {
         StepParams P = step_params(c, ci, 0u);
         P.r = c->W;
@@ -273,6 +319,20 @@ gs_status gs_cache_init(const gs_graph* g, int32_t num_hops, const int32_t* fano
     if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "cudaMemsetAsync"); }
     *out = c;
     return GS_OK;
+}
+
+gs_status gs_cache_init(const gs_graph* g, int32_t num_hops, const int32_t* fanouts, int32_t cache_width, uint64_t seed,
+                        int32_t shared, void* d_cache_storage, size_t cache_bytes, void* stream, gs_cache** out) {
+    return cache_init_impl(g, num_hops, fanouts, cache_width, seed, shared, -1, g ? g->num_nodes : 0, d_cache_storage,
+                           cache_bytes, stream, out);
+}
+
+gs_status gs_cache_init_split(const gs_graph* g, int32_t num_hops, const int32_t* fanouts, int32_t cache_width,
+                              uint64_t seed, int32_t shared, int32_t theta, int64_t dense_rows, void* d_cache_storage,
+                              size_t cache_bytes, void* stream, gs_cache** out) {
+    if (theta < 0) return fail(GS_ERR_ARG, "theta must be >= 0");
+    return cache_init_impl(g, num_hops, fanouts, cache_width, seed, shared, theta, dense_rows, d_cache_storage,
+                           cache_bytes, stream, out);
 }
 
 void gs_cache_destroy(gs_cache* c) {
@@ -410,9 +470,9 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         // every mode that scans rows runs as scan + finish kernels; only a batch that refreshes
         // nothing (OTF with r = 0, OTF Fetch with no fetch at this layer) needs the pick alone
         const bool fbl = (mode == GS_MODE_FBL);
-        const bool split = fbl || r > 0 || n_fetch > 0;
+        const bool split = fbl || r > 0 || n_fetch > 0 || c->theta >= 0;
         C.split = split ? 1 : 0;
-        C.W = fbl ? c->fanouts[layer] : c->W;
+        C.W = fbl ? c->fanouts[layer] : (c->theta > c->W ? c->theta : c->W);   // rows above this degree are refreshed
         C.r = n_fetch > 0 ? n_fetch : (fbl ? c->fanouts[layer] : r);
         C.d_refresh_from = (c->shared && k > 0 && mode != GS_MODE_OTF_FETCH && !fbl) ? c->d_hdr + HDR_N + (k - 1) : nullptr;
         C.tile_sums2 = (int32_t*)(ws + w.tiles_a2);
@@ -618,8 +678,8 @@ gs_status gs_cache_read_rows(const gs_cache* c, int32_t layer, const int32_t* d_
     if (layer < 0 || layer >= c->L) return fail(GS_ERR_ARG, "layer %d outside [0, %d)", layer, c->L);
     if (n < 0 || (n > 0 && (!d_nodes || !d_out))) return fail(GS_ERR_ARG, "bad node list");
     const int32_t ci = c->shared ? 0 : layer;
-    const int32_t* slots = c->d_slots + (size_t)ci * (size_t)c->graph->num_nodes * c->pitch;
-    GS_CUDA(launch_read_rows(slots, c->pitch, c->W, d_nodes, n, d_out, (cudaStream_t)stream));
+    const int32_t* slots = c->d_slots + (size_t)ci * (size_t)c->rows * c->pitch;
+    GS_CUDA(launch_read_rows(slots, c->d_row_index, c->pitch, c->W, d_nodes, n, d_out, (cudaStream_t)stream));
     return GS_OK;
 }
 

@@ -123,7 +123,10 @@ struct GraphView {
 
 struct StepParams {
     GraphView g;
-    int32_t* slots;        // this step's cache: [num_nodes][pitch]
+    int32_t* slots;        // this step's cache: [rows][pitch]; row of node v = v, or row_index[v] in a split cache
+    const int32_t* row_index;  // split cache only: cache row of each node, -1 for the sparse part (degree <= theta)
+    int32_t theta;         // split cache: nodes with degree <= theta are sampled from the graph; -1 = no split
+    uint32_t word_fetch;   // (FETCH << 8) | layer, the key word of the sparse part
     int32_t pitch, W, f, r;
     uint32_t step, key0, key1;
     uint32_t rk[20];       // Philox round keys derived from (key0, key1)
@@ -228,7 +231,9 @@ cudaError_t launch_relabel(const RelabelParams& p, int64_t m_bound, cudaStream_t
 cudaError_t launch_gather(const void* src, int64_t src_ld_bytes, int64_t row_bytes, const int32_t* ids,
                           const int32_t* d_count, int32_t count_bound, void* dst, int64_t dst_ld_bytes,
                           cudaStream_t s);
-cudaError_t launch_read_rows(const int32_t* slots, int32_t pitch, int32_t W, const int32_t* nodes, int32_t n,
-                             int32_t* out, cudaStream_t s);
+cudaError_t launch_read_rows(const int32_t* slots, const int32_t* row_index, int32_t pitch, int32_t W,
+                             const int32_t* nodes, int32_t n, int32_t* out, cudaStream_t s);
+cudaError_t launch_build_row_index(const GraphView& g, int32_t theta, int32_t* row_index, int32_t* tile_sums,
+                                   int32_t* d_dense_rows, cudaStream_t s);
 
 }  // namespace gs

@@ -42,6 +42,12 @@ constexpr int RP_WARPS = RP_THREADS / 32;
 constexpr int RETRY_QUEUE_DEGREE = 2048;  // split path: longer rows that need a rescan go to the hub kernel
 static_assert(CAND_CAP == HUB_CAND_CAP, "hub buffers are copied into a warp buffer");
 
+// First slot of node v's cache row; negative for a node of the sparse part of a split cache.
+__device__ __forceinline__ int64_t row_offset(const StepParams& P, int32_t v) {
+    const int64_t r = P.row_index ? (int64_t)__ldg(P.row_index + v) : (int64_t)v;
+    return r * P.pitch;
+}
+
 __device__ __forceinline__ uint32_t threshold_for(float lambda, uint32_t deg) {
     // inclusive key threshold: about lambda of deg uniform 32-bit keys fall at or below it
     if (deg <= (uint32_t)CAND_CAP) return 0xFFFFFFFFu;
@@ -478,11 +484,11 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick(const __grid_con
         // the current cache row of a node (nothing to read when the rows are being initialised)
         auto fetch_row = [&](int i) -> int32_t {
             const int32_t v = __shfl_sync(FULL, v_l, i);
-            return (!P.init_rows && !P.fbl && lane < W) ? P.slots[(int64_t)v * P.pitch + lane] : -1;
+            return (!P.init_rows && !P.fbl && lane < W) ? P.slots[row_offset(P, v) + lane] : -1;
         };
         // nodes of the chunk this kernel has work for: all of them when picking; when initialising only
         // the rows that need a selection (rows that hold their whole adjacency are written by k_init_low_rows)
-        uint32_t todo = __ballot_sync(FULL, lane < cnt && (!P.init_rows || hi_l - lo_l > (long long)W));
+        uint32_t todo = __ballot_sync(FULL, lane < cnt && (!P.init_rows || hi_l - lo_l > (long long)(P.theta > W ? P.theta : W)));
         auto next_node = [&]() -> int {
             if (!todo) return -1;
             const int b = __ffs(todo) - 1;
@@ -536,7 +542,7 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick(const __grid_con
                 if (P.fbl) {
                     warp_emit_sorted(P, prev.deg < (uint32_t)W ? (int)prev.deg : W, prev.e_base, n_base, prev.slot, lane);
                 } else {
-                    if (prev.refresh) store_row(P, P.slots + (int64_t)prev.v * P.pitch, prev.evict, prev.slot, lane);
+                    if (prev.refresh) store_row(P, P.slots + row_offset(P, prev.v), prev.evict, prev.slot, lane);
                     if (P.do_pick) warp_pick(P, prev.v, prev.deg, prev.e_base, n_base, prev.slot, lane);
                 }
             }
@@ -616,7 +622,7 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick_hub(const __grid
         for (int j = lane; j < CAND_CAP; j += 32)
             if (j < c) buf[j] = __ldcg(cand + j);
         __syncwarp();
-        int32_t* row = P.slots + (int64_t)v * P.pitch;
+        int32_t* row = P.slots + row_offset(P, v);
         int32_t slot = (!P.init_rows && !P.fbl && lane < W) ? row[lane] : -1;
         const uint32_t evict = evict_mask_for(P, v, lane);
         Quick Q;
@@ -870,7 +876,8 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
         auto prefetch = [&](int i) {
             const int32_t v = __shfl_sync(FULL, v_l, i);
             const int cc = __shfl_sync(FULL, cc_l, i);
-            row_next = (!P.fbl && lane < W) ? P.slots[(int64_t)v * P.pitch + lane] : -1;
+            const int64_t ro = P.fbl ? -1 : row_offset(P, v);
+            row_next = (ro >= 0 && lane < W) ? P.slots[ro + lane] : -1;
             const unsigned long long* cl = P.cand + (size_t)(base + i) * SPLIT_CAND_CAP;
             cand_next = (lane < cc) ? __ldcg(cl + lane) : ~0ull;
             cand_next2 = (lane + 32 < cc && lane + 32 < SPLIT_CAND_CAP) ? __ldcg(cl + lane + 32) : ~0ull;
@@ -886,8 +893,29 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
             int32_t slot = row_next;
             unsigned long long cand = cand_next, cand2 = cand_next2;
             if (i + 1 < cnt) prefetch(i + 1);
-            const bool refresh = deg > (uint32_t)W && p >= refresh_from;
+            const bool refresh = deg > (uint32_t)W && P.r > 0 && p >= refresh_from;
             const int ncached = deg < (uint32_t)W ? (int)deg : W;
+            if (!P.fbl && P.theta >= 0 && deg <= (uint32_t)P.theta) {
+                // Sparse part of a split cache (degree <= theta <= SMALL_DEGREE): no cache row exists;
+                // the node is sampled from the graph by the Full Batch Load rule, in every mode.
+                const int f = P.f;
+                int32_t id = -1;
+                if ((int)deg <= f) {
+                    if (lane < (int)deg) id = __ldg(P.g.indices + rs + lane);
+                } else {
+                    const uint4 o = philox4x32_10((uint32_t)lane, (uint32_t)v, P.step, P.word_fetch, P.key0, P.key1);
+                    const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (4u * lane + j < deg) buf[4 * lane + j] = ((unsigned long long)kk[j] << 32) | (4u * lane + j);
+                    __syncwarp();
+                    const unsigned long long x = warp_top_sorted(buf, (int)deg, f, 0xFFFFFFFFu, lane);
+                    if (lane < f) id = __ldg(P.g.indices + rs + (uint32_t)x);
+                    __syncwarp();
+                }
+                warp_emit_sorted(P, (int)deg < f ? (int)deg : f, e_base, n_base, id, lane);
+                continue;
+            }
             if (P.fbl && !refresh) {
                 // Full Batch Load of a short row: the whole adjacency, already in ascending offset
                 if (lane < (int)deg) {
@@ -934,7 +962,7 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
                     warp_emit_sorted(P, W, e_base, n_base, slot, lane);
                     continue;
                 }
-                if (lane < W) P.slots[(int64_t)v * P.pitch + lane] = slot;
+                if (lane < W) P.slots[row_offset(P, v) + lane] = slot;
             } else if (refresh) {
                 uint32_t evict;
                 if (P.fetch) {
@@ -1018,7 +1046,7 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
                     }
                     continue;
                 }
-                if ((evict >> lane) & 1u) P.slots[(int64_t)v * P.pitch + lane] = slot;
+                if ((evict >> lane) & 1u) P.slots[row_offset(P, v) + lane] = slot;
             }
             // S2 pick
             const uint32_t cmask = ncached >= 32 ? FULL : ((1u << ncached) - 1u);

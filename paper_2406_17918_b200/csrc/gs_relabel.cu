@@ -64,12 +64,12 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
         if (v >= 0) {
             const int64_t deg = P.g.indptr[v + 1] - P.g.indptr[v];
             c = deg < (int64_t)P.f ? (int)deg : P.f;
-            if (P.split && deg > (int64_t)SMALL_DEGREE && deg > (int64_t)P.W && p >= refresh_from) {
+            if (P.split && P.r > 0 && deg > (int64_t)SMALL_DEGREE && deg > (int64_t)P.W && p >= refresh_from) {
                 const int64_t nq = (deg + 3) >> 2;
                 nch = (int)((nq + HUB_CHUNK_QUADS - 1) / HUB_CHUNK_QUADS);
                 quads = (unsigned)nq;
             }
-            if (P.split && deg > (int64_t)P.W && p >= refresh_from) refreshed = 1;
+            if (P.split && P.r > 0 && deg > (int64_t)P.W && p >= refresh_from) refreshed = 1;
         }
     }
     int total;
@@ -293,18 +293,60 @@ cudaError_t launch_relabel(const RelabelParams& p, int64_t m_bound, cudaStream_t
 }
 
 // ---------------------------------------------------------------- logical cache rows (parity / debug)
-__global__ void k_read_rows(const int32_t* slots, int pitch, int W, const int32_t* nodes, int n, int32_t* out) {
+__global__ void k_read_rows(const int32_t* slots, const int32_t* row_index, int pitch, int W, const int32_t* nodes,
+                            int n, int32_t* out) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n * W) return;
     const int row = i / W, j = i - row * W;
-    out[i] = slots[(int64_t)nodes[row] * pitch + j];
+    const int64_t r = row_index ? (int64_t)row_index[nodes[row]] : (int64_t)nodes[row];
+    out[i] = r >= 0 ? slots[r * pitch + j] : -1;   // nodes of the sparse part have no cache row
 }
 
-cudaError_t launch_read_rows(const int32_t* slots, int32_t pitch, int32_t W, const int32_t* nodes, int32_t n,
-                             int32_t* out, cudaStream_t s) {
+// Split cache: row_index[v] = rank of v among the nodes with degree > theta, -1 for the others.
+// Same pattern as the other scans: tile-local scan, the last block scans the tile sums; a second
+// kernel adds the tile offsets.
+__global__ void __launch_bounds__(1024) k_row_index_local(GraphView g, int theta, int32_t* row_index,
+                                                          int32_t* tile_sums, int32_t* ticket_and_total) {
+    __shared__ int warp_sums[33];
+    __shared__ int is_last;
+    const int64_t v = (int64_t)blockIdx.x * 1024 + threadIdx.x;
+    int dense = 0;
+    if (v < g.num_nodes) dense = (g.indptr[v + 1] - g.indptr[v] > (int64_t)theta) ? 1 : 0;
+    int total;
+    const int excl = block_exclusive_scan<1024>(dense, warp_sums, &total);
+    if (v < g.num_nodes) row_index[v] = dense ? excl : -1;
+    if (threadIdx.x == 0) {
+        tile_sums[blockIdx.x] = total;
+        __threadfence();
+        is_last = (atomicAdd(ticket_and_total, 1) == (int)gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const int rows = scan_tiles_in_place<1024>(tile_sums, (int)gridDim.x, warp_sums);
+    if (threadIdx.x == 0) ticket_and_total[1] = rows;
+}
+
+__global__ void __launch_bounds__(1024) k_row_index_offsets(int64_t num_nodes, int32_t* row_index, const int32_t* tile_sums) {
+    const int64_t v = (int64_t)blockIdx.x * 1024 + threadIdx.x;
+    if (v < num_nodes && row_index[v] >= 0) row_index[v] += tile_sums[blockIdx.x];
+}
+
+// d_dense_rows: two zeroed ints (ticket, result).
+cudaError_t launch_build_row_index(const GraphView& g, int32_t theta, int32_t* row_index, int32_t* tile_sums,
+                                   int32_t* d_dense_rows, cudaStream_t s) {
+    const int tiles = (int)((g.num_nodes + 1023) / 1024);
+    k_row_index_local<<<tiles, 1024, 0, s>>>(g, theta, row_index, tile_sums, d_dense_rows);
+    k_row_index_offsets<<<tiles, 1024, 0, s>>>(g.num_nodes, row_index, tile_sums);
+    count_launches(2);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_read_rows(const int32_t* slots, const int32_t* row_index, int32_t pitch, int32_t W,
+                             const int32_t* nodes, int32_t n, int32_t* out, cudaStream_t s) {
     if (n <= 0) return cudaSuccess;
     const int64_t total = (int64_t)n * W;
-    k_read_rows<<<(int)((total + 255) / 256), 256, 0, s>>>(slots, pitch, W, nodes, n, out);
+    k_read_rows<<<(int)((total + 255) / 256), 256, 0, s>>>(slots, row_index, pitch, W, nodes, n, out);
     count_launches(1);
     return cudaGetLastError();
 }

@@ -33,16 +33,28 @@ class Pair:
         self.G = gs.gs_graph_create(self.g_dev.indptr, self.g_dev.indices, self.X)
         self.seed = seed
 
-    def samplers(self, max_seeds, tuning=None):
-        C = gs.gs_cache_init(self.G, self.cfg["fanouts"], self.W, self.seed, self.shared)
+    def samplers(self, max_seeds, tuning=None, theta=None):
+        self.theta = theta
+        if theta is None:
+            C = gs.gs_cache_init(self.G, self.cfg["fanouts"], self.W, self.seed, self.shared)
+        else:
+            C = gs.gs_cache_init_split(self.G, self.cfg["fanouts"], self.W, self.seed, self.shared, theta)
         if tuning:
             gs.gs_cache_set_tuning(C, **tuning)
         ws = torch.empty(gs.gs_workspace_bytes(self.G, self.cfg["fanouts"], max_seeds), dtype=torch.uint8, device="cuda")
         O = oracle.Sampler(self.indptr, self.indices, self.cfg["fanouts"], self.W, self.seed, self.shared)
+        if theta is not None:
+            O.set_theta(theta)
         return C, ws, O
 
     def check_rows(self, C, O, nodes):
         nodes = np.asarray(nodes, dtype=np.int32)
+        if getattr(self, "theta", None) is not None:      # a split cache has rows for the dense part only
+            sparse = nodes[self.deg[nodes] <= self.theta]
+            nodes = nodes[self.deg[nodes] > self.theta]
+            if len(sparse):
+                got = gs.gs_cache_read_rows(C, 0, torch.from_numpy(sparse).cuda()).cpu().numpy()
+                assert (got == -1).all()
         for layer in range(1 if self.shared else self.L):
             got = gs.gs_cache_read_rows(C, layer, torch.from_numpy(nodes).cuda()).cpu().numpy()
             want = O.cache_rows(layer, nodes)
@@ -83,9 +95,9 @@ class Pair:
                 assert bool((out[n[self.L]:] == 7).all())
         return n, m
 
-    def run(self, mode, gamma, batches, batch_size=None, tuning=None, first_step=1, **kw):
+    def run(self, mode, gamma, batches, batch_size=None, tuning=None, first_step=1, theta=None, **kw):
         B = batch_size or self.cfg["batch"]
-        C, ws, O = self.samplers(B, tuning)
+        C, ws, O = self.samplers(B, tuning, theta)
         out = []
         for b in range(batches):
             seeds = batch_seeds(self.perm, b, B)

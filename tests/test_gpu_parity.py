@@ -90,6 +90,34 @@ def test_otf_fetch_mode_internal_paths_and_shared(mid, shared_cfg):
         mid.check_batch(C, ws, O, batch_seeds(mid.perm, b, mid.cfg["batch"]), mode, rate, b + 1)
 
 
+@pytest.mark.parametrize("theta", [10, 16, 128])
+def test_dense_sparse_split_tiny(tiny, theta):
+    C, ws, O, _ = tiny.run("otf", 0.25, 4, theta=theta)
+    tiny.check_rows(C, O, np.arange(tiny.cfg["num_nodes"], dtype=np.int32))
+    tiny.run("fcr", 0.0, 2, theta=theta)
+
+
+def test_dense_sparse_split_other_modes_and_graphs(mid, shared_cfg):
+    import paper_2406_17918_b200 as gs
+    mid.run("otf", 0.3, 3, theta=20)
+    mid.run("otf", 0.0, 1, theta=64)
+    mid.run("fetch", 0.4, 2, theta=48)
+    mid.run("fbl", 0.0, 1, theta=48)
+    mid.run("fcr", 1.0, 1, theta=128, tuning=dict(lambda_full=1.0))
+    shared_cfg.run("otf", 0.3, 2, theta=32)
+    # the split cache is much smaller: rows only for the dense part
+    G = mid.G
+    dense = int((mid.deg > 20).sum())
+    full = gs.gs_cache_bytes(G, 3, 20, False)
+    split = gs.gs_cache_bytes_split(G, 3, 20, False, dense)
+    assert split < 0.25 * full
+    with pytest.raises(gs.GsError) as e:
+        gs.gs_cache_init_split(G, [15, 10, 5], 20, 1, False, 20, dense_rows=dense + 1)
+    assert e.value.status == 1 and "dense_rows" in str(e.value)
+    with pytest.raises(gs.GsError):
+        gs.gs_cache_init_split(G, [15, 10, 5], 20, 1, False, 129)
+
+
 def test_shared_cache_mode(shared_cfg):
     shared_cfg.run("otf", 0.3, 3)
     shared_cfg.run("fcr", 0.0, 1)
