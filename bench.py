@@ -128,7 +128,8 @@ def algorithmic_bytes(cfg, n, m_by_step, refreshed_by_step, r):
     return total + feat, feat
 
 
-def cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, budget_s=32.0, reps=1, first_seeds=None):
+def cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, budget_s=32.0, reps=1, first_seeds=None,
+                        theta=None):
     """Times the CPU oracle, as it stands, on the first `s` seeds of batch 0 (s grown until one
     batch takes a few seconds).  Returns (edges/s, feature GB/s, description, seconds per batch)."""
     import numpy as np
@@ -137,6 +138,8 @@ def cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, budget_s=32
     from workloads import feature_rows
 
     O = oracle.Sampler(indptr_h, indices_h, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED, cfg["shared"])
+    if theta is not None:
+        O.set_theta(theta)
     om = {"otf": oracle.MODE_OTF, "fcr": oracle.MODE_FCR, "fbl": oracle.MODE_FBL, "fetch": oracle.MODE_OTF_FETCH}[mode]
     B = cfg["batch"]
     s = first_seeds or max(1, min(B, 16))
@@ -182,6 +185,8 @@ def main():
                     help="sampling mode (default: the config's OTF run); fbl = no cache, the paper's baseline "
                          "sampler; fetch = OTF Fetch")
     ap.add_argument("--rate", type=float, default=None, help="gamma (otf) or delta (fetch); default: the config's")
+    ap.add_argument("--theta", type=int, default=None,
+                    help="dense/sparse split: cache rows only for nodes with degree > theta (default: one row per node)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -224,7 +229,13 @@ def main():
     G = gs.gs_graph_create(g.indptr, g.indices, X)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
-    C = gs.gs_cache_init(G, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED, cfg["shared"])
+    if args.theta is None:
+        C = gs.gs_cache_init(G, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED, cfg["shared"])
+    else:
+        dense_rows = int((g.degrees() > args.theta).sum().item())
+        ev0.record()
+        C = gs.gs_cache_init_split(G, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED, cfg["shared"], args.theta,
+                                   dense_rows)
     ev1.record()
     torch.cuda.synchronize()
     presample_ms = ev0.elapsed_time(ev1)
@@ -293,7 +304,7 @@ def main():
     deg = g.degrees()
     n_last = [int(counts[K - 1][w]) for w in n_words]
     fr = input_nodes[: n_last[L]].long()
-    over = (deg[fr] > cfg["cache_width"])
+    over = (deg[fr] > (cfg["cache_width"] if args.theta is None else args.theta))
     refreshed_frac = []
     for k in range(L):
         lo = n_last[k - 1] if (cfg["shared"] and k > 0) else 0
@@ -379,6 +390,7 @@ def main():
         "config": {"workload": cfg["name"], "num_nodes": g.num_nodes, "num_edges": g.num_edges,
                    "fanouts": cfg["fanouts"], "cache_width": cfg["cache_width"], "mode": mode, "gamma": gamma,
                    "batch": B, "shared_cache": cfg["shared"], "feat_dim": cfg["feat_dim"],
+                   "theta": args.theta, "cache_bytes": C.storage.numel(),
                    "parallelism": "replicas x%d" % world, "l2": "inputs_larger_than_L2",
                    "sampled_edges_per_batch": edges / K, "input_nodes_per_batch": feat_rows / K},
         "breakdown_ms_per_step": {"sample_batch": sample_ms / K, "gather_features": gather_ms / K,
@@ -399,7 +411,7 @@ def main():
         indptr_h, indices_h = g.indptr.cpu().numpy(), g.indices.cpu().numpy()
         if cfg["feat_kind"] != "hash":
             cpu_oracle_baseline.features = X.cpu()
-        v, fg, desc, _ = cpu_oracle_baseline(cfg, indptr_h, indices_h, perm.cpu(), mode, gamma)
+        v, fg, desc, _ = cpu_oracle_baseline(cfg, indptr_h, indices_h, perm.cpu(), mode, gamma, theta=args.theta)
         result["cpu_baseline"] = {"value": v, "unit": "edges/s", "feature_gbs": fg, "cores": 1,
                                   "host_cores": os.cpu_count(), "kind": "oracle", "sample": desc}
     print(json.dumps(result))
@@ -416,13 +428,13 @@ def reference_arm(args, cfg, mode, gamma):
     if cfg["feat_kind"] != "hash":
         cpu_oracle_baseline.features = build_features(cfg)
     # size the per-step sample once, then time warm-up + K steps at that size
-    v, fg, desc, dt = cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, budget_s=8.0)
+    v, fg, desc, dt = cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, budget_s=8.0, theta=args.theta)
     s = int(desc.split("first ")[1].split(" ")[0])
     per_step_budget = max(1, min(args.steps, int(120.0 / max(dt, 1e-3))))
     K = per_step_budget
     tot_edges, tot_t, fgs = 0.0, 0.0, []
     for i in range(min(args.warmup, 1) + K):
-        vv, ff, _, tt = cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, first_seeds=s)
+        vv, ff, _, tt = cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, first_seeds=s, theta=args.theta)
         if i >= min(args.warmup, 1):
             tot_edges += vv * tt
             tot_t += tt
