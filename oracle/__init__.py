@@ -64,6 +64,7 @@ def lib():
                                      ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32)]
         L.gso_fetch_count.argtypes = [ctypes.c_double, ctypes.c_int32]
         L.gso_fetch_count.restype = ctypes.c_int32
+        L.gso_refresh_all.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_double, ctypes.c_uint32]
         L.gso_sample_batch.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int,
                                        ctypes.c_double, ctypes.c_uint32]
         for name in ("gso_num_nodes", "gso_num_edges"):
@@ -173,6 +174,10 @@ class Sampler:
 
     def refresh_node(self, layer, v, step, r):
         if lib().gso_refresh_node(self._h, layer, int(v), step, r):
+            raise ValueError("bad arguments")
+
+    def refresh_all(self, mode, gamma, step):
+        if lib().gso_refresh_all(self._h, mode, float(gamma), step):
             raise ValueError("bad arguments")
 
     def pick_node(self, layer, v, step):

@@ -310,6 +310,21 @@ int gso_refresh_node(gso_sampler* s, int32_t layer, int32_t v, uint32_t step, in
     return 0;
 }
 
+/* The refresh as Algorithms 2 and 3 state it ("if t mod T = 0": RefreshCache / CacheRefresh for
+ * l = 1..L): every row of every layer's cache, not only the rows of the batch's frontier.
+ * With a dense/sparse split only the dense part has rows. */
+int gso_refresh_all(gso_sampler* s, int mode, double gamma, uint32_t step) {
+    if (!s || step == 0) return 1;
+    if (mode != GSO_MODE_FCR && mode != GSO_MODE_OTF) return 1;
+    if (mode == GSO_MODE_OTF && !(gamma >= 0.0 && gamma <= 1.0)) return 1;
+    int32_t r = gso_refresh_count(mode, gamma, s->W);
+    int32_t caches = s->shared ? 1 : s->L;
+    for (int32_t layer = 0; layer < caches; ++layer)
+        for (int64_t v = 0; v < s->N; ++v)
+            if (degree(s, (int32_t)v) > s->theta) refresh_row(s, layer, (int32_t)v, step, r);
+    return 0;
+}
+
 int gso_fbl_node(gso_sampler* s, int32_t layer, int32_t v, uint32_t step, int32_t* out, int32_t* count) {
     if (bad_node(s, layer, v) || !out || !count) return 1;
     *count = fbl_row(s, layer, v, step, out);

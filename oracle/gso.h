@@ -74,6 +74,12 @@ int32_t gso_fetch_count(double delta, int32_t f);
 /* Full Batch Load pick of one node (no cache involved); out has room for fanout entries. */
 int gso_fbl_node(gso_sampler*, int32_t layer, int32_t v, uint32_t step, int32_t* out, int32_t* count);
 
+/* Whole-cache refresh, the literal reading of Algorithms 2 and 3 (every T-th batch, all layers, all
+ * rows): mode GSO_MODE_FCR replaces every row, GSO_MODE_OTF replaces refresh_count(gamma) slots of
+ * every row, with the keys of `step` (>= 1).  Batches between two such refreshes sample with
+ * GSO_MODE_OTF and gamma = 0 (SampleFromCache only). */
+int gso_refresh_all(gso_sampler*, int mode, double gamma, uint32_t step);
+
 /* One batch.  mode/gamma as in the paper (gamma ignored for FCR and FBL).  GSO_MODE_FBL samples
  * every hop straight from the graph and leaves the cache untouched; for GSO_MODE_OTF_FETCH
  * `gamma` carries the fetch rate delta, and the cache is not modified either.  step >= 1.  Seeds must be distinct.
