@@ -108,6 +108,21 @@ gs_status gs_cache_init_split(const gs_graph*, int32_t num_hops, const int32_t* 
                               uint64_t seed, int32_t shared, int32_t theta, int64_t dense_rows,
                               void* d_cache_storage, size_t cache_bytes, void* stream, gs_cache** out);
 
+/* Whole-cache refresh: the refresh exactly as Algorithms 2 and 3 write it ("if t mod T = 0":
+ * RefreshCache / CacheRefresh for l = 1..L) - every cached row of every layer's cache, not only the
+ * rows of a batch's frontier.  The caller owns the schedule: every T-th batch it calls this with
+ * that batch's step, and samples all batches with gs_sample_batch(GS_MODE_OTF, gamma = 0), which is
+ * SampleFromCache alone.
+ *   mode   GS_MODE_FCR: all W slots of every row are replaced; GS_MODE_OTF: floor(gamma*W + 0.5)
+ *          slots per row (Section "OTF Refresh"); other modes: GS_ERR_ARG
+ *   step   >= 1; keys of (node, layer, step) as in gs_sample_batch, so refreshing a node here or
+ *          through a batch of the same step gives the same row
+ * Rows holding their whole adjacency (degree <= cache_width) and the sparse part of a split cache
+ * are left alone.  Asynchronous on `stream`; needs no workspace (between batches the cache's own
+ * relabel table is idle and serves as scratch).  Must not overlap a batch on the same cache, and
+ * it clears the counts of the previous batch (gs_batch_counts, gs_batch_stats). */
+gs_status gs_cache_refresh_all(gs_cache*, gs_mode mode, double gamma, uint32_t step, void* stream);
+
 /* One hop's message-flow graph ("blocks" of Algorithm 2/3), stored destination-major.  The
  * destination nodes are the first *d_num_dst entries of the input-node list, the source nodes its
  * first *d_num_src entries (so sources begin with the destinations).  Counts are device scalars;

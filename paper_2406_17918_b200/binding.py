@@ -70,6 +70,7 @@ def _load():
         "gs_cache_bytes": [vp, i32, i32, i32, psz],
         "gs_workspace_bytes": [vp, i32, vp, i32, psz],
         "gs_cache_init": [vp, i32, vp, i32, u64, i32, vp, sz, vp, pvp],
+        "gs_cache_refresh_all": [vp, ctypes.c_int, ctypes.c_double, ctypes.c_uint32, vp],
         "gs_cache_bytes_split": [vp, i32, i32, i32, i64, psz],
         "gs_cache_init_split": [vp, i32, vp, i32, u64, i32, i32, i64, vp, sz, vp, pvp],
         "gs_sample_batch": [vp, vp, i32, ctypes.c_int, dbl, u32, vp, sz, vp, vp, pvp, pvp],
@@ -264,6 +265,11 @@ def gs_cache_init_split(graph: Graph, fanouts, cache_width: int, seed: int, shar
                                   int(shared), int(theta), int(dense_rows), _ptr(storage), storage.numel(),
                                   _stream(stream), ctypes.byref(h)))
     return Cache(h, graph, storage, fanouts, cache_width, shared)
+
+
+def gs_cache_refresh_all(cache: Cache, mode: int, gamma: float, step: int, stream=None) -> None:
+    """Refresh every cached row of every layer (the 't mod T = 0' branch of Algorithms 2 and 3)."""
+    _check(_L.gs_cache_refresh_all(cache.handle, mode, float(gamma), step, _stream(stream)))
 
 
 def _blocks_out(cache: Cache, cblocks, workspace):

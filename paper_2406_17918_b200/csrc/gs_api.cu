@@ -206,6 +206,55 @@ gs_status gs_cache_bytes_split(const gs_graph* g, int32_t num_hops, int32_t cach
     return GS_OK;
 }
 
+// Refreshes r slots of every cached row (all caches) with the keys of `step`: the fused per-node
+// kernels over the node range instead of a frontier.  init = 1 writes whole rows (the pre-sample).
+// The relabel table is idle between batches and serves as the hub storage of these launches (the
+// hub degree is raised until the hubs it can produce fit there); it is reset afterwards, which is
+// the state every batch expects of entries it has not stamped.
+static cudaError_t refresh_every_row(gs_cache* c, int32_t r, uint32_t step, int init, cudaStream_t s) {
+    const gs_graph* g = c->graph;
+    const size_t table_room = (size_t)g->num_nodes * 8;
+    int64_t hub_degree0 = c->hub_degree < HUB_MIN_DEGREE ? HUB_MIN_DEGREE : c->hub_degree;
+    int64_t cap0 = 0, items0 = 0;
+    size_t o_entry = 0, o_state = 0, o_items = 0, o_cand = 0;
+    for (int tries = 0; tries < 40; ++tries, hub_degree0 *= 2) {
+        cap0 = g->num_edges / hub_degree0 + 1;
+        if (cap0 > g->num_nodes) cap0 = g->num_nodes;
+        items0 = g->num_edges / (4 * (int64_t)HUB_CHUNK_QUADS) + cap0 + 1;
+        o_entry = 0;
+        o_state = align_up(o_entry + (size_t)cap0 * 8, 256);
+        o_items = align_up(o_state + (size_t)cap0 * 8, 256);
+        o_cand = align_up(o_items + (size_t)items0 * 4, 256);
+        if (o_cand + (size_t)cap0 * HUB_CAND_CAP * 8 <= table_room) break;
+        cap0 = 0;
+    }
+    cudaError_t e = cudaSuccess;
+    for (int ci = 0; ci < c->num_caches; ++ci) {
+        StepParams P = step_params(c, ci, step);
+        P.r = r;
+        P.frontier = nullptr;
+        P.d_n = nullptr;
+        P.n_host = (int32_t)g->num_nodes;
+        P.d_refresh_from = nullptr;
+        P.do_pick = 0;
+        P.init_rows = init;
+        char* hub_base = (char*)c->d_table;
+        P.hub_entry = (int2*)(hub_base + o_entry);
+        P.hub_state = (int2*)(hub_base + o_state);
+        P.hub_items = (int32_t*)(hub_base + o_items);
+        P.hub_cand = (unsigned long long*)(hub_base + o_cand);
+        P.hub_counter = (unsigned long long*)(c->d_hdr + HDR_HUB64 + 2 * ci);
+        P.hub_cap = (int32_t)cap0;          // 0: the table is too small, every node is done by one warp
+        P.item_cap = (int32_t)items0;
+        P.hub_degree = cap0 > 0 ? (int32_t)(hub_degree0 > 0x7FFFFFFF ? 0x7FFFFFFF : hub_degree0) : 0x7FFFFFFF;
+        P.work_counter = c->d_hdr + HDR_WORK + ci;
+        P.work_counter2 = c->d_hdr + HDR_WORK2 + ci;
+        e = launch_refresh_pick(P, g->num_nodes, s);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaMemsetAsync(c->d_table, 0xFF, (size_t)g->num_nodes * 8, s);
+}
+
 static gs_status cache_init_impl(const gs_graph* g, int32_t num_hops, const int32_t* fanouts, int32_t cache_width,
                                  uint64_t seed, int32_t shared, int32_t theta, int64_t dense_rows,
                                  void* d_cache_storage, size_t cache_bytes, void* stream, gs_cache** out) {
@@ -254,24 +303,6 @@ static gs_status cache_init_impl(const gs_graph* g, int32_t num_hops, const int3
     cudaStream_t s = (cudaStream_t)stream;
     e = cudaMemsetAsync(c->d_hdr, 0, HDR_BYTES, s);
     if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "cudaMemsetAsync"); }
-    // S0: a full refresh (r = W) of every node at step 0, rows with deg <= W copied verbatim.
-    // The relabel table is not in use yet and serves as the hub storage of these launches; the
-    // hub degree is raised until the hubs it can produce fit there.
-    const size_t table_room = (size_t)g->num_nodes * 8;
-    int64_t hub_degree0 = c->hub_degree < HUB_MIN_DEGREE ? HUB_MIN_DEGREE : c->hub_degree;
-    int64_t cap0 = 0, items0 = 0;
-    size_t o_entry = 0, o_state = 0, o_items = 0, o_cand = 0;
-    for (int tries = 0; tries < 40; ++tries, hub_degree0 *= 2) {
-        cap0 = g->num_edges / hub_degree0 + 1;
-        if (cap0 > g->num_nodes) cap0 = g->num_nodes;
-        items0 = g->num_edges / (4 * (int64_t)HUB_CHUNK_QUADS) + cap0 + 1;
-        o_entry = 0;
-        o_state = align_up(o_entry + (size_t)cap0 * 8, 256);
-        o_items = align_up(o_state + (size_t)cap0 * 8, 256);
-        o_cand = align_up(o_items + (size_t)items0 * 4, 256);
-        if (o_cand + (size_t)cap0 * HUB_CAND_CAP * 8 <= table_room) break;
-        cap0 = 0;
-    }
     if (split_cache) {
         // Row index of the dense part (tile sums live in the not yet used relabel table); the number
         // of dense nodes the caller sized the storage for must be the graph's.
@@ -292,31 +323,8 @@ static gs_status cache_init_impl(const gs_graph* g, int32_t num_hops, const int3
                                  c->num_caches, s);
         if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "pre-sample launch"); }
     }
-    for (int ci = 0; ci < c->num_caches; ++ci) {
-        StepParams P = step_params(c, ci, 0u);
-        P.r = c->W;
-        P.frontier = nullptr;
-        P.d_n = nullptr;
-        P.n_host = (int32_t)g->num_nodes;
-        P.d_refresh_from = nullptr;
-        P.do_pick = 0;
-        P.init_rows = 1;
-        char* hub_base = (char*)c->d_table;
-        P.hub_entry = (int2*)(hub_base + o_entry);
-        P.hub_state = (int2*)(hub_base + o_state);
-        P.hub_items = (int32_t*)(hub_base + o_items);
-        P.hub_cand = (unsigned long long*)(hub_base + o_cand);
-        P.hub_counter = (unsigned long long*)(c->d_hdr + HDR_HUB64 + 2 * ci);
-        P.hub_cap = (int32_t)cap0;          // 0: the table is too small, every node is done by one warp
-        P.item_cap = (int32_t)items0;
-        P.hub_degree = cap0 > 0 ? (int32_t)(hub_degree0 > 0x7FFFFFFF ? 0x7FFFFFFF : hub_degree0) : 0x7FFFFFFF;
-        P.work_counter = c->d_hdr + HDR_WORK + ci;
-        P.work_counter2 = c->d_hdr + HDR_WORK2 + ci;
-        e = launch_refresh_pick(P, g->num_nodes, s);
-        if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "pre-sample launch"); }
-    }
-    e = cudaMemsetAsync(c->d_table, 0xFF, (size_t)g->num_nodes * 8, s);
-    if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "cudaMemsetAsync"); }
+    e = refresh_every_row(c, c->W, 0u, 1, s);
+    if (e != cudaSuccess) { cudaFreeHost(c->h_pinned); delete c; return cuda_fail(e, "pre-sample launch"); }
     *out = c;
     return GS_OK;
 }
@@ -611,6 +619,24 @@ gs_status gs_sample_batch(gs_cache* c, const int32_t* d_seeds, int32_t num_seeds
     if (!aligned(d_seeds, 4)) return fail(GS_ERR_ALIGN, "d_seeds must be 4-byte aligned");
     return sample_impl(c, d_seeds, num_seeds, mode, gamma, step, d_workspace, workspace_bytes, (cudaStream_t)stream,
                        blocks, d_input_nodes, d_num_input_nodes);
+}
+
+gs_status gs_cache_refresh_all(gs_cache* c, gs_mode mode, double gamma, uint32_t step, void* stream) {
+    if (!c) return fail(GS_ERR_ARG, "cache is NULL");
+    if (mode != GS_MODE_FCR && mode != GS_MODE_OTF) return fail(GS_ERR_ARG, "only FCR and OTF refresh the cache");
+    if (mode == GS_MODE_OTF && !(gamma >= 0.0 && gamma <= 1.0)) return fail(GS_ERR_ARG, "gamma outside [0, 1]");
+    if (step == 0) return fail(GS_ERR_ARG, "step 0 is reserved for the pre-sample");
+    int32_t r = c->W;
+    if (mode == GS_MODE_OTF) {
+        double rr = std::floor(gamma * (double)c->W + 0.5);
+        r = rr < 0 ? 0 : (rr > c->W ? c->W : (int32_t)rr);
+    }
+    if (r == 0) return GS_OK;
+    cudaStream_t s = (cudaStream_t)stream;
+    GS_CUDA(cudaMemsetAsync(c->d_hdr, 0, HDR_BYTES, s));
+    GS_CUDA(refresh_every_row(c, r, step, 0, s));
+    c->serial = 0;   // the table was reset: stamps start over
+    return GS_OK;
 }
 
 gs_status gs_batch_counts(gs_cache* c, void* stream, int32_t* h_num_nodes, int32_t* h_num_edges) {

@@ -486,9 +486,10 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick(const __grid_con
             const int32_t v = __shfl_sync(FULL, v_l, i);
             return (!P.init_rows && !P.fbl && lane < W) ? P.slots[row_offset(P, v) + lane] : -1;
         };
-        // nodes of the chunk this kernel has work for: all of them when picking; when initialising only
-        // the rows that need a selection (rows that hold their whole adjacency are written by k_init_low_rows)
-        uint32_t todo = __ballot_sync(FULL, lane < cnt && (!P.init_rows || hi_l - lo_l > (long long)(P.theta > W ? P.theta : W)));
+        // nodes of the chunk this kernel has work for: all of them when picking; otherwise (pre-sample,
+        // whole-cache refresh) only the rows that need a selection - rows that hold their whole adjacency
+        // were written by k_init_low_rows, and the sparse part of a split cache has no rows
+        uint32_t todo = __ballot_sync(FULL, lane < cnt && (P.do_pick || hi_l - lo_l > (long long)(P.theta > W ? P.theta : W)));
         auto next_node = [&]() -> int {
             if (!todo) return -1;
             const int b = __ffs(todo) - 1;

@@ -95,6 +95,22 @@ class Pair:
                 assert bool((out[n[self.L]:] == 7).all())
         return n, m
 
+    def run_periodic(self, mode, gamma, T, batches, batch_size=None, tuning=None, theta=None, **kw):
+        """Algorithms 2/3 as written: every T-th batch refreshes the whole cache, all batches only pick."""
+        B = batch_size or self.cfg["batch"]
+        C, ws, O = self.samplers(B, tuning, theta)
+        gm, om = MODES[mode]
+        all_nodes = np.arange(self.cfg["num_nodes"], dtype=np.int32)
+        for t in range(1, batches + 1):
+            if t % T == 0:
+                gs.gs_cache_refresh_all(C, gm, gamma, t)
+                O.refresh_all(om, gamma, t)
+                gs.gs_sync_status(C)
+                self.check_rows(C, O, all_nodes)
+            self.check_batch(C, ws, O, batch_seeds(self.perm, t, B), "otf", 0.0, t, **kw)
+        self.check_rows(C, O, all_nodes)
+        return C, ws, O
+
     def run(self, mode, gamma, batches, batch_size=None, tuning=None, first_step=1, theta=None, **kw):
         B = batch_size or self.cfg["batch"]
         C, ws, O = self.samplers(B, tuning, theta)

@@ -118,6 +118,21 @@ def test_dense_sparse_split_other_modes_and_graphs(mid, shared_cfg):
         gs.gs_cache_init_split(G, [15, 10, 5], 20, 1, False, 129)
 
 
+def test_periodic_whole_cache_refresh(tiny, mid, shared_cfg):
+    import paper_2406_17918_b200 as gs
+    tiny.run_periodic("otf", 0.3, 2, 6)
+    tiny.run_periodic("fcr", 0.0, 3, 6)
+    tiny.run_periodic("otf", 0.5, 2, 4, theta=16)
+    mid.run_periodic("otf", 0.25, 2, 4, rows=64, features=False)
+    mid.run_periodic("fcr", 0.0, 2, 2, rows=64, features=False, tuning=dict(hub_degree=64))
+    C, ws, O = shared_cfg.run_periodic("otf", 0.3, 2, 2, rows=64, features=False)
+    # a whole-cache refresh followed by per-batch refreshes keeps working (stamps restart cleanly)
+    shared_cfg.check_batch(C, ws, O, batch_seeds(shared_cfg.perm, 7, shared_cfg.cfg["batch"]), "otf", 0.3, 3, rows=64)
+    for bad in [(gs.GS_MODE_FBL, 0.0, 1), (gs.GS_MODE_OTF_FETCH, 0.5, 1), (gs.GS_MODE_OTF, 1.5, 1), (gs.GS_MODE_FCR, 0.0, 0)]:
+        with pytest.raises(gs.GsError):
+            gs.gs_cache_refresh_all(C, *bad)
+
+
 def test_shared_cache_mode(shared_cfg):
     shared_cfg.run("otf", 0.3, 3)
     shared_cfg.run("fcr", 0.0, 1)
