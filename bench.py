@@ -187,6 +187,10 @@ def main():
     ap.add_argument("--rate", type=float, default=None, help="gamma (otf) or delta (fetch); default: the config's")
     ap.add_argument("--theta", type=int, default=None,
                     help="dense/sparse split: cache rows only for nodes with degree > theta (default: one row per node)")
+    ap.add_argument("--period", type=int, default=None,
+                    help="T: the schedule of Algorithms 2/3 as written - every T-th batch refreshes the whole cache "
+                         "(--mode otf/fcr, --rate), every batch only samples from the cache; no CPU baseline "
+                         "(the oracle's whole-cache refresh of this graph takes hours)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -246,13 +250,28 @@ def main():
     hdr = C.storage[:512].view(torch.int32)
     stat0 = gs.gs_stats_word_offset()
 
+    if args.period:
+        if mode not in ("otf", "fcr"):
+            raise SystemExit("--period needs --mode otf or fcr")
+        args.no_cpu_baseline = True
+        refresh_mode, refresh_gamma = gm, gamma
+        gm, gamma, r = gs.GS_MODE_OTF, 0.0, 0
+
     K, Wm = args.steps, args.warmup
     seeds_all = [batch_seeds(perm, b, B, rank, world) for b in range(Wm + 2 * K)]
     pinned_counts = torch.zeros((K, 128), dtype=torch.int32).pin_memory()
     out = None
 
+    refresh_events = []
+
     def one_step(b, step):
         nonlocal out
+        if args.period and step % args.period == 0:
+            ra, rb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ra.record()
+            gs.gs_cache_refresh_all(C, refresh_mode, refresh_gamma, step)
+            rb.record()
+            refresh_events.append((ra, rb))
         blocks, input_nodes, cnt = gs.gs_sample_batch(C, seeds_all[b], gm, gamma, step, ws)
         if out is None:
             out = torch.empty((blocks[0].max_src, cfg["feat_dim"]), dtype=X.dtype, device=device)
@@ -332,6 +351,8 @@ def main():
         e0.record()
         for i in range(K):
             step = Wm + K + i + 1
+            if args.period and step % args.period == 0:
+                gs.gs_cache_refresh_all(C, refresh_mode, refresh_gamma, step)
             blocks, input_nodes, n, m = gs.gs_sample_batch_host(C, host_seeds[i], gm, gamma, step, ws)
             gs.gs_gather_features(G, input_nodes, None, out[: n[L]])
             e_edges += sum(m)
@@ -390,7 +411,8 @@ def main():
         "config": {"workload": cfg["name"], "num_nodes": g.num_nodes, "num_edges": g.num_edges,
                    "fanouts": cfg["fanouts"], "cache_width": cfg["cache_width"], "mode": mode, "gamma": gamma,
                    "batch": B, "shared_cache": cfg["shared"], "feat_dim": cfg["feat_dim"],
-                   "theta": args.theta, "cache_bytes": C.storage.numel(),
+                   "theta": args.theta, "period": args.period,
+                   "refresh": ({"mode": mode, "gamma": refresh_gamma} if args.period else "per batch, frontier rows"), "cache_bytes": C.storage.numel(),
                    "parallelism": "replicas x%d" % world, "l2": "inputs_larger_than_L2",
                    "sampled_edges_per_batch": edges / K, "input_nodes_per_batch": feat_rows / K},
         "breakdown_ms_per_step": {"sample_batch": sample_ms / K, "gather_features": gather_ms / K,
@@ -398,6 +420,7 @@ def main():
         "philox_blocks_per_batch": philox_blocks / K,
         "slow_refills_per_batch": slow_refills / K,
         "presample_ms": presample_ms,
+        "whole_cache_refresh_ms": ([a.elapsed_time(b) for a, b in refresh_events] if args.period else None),
         "setup_s": {"graph_and_features": t_graph},
         "roofline": roof_scan if (dominant == "scan" and roof_scan) else roof_gather,
         "roofline_gather": roof_gather,

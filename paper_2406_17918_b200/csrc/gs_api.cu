@@ -475,11 +475,11 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
             double nf = std::floor(gamma * (double)c->fanouts[layer] + 0.5);
             n_fetch = nf < 0 ? 0 : (nf > c->fanouts[layer] ? c->fanouts[layer] : (int32_t)nf);
         }
-        // every mode that scans rows runs as scan + finish kernels; only a batch that refreshes
-        // nothing (OTF with r = 0, OTF Fetch with no fetch at this layer) needs the pick alone
+        // every batch runs as scan + finish kernels; a step that refreshes and fetches nothing (OTF
+        // with r = 0, OTF Fetch with no fetch at this layer) has no scan items and skips the scan launch
         const bool fbl = (mode == GS_MODE_FBL);
-        const bool split = fbl || r > 0 || n_fetch > 0 || c->theta >= 0;
-        C.split = split ? 1 : 0;
+        const bool scans = fbl || r > 0 || n_fetch > 0;
+        C.split = 1;
         C.W = fbl ? c->fanouts[layer] : (c->theta > c->W ? c->theta : c->W);   // rows above this degree are refreshed
         C.r = n_fetch > 0 ? n_fetch : (fbl ? c->fanouts[layer] : r);
         C.d_refresh_from = (c->shared && k > 0 && mode != GS_MODE_OTF_FETCH && !fbl) ? c->d_hdr + HDR_N + (k - 1) : nullptr;
@@ -534,15 +534,12 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         P.d_items_total = c->d_hdr + HDR_ITEMS + k;
         P.cand_count = C.cand_count;
         P.cand = (unsigned long long*)(ws + w.cand);
-        if (split) {
+        if (scans) {
             int64_t item_bound = b.nb[k] + g->num_edges / (4 * (int64_t)HUB_CHUNK_QUADS) + 1;
             GS_CUDA(launch_scan(P, item_bound, s));
-            if (ev) GS_CUDA(cudaEventRecord(ev[2], s));
-            GS_CUDA(launch_finish(P, b.nb[k], s));
-        } else {
-            if (ev) GS_CUDA(cudaEventRecord(ev[2], s));
-            GS_CUDA(launch_refresh_pick(P, b.nb[k], s));
         }
+        if (ev) GS_CUDA(cudaEventRecord(ev[2], s));
+        GS_CUDA(launch_finish(P, b.nb[k], s));
         if (ev) GS_CUDA(cudaEventRecord(ev[3], s));
 
         RelabelParams R{};
