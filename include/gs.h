@@ -238,6 +238,63 @@ gs_status gs_batch_counts(gs_cache*, void* stream, int32_t* h_num_nodes, int32_t
 gs_status gs_gather_features(const gs_graph*, const int32_t* d_ids, const int32_t* d_count_or_null,
                              int32_t count_bound, void* d_out, int64_t out_ld, void* stream);
 
+/* out[i, :] = src[ids[i] - first_row, :] for any row-major matrix on the device (the copy kernel
+ * of gs_gather_features).  `src` holds rows first_row, first_row + 1, ... of a larger matrix - a
+ * feature shard - and ids are global; every id must lie inside the rows that `src` holds (not
+ * checked); negative ids are skipped.  row_elems, src_ld, out_ld in elements of `dtype`. */
+gs_status gs_gather_rows(const void* d_src, gs_dtype dtype, int32_t row_elems, int64_t src_ld, int64_t first_row,
+                         const int32_t* d_ids, const int32_t* d_count_or_null, int32_t count_bound, void* d_out,
+                         int64_t out_ld, void* stream);
+
+/* ---- Node-sharded sampling over several GPUs (the paper's Section "Shared Cache Mode" speaks of a
+ * cache that serves multiple computation processes; the partition and the exchange are this
+ * library's).  Nodes are partitioned by id range: shard o of `world` owns the nodes
+ * [o*S, (o+1)*S), S = ceil(num_nodes / world), with their CSR rows, cache rows and feature rows.
+ * A shard's gs_graph has the full num_nodes and an indptr in which only the owned rows are
+ * non-empty; its cache is created with gs_cache_init_split, so only owned dense rows use memory.
+ * One hop (sampling step k, layer L-1-k) of a rank's batch:
+ *   1. gs_shard_bucket           frontier_k grouped by owner            (requester)
+ *   2. exchange the groups (all-to-all; the caller's, e.g. NCCL)
+ *   3. gs_shard_sample_rows      refresh + pick for each received list  (owner)
+ *   4. exchange the rows of picks back
+ *   5. gs_shard_extend           dedup + relabel + block CSR            (requester)
+ * and after the last hop the same exchange with gs_gather_rows for the feature rows.  Every
+ * random choice is keyed by (seed, node, item, step), so the rows an owner returns are the rows
+ * a single device would compute, and refreshing a node twice in one step (two ranks ask for it)
+ * gives the same row as once.  A sharded run therefore equals one sampler, with dense/sparse
+ * split theta, that takes the ranks' batches of a step one after the other.  All ranks use the
+ * same step for the batches they run together. */
+
+/* Groups n node ids by owner.  d_sorted[n]: the ids, owner 0's first (order inside a group is
+ * unspecified); d_slot[n]: position of d_nodes[i] in d_sorted; d_counts: int32[2*world + 1], on
+ * return words [0, world) hold the group sizes and word 2*world is 0 or GS_ERR_RANGE (an id outside
+ * [0, num_nodes)); the words between are scratch.  world <= 64.  Asynchronous on `stream`. */
+gs_status gs_shard_bucket(const int32_t* d_nodes, int32_t n, int64_t num_nodes, int32_t world, int32_t* d_sorted,
+                          int32_t* d_slot, int32_t* d_counts, void* stream);
+
+/* Owner side.  For n distinct nodes of this shard: refresh (per mode / rate, exactly as
+ * gs_sample_batch does for a frontier at `layer`) and pick; d_picks[n][fanout(layer)] receives the
+ * picks of node i in the order a local batch would emit them, padded with -1.  Works on state of
+ * its own (a second header) and does not touch the relabel table, so it may run between the hops
+ * of this rank's own batch.  Lists of different requesters go in separate calls (a node may
+ * appear in several of them).  Workspace: gs_shard_workspace_bytes(graph, fanout(layer), n).
+ * gs_shard_status synchronises `stream` and reports a bad node id met by the last call. */
+gs_status gs_shard_workspace_bytes(const gs_graph*, int32_t fanout, int32_t max_nodes, size_t* bytes);
+gs_status gs_shard_sample_rows(gs_cache*, const int32_t* d_nodes, int32_t n, int32_t layer, gs_mode mode, double rate,
+                               uint32_t step, void* d_workspace, size_t workspace_bytes, void* stream, int32_t* d_picks);
+gs_status gs_shard_status(gs_cache*, void* stream);
+
+/* Requester side, hop k = 0 .. num_hops-1 in order.  d_reply[n_k][fanout(L-1-k)]: the owners' rows
+ * in d_sorted order; d_slot[n_k] as returned by gs_shard_bucket for frontier_k.  k = 0 starts a new
+ * batch and takes the seeds (distinct, as for gs_sample_batch); later hops ignore d_seeds and
+ * num_seeds.  The workspace is the one of gs_sample_batch (gs_workspace_bytes for num_seeds) and
+ * must stay untouched between the hops of a batch.  Fills *block like gs_sample_batch fills
+ * blocks[L-1-k]; *d_frontier is the frontier array (frontier_{k+1} is its prefix of
+ * *block->d_num_src ids).  Counts: gs_batch_counts, as after gs_sample_batch. */
+gs_status gs_shard_extend(gs_cache*, int32_t k, const int32_t* d_seeds, int32_t num_seeds, const int32_t* d_reply,
+                          const int32_t* d_slot, void* d_workspace, size_t workspace_bytes, void* stream, gs_block* block,
+                          const int32_t** d_frontier);
+
 /* Copy n logical cache rows (cache_width slots each, -1 = empty) of `layer` into d_out[n][cache_width]. */
 gs_status gs_cache_read_rows(const gs_cache*, int32_t layer, const int32_t* d_nodes, int32_t n,
                              int32_t* d_out, void* stream);

@@ -83,6 +83,12 @@ def _load():
         "gs_cache_export": [vp, vp, sz, vp],
         "gs_cache_import": [vp, vp, sz, vp],
         "gs_sync_status": [vp, vp],
+        "gs_gather_rows": [vp, ctypes.c_int, i32, i64, i64, vp, vp, i32, vp, i64, vp],
+        "gs_shard_bucket": [vp, i32, i64, i32, vp, vp, vp, vp],
+        "gs_shard_workspace_bytes": [vp, i32, i32, psz],
+        "gs_shard_sample_rows": [vp, vp, i32, i32, ctypes.c_int, dbl, u32, vp, sz, vp, vp],
+        "gs_shard_status": [vp, vp],
+        "gs_shard_extend": [vp, i32, vp, i32, vp, vp, vp, sz, vp, vp, pvp],
         "gs_batch_stats": [vp, vp, vp],
         "gs_cache_profile_begin": [vp, i32],
         "gs_cache_profile_end": [vp, vp, vp, vp],
@@ -365,6 +371,67 @@ def gs_gather_features(graph: Graph, ids: torch.Tensor, count, out: torch.Tensor
     _check(_L.gs_gather_features(graph.handle, _ptr(ids), _ptr(count), bound, _ptr(out), out.stride(0),
                                  _stream(stream)))
     return out
+
+
+def gs_gather_rows(src: torch.Tensor, ids: torch.Tensor, out: torch.Tensor, first_row: int = 0, count=None, stream=None):
+    """out[i] = src[ids[i] - first_row] for a row-major 2-D f32 / bf16 CUDA tensor."""
+    if src.dim() != 2 or src.stride(1) != 1 or out.dim() != 2 or out.stride(1) != 1 or out.dtype != src.dtype:
+        raise TypeError("src and out must be row-major 2-D tensors of one dtype")
+    if ids.dtype != torch.int32 or not ids.is_cuda:
+        raise TypeError("ids must be an int32 CUDA tensor")
+    dtype = {torch.float32: GS_F32, torch.bfloat16: GS_BF16}[src.dtype]
+    bound = min(out.shape[0], ids.numel())
+    _check(_L.gs_gather_rows(_ptr(src), dtype, src.shape[1], src.stride(0), int(first_row), _ptr(ids), _ptr(count), bound,
+                             _ptr(out), out.stride(0), _stream(stream)))
+    return out
+
+
+def gs_shard_bucket(nodes: torch.Tensor, num_nodes: int, world: int, stream=None):
+    """Group node ids by owner.  Returns (sorted ids, slot of every input id, int32[2*world+1] device counts)."""
+    if nodes.dtype != torch.int32 or not nodes.is_cuda or not nodes.is_contiguous():
+        raise TypeError("nodes must be a contiguous int32 CUDA tensor")
+    sorted_ids = torch.empty_like(nodes)
+    slot = torch.empty_like(nodes)
+    counts = torch.empty(2 * world + 1, dtype=torch.int32, device=nodes.device)
+    _check(_L.gs_shard_bucket(_ptr(nodes), nodes.numel(), int(num_nodes), int(world), _ptr(sorted_ids), _ptr(slot),
+                              _ptr(counts), _stream(stream)))
+    return sorted_ids, slot, counts
+
+
+def gs_shard_workspace_bytes(graph: Graph, fanout: int, max_nodes: int) -> int:
+    out = ctypes.c_size_t()
+    _check(_L.gs_shard_workspace_bytes(graph.handle, int(fanout), int(max_nodes), ctypes.byref(out)))
+    return out.value
+
+
+def gs_shard_sample_rows(cache: Cache, nodes: torch.Tensor, layer: int, mode: int, rate: float, step: int,
+                         workspace: torch.Tensor, picks: torch.Tensor = None, stream=None) -> torch.Tensor:
+    """Owner side of one hop: picks[n, fanout(layer)] (-1 padded) for n distinct nodes of this shard."""
+    if nodes.dtype != torch.int32 or not nodes.is_cuda or not nodes.is_contiguous():
+        raise TypeError("nodes must be a contiguous int32 CUDA tensor")
+    f = cache.fanouts[layer]
+    if picks is None:
+        picks = torch.empty((nodes.numel(), f), dtype=torch.int32, device=nodes.device)
+    _check(_L.gs_shard_sample_rows(cache.handle, _ptr(nodes), nodes.numel(), int(layer), mode, float(rate), step,
+                                   _ptr(workspace), workspace.numel(), _stream(stream), _ptr(picks)))
+    return picks
+
+
+def gs_shard_status(cache: Cache, stream=None):
+    _check(_L.gs_shard_status(cache.handle, _stream(stream)))
+
+
+def gs_shard_extend(cache: Cache, k: int, seeds, reply: torch.Tensor, slot: torch.Tensor, workspace: torch.Tensor,
+                    stream=None):
+    """Requester side of hop k.  Returns (block of layer L-1-k, frontier array aliasing the workspace)."""
+    cb = _CBlock()
+    d_fr = ctypes.c_void_p()
+    _check(_L.gs_shard_extend(cache.handle, int(k), _ptr(seeds), 0 if seeds is None else seeds.numel(), _ptr(reply),
+                              _ptr(slot), _ptr(workspace), workspace.numel(), _stream(stream), ctypes.byref(cb),
+                              ctypes.byref(d_fr)))
+    block = Block(cb, workspace, cache.storage)
+    off = d_fr.value - workspace.data_ptr()
+    return block, workspace[off:off + 4 * block.max_src].view(torch.int32)
 
 
 def gs_cache_read_rows(cache: Cache, layer: int, nodes: torch.Tensor, stream=None) -> torch.Tensor:

@@ -30,6 +30,8 @@ struct gs_cache {
     int32_t* d_slots;
     size_t slot_bytes;        // all caches
     uint32_t serial;          // batches run; the relabel stamp is derived from it
+    uint32_t shard_stamp;     // stamp of the sharded batch in progress (gs_shard_extend)
+    int32_t shard_seeds;      // its number of seeds
     float lambda_otf, lambda_full;
     int32_t hub_degree;
     int32_t theta;            // split cache: nodes with degree <= theta have no row (-1: every node has one)
@@ -404,12 +406,31 @@ gs_status gs_cache_set_tuning(gs_cache* c, double lambda_otf, double lambda_full
     return GS_OK;
 }
 
+// The stamp of a new batch: newer batches always win the atomicMin on the relabel table.
+static uint32_t next_stamp(gs_cache* c, cudaStream_t s) {
+    if (c->serial == 0xFFFFFFFEu) {  // stamp space used up: start over with a clean table
+        if (cudaMemsetAsync(c->d_table, 0xFF, (size_t)c->graph->num_nodes * 8, s) != cudaSuccess) return 0;
+        c->serial = 0;
+    }
+    c->serial += 1;
+    return 0xFFFFFFFFu - c->serial;
+}
+
+// One hop of a node-sharded run, owner side: refresh + pick for a list of distinct nodes at one
+// layer, the picks exported as rows of f ids.  Runs on the second header and leaves the relabel
+// table alone, so it may come between the hops of this rank's own batch.
+struct HopArgs {
+    int32_t layer;
+    int32_t* d_picks;   // [n][f], -1 padded
+};
+
 static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_seeds, gs_mode mode, double gamma,
                              uint32_t step, void* d_workspace, size_t workspace_bytes, cudaStream_t s,
                              gs_block* blocks, const int32_t** d_input_nodes, const int32_t** d_num_input_nodes,
-                             const OutputBuffers* out = nullptr) {
+                             const OutputBuffers* out = nullptr, const HopArgs* hop = nullptr) {
     const gs_graph* g = c->graph;
-    const int L = c->L;
+    const int L = hop ? 1 : c->L;
+    int32_t* const hdr = hop ? c->d_hdr + HDR_OWNER : c->d_hdr;
     int32_t r;
     if (mode == GS_MODE_FCR || mode == GS_MODE_FBL) {
         r = c->W;
@@ -419,7 +440,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         double rr = std::floor(gamma * (double)c->W + 0.5);
         r = rr < 0 ? 0 : (rr > c->W ? c->W : (int32_t)rr);
     }
-    const Bounds b = make_bounds(g->num_nodes, L, c->fanouts, num_seeds);
+    const Bounds b = make_bounds(g->num_nodes, L, hop ? c->fanouts + hop->layer : c->fanouts, num_seeds);
     const WorkspaceLayout w = make_layout(b, g->num_edges);
     if (workspace_bytes < w.total) return fail(GS_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, w.total);
     char* ws = (char*)d_workspace;
@@ -441,17 +462,16 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         frontier = out->input_nodes;
     }
 
-    if (c->serial == 0xFFFFFFFEu) {  // stamp space used up: start over with a clean table
-        GS_CUDA(cudaMemsetAsync(c->d_table, 0xFF, (size_t)g->num_nodes * 8, s));
-        c->serial = 0;
+    uint32_t stamp = 0;
+    if (!hop) {
+        stamp = next_stamp(c, s);
+        if (!stamp) return cuda_fail(cudaGetLastError(), "cudaMemsetAsync");
     }
-    c->serial += 1;
-    const uint32_t stamp = 0xFFFFFFFFu - c->serial;  // newer batches always win the atomicMin
-    GS_CUDA(cudaMemsetAsync(c->d_hdr, 0, HDR_BYTES, s));
+    GS_CUDA(cudaMemsetAsync(hdr, 0, HDR_ONE, s));
 
-    const bool prof = c->prof_events && c->prof_used < c->prof_cap;
+    const bool prof = !hop && c->prof_events && c->prof_used < c->prof_cap;
     for (int k = 0; k < L; ++k) {
-        const int layer = L - 1 - k;
+        const int layer = hop ? hop->layer : L - 1 - k;
         cudaEvent_t* ev = prof ? c->prof_events + ((size_t)c->prof_used * L + k) * PROF_EVENTS_PER_STEP : nullptr;
         if (ev) GS_CUDA(cudaEventRecord(ev[0], s));
         int32_t* blk_indptr = out ? out->indptr[layer] : (int32_t*)(ws + w.blk_indptr[k]);
@@ -461,7 +481,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         C.g = GraphView{g->d_indptr, g->d_indices, g->num_nodes};
         C.seeds = (k == 0) ? d_seeds : nullptr;
         C.frontier = frontier;
-        C.hdr = c->d_hdr;
+        C.hdr = hdr;
         C.k = k;
         C.f = c->fanouts[layer];
         C.n_host = num_seeds;
@@ -469,6 +489,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         C.tile_sums = tiles_a;
         C.table = c->d_table;
         C.stamp = stamp;
+        C.no_stamp = hop ? 1 : 0;
         // a partial refresh runs as scan + finish kernels; FCR (and r = 0) use the fused kernels
         int32_t n_fetch = 0;
         if (mode == GS_MODE_OTF_FETCH) {
@@ -482,7 +503,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         C.split = 1;
         C.W = fbl ? c->fanouts[layer] : (c->theta > c->W ? c->theta : c->W);   // rows above this degree are refreshed
         C.r = n_fetch > 0 ? n_fetch : (fbl ? c->fanouts[layer] : r);
-        C.d_refresh_from = (c->shared && k > 0 && mode != GS_MODE_OTF_FETCH && !fbl) ? c->d_hdr + HDR_N + (k - 1) : nullptr;
+        C.d_refresh_from = (c->shared && k > 0 && mode != GS_MODE_OTF_FETCH && !fbl) ? hdr + HDR_N + (k - 1) : nullptr;   // k = 0 for a single hop
         C.tile_sums2 = (int32_t*)(ws + w.tiles_a2);
         C.item_start = (int32_t*)(ws + w.item_start);
         C.items = (int32_t*)(ws + w.items);
@@ -494,9 +515,9 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         StepParams P = step_params(c, layer, step);
         P.r = r;
         P.frontier = frontier;
-        P.d_n = c->d_hdr + HDR_N + k;
+        P.d_n = hdr + HDR_N + k;
         P.n_host = 0;
-        P.d_refresh_from = (c->shared && k > 0) ? c->d_hdr + HDR_N + (k - 1) : nullptr;
+        P.d_refresh_from = (c->shared && k > 0) ? hdr + HDR_N + (k - 1) : nullptr;
         P.blk_indptr = blk_indptr;
         P.picked = picked;
         P.stamp = stamp;
@@ -504,14 +525,20 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         P.hub_state = (int2*)(ws + w.hub_state);
         P.hub_items = (int32_t*)(ws + w.hub_items);
         P.hub_cand = (unsigned long long*)(ws + w.hub_cand);
-        P.hub_counter = (unsigned long long*)(c->d_hdr + HDR_HUB64 + 2 * k);
+        P.hub_counter = (unsigned long long*)(hdr + HDR_HUB64 + 2 * k);
         P.hub_cap = (int32_t)w.hub_cap;
         P.item_cap = (int32_t)w.item_cap;
-        P.work_counter = c->d_hdr + HDR_WORK + k;
-        P.work_counter2 = c->d_hdr + HDR_WORK2 + k;
-        P.work_counter_scan = c->d_hdr + HDR_WORK3 + k;
+        P.work_counter = hdr + HDR_WORK + k;
+        P.work_counter2 = hdr + HDR_WORK2 + k;
+        P.work_counter_scan = hdr + HDR_WORK3 + k;
         P.do_pick = 1;
         P.init_rows = 0;
+        if (hop) {   // a shared cache refreshes every requested node: the same keys give the same row again
+            P.table = nullptr;
+            P.status = hdr + HDR_STATUS;
+            P.stats = hdr + HDR_STAT_SLOW;
+            P.d_refresh_from = nullptr;
+        }
         if (n_fetch > 0) {           // scan + finish with FETCH keys; the finish kernel emits cache part + fetched part
             P.fetch = 1;
             P.r = n_fetch;
@@ -531,7 +558,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         }
         P.item_start = C.item_start;
         P.items = C.items;
-        P.d_items_total = c->d_hdr + HDR_ITEMS + k;
+        P.d_items_total = hdr + HDR_ITEMS + k;
         P.cand_count = C.cand_count;
         P.cand = (unsigned long long*)(ws + w.cand);
         if (scans) {
@@ -541,9 +568,13 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         if (ev) GS_CUDA(cudaEventRecord(ev[2], s));
         GS_CUDA(launch_finish(P, b.nb[k], s));
         if (ev) GS_CUDA(cudaEventRecord(ev[3], s));
+        if (hop) {
+            GS_CUDA(launch_export_picks(blk_indptr, picked, num_seeds, c->fanouts[layer], hop->d_picks, s));
+            break;
+        }
 
         RelabelParams R{};
-        R.hdr = c->d_hdr;
+        R.hdr = hdr;
         R.k = k;
         R.picked = picked;
         R.aux = aux;
@@ -560,15 +591,15 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         B.max_dst = (int32_t)b.nb[k];
         B.max_src = (int32_t)b.nb[k + 1];
         B.max_edges = (int32_t)b.mb[k];
-        B.d_num_dst = c->d_hdr + HDR_N + k;
-        B.d_num_src = c->d_hdr + HDR_N + k + 1;
-        B.d_num_edges = c->d_hdr + HDR_M + k;
+        B.d_num_dst = hdr + HDR_N + k;
+        B.d_num_src = hdr + HDR_N + k + 1;
+        B.d_num_edges = hdr + HDR_M + k;
         B.d_indptr = blk_indptr;
         B.d_indices = blk_indices;
     }
     if (prof) c->prof_used += 1;
     if (d_input_nodes) *d_input_nodes = frontier;
-    if (d_num_input_nodes) *d_num_input_nodes = c->d_hdr + HDR_N + L;
+    if (d_num_input_nodes) *d_num_input_nodes = hdr + HDR_N + L;
     return GS_OK;
 }
 
@@ -630,9 +661,152 @@ gs_status gs_cache_refresh_all(gs_cache* c, gs_mode mode, double gamma, uint32_t
     }
     if (r == 0) return GS_OK;
     cudaStream_t s = (cudaStream_t)stream;
-    GS_CUDA(cudaMemsetAsync(c->d_hdr, 0, HDR_BYTES, s));
+    GS_CUDA(cudaMemsetAsync(c->d_hdr, 0, HDR_ONE, s));
     GS_CUDA(refresh_every_row(c, r, step, 0, s));
     c->serial = 0;   // the table was reset: stamps start over
+    return GS_OK;
+}
+
+/* ---------------------------------------------------------------- node-sharded sampling */
+
+gs_status gs_shard_bucket(const int32_t* d_nodes, int32_t n, int64_t num_nodes, int32_t world, int32_t* d_sorted,
+                          int32_t* d_slot, int32_t* d_counts, void* stream) {
+    if (world < 1 || world > 64) return fail(GS_ERR_ARG, "world %d outside [1, 64]", world);
+    if (num_nodes < 1 || num_nodes >= ((int64_t)1 << 31)) return fail(GS_ERR_ARG, "num_nodes outside [1, 2^31)");
+    if (n < 0) return fail(GS_ERR_ARG, "n is negative");
+    if (!d_counts || (n > 0 && (!d_nodes || !d_sorted || !d_slot))) return fail(GS_ERR_ARG, "NULL argument");
+    const int32_t rows_per_shard = (int32_t)((num_nodes + world - 1) / world);
+    GS_CUDA(launch_shard_bucket(d_nodes, n, rows_per_shard, world, d_sorted, d_slot, d_counts, d_counts + 2 * world,
+                                (cudaStream_t)stream));
+    return GS_OK;
+}
+
+gs_status gs_shard_workspace_bytes(const gs_graph* g, int32_t fanout, int32_t max_nodes, size_t* bytes) {
+    return gs_workspace_bytes(g, 1, &fanout, max_nodes, bytes);
+}
+
+gs_status gs_shard_sample_rows(gs_cache* c, const int32_t* d_nodes, int32_t n, int32_t layer, gs_mode mode, double rate,
+                               uint32_t step, void* d_workspace, size_t workspace_bytes, void* stream, int32_t* d_picks) {
+    if (!c) return fail(GS_ERR_ARG, "cache is NULL");
+    if (layer < 0 || layer >= c->L) return fail(GS_ERR_ARG, "layer %d outside [0, %d)", layer, c->L);
+    if (n == 0) return GS_OK;
+    if (!d_picks) return fail(GS_ERR_ARG, "d_picks is NULL");
+    gs_block unused[GS_MAX_HOPS];
+    gs_status st = check_batch_args(c, d_nodes, n, mode, rate, step, d_workspace, unused);
+    if (st != GS_OK) return st;
+    if (!aligned(d_nodes, 4) || !aligned(d_picks, 4)) return fail(GS_ERR_ALIGN, "node and pick arrays must be 4-byte aligned");
+    HopArgs hop{layer, d_picks};
+    return sample_impl(c, d_nodes, n, mode, rate, step, d_workspace, workspace_bytes, (cudaStream_t)stream, unused, nullptr,
+                       nullptr, nullptr, &hop);
+}
+
+gs_status gs_shard_status(gs_cache* c, void* stream) {
+    if (!c) return fail(GS_ERR_ARG, "cache is NULL");
+    cudaStream_t s = (cudaStream_t)stream;
+    GS_CUDA(cudaMemcpyAsync(c->h_pinned, c->d_hdr + HDR_OWNER + HDR_STATUS, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    GS_CUDA(cudaStreamSynchronize(s));
+    const int status = c->h_pinned[0];
+    if (status == GS_ERR_RANGE) return fail(GS_ERR_RANGE, "a requested node id is outside [0, num_nodes)");
+    if (status != 0) return fail(GS_ERR_CUDA, "unexpected device status %d", status);
+    return GS_OK;
+}
+
+gs_status gs_shard_extend(gs_cache* c, int32_t k, const int32_t* d_seeds, int32_t num_seeds, const int32_t* d_reply,
+                          const int32_t* d_slot, void* d_workspace, size_t workspace_bytes, void* stream, gs_block* block,
+                          const int32_t** d_frontier) {
+    if (!c) return fail(GS_ERR_ARG, "cache is NULL");
+    if (k < 0 || k >= c->L) return fail(GS_ERR_ARG, "hop %d outside [0, %d)", k, c->L);
+    if (!d_reply || !block) return fail(GS_ERR_ARG, "NULL argument");
+    if (!d_workspace || !aligned(d_workspace, 256)) return fail(GS_ERR_ALIGN, "d_workspace must be 256-byte aligned");
+    const gs_graph* g = c->graph;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (k == 0) {
+        if (!d_seeds) return fail(GS_ERR_ARG, "seeds is NULL");
+        if (num_seeds < 1 || (int64_t)num_seeds > g->num_nodes) return fail(GS_ERR_ARG, "num_seeds outside [1, num_nodes]");
+        const uint32_t stamp = next_stamp(c, s);
+        if (!stamp) return cuda_fail(cudaGetLastError(), "cudaMemsetAsync");
+        c->shard_stamp = stamp;
+        c->shard_seeds = num_seeds;
+        GS_CUDA(cudaMemsetAsync(c->d_hdr, 0, HDR_ONE, s));
+    } else if (c->shard_seeds < 1) {
+        return fail(GS_ERR_ARG, "hop %d before hop 0", k);
+    }
+    const int L = c->L, layer = L - 1 - k;
+    const Bounds b = make_bounds(g->num_nodes, L, c->fanouts, c->shard_seeds);
+    const WorkspaceLayout w = make_layout(b, g->num_edges);
+    if (workspace_bytes < w.total) return fail(GS_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, w.total);
+    char* ws = (char*)d_workspace;
+    int32_t* frontier = (int32_t*)(ws + w.frontier);
+    int32_t* picked = (int32_t*)(ws + w.picked);
+    int32_t* blk_indptr = (int32_t*)(ws + w.blk_indptr[k]);
+    int32_t* blk_indices = (int32_t*)(ws + w.blk_indices[k]);
+
+    CountParams C{};
+    C.g = GraphView{g->d_indptr, g->d_indices, g->num_nodes};
+    C.seeds = (k == 0) ? d_seeds : nullptr;
+    C.frontier = frontier;
+    C.hdr = c->d_hdr;
+    C.k = k;
+    C.f = c->fanouts[layer];
+    C.n_host = c->shard_seeds;
+    C.blk_indptr = blk_indptr;
+    C.tile_sums = (int32_t*)(ws + w.tiles_a);
+    C.table = c->d_table;
+    C.stamp = c->shard_stamp;
+    C.split = 1;                 // lays out (empty) scan item lists; nothing is scanned on this side
+    C.W = c->W;
+    C.r = 0;
+    C.tile_sums2 = (int32_t*)(ws + w.tiles_a2);
+    C.item_start = (int32_t*)(ws + w.item_start);
+    C.items = (int32_t*)(ws + w.items);
+    C.cand_count = (int32_t*)(ws + w.cand_count);
+    C.scan_item_cap = w.scan_item_cap;
+    C.reply = d_reply;
+    C.slot = d_slot;
+    GS_CUDA(launch_row_counts(C, b.nb[k], s));
+    GS_CUDA(launch_import_picks(c->d_hdr, k, (int32_t)b.nb[k], C.f, d_reply, d_slot, blk_indptr, picked, c->d_table,
+                                c->shard_stamp, g->num_nodes, c->d_hdr + HDR_STATUS, s));
+    RelabelParams R{};
+    R.hdr = c->d_hdr;
+    R.k = k;
+    R.picked = picked;
+    R.aux = (int32_t*)(ws + w.aux);
+    R.tile_sums = (int32_t*)(ws + w.tiles_e);
+    R.frontier = frontier;
+    R.local = blk_indices;
+    R.table = c->d_table;
+    R.stamp = c->shard_stamp;
+    R.n_cap = b.nb[k + 1];
+    GS_CUDA(launch_relabel(R, b.mb[k], s));
+
+    gs_block& B = *block;
+    B.max_dst = (int32_t)b.nb[k];
+    B.max_src = (int32_t)b.nb[k + 1];
+    B.max_edges = (int32_t)b.mb[k];
+    B.d_num_dst = c->d_hdr + HDR_N + k;
+    B.d_num_src = c->d_hdr + HDR_N + k + 1;
+    B.d_num_edges = c->d_hdr + HDR_M + k;
+    B.d_indptr = blk_indptr;
+    B.d_indices = blk_indices;
+    if (d_frontier) *d_frontier = frontier;
+    return GS_OK;
+}
+
+gs_status gs_gather_rows(const void* d_src, gs_dtype dtype, int32_t row_elems, int64_t src_ld, int64_t first_row,
+                         const int32_t* d_ids, const int32_t* d_count_or_null, int32_t count_bound, void* d_out,
+                         int64_t out_ld, void* stream) {
+    if (dtype != GS_F32 && dtype != GS_BF16) return fail(GS_ERR_ARG, "unknown dtype %d", (int)dtype);
+    const int64_t eb = dtype == GS_BF16 ? 2 : 4;
+    if (count_bound < 0) return fail(GS_ERR_ARG, "count_bound is negative");
+    if (count_bound == 0) return GS_OK;
+    if (!d_src || !d_ids || !d_out) return fail(GS_ERR_ARG, "NULL argument");
+    if (row_elems < 1 || src_ld < row_elems || out_ld < row_elems) return fail(GS_ERR_ARG, "bad row size or pitch");
+    if (first_row < 0) return fail(GS_ERR_ARG, "first_row is negative");
+    if (!aligned(d_src, (size_t)eb) || !aligned(d_out, (size_t)eb) || !aligned(d_ids, 4)) return fail(GS_ERR_ALIGN, "misaligned argument");
+    // ids are global; the source holds rows first_row, first_row + 1, ...: address row 0 where it would be
+    const uintptr_t base = (uintptr_t)d_src - (uintptr_t)(first_row * src_ld * eb);
+    GS_CUDA(launch_gather((const void*)base, src_ld * eb, (int64_t)row_elems * eb, d_ids, d_count_or_null, count_bound, d_out,
+                          out_ld * eb, (cudaStream_t)stream));
     return GS_OK;
 }
 

@@ -25,9 +25,11 @@ constexpr int HDR_STAT_REFRESHED = HDR_STAT_QUEUED + 1;   // nodes refreshed
 constexpr int HDR_STAT_QUADS = HDR_STAT_REFRESHED + 1;    // Philox blocks the scan kernel has to evaluate
 constexpr int HDR_WORDS = HDR_STAT_QUADS + 1;
 constexpr int HDR_HUB64 = 128;                   // 64-bit (hubs << 32 | chunks) counters, one per launch
-constexpr size_t HDR_BYTES = 1024;
+constexpr size_t HDR_ONE = 1024;                 // bytes of one header
+constexpr int HDR_OWNER = (int)(HDR_ONE / 4);    // word offset of the second header: owner-side hops of a sharded run
+constexpr size_t HDR_BYTES = 2 * HDR_ONE;        // both headers, at the start of the cache storage
 static_assert(HDR_WORDS <= HDR_HUB64, "header words overlap the 64-bit counters");
-static_assert((HDR_HUB64 + 2 * GS_MAX_HOPS) * 4 <= HDR_BYTES, "header too small");
+static_assert((HDR_HUB64 + 2 * GS_MAX_HOPS) * 4 <= HDR_ONE, "header too small");
 
 #ifndef GS_SCAN_CHUNK_QUADS
 #define GS_SCAN_CHUNK_QUADS 1024
@@ -137,7 +139,7 @@ struct StepParams {
     const int32_t* d_refresh_from;  // device scalar: positions below it are not refreshed; NULL -> 0
     const int32_t* blk_indptr;   // final offsets of each node's picks
     int32_t* picked;             // global ids of the picks
-    unsigned long long* table;   // relabel table, (stamp << 32) | position
+    unsigned long long* table;   // relabel table, (stamp << 32) | position; NULL: picks are not registered (owner side of a sharded run)
     uint32_t stamp;
     // hubs: nodes whose scan is split into chunks over many warps
     int2* hub_entry;                 // (frontier position, first chunk)
@@ -185,6 +187,10 @@ struct CountParams {
     int32_t* items;
     int32_t* cand_count;
     int64_t scan_item_cap;
+    // sharded sampling
+    int32_t no_stamp;        // owner side: step 0 neither checks duplicates nor touches the relabel table
+    const int32_t* reply;    // requester side: picks by row [rows][f], -1 padded; row lengths come from here, not from degrees
+    const int32_t* slot;     // requester side: row of `reply` that belongs to frontier position p
 };
 
 struct RelabelParams {
@@ -233,6 +239,13 @@ cudaError_t launch_gather(const void* src, int64_t src_ld_bytes, int64_t row_byt
                           cudaStream_t s);
 cudaError_t launch_read_rows(const int32_t* slots, const int32_t* row_index, int32_t pitch, int32_t W,
                              const int32_t* nodes, int32_t n, int32_t* out, cudaStream_t s);
+cudaError_t launch_shard_bucket(const int32_t* nodes, int32_t n, int32_t rows_per_shard, int32_t world, int32_t* sorted,
+                                int32_t* slot, int32_t* counts_and_scratch, int32_t* status, cudaStream_t s);
+cudaError_t launch_export_picks(const int32_t* blk_indptr, const int32_t* picked, int32_t n, int32_t f, int32_t* out,
+                                cudaStream_t s);
+cudaError_t launch_import_picks(const int32_t* hdr, int32_t k, int32_t n_bound, int32_t f, const int32_t* reply,
+                                const int32_t* slot, const int32_t* blk_indptr, int32_t* picked, unsigned long long* table,
+                                uint32_t stamp, int64_t num_nodes, int32_t* status, cudaStream_t s);
 cudaError_t launch_build_row_index(const GraphView& g, int32_t theta, int32_t* row_index, int32_t* tile_sums,
                                    int32_t* d_dense_rows, cudaStream_t s);
 

@@ -356,6 +356,11 @@ __device__ __forceinline__ uint32_t evict_mask_for(const StepParams& P, int32_t 
     return warp_smallest_k(word_of(o, lane & 3), wmask, P.r, lane);
 }
 
+// First half of S3, fused into the pick: the pick at edge position e claims its id in the relabel table.
+__device__ __forceinline__ void register_pick(const StepParams& P, int32_t id, uint32_t n_base, int e) {
+    if (P.table) atomicMin(P.table + id, ((unsigned long long)P.stamp << 32) | (n_base + (uint32_t)e));
+}
+
 // S2: choose and emit the picks of one node; registers their positions in the relabel table.
 __device__ __forceinline__ void warp_pick(const StepParams& P, int32_t v, uint32_t deg, int e_base, uint32_t n_base,
                                           int32_t slot, int lane) {
@@ -369,7 +374,7 @@ __device__ __forceinline__ void warp_pick(const StepParams& P, int32_t v, uint32
     if ((pm >> lane) & 1u) {
         const int e = e_base + __popc(pm & lanemask_lt());
         P.picked[e] = slot;
-        atomicMin(P.table + slot, ((unsigned long long)P.stamp << 32) | (n_base + (uint32_t)e));
+        register_pick(P, slot, n_base, e);
     }
 }
 
@@ -385,7 +390,7 @@ __device__ __forceinline__ void warp_emit_sorted(const StepParams& P, int cnt, i
     if (lane < cnt) {
         const int e = e_base + rank;
         P.picked[e] = id;
-        atomicMin(P.table + id, ((unsigned long long)P.stamp << 32) | (n_base + (uint32_t)e));
+        register_pick(P, id, n_base, e);
     }
 }
 
@@ -923,7 +928,7 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
                     const int32_t id = __ldg(P.g.indices + rs + lane);
                     const int e = e_base + lane;
                     P.picked[e] = id;
-                    atomicMin(P.table + id, ((unsigned long long)P.stamp << 32) | (n_base + (uint32_t)e));
+                    register_pick(P, id, n_base, e);
                 }
                 continue;
             }
@@ -1043,7 +1048,7 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
                     else if ((evict >> lane) & 1u) e = e_base + (P.f - P.r) + __popc(evict & lt);
                     if (e >= 0) {
                         P.picked[e] = slot;
-                        atomicMin(P.table + slot, ((unsigned long long)P.stamp << 32) | (n_base + (uint32_t)e));
+                        register_pick(P, slot, n_base, e);
                     }
                     continue;
                 }
@@ -1056,7 +1061,7 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
             if ((pm >> lane) & 1u) {
                 const int e = e_base + __popc(pm & lanemask_lt());
                 P.picked[e] = slot;
-                atomicMin(P.table + slot, ((unsigned long long)P.stamp << 32) | (n_base + (uint32_t)e));
+                register_pick(P, slot, n_base, e);
             }
         }
     }

@@ -54,14 +54,20 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
                 v = -1;
             } else {
                 P.frontier[p] = v;
-                const unsigned long long mine = ((unsigned long long)P.stamp << 32) | (unsigned)p;
-                const unsigned long long old = atomicMin(P.table + v, mine);
-                if ((uint32_t)(old >> 32) == P.stamp) raise_status(status, GS_ERR_DUP_SEED);
+                if (!P.no_stamp) {
+                    const unsigned long long mine = ((unsigned long long)P.stamp << 32) | (unsigned)p;
+                    const unsigned long long old = atomicMin(P.table + v, mine);
+                    if ((uint32_t)(old >> 32) == P.stamp) raise_status(status, GS_ERR_DUP_SEED);
+                }
             }
         } else {
             v = P.frontier[p];
         }
-        if (v >= 0) {
+        if (v >= 0 && P.reply) {
+            // sharded run, requester side: the owners have sampled; a row's picks are the non-negative prefix
+            const int32_t* row = P.reply + (int64_t)(P.slot ? P.slot[p] : p) * P.f;
+            while (c < P.f && __ldg(row + c) >= 0) ++c;
+        } else if (v >= 0) {
             const int64_t deg = P.g.indptr[v + 1] - P.g.indptr[v];
             c = deg < (int64_t)P.f ? (int)deg : P.f;
             if (P.split && P.r > 0 && deg > (int64_t)SMALL_DEGREE && deg > (int64_t)P.W && p >= refresh_from) {

@@ -1,0 +1,192 @@
+"""Node-sharded sampling over several GPUs: one exchange per hop.
+
+Nodes are partitioned by id range; rank o owns the CSR rows, cache rows and feature rows of
+``[o*S, (o+1)*S)``, ``S = ceil(N / world)``.  Every random choice of the sampler is keyed by
+(seed, node, item, step), so the picks an owner computes for a node are the picks a single
+device would compute, and a sharded run equals one sampler (with the dense/sparse split the
+shards' caches use) that takes the ranks' batches of a step one after the other.
+
+One hop of a rank's batch (sampling step k, layer L-1-k):
+
+    bucket frontier_k by owner  ->  all-to-all(v) ids  ->  owners refresh + pick
+                                <-  all-to-all(v) rows of f picks  <-
+    dedup + relabel + block CSR
+
+and after the last hop one more round trip for the feature rows.  The per-rank phases live in
+:class:`ShardRank`; two drivers run them: :func:`sample_batch` (one process per GPU, the
+exchange is ``torch.distributed.all_to_all_single`` over NCCL / NVLink) and
+:func:`sample_batch_local` (all ranks in one process, the exchange is a copy; used to check a
+multi-rank run on one GPU - the ranks' kernels run one after the other, nothing waits).
+This module only moves arguments: every step of the path runs in the library's kernels
+(``ops`` is the binding; tests may pass a stand-in with the same functions).
+"""
+from __future__ import annotations
+
+import torch
+import torch.distributed as dist
+
+
+def rows_per_shard(num_nodes: int, world: int) -> int:
+    return (num_nodes + world - 1) // world
+
+
+def shard_range(num_nodes: int, rank: int, world: int):
+    s = rows_per_shard(num_nodes, world)
+    return min(num_nodes, rank * s), min(num_nodes, (rank + 1) * s)
+
+
+def shard_csr(indptr: torch.Tensor, indices: torch.Tensor, rank: int, world: int):
+    """The shard's CSR: full-length indptr in which only the owned rows are non-empty, and the
+    owned rows' neighbour ids (global)."""
+    n = indptr.numel() - 1
+    lo, hi = shard_range(n, rank, world)
+    e0, e1 = int(indptr[lo].item()), int(indptr[hi].item())
+    ip = torch.empty_like(indptr)
+    ip[: lo + 1] = 0
+    ip[lo:hi + 1] = indptr[lo:hi + 1] - e0
+    ip[hi + 1:] = e1 - e0
+    return ip.contiguous(), indices[e0:e1].contiguous()
+
+
+class ShardRank:
+    """One rank of a sharded run: its shard's graph, split cache, feature rows and workspaces."""
+
+    def __init__(self, ops, rank, world, indptr_shard, indices_shard, features_shard, fanouts, cache_width, seed,
+                 shared, theta, max_seeds, max_requests):
+        self.ops, self.rank, self.world = ops, rank, world
+        self.num_nodes = indptr_shard.numel() - 1
+        self.first_row = shard_range(self.num_nodes, rank, world)[0]
+        self.fanouts, self.L = list(fanouts), len(fanouts)
+        self.features = features_shard
+        self.graph = ops.gs_graph_create(indptr_shard, indices_shard, None)
+        self.cache = ops.gs_cache_init_split(self.graph, fanouts, cache_width, seed, shared, theta)
+        dev = indptr_shard.device
+        self.ws = torch.empty(ops.gs_workspace_bytes(self.graph, fanouts, max_seeds), dtype=torch.uint8, device=dev)
+        self.max_requests = max_requests
+        self.ws_owner = torch.empty(ops.gs_shard_workspace_bytes(self.graph, max(fanouts), max_requests),
+                                    dtype=torch.uint8, device=dev)
+        self.blocks = [None] * self.L
+        self.n = []
+
+    # ---- requester side
+    def begin(self, seeds):
+        self.seeds = seeds
+        self.frontier, self.n = seeds, [seeds.numel()]
+        self.blocks = [None] * self.L
+
+    def requests(self, nodes):
+        """Bucket `nodes` by owner -> (ids grouped by owner, group sizes as a list); remembers the slots."""
+        sorted_ids, self.slot, counts = self.ops.gs_shard_bucket(nodes, self.num_nodes, self.world)
+        c = counts.cpu().tolist()                      # the all-to-all needs the sizes on the host
+        if c[2 * self.world] != 0:
+            raise ValueError("a node id is outside [0, num_nodes)")
+        return sorted_ids, c[: self.world]
+
+    def hop_requests(self, k):
+        return self.requests(self.frontier[: self.n[k]])
+
+    def hop_finish(self, k, reply):
+        """`reply`: [n_k, f] rows of picks in the order the requests were sent."""
+        block, frontier = self.ops.gs_shard_extend(self.cache, k, self.seeds if k == 0 else None, reply, self.slot, self.ws)
+        n, m = self.ops.gs_batch_counts(self.cache)   # n_{k+1} sizes the next hop's exchange
+        self.blocks[self.L - 1 - k] = block
+        self.frontier, self.n, self.m = frontier, n[: k + 2], m
+        return n[k + 1]
+
+    def feature_requests(self):
+        return self.requests(self.frontier[: self.n[self.L]])
+
+    def feature_finish(self, rows):
+        out = torch.empty((self.n[self.L], rows.shape[1]), dtype=rows.dtype, device=rows.device)
+        return self.ops.gs_gather_rows(rows, self.slot, out)
+
+    # ---- owner side
+    def hop_serve(self, layer, lists, mode, rate, step):
+        """One list of distinct nodes per requester -> one [len, f] tensor of picks each."""
+        out = []
+        for nodes in lists:
+            if nodes.numel() > self.max_requests:
+                raise ValueError("a request list of %d nodes exceeds max_requests %d" % (nodes.numel(), self.max_requests))
+            out.append(self.ops.gs_shard_sample_rows(self.cache, nodes.contiguous(), layer, mode, rate, step, self.ws_owner))
+        self.ops.gs_shard_status(self.cache)
+        return out
+
+    def feature_serve(self, lists):
+        out = []
+        for nodes in lists:
+            rows = torch.empty((nodes.numel(), self.features.shape[1]), dtype=self.features.dtype, device=self.features.device)
+            out.append(self.ops.gs_gather_rows(self.features, nodes.contiguous(), rows, first_row=self.first_row))
+        return out
+
+
+def _split(t, counts):
+    return list(torch.split(t, counts)) if t.numel() else [t[:0] for _ in counts]
+
+
+# --------------------------------------------------------------------------- all ranks in one process
+def sample_batch_local(ranks, seeds_per_rank, mode, rate, step, features=True):
+    """Runs one batch per rank, phase by phase; the exchange is a local copy.  Returns, per rank,
+    (blocks by layer, frontier tensor, n list, m list, feature rows or None)."""
+    R = len(ranks)
+    L = ranks[0].L
+    for r, seeds in zip(ranks, seeds_per_rank):
+        r.begin(seeds)
+
+    def round_trip(req, serve):
+        sent = [_split(ids, counts) for ids, counts in req]                 # sent[r][o]
+        served = [serve(ranks[o], [sent[r][o] for r in range(R)]) for o in range(R)]   # served[o][r]
+        return [torch.cat([served[o][r] for o in range(R)]) for r in range(R)]
+
+    for k in range(L):
+        layer = L - 1 - k
+        replies = round_trip([r.hop_requests(k) for r in ranks],
+                             lambda owner, lists: owner.hop_serve(layer, lists, mode, rate, step))
+        for r, reply in zip(ranks, replies):
+            r.hop_finish(k, reply.contiguous())
+    feats = [None] * R
+    if features:
+        rows = round_trip([r.feature_requests() for r in ranks], lambda owner, lists: owner.feature_serve(lists))
+        feats = [r.feature_finish(x.contiguous()) for r, x in zip(ranks, rows)]
+    return [(r.blocks, r.frontier, r.n, r.m, f) for r, f in zip(ranks, feats)]
+
+
+# --------------------------------------------------------------------------- one process per rank
+def _all_to_all_v(send, send_counts, width, group):
+    """send: [sum(send_counts), *width] grouped by destination -> (received tensor, receive counts)."""
+    dev = send.device
+    sc = torch.tensor(send_counts, dtype=torch.int64, device=dev)
+    rc = torch.empty_like(sc)
+    dist.all_to_all_single(rc, sc, group=group)
+    recv_counts = rc.cpu().tolist()
+    recv = torch.empty((sum(recv_counts),) + tuple(width), dtype=send.dtype, device=dev)
+    dist.all_to_all_single(recv, send.contiguous(), recv_counts, send_counts, group=group)
+    return recv, recv_counts
+
+
+def sample_batch(rank_state: ShardRank, seeds, mode, rate, step, features=True, group=None):
+    """This rank's part of a sharded batch (every rank of `group` calls it with the same mode, rate
+    and step).  Returns (blocks by layer, frontier tensor, n list, m list, feature rows or None)."""
+    me = rank_state
+    L = me.L
+    me.begin(seeds)
+
+    def round_trip(ids, counts, serve, width, dtype):
+        recv, recv_counts = _all_to_all_v(ids, counts, (), group)
+        served = serve(_split(recv, recv_counts))
+        back = torch.cat(served) if served else torch.empty((0,) + width, dtype=dtype, device=ids.device)
+        reply = torch.empty((ids.numel(),) + width, dtype=dtype, device=ids.device)
+        dist.all_to_all_single(reply, back.contiguous(), counts, recv_counts, group=group)
+        return reply
+
+    for k in range(L):
+        layer = L - 1 - k
+        ids, counts = me.hop_requests(k)
+        reply = round_trip(ids, counts, lambda lists: me.hop_serve(layer, lists, mode, rate, step),
+                           (me.fanouts[layer],), torch.int32)
+        me.hop_finish(k, reply)
+    feats = None
+    if features:
+        ids, counts = me.feature_requests()
+        rows = round_trip(ids, counts, me.feature_serve, (me.features.shape[1],), me.features.dtype)
+        feats = me.feature_finish(rows)
+    return me.blocks, me.frontier, me.n, me.m, feats

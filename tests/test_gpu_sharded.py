@@ -1,0 +1,124 @@
+"""Node-sharded sampling on one GPU (all ranks in one process, run phase by phase) vs the CPU oracle.
+
+A sharded run must equal ONE sampler with the shards' dense/sparse split that takes the ranks'
+batches of a step one after the other: every choice is keyed by (seed, node, item, step)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from workloads import batch_seeds, build_features, build_graph, get_config, seed_permutation
+
+pytestmark = pytest.mark.gpu
+
+MODES = {"fcr": (0, oracle.MODE_FCR), "otf": (1, oracle.MODE_OTF), "fbl": (2, oracle.MODE_FBL),
+         "fetch": (3, oracle.MODE_OTF_FETCH)}
+
+
+class Setup:
+    def __init__(self, name, world, theta, seed=5, B=None):
+        import paper_2406_17918_b200 as gs
+        from paper_2406_17918_b200 import sharded
+        self.gs, self.sharded = gs, sharded
+        cfg = self.cfg = get_config(name)
+        g = build_graph(cfg)
+        self.indptr, self.indices = g.indptr.numpy(), g.indices.numpy()
+        self.deg = self.indptr[1:] - self.indptr[:-1]
+        self.X = build_features(cfg)
+        self.perm = seed_permutation(cfg)
+        self.world, self.theta = world, theta
+        self.B = B or cfg["batch"]
+        N = cfg["num_nodes"]
+        self.ranks = []
+        for r in range(world):
+            ip, idx = sharded.shard_csr(g.indptr, g.indices, r, world)
+            lo, hi = sharded.shard_range(N, r, world)
+            self.ranks.append(sharded.ShardRank(gs, r, world, ip.cuda(), idx.cuda(), self.X[lo:hi].cuda().contiguous(),
+                                                cfg["fanouts"], cfg["cache_width"], seed, cfg["shared"], theta,
+                                                max_seeds=self.B, max_requests=min(N, self.B * 400)))
+        self.O = oracle.Sampler(self.indptr, self.indices, cfg["fanouts"], cfg["cache_width"], seed, cfg["shared"])
+        self.O.set_theta(theta)
+
+    def step(self, mode, rate, t, features=True):
+        gm, om = MODES[mode]
+        L = len(self.cfg["fanouts"])
+        seeds = [batch_seeds(self.perm, t, self.B, r, self.world) for r in range(self.world)]
+        res = self.sharded.sample_batch_local(self.ranks, [s.cuda() for s in seeds], gm, rate, t, features=features)
+        for r in range(self.world):
+            blocks, frontier, n, m, feats = res[r]
+            fr_o, n_o, blocks_o = self.O.sample_batch(seeds[r].numpy(), om, rate, t)
+            assert n == n_o, (r, n, n_o)
+            assert np.array_equal(frontier[: n[L]].cpu().numpy(), fr_o)
+            for layer in range(L):
+                k = L - 1 - layer
+                assert m[layer] == blocks_o[layer].num_edges
+                assert np.array_equal(blocks[layer].indptr(n[k]).cpu().numpy(), blocks_o[layer].indptr)
+                assert np.array_equal(blocks[layer].indices(m[layer]).cpu().numpy(), blocks_o[layer].indices)
+            if features:
+                want = self.X[torch.from_numpy(fr_o.astype(np.int64))]
+                assert torch.equal(feats.cpu().view(torch.int32 if want.element_size() == 4 else torch.int16),
+                                   want.view(torch.int32 if want.element_size() == 4 else torch.int16))
+        return res
+
+    def check_rows(self, sample=None):
+        """Cache rows of the dense nodes, read from their owners."""
+        N = self.cfg["num_nodes"]
+        nodes = np.nonzero(self.deg > self.theta)[0].astype(np.int32)
+        if sample and len(nodes) > sample:
+            nodes = np.sort(np.random.default_rng(1).choice(nodes, sample, replace=False))
+        S = self.sharded.rows_per_shard(N, self.world)
+        for layer in range(1 if self.cfg["shared"] else len(self.cfg["fanouts"])):
+            want = self.O.cache_rows(layer, nodes)
+            for r in range(self.world):
+                mine = nodes[(nodes // S) == r]
+                if len(mine) == 0:
+                    continue
+                got = self.gs.gs_cache_read_rows(self.ranks[r].cache, layer, torch.from_numpy(mine).cuda()).cpu().numpy()
+                assert np.array_equal(got, want[(nodes // S) == r]), (layer, r)
+
+
+@pytest.mark.parametrize("world", [1, 2, 3])
+def test_sharded_tiny_all_modes(world):
+    s = Setup("tiny", world, theta=12)
+    t = 1
+    for mode, rate in [("otf", 0.25), ("otf", 0.25), ("fcr", 0.0), ("fetch", 0.5), ("fbl", 0.0), ("otf", 0.0), ("otf", 1.0)]:
+        s.step(mode, rate, t)
+        t += 1
+    s.check_rows()
+
+
+def test_sharded_mid_and_shared_cache():
+    s = Setup("mid", 4, theta=24, B=512)
+    for t in (1, 2):
+        s.step("otf", 0.3, t)
+    s.step("fcr", 0.0, 3, features=False)
+    s.check_rows(sample=4000)
+    s = Setup("shared", 2, theta=32, B=1024)
+    for t in (1, 2):
+        s.step("otf", 0.3, t)
+    s.check_rows(sample=4000)
+
+
+def test_bucket_and_gather_rows_primitives():
+    import paper_2406_17918_b200 as gs
+    rng = np.random.default_rng(3)
+    N, world = 100003, 7
+    nodes = torch.from_numpy(rng.choice(N, 50001, replace=False).astype(np.int32)).cuda()
+    sorted_ids, slot, counts = gs.gs_shard_bucket(nodes, N, world)
+    S = (N + world - 1) // world
+    c = counts.cpu().numpy()
+    owner = (nodes.cpu().numpy() // S)
+    assert c[2 * world] == 0 and np.array_equal(c[:world], np.bincount(owner, minlength=world))
+    so = sorted_ids.cpu().numpy()
+    assert np.array_equal(so // S, np.sort(owner))                              # grouped by owner
+    assert np.array_equal(so[slot.cpu().numpy()], nodes.cpu().numpy())          # slot ties each id to its place
+    assert len(np.unique(slot.cpu().numpy())) == nodes.numel()
+    bad = nodes.clone()
+    bad[17] = N + 5 * S
+    assert gs.gs_shard_bucket(bad, N, world)[2].cpu().numpy()[2 * world] == 3   # GS_ERR_RANGE
+    # rows of a shard addressed by global ids
+    X = torch.randn(1000, 24, device="cuda").to(torch.bfloat16)
+    ids = torch.from_numpy(rng.integers(400, 700, 333).astype(np.int32)).cuda()
+    out = torch.empty((333, 24), dtype=torch.bfloat16, device="cuda")
+    gs.gs_gather_rows(X[400:700], ids, out, first_row=400)
+    assert torch.equal(out, X[ids.long()])
