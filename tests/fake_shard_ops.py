@@ -1,0 +1,116 @@
+"""A CPU stand-in for the binding's sharded entry points, built from the oracle's per-node
+primitives: lets the multi-rank drivers of `paper_2406_17918_b200.sharded` run under gloo
+without a GPU.  Test infrastructure only."""
+import numpy as np
+import torch
+
+import oracle
+
+GS_MODE_FCR, GS_MODE_OTF, GS_MODE_FBL, GS_MODE_OTF_FETCH = 0, 1, 2, 3
+_OM = {0: oracle.MODE_FCR, 1: oracle.MODE_OTF, 2: oracle.MODE_FBL, 3: oracle.MODE_OTF_FETCH}
+
+
+class _Graph:
+    def __init__(self, indptr, indices):
+        self.indptr, self.indices = indptr.numpy().copy(), indices.numpy().copy()
+        self.deg = self.indptr[1:] - self.indptr[:-1]
+
+
+class _Block:
+    def __init__(self, indptr, indices):
+        self._indptr, self._indices = indptr, indices
+
+    def indptr(self, n):
+        return torch.from_numpy(self._indptr[: n + 1])
+
+    def indices(self, m):
+        return torch.from_numpy(self._indices[:m])
+
+
+class _Cache:
+    pass
+
+
+def gs_graph_create(indptr, indices, features):
+    return _Graph(indptr, indices)
+
+
+def gs_cache_init_split(graph, fanouts, W, seed, shared, theta):
+    c = _Cache()
+    c.graph, c.fanouts, c.W, c.theta = graph, list(fanouts), W, theta
+    c.O = oracle.Sampler(graph.indptr, graph.indices, fanouts, W, seed, shared)
+    c.O.set_theta(theta)
+    return c
+
+
+def gs_workspace_bytes(graph, fanouts, max_seeds):
+    return 256
+
+
+def gs_shard_workspace_bytes(graph, fanout, max_nodes):
+    return 256
+
+
+def gs_shard_bucket(nodes, num_nodes, world):
+    v = nodes.numpy()
+    S = (num_nodes + world - 1) // world
+    owner = v // S
+    order = np.argsort(owner, kind="stable")
+    slot = np.empty(len(v), dtype=np.int32)
+    slot[order] = np.arange(len(v), dtype=np.int32)
+    counts = np.zeros(2 * world + 1, dtype=np.int32)
+    counts[:world] = np.bincount(owner, minlength=world)
+    return torch.from_numpy(v[order].copy()), torch.from_numpy(slot), torch.from_numpy(counts)
+
+
+def gs_shard_sample_rows(cache, nodes, layer, mode, rate, step, ws):
+    f = cache.fanouts[layer]
+    out = np.full((nodes.numel(), f), -1, dtype=np.int32)
+    O, om = cache.O, _OM[mode]
+    for i, v in enumerate(nodes.numpy().tolist()):
+        if om == oracle.MODE_FBL or cache.graph.deg[v] <= cache.theta:
+            row = O.fbl_node(layer, v, step)
+        elif om == oracle.MODE_OTF_FETCH:
+            row = O.fetch_node(layer, v, step, oracle.fetch_count(rate, f))
+        else:
+            O.refresh_node(layer, v, step, oracle.refresh_count(om, rate, cache.W))
+            row = O.pick_node(layer, v, step)
+        out[i, : len(row)] = row
+    return torch.from_numpy(out)
+
+
+def gs_shard_status(cache):
+    pass
+
+
+def gs_shard_extend(cache, k, seeds, reply, slot, ws):
+    L = len(cache.fanouts)
+    if k == 0:
+        cache.frontier = seeds.numpy().tolist()
+        cache.pos = {v: i for i, v in enumerate(cache.frontier)}
+        cache.n, cache.m = [len(cache.frontier)], [0] * L
+    rows, sl = reply.numpy(), slot.numpy()
+    n_k = cache.n[k]
+    indptr, local = [0], []
+    for p in range(n_k):
+        for u in rows[sl[p]]:
+            if u < 0:
+                break
+            if u not in cache.pos:
+                cache.pos[int(u)] = len(cache.frontier)
+                cache.frontier.append(int(u))
+            local.append(cache.pos[int(u)])
+        indptr.append(len(local))
+    cache.n.append(len(cache.frontier))
+    cache.m[L - 1 - k] = len(local)
+    return _Block(np.array(indptr, dtype=np.int32), np.array(local, dtype=np.int32)), \
+        torch.tensor(cache.frontier, dtype=torch.int32)
+
+
+def gs_batch_counts(cache):
+    return list(cache.n), list(cache.m)
+
+
+def gs_gather_rows(src, ids, out, first_row=0):
+    out.copy_(src[ids.long() - first_row])
+    return out
