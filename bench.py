@@ -191,6 +191,10 @@ def main():
                     help="T: the schedule of Algorithms 2/3 as written - every T-th batch refreshes the whole cache "
                          "(--mode otf/fcr, --rate), every batch only samples from the cache; no CPU baseline "
                          "(the oracle's whole-cache refresh of this graph takes hours)")
+    ap.add_argument("--sharded", action="store_true",
+                    help="node-sharded run: rank o owns the CSR, cache and feature rows of an id range, one "
+                         "all-to-all round trip per hop (needs --theta; default 32); at 1 GPU it measures the "
+                         "protocol's overhead, the exchange being a local copy")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -222,6 +226,8 @@ def main():
     rank, local_rank, world = replicas.init("nccl", device)
     if world != args.gpus:
         print("warning: --gpus %d but WORLD_SIZE=%d" % (args.gpus, world), file=sys.stderr)
+    if args.sharded:
+        return sharded_arm(args, cfg, mode, gamma, rank, local_rank, world, device)
 
     # ---- inputs, resident in HBM before anything is timed
     t_setup = time.time()
@@ -438,6 +444,79 @@ def main():
         result["cpu_baseline"] = {"value": v, "unit": "edges/s", "feature_gbs": fg, "cores": 1,
                                   "host_cores": os.cpu_count(), "kind": "oracle", "sample": desc}
     print(json.dumps(result))
+    replicas.shutdown()
+    return 0
+
+
+def sharded_arm(args, cfg, mode, gamma, rank, local_rank, world, device):
+    """Node-sharded sampling: every rank samples its own batch per step; frontier nodes are served by
+    their owners.  Same metric, whole-job edges/s; host syncs of the exchange are inside the timed region."""
+    import paper_2406_17918_b200 as gs
+    from paper_2406_17918_b200 import replicas, sharded
+
+    theta = 32 if args.theta is None else args.theta
+    g = build_graph(cfg, device=device)
+    N = cfg["num_nodes"]
+    lo, hi = sharded.shard_range(N, rank, world)
+    ip, idx = sharded.shard_csr(g.indptr, g.indices, rank, world)
+    num_edges = g.num_edges
+    del g
+    X = build_features(cfg, device=device, row_range=(lo, hi))
+    perm = seed_permutation(cfg, device=device)
+    B, L = cfg["batch"], len(cfg["fanouts"])
+    bound = B
+    for k in range(L - 1):
+        bound = min(N, bound * (1 + cfg["fanouts"][L - 1 - k]))
+    me = sharded.ShardRank(gs, rank, world, ip, idx, X, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED, cfg["shared"],
+                           theta, max_seeds=B, max_requests=bound)
+    gm = {"otf": gs.GS_MODE_OTF, "fcr": gs.GS_MODE_FCR, "fbl": gs.GS_MODE_FBL, "fetch": gs.GS_MODE_OTF_FETCH}[mode]
+    K, Wm = args.steps, args.warmup
+
+    def one(step):
+        seeds = batch_seeds(perm, step, B, rank, world)
+        if world > 1:
+            return sharded.sample_batch(me, seeds, gm, gamma, step)
+        return sharded.sample_batch_local([me], [seeds], gm, gamma, step)[0]
+
+    for t in range(1, Wm + 1):
+        one(t)
+    clocks = ClockSampler(local_rank) if rank == 0 else None
+    time.sleep(0.3)
+    replicas.barrier()
+    torch.cuda.synchronize()
+    launches0 = gs.gs_kernel_launches()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wall0 = time.time()
+    edges = rows = 0
+    e0.record()
+    for t in range(Wm + 1, Wm + K + 1):
+        blocks, frontier, n, m, feats = one(t)
+        edges += sum(m)
+        rows += n[L]
+    e1.record()
+    torch.cuda.synchronize()
+    replicas.barrier()
+    wall1 = time.time()
+    launches = gs.gs_kernel_launches() - launches0
+    t_ms, (edges_all, rows_all) = replicas.aggregate(e0.elapsed_time(e1), [edges, rows], device)
+    if clocks:
+        clocks.stop()
+    if rank == 0:
+        esize = 4 if cfg["feat_dtype"] == "f32" else 2
+        print(json.dumps({
+            "metric": METRIC, "value": edges_all / (t_ms * 1e-3), "unit": "edges/s",
+            "feature_gbs": rows_all * cfg["feat_dim"] * esize / (t_ms * 1e-3) / 1e9,
+            "n_gpus": world, "steps": K, "warmup": Wm, "ms_per_step": t_ms / K, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int32 ids + %s feature copy" % cfg["feat_dtype"],
+            "data": "synthetic",
+            "config": {"workload": cfg["name"], "num_nodes": N, "num_edges": num_edges, "fanouts": cfg["fanouts"],
+                       "cache_width": cfg["cache_width"], "mode": mode, "gamma": gamma, "batch": B, "theta": theta,
+                       "shared_cache": cfg["shared"], "feat_dim": cfg["feat_dim"],
+                       "parallelism": "node-sharded x%d (one all-to-all round trip per hop%s)"
+                                      % (world, "" if world > 1 else "; 1 rank: local copy"),
+                       "l2": "inputs_larger_than_L2", "cache_bytes_per_rank": me.cache.storage.numel()},
+            "roofline": None, "e2e": None, "gpu_launches": launches,
+            "clocks": clocks.summary(wall0, wall1) if clocks else None}))
     replicas.shutdown()
     return 0
 

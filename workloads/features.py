@@ -55,17 +55,21 @@ def feature_rows(cfg: dict, ids: torch.Tensor) -> torch.Tensor:
     return _hash_rows(cfg, ids.to(torch.int64))
 
 
-def build_features(cfg: dict, device="cpu", rows_per_chunk: int = 1 << 19) -> torch.Tensor:
-    """The [num_nodes, feat_dim] feature matrix on `device` (row-major, contiguous)."""
+def build_features(cfg: dict, device="cpu", rows_per_chunk: int = 1 << 19, row_range=None) -> torch.Tensor:
+    """The [num_nodes, feat_dim] feature matrix on `device` (row-major, contiguous), or its rows
+    [row_range[0], row_range[1]) - a shard."""
     n, d = cfg["num_nodes"], cfg["feat_dim"]
     seed = cfg["graph_seed"]
     kind = cfg["feat_kind"]
+    first, last = row_range if row_range is not None else (0, n)
     if kind == "hash":
-        out = torch.empty((n, d), dtype=_torch_dtype(cfg), device=device)
-        for lo in range(0, n, rows_per_chunk):
-            hi = min(n, lo + rows_per_chunk)
-            out[lo:hi] = _hash_rows(cfg, torch.arange(lo, hi, dtype=torch.int64, device=device))
+        out = torch.empty((last - first, d), dtype=_torch_dtype(cfg), device=device)
+        for lo in range(first, last, rows_per_chunk):
+            hi = min(last, lo + rows_per_chunk)
+            out[lo - first:hi - first] = _hash_rows(cfg, torch.arange(lo, hi, dtype=torch.int64, device=device))
         return out
+    if row_range is not None:
+        return build_features(cfg, "cpu", rows_per_chunk)[first:last].contiguous().to(device)
     idx = torch.arange(n * d, dtype=torch.int64)
     if kind == "normal":
         u1 = (lsr(hash_u64(seed, _STREAM_FEAT, 2 * idx), 11).to(torch.float64) + 1.0) * (1.0 / (1 << 53))
