@@ -500,7 +500,6 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         // with r = 0, OTF Fetch with no fetch at this layer) has no scan items and skips the scan launch
         const bool fbl = (mode == GS_MODE_FBL);
         const bool scans = fbl || r > 0 || n_fetch > 0;
-        C.split = 1;
         C.W = fbl ? c->fanouts[layer] : (c->theta > c->W ? c->theta : c->W);   // rows above this degree are refreshed
         C.r = n_fetch > 0 ? n_fetch : (fbl ? c->fanouts[layer] : r);
         C.d_refresh_from = (c->shared && k > 0 && mode != GS_MODE_OTF_FETCH && !fbl) ? hdr + HDR_N + (k - 1) : nullptr;   // k = 0 for a single hop
@@ -753,7 +752,6 @@ gs_status gs_shard_extend(gs_cache* c, int32_t k, const int32_t* d_seeds, int32_
     C.tile_sums = (int32_t*)(ws + w.tiles_a);
     C.table = c->d_table;
     C.stamp = c->shard_stamp;
-    C.split = 1;                 // lays out (empty) scan item lists; nothing is scanned on this side
     C.W = c->W;
     C.r = 0;
     C.tile_sums2 = (int32_t*)(ws + w.tiles_a2);

@@ -179,8 +179,8 @@ struct CountParams {
     int32_t* tile_sums;
     unsigned long long* table;
     uint32_t stamp;
-    // split OTF path: also lays out the scan work items of the refreshed nodes
-    int32_t split, W, r;
+    // also lays out the scan work items of the refreshed nodes (rows above SMALL_DEGREE, r > 0)
+    int32_t W, r;
     const int32_t* d_refresh_from;
     int32_t* tile_sums2;
     int32_t* item_start;

@@ -42,9 +42,9 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
     if ((int)blockIdx.x >= tiles) return;
     const int p = blockIdx.x * SCAN_A_TILE + threadIdx.x;
     int c = 0;
-    int nch = 0;   // scan work items of this node (split path only)
+    int nch = 0;   // scan work items of this node
     unsigned quads = 0, refreshed = 0;
-    const int refresh_from = (P.split && P.d_refresh_from) ? __ldcg(P.d_refresh_from) : 0;
+    const int refresh_from = P.d_refresh_from ? __ldcg(P.d_refresh_from) : 0;
     if (p < n) {
         int v;
         if (P.k == 0) {
@@ -70,19 +70,19 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
         } else if (v >= 0) {
             const int64_t deg = P.g.indptr[v + 1] - P.g.indptr[v];
             c = deg < (int64_t)P.f ? (int)deg : P.f;
-            if (P.split && P.r > 0 && deg > (int64_t)SMALL_DEGREE && deg > (int64_t)P.W && p >= refresh_from) {
+            if (P.r > 0 && deg > (int64_t)SMALL_DEGREE && deg > (int64_t)P.W && p >= refresh_from) {
                 const int64_t nq = (deg + 3) >> 2;
                 nch = (int)((nq + HUB_CHUNK_QUADS - 1) / HUB_CHUNK_QUADS);
                 quads = (unsigned)nq;
             }
-            if (P.split && P.r > 0 && deg > (int64_t)P.W && p >= refresh_from) refreshed = 1;
+            if (P.r > 0 && deg > (int64_t)P.W && p >= refresh_from) refreshed = 1;
         }
     }
     int total;
     const int excl = block_exclusive_scan<SCAN_A_TILE>(c, warp_sums, &total);
     if (p < n) P.blk_indptr[p] = excl;
     int total2 = 0;
-    if (P.split) {
+    {
         const unsigned wq = __reduce_add_sync(FULL, quads), wr = __reduce_add_sync(FULL, refreshed);
         if ((threadIdx.x & 31) == 0 && wr) {
             atomicAdd((unsigned*)(P.hdr + HDR_STAT_QUADS), wq);
@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
         if (p < n) P.item_start[p] = excl2;
     }
     if (threadIdx.x == 0) {
-        if (P.split) P.tile_sums2[blockIdx.x] = total2;
+        P.tile_sums2[blockIdx.x] = total2;
         P.tile_sums[blockIdx.x] = total;
         __threadfence();
         const int ticket = atomicAdd(P.hdr + HDR_TICKET_A + P.k, 1);
@@ -102,8 +102,7 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
     if (!is_last) return;
     __threadfence();
     const int m = scan_tiles_in_place<SCAN_A_TILE>(P.tile_sums, tiles, warp_sums);
-    int items = 0;
-    if (P.split) items = scan_tiles_in_place<SCAN_A_TILE>(P.tile_sums2, tiles, warp_sums);
+    const int items = scan_tiles_in_place<SCAN_A_TILE>(P.tile_sums2, tiles, warp_sums);
     if (threadIdx.x == 0) {
         P.hdr[HDR_M + P.k] = m;
         P.hdr[HDR_ITEMS + P.k] = items;
@@ -117,7 +116,6 @@ __global__ void __launch_bounds__(1024) k_row_offsets(CountParams P) {
     const int p = blockIdx.x * SCAN_A_TILE + threadIdx.x;
     if (p < n) P.blk_indptr[p] += P.tile_sums[p / SCAN_A_TILE];
     else if (p == n) P.blk_indptr[n] = __ldcg(P.hdr + HDR_M + P.k);
-    if (!P.split) return;
     // scan work items: node p owns items [item_start[p], item_start[p+1]), one per chunk of its row
     int first = 0, next = 0;
     if (p < n) {
