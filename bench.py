@@ -35,6 +35,17 @@ FALLBACK_HBM_GBS = 6650.0
 ALU_LANE_OPS = 148 * 128 * 1.965e9
 PHILOX_LANE_OPS = 60.0
 SAMPLER_SEED = 0x6A09E667F3BCC908
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one captured launch, from the ncu summaries under
+# profiles/ (captures on the small workloads; scaled to a launch of the benchmarked workload by the units processed).
+#   k_scan, workload large, sampling step 2 of batch 0: 5,650,688 B read + 12,032 B written for 16,380,004 Philox
+#     blocks in 45,281 work items.  The traffic is the items' descriptors, so it follows the number of items; larger
+#     rows mean fewer items per block, which makes the per-block scaling an upper estimate for the scale workload.
+#   k_gather with 256-byte bf16 rows, workload shared, batch 0: 13,165,312 B read for 50,620 rows (260 B per row: the
+#     row and its id); the 256 B written per row were still in L2 when that short launch ended, so the written bytes
+#     are counted as the algorithmic ones.  400-byte fp32 rows (workload large): 144,165,376 B read + 68,206,592 B
+#     written (the rest still in L2) for 282 K rows: 1.28 x the algorithmic read (rows start on 16-byte boundaries).
+NCU_SCAN_BYTES_PER_BLOCK = (5650688 + 12032) / 16380004
+NCU_GATHER_READ_BYTES_PER_256B_ROW = 13165312 / 50620
 
 
 def measured_peak():
@@ -238,14 +249,18 @@ def main():
     t_graph = time.time() - t_setup
     G = gs.gs_graph_create(g.indptr, g.indices, X)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
+    L_hops = len(cfg["fanouts"])
     if args.theta is None:
-        C = gs.gs_cache_init(G, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED, cfg["shared"])
+        storage = torch.empty(gs.gs_cache_bytes(G, L_hops, cfg["cache_width"], cfg["shared"]), dtype=torch.uint8, device=device)
+        ev0.record()
+        C = gs.gs_cache_init(G, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED, cfg["shared"], storage=storage)
     else:
         dense_rows = int((g.degrees() > args.theta).sum().item())
+        storage = torch.empty(gs.gs_cache_bytes_split(G, L_hops, cfg["cache_width"], cfg["shared"], dense_rows),
+                              dtype=torch.uint8, device=device)
         ev0.record()
         C = gs.gs_cache_init_split(G, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED, cfg["shared"], args.theta,
-                                   dense_rows)
+                                   dense_rows, storage=storage)
     ev1.record()
     torch.cuda.synchronize()
     presample_ms = ev0.elapsed_time(ev1)
@@ -382,9 +397,16 @@ def main():
     gather_bytes_per_launch = alg_feat / K
     gather_ms_per_launch = gather_ms / K
     achieved = gather_bytes_per_launch / (gather_ms_per_launch * 1e-3) / 1e9
+    row_bytes = cfg["feat_dim"] * esize
+    gather_traffic = None   # only the 256-byte-row capture scales cleanly (no sector over-fetch, see above)
+    if row_bytes == 256:
+        gather_traffic = (feat_rows / K) * (NCU_GATHER_READ_BYTES_PER_256B_ROW + row_bytes)
     roof_gather = {"kernel": "k_gather (feature rows), 1 launch per step", "bound": "hbm", "achieved": achieved,
                    "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                   "ms_per_launch": gather_ms_per_launch, "traffic": None}
+                   "ms_per_launch": gather_ms_per_launch, "traffic": gather_traffic,
+                   "traffic_note": "bytes per launch; read bytes scaled by rows from the ncu capture of workload shared "
+                                   "(same 256-byte rows), written bytes algorithmic" if gather_traffic else
+                                   "no capture with this row size scales by rows; see profiles/"}
     # the threshold scan (k_scan, one launch per sampling step) is bound by integer ALU work: Philox blocks
     scan_launches = K * L
     roof_scan = None
@@ -394,7 +416,11 @@ def main():
         roof_scan = {"kernel": "k_scan (Philox threshold scan), %d launches per step" % L, "bound": "alu",
                      "achieved": a_scan, "peak": p_scan, "peak_kind": "derived: 148 SMs x 128 lanes x 1.965 GHz / 60 lane-ops per block",
                      "unit": "G Philox4x32-10 blocks/s", "frac": a_scan / p_scan,
-                     "ms_per_launch": group_ms["scan"] / scan_launches, "traffic": None}
+                     "ms_per_launch": group_ms["scan"] / scan_launches,
+                     "traffic": NCU_SCAN_BYTES_PER_BLOCK * philox_blocks / scan_launches,
+                     "traffic_note": "DRAM bytes per launch, scaled by Philox blocks from the ncu capture of workload "
+                                     "large (an upper estimate: the traffic follows work items, and larger rows have "
+                                     "fewer items per block); the scan reads no CSR bytes"}
     groups = dict(group_ms)
     groups["gather"] = gather_ms
     dominant = max(groups, key=groups.get)
