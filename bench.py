@@ -206,6 +206,9 @@ def main():
                     help="node-sharded run: rank o owns the CSR, cache and feature rows of an id range, one "
                          "all-to-all round trip per hop (needs --theta; default 32); at 1 GPU it measures the "
                          "protocol's overhead, the exchange being a local copy")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="run the feature gather of a batch on the sampling stream instead of a second stream "
+                         "(where it overlaps the first, latency-bound hops of the next batch)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -281,53 +284,104 @@ def main():
     K, Wm = args.steps, args.warmup
     seeds_all = [batch_seeds(perm, b, B, rank, world) for b in range(Wm + 2 * K)]
     pinned_counts = torch.zeros((K, 128), dtype=torch.int32).pin_memory()
-    out = None
 
+    # Batches are independent once sampled, so the gather of batch t (HBM-bound) runs on a second, lower-priority
+    # stream while the sampling stream already works on the first hops of batch t+1 (small, latency-bound kernels).
+    # Two workspaces / output buffers alternate; the batch's row count is copied out of the state header before the
+    # next batch clears it.
+    overlap = not args.no_overlap
+    nbuf = 2 if overlap else 1
+    ws_list = [ws] + [torch.empty_like(ws) for _ in range(nbuf - 1)]
+    out_list = [None] * nbuf
+    cnt_copy = [torch.zeros((), dtype=torch.int32, device=device) for _ in range(nbuf)]
+    s_main = torch.cuda.Stream(device=device, priority=-1)
+    s_gather = torch.cuda.Stream(device=device, priority=0) if overlap else s_main
+    ready = [torch.cuda.Event() for _ in range(nbuf)]
+    done = [torch.cuda.Event() for _ in range(nbuf)]
     refresh_events = []
 
-    def one_step(b, step):
-        nonlocal out
+    def one_step(b, step, j):
         if args.period and step % args.period == 0:
             ra, rb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             ra.record()
             gs.gs_cache_refresh_all(C, refresh_mode, refresh_gamma, step)
             rb.record()
             refresh_events.append((ra, rb))
-        blocks, input_nodes, cnt = gs.gs_sample_batch(C, seeds_all[b], gm, gamma, step, ws)
-        if out is None:
-            out = torch.empty((blocks[0].max_src, cfg["feat_dim"]), dtype=X.dtype, device=device)
+        blocks, input_nodes, cnt = gs.gs_sample_batch(C, seeds_all[b], gm, gamma, step, ws_list[j])
+        if out_list[j] is None:
+            out_list[j] = torch.empty((blocks[0].max_src, cfg["feat_dim"]), dtype=X.dtype, device=device)
         return blocks, input_nodes, cnt
 
-    for b in range(Wm):
-        blocks, input_nodes, cnt = one_step(b, b + 1)
-        gs.gs_gather_features(G, input_nodes, cnt, out)
-    gs.gs_sync_status(C)
+    def gather_step(j, input_nodes, cnt, ev_a=None, ev_b=None):
+        if overlap:
+            cnt_copy[j].copy_(cnt)
+            ready[j].record()
+            s_gather.wait_event(ready[j])
+            cnt = cnt_copy[j]
+        if ev_a is not None:
+            ev_a.record(s_gather)
+        gs.gs_gather_features(G, input_nodes, cnt, out_list[j], stream=s_gather)
+        if ev_b is not None:
+            ev_b.record(s_gather)
+        if overlap:
+            done[j].record(s_gather)
 
-    events = [torch.cuda.Event(enable_timing=True) for _ in range(3 * K)]
-    clocks = ClockSampler(local_rank) if rank == 0 else None
-    time.sleep(0.3)
-    replicas.barrier()
     torch.cuda.synchronize()
-    launches0 = gs.gs_kernel_launches()
-    gs.gs_cache_profile_begin(C, K)     # CUDA events around the batch's kernel groups, on the launching stream
-    wall0 = time.time()
-    for i in range(K):
-        b = Wm + i
-        events[3 * i].record()
-        blocks, input_nodes, cnt = one_step(b, b + 1)
-        events[3 * i + 1].record()
-        gs.gs_gather_features(G, input_nodes, cnt, out)
-        events[3 * i + 2].record()
-        pinned_counts[i].copy_(hdr, non_blocking=True)
-    end = torch.cuda.Event(enable_timing=True)
-    end.record()
+    with torch.cuda.stream(s_main):
+        for b in range(Wm):
+            j = b % nbuf
+            if overlap:
+                s_main.wait_event(done[j])
+            blocks, input_nodes, cnt = one_step(b, b + 1, j)
+            gather_step(j, input_nodes, cnt)
+        gs.gs_sync_status(C)
+        torch.cuda.synchronize()
+
+        events = [torch.cuda.Event(enable_timing=True) for _ in range(4 * K)]
+        clocks = ClockSampler(local_rank) if rank == 0 else None
+        time.sleep(0.3)
+        replicas.barrier()
+        torch.cuda.synchronize()
+        launches0 = gs.gs_kernel_launches()
+        gs.gs_cache_profile_begin(C, K)     # CUDA events around the batch's kernel groups, on the launching stream
+        wall0 = time.time()
+        for i in range(K):
+            b = Wm + i
+            j = b % nbuf
+            if overlap:
+                s_main.wait_event(done[j])          # the gather that last read this workspace has finished
+            events[4 * i].record()
+            blocks, input_nodes, cnt = one_step(b, b + 1, j)
+            events[4 * i + 1].record()
+            pinned_counts[i].copy_(hdr, non_blocking=True)
+            gather_step(j, input_nodes, cnt, events[4 * i + 2], events[4 * i + 3])
+        if overlap:
+            for j in range(nbuf):
+                s_main.wait_event(done[j])
+        end = torch.cuda.Event(enable_timing=True)
+        end.record()
+        torch.cuda.synchronize()
+        replicas.barrier()
+        wall1 = time.time()
+        launches = gs.gs_kernel_launches() - launches0
+        total_ms = events[0].elapsed_time(end)
+        group_ms, _ = gs.gs_cache_profile_end(C)
+        gs.gs_sync_status(C)
+    out = out_list[0]
+    # the gather alone (nothing else on the GPU), on the last batch's input nodes: the kernel's own rate
+    jl = (Wm + K - 1) % nbuf
+    iso = []
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)    # larger than L2: no row survives between launches
+    for _ in range(8):
+        flush.zero_()
+        ia, ib = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ia.record()
+        gs.gs_gather_features(G, input_nodes, cnt_copy[jl] if overlap else cnt, out_list[jl])
+        ib.record()
+        iso.append((ia, ib))
     torch.cuda.synchronize()
-    replicas.barrier()
-    wall1 = time.time()
-    launches = gs.gs_kernel_launches() - launches0
-    total_ms = events[0].elapsed_time(end)
-    group_ms, _ = gs.gs_cache_profile_end(C)
-    gs.gs_sync_status(C)
+    gather_alone_ms = sorted(a.elapsed_time(b) for a, b in iso[2:])[len(iso[2:]) // 2]
+    del flush
     if clocks:
         time.sleep(0.1)
         clocks.stop()
@@ -338,8 +392,8 @@ def main():
     counts = pinned_counts.numpy()
     edges = 0
     feat_rows = 0
-    sample_ms = sum(events[3 * i].elapsed_time(events[3 * i + 1]) for i in range(K))
-    gather_ms = sum(events[3 * i + 1].elapsed_time(events[3 * i + 2]) for i in range(K))
+    sample_ms = sum(events[4 * i].elapsed_time(events[4 * i + 1]) for i in range(K))
+    gather_ms = sum(events[4 * i + 2].elapsed_time(events[4 * i + 3]) for i in range(K))
     # refreshed nodes per step, from the last batch's frontier (outside the timed region)
     deg = g.degrees()
     n_last = [int(counts[K - 1][w]) for w in n_words]
@@ -397,6 +451,8 @@ def main():
     gather_bytes_per_launch = alg_feat / K
     gather_ms_per_launch = gather_ms / K
     achieved = gather_bytes_per_launch / (gather_ms_per_launch * 1e-3) / 1e9
+    last_rows = int(counts[K - 1][n_words[L]])
+    alone_gbs = last_rows * (4 + 2 * cfg["feat_dim"] * esize) / (gather_alone_ms * 1e-3) / 1e9
     row_bytes = cfg["feat_dim"] * esize
     gather_traffic = None   # only the 256-byte-row capture scales cleanly (no sector over-fetch, see above)
     if row_bytes == 256:
@@ -404,6 +460,9 @@ def main():
     roof_gather = {"kernel": "k_gather (feature rows), 1 launch per step", "bound": "hbm", "achieved": achieved,
                    "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
                    "ms_per_launch": gather_ms_per_launch, "traffic": gather_traffic,
+                   "concurrent_with_next_batch": overlap,
+                   "alone": {"achieved": alone_gbs, "frac": alone_gbs / peak, "ms_per_launch": gather_alone_ms,
+                             "what": "the same launch with nothing else running, L2 flushed before each, median of 6"},
                    "traffic_note": "bytes per launch; read bytes scaled by rows from the ncu capture of workload shared "
                                    "(same 256-byte rows), written bytes algorithmic" if gather_traffic else
                                    "no capture with this row size scales by rows; see profiles/"}
@@ -446,6 +505,7 @@ def main():
                    "theta": args.theta, "period": args.period,
                    "refresh": ({"mode": mode, "gamma": refresh_gamma} if args.period else "per batch, frontier rows"), "cache_bytes": C.storage.numel(),
                    "parallelism": "replicas x%d" % world, "l2": "inputs_larger_than_L2",
+                   "gather_stream": "second stream, overlapping the next batch's first hops" if overlap else "sampling stream",
                    "sampled_edges_per_batch": edges / K, "input_nodes_per_batch": feat_rows / K},
         "breakdown_ms_per_step": {"sample_batch": sample_ms / K, "gather_features": gather_ms / K,
                                   "kernel_groups": {k: v / K for k, v in groups.items()}, "dominant": dominant},
