@@ -423,15 +423,26 @@ def main():
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e_edges = 0
-        e0.record()
-        for i in range(K):
-            step = Wm + K + i + 1
-            if args.period and step % args.period == 0:
-                gs.gs_cache_refresh_all(C, refresh_mode, refresh_gamma, step)
-            blocks, input_nodes, n, m = gs.gs_sample_batch_host(C, host_seeds[i], gm, gamma, step, ws)
-            gs.gs_gather_features(G, input_nodes, None, out[: n[L]])
-            e_edges += sum(m)
-        e1.record()
+        done_e = [torch.cuda.Event() for _ in range(nbuf)]
+        with torch.cuda.stream(s_main):
+            e0.record()
+            for i in range(K):
+                step = Wm + K + i + 1
+                j = i % nbuf
+                if overlap:
+                    s_main.wait_event(done_e[j])      # the gather that last read this workspace has finished
+                if args.period and step % args.period == 0:
+                    gs.gs_cache_refresh_all(C, refresh_mode, refresh_gamma, step)
+                # returns once the batch's counts are on the host (synchronises the sampling stream only)
+                blocks, input_nodes, n, m = gs.gs_sample_batch_host(C, host_seeds[i], gm, gamma, step, ws_list[j])
+                gs.gs_gather_features(G, input_nodes, None, out_list[j][: n[L]], stream=s_gather)
+                if overlap:
+                    done_e[j].record(s_gather)
+                e_edges += sum(m)
+            if overlap:
+                for j in range(nbuf):
+                    s_main.wait_event(done_e[j])
+            e1.record()
         torch.cuda.synchronize()
         replicas.barrier()
         e_ms, (e_edges_all,) = replicas.aggregate(e0.elapsed_time(e1), [e_edges], device)
