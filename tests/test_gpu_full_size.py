@@ -25,6 +25,69 @@ def test_large_one_whole_batch():
     pair.check_batch(C, ws, O, seeds, "otf", 0.2, 1, features=False, rows=3000)
 
 
+def test_large_split_cache_whole_batch_then_whole_cache_refresh():
+    """Dense/sparse split (theta = 32) at full size: one whole batch element by element, then the
+    whole-cache refresh checked on sampled nodes the oracle refreshes one by one."""
+    import paper_2406_17918_b200 as gs
+    from parity import Pair
+
+    pair = Pair(get_config("large"), features=False)
+    theta = 32
+    C, ws, O = pair.samplers(pair.cfg["batch"], theta=theta)
+    full = gs.gs_cache_bytes(pair.G, pair.L, pair.W, False)
+    assert C.storage.numel() < 0.6 * full
+    seeds = batch_seeds(pair.perm, 0, pair.cfg["batch"])
+    pair.check_batch(C, ws, O, seeds, "otf", 0.2, 1, features=False, rows=2000)
+    rng = np.random.default_rng(11)
+    dense = np.nonzero(pair.deg > theta)[0]
+    nodes = np.concatenate([np.argsort(-pair.deg)[:16], rng.choice(dense, 1500, replace=False)]).astype(np.int32)
+    for mode, gamma, step in (("otf", 0.2, 2), ("fcr", 0.0, 3)):
+        gm, om = {"otf": (gs.GS_MODE_OTF, oracle.MODE_OTF), "fcr": (gs.GS_MODE_FCR, oracle.MODE_FCR)}[mode]
+        gs.gs_cache_refresh_all(C, gm, gamma, step)
+        gs.gs_sync_status(C)
+        r = oracle.refresh_count(om, gamma, pair.W)
+        for layer in range(pair.L):
+            for v in nodes:
+                O.refresh_node(layer, int(v), step, r)
+        pair.check_rows(C, O, nodes)
+    # a sparse node has no row, before and after
+    sparse = np.nonzero(pair.deg <= theta)[0][:100].astype(np.int32)
+    assert (gs.gs_cache_read_rows(C, 0, torch.from_numpy(sparse).cuda()).cpu().numpy() == -1).all()
+
+
+def test_large_two_shards_one_step():
+    """Node-sharded sampling at full size: two ranks run phase by phase on this GPU; each rank's whole
+    batch must equal what one sampler (theta = 32) gives when it takes the two batches in turn."""
+    import paper_2406_17918_b200 as gs
+    from paper_2406_17918_b200 import sharded
+
+    cfg = get_config("large")
+    g = build_graph(cfg)
+    perm = seed_permutation(cfg)
+    N, B, L, theta, seed, world = cfg["num_nodes"], cfg["batch"], len(cfg["fanouts"]), 32, 7, 2
+    X = torch.arange(N, dtype=torch.float32).reshape(N, 1).repeat(1, 4).contiguous()    # row v holds v: cheap to check
+    ranks = []
+    for r in range(world):
+        ip, idx = sharded.shard_csr(g.indptr, g.indices, r, world)
+        lo, hi = sharded.shard_range(N, r, world)
+        ranks.append(sharded.ShardRank(gs, r, world, ip.cuda(), idx.cuda(), X[lo:hi].cuda().contiguous(), cfg["fanouts"],
+                                       cfg["cache_width"], seed, False, theta, max_seeds=B, max_requests=B * 6 * 11))
+    O = oracle.Sampler(g.indptr.numpy(), g.indices.numpy(), cfg["fanouts"], cfg["cache_width"], seed, False)
+    O.set_theta(theta)
+    seeds = [batch_seeds(perm, 1, B, r, world) for r in range(world)]
+    res = sharded.sample_batch_local(ranks, [s.cuda() for s in seeds], gs.GS_MODE_OTF, 0.2, 1)
+    for r in range(world):
+        blocks, frontier, n, m, feats = res[r]
+        fr_o, n_o, blocks_o = O.sample_batch(seeds[r].numpy(), oracle.MODE_OTF, 0.2, 1)
+        assert n == n_o
+        assert np.array_equal(frontier[: n[L]].cpu().numpy(), fr_o)
+        for layer in range(L):
+            k = L - 1 - layer
+            assert np.array_equal(blocks[layer].indptr(n[k]).cpu().numpy(), blocks_o[layer].indptr)
+            assert np.array_equal(blocks[layer].indices(m[layer]).cpu().numpy(), blocks_o[layer].indices)
+        assert torch.equal(feats[:, 0].cpu(), torch.from_numpy(fr_o.astype(np.float32)))
+
+
 def _is_neighbour(indptr, indices, dst, src):
     """Vectorised binary search of src in the sorted CSR row of dst (all on the GPU)."""
     lo = indptr[dst]
