@@ -246,6 +246,17 @@ gs_status gs_gather_rows(const void* d_src, gs_dtype dtype, int32_t row_elems, i
                          const int32_t* d_ids, const int32_t* d_count_or_null, int32_t count_bound, void* d_out,
                          int64_t out_ld, void* stream);
 
+/* The feature step of a sharded run as ONE kernel over peer memory: out[i, :] = row ids[i] of a
+ * matrix whose rows are split over `world` shards of S = ceil(num_rows / world) rows; shard o holds
+ * rows [o*S, (o+1)*S) and starts at h_shard_bases[o] (a HOST array of DEVICE addresses - this
+ * GPU's own memory or peer GPUs' memory mapped into this process, e.g. CUDA IPC or a symmetric
+ * allocation; mapping is the caller's).  Each row is read with plain 16-byte streaming loads
+ * straight from its owner and written to `d_out`: the row crosses NVLink once, no staging buffer,
+ * no exchange of ids.  ids outside [0, num_rows) are skipped.  All shards share src_ld. */
+gs_status gs_gather_rows_peer(const void* const* h_shard_bases, int32_t world, int64_t num_rows, gs_dtype dtype,
+                              int32_t row_elems, int64_t src_ld, const int32_t* d_ids, const int32_t* d_count_or_null,
+                              int32_t count_bound, void* d_out, int64_t out_ld, void* stream);
+
 /* ---- Node-sharded sampling over several GPUs (the paper's Section "Shared Cache Mode" speaks of a
  * cache that serves multiple computation processes; the partition and the exchange are this
  * library's).  Nodes are partitioned by id range: shard o of `world` owns the nodes

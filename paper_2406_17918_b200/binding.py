@@ -84,6 +84,7 @@ def _load():
         "gs_cache_import": [vp, vp, sz, vp],
         "gs_sync_status": [vp, vp],
         "gs_gather_rows": [vp, ctypes.c_int, i32, i64, i64, vp, vp, i32, vp, i64, vp],
+        "gs_gather_rows_peer": [vp, i32, i64, ctypes.c_int, i32, i64, vp, vp, i32, vp, i64, vp],
         "gs_shard_bucket": [vp, i32, i64, i32, vp, vp, vp, vp],
         "gs_shard_workspace_bytes": [vp, i32, i32, psz],
         "gs_shard_sample_rows": [vp, vp, i32, i32, ctypes.c_int, dbl, u32, vp, sz, vp, vp],
@@ -383,6 +384,23 @@ def gs_gather_rows(src: torch.Tensor, ids: torch.Tensor, out: torch.Tensor, firs
     bound = min(out.shape[0], ids.numel())
     _check(_L.gs_gather_rows(_ptr(src), dtype, src.shape[1], src.stride(0), int(first_row), _ptr(ids), _ptr(count), bound,
                              _ptr(out), out.stride(0), _stream(stream)))
+    return out
+
+
+def gs_gather_rows_peer(shard_bases, num_rows: int, dtype: torch.dtype, row_elems: int, src_ld: int, ids: torch.Tensor,
+                        out: torch.Tensor, count=None, stream=None):
+    """out[i] = row ids[i] of a matrix split over len(shard_bases) row shards; `shard_bases` are device
+    addresses (ints), local or peer-mapped.  One kernel: the rows are pulled straight from their owners."""
+    if ids.dtype != torch.int32 or not ids.is_cuda:
+        raise TypeError("ids must be an int32 CUDA tensor")
+    if out.dim() != 2 or out.stride(1) != 1 or out.dtype != dtype:
+        raise TypeError("out must be a row-major 2-D tensor of the given dtype")
+    world = len(shard_bases)
+    arr = (ctypes.c_void_p * world)(*[ctypes.c_void_p(int(b)) for b in shard_bases])
+    bound = min(out.shape[0], ids.numel())
+    _check(_L.gs_gather_rows_peer(arr, world, int(num_rows), {torch.float32: GS_F32, torch.bfloat16: GS_BF16}[dtype],
+                                  int(row_elems), int(src_ld), _ptr(ids), _ptr(count), bound, _ptr(out), out.stride(0),
+                                  _stream(stream)))
     return out
 
 

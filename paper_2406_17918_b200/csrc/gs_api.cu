@@ -808,6 +808,29 @@ gs_status gs_gather_rows(const void* d_src, gs_dtype dtype, int32_t row_elems, i
     return GS_OK;
 }
 
+gs_status gs_gather_rows_peer(const void* const* h_shard_bases, int32_t world, int64_t num_rows, gs_dtype dtype,
+                              int32_t row_elems, int64_t src_ld, const int32_t* d_ids, const int32_t* d_count_or_null,
+                              int32_t count_bound, void* d_out, int64_t out_ld, void* stream) {
+    if (dtype != GS_F32 && dtype != GS_BF16) return fail(GS_ERR_ARG, "unknown dtype %d", (int)dtype);
+    const int64_t eb = dtype == GS_BF16 ? 2 : 4;
+    if (world < 1 || world > 64) return fail(GS_ERR_ARG, "world %d outside [1, 64]", world);
+    if (num_rows < 1 || num_rows >= ((int64_t)1 << 31)) return fail(GS_ERR_ARG, "num_rows outside [1, 2^31)");
+    if (count_bound < 0) return fail(GS_ERR_ARG, "count_bound is negative");
+    if (count_bound == 0) return GS_OK;
+    if (!h_shard_bases || !d_ids || !d_out) return fail(GS_ERR_ARG, "NULL argument");
+    if (row_elems < 1 || src_ld < row_elems || out_ld < row_elems) return fail(GS_ERR_ARG, "bad row size or pitch");
+    const int64_t rows_per_shard = (num_rows + world - 1) / world;
+    for (int o = 0; o < world; ++o) {
+        const bool empty = (int64_t)o * rows_per_shard >= num_rows;   // a trailing shard may own no row
+        if (!h_shard_bases[o] && !empty) return fail(GS_ERR_ARG, "shard %d has no base address", o);
+        if (!aligned(h_shard_bases[o], (size_t)eb)) return fail(GS_ERR_ALIGN, "shard %d is misaligned", o);
+    }
+    if (!aligned(d_out, (size_t)eb) || !aligned(d_ids, 4)) return fail(GS_ERR_ALIGN, "misaligned argument");
+    GS_CUDA(launch_gather_sharded(h_shard_bases, world, num_rows, rows_per_shard, src_ld * eb, (int64_t)row_elems * eb, d_ids,
+                                  d_count_or_null, count_bound, d_out, out_ld * eb, (cudaStream_t)stream));
+    return GS_OK;
+}
+
 gs_status gs_batch_counts(gs_cache* c, void* stream, int32_t* h_num_nodes, int32_t* h_num_edges) {
     if (!c) return fail(GS_ERR_ARG, "cache is NULL");
     cudaStream_t s = (cudaStream_t)stream;

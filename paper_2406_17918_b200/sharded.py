@@ -96,6 +96,14 @@ class ShardRank:
     def feature_requests(self):
         return self.requests(self.frontier[: self.n[self.L]])
 
+    def feature_pull(self, shard_bases):
+        """The feature step as one kernel: every input node's row is read straight from its owner's
+        memory (`shard_bases[o]`: device address of rank o's feature rows, peer-mapped where o is another GPU)."""
+        n = self.n[self.L]
+        out = torch.empty((n, self.features.shape[1]), dtype=self.features.dtype, device=self.features.device)
+        return self.ops.gs_gather_rows_peer(shard_bases, self.num_nodes, self.features.dtype, self.features.shape[1],
+                                            self.features.stride(0), self.frontier[:n], out)
+
     def feature_finish(self, rows):
         out = torch.empty((self.n[self.L], rows.shape[1]), dtype=rows.dtype, device=rows.device)
         return self.ops.gs_gather_rows(rows, self.slot, out)
@@ -144,7 +152,10 @@ def sample_batch_local(ranks, seeds_per_rank, mode, rate, step, features=True):
         for r, reply in zip(ranks, replies):
             r.hop_finish(k, reply.contiguous())
     feats = [None] * R
-    if features:
+    if features == "peer":     # all shards live in this process: their addresses are the "peer" mappings
+        bases = [r.features.data_ptr() for r in ranks]
+        feats = [r.feature_pull(bases) for r in ranks]
+    elif features:
         rows = round_trip([r.feature_requests() for r in ranks], lambda owner, lists: owner.feature_serve(lists))
         feats = [r.feature_finish(x.contiguous()) for r, x in zip(ranks, rows)]
     return [(r.blocks, r.frontier, r.n, r.m, f) for r, f in zip(ranks, feats)]
@@ -163,9 +174,12 @@ def _all_to_all_v(send, send_counts, width, group):
     return recv, recv_counts
 
 
-def sample_batch(rank_state: ShardRank, seeds, mode, rate, step, features=True, group=None):
+def sample_batch(rank_state: ShardRank, seeds, mode, rate, step, features=True, group=None, feature_bases=None):
     """This rank's part of a sharded batch (every rank of `group` calls it with the same mode, rate
-    and step).  Returns (blocks by layer, frontier tensor, n list, m list, feature rows or None)."""
+    and step).  Returns (blocks by layer, frontier tensor, n list, m list, feature rows or None).
+    `feature_bases`: device addresses of every rank's feature rows as mapped into this process (CUDA
+    IPC, symmetric memory, ...); when given, the feature step is one kernel of peer loads instead of an
+    all-to-all round trip."""
     me = rank_state
     L = me.L
     me.begin(seeds)
@@ -185,7 +199,9 @@ def sample_batch(rank_state: ShardRank, seeds, mode, rate, step, features=True, 
                            (me.fanouts[layer],), torch.int32)
         me.hop_finish(k, reply)
     feats = None
-    if features:
+    if features and feature_bases is not None:
+        feats = me.feature_pull(feature_bases)
+    elif features:
         ids, counts = me.feature_requests()
         rows = round_trip(ids, counts, me.feature_serve, (me.features.shape[1],), me.features.dtype)
         feats = me.feature_finish(rows)

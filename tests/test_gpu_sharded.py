@@ -85,12 +85,13 @@ def test_sharded_tiny_all_modes(world):
         s.step(mode, rate, t)
         t += 1
     s.check_rows()
+    s.step("otf", 0.25, t, features="peer")     # the feature rows pulled from their owners by one kernel
 
 
 def test_sharded_mid_and_shared_cache():
     s = Setup("mid", 4, theta=24, B=512)
     for t in (1, 2):
-        s.step("otf", 0.3, t)
+        s.step("otf", 0.3, t, features="peer" if t == 2 else True)
     s.step("fcr", 0.0, 3, features=False)
     s.check_rows(sample=4000)
     s = Setup("shared", 2, theta=32, B=1024)
@@ -122,3 +123,14 @@ def test_bucket_and_gather_rows_primitives():
     out = torch.empty((333, 24), dtype=torch.bfloat16, device="cuda")
     gs.gs_gather_rows(X[400:700], ids, out, first_row=400)
     assert torch.equal(out, X[ids.long()])
+    # the same matrix as three shards of ceil(1000/3) rows, each at its own address
+    parts = [X[0:334].clone(), X[334:668].clone(), X[668:1000].clone()]
+    ids = torch.from_numpy(rng.integers(0, 1000, 4001).astype(np.int32)).cuda()
+    ids[5] = -1
+    ids[6] = 1000
+    out = torch.full((4001, 24), 7, dtype=torch.bfloat16, device="cuda")
+    gs.gs_gather_rows_peer([p.data_ptr() for p in parts], 1000, torch.bfloat16, 24, 24, ids, out)
+    ok = (ids >= 0) & (ids < 1000)
+    assert torch.equal(out[ok], X[ids[ok].long()]) and bool((out[~ok] == 7).all())
+    with pytest.raises(gs.GsError):
+        gs.gs_gather_rows_peer([parts[0].data_ptr(), 0, parts[2].data_ptr()], 1000, torch.bfloat16, 24, 24, ids, out)
