@@ -935,7 +935,7 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
             uint32_t ekey = 0, pkey = 0;
             if (!P.fbl && (refresh || ncached > P.f)) evict_pick_keys(P, v, lane, ekey, pkey);
             uint32_t cache_part = 0;   // OTF Fetch: lanes of the cache slots that are part of the sample
-            if (refresh && P.r >= W) {
+            if (refresh && P.r >= W && !P.fetch) {
                 // Full refill (FCR, and Full Batch Load with W = f): the W offsets first in key order,
                 // in that order.  Short rows take every offset as a candidate, longer ones the list
                 // the scan kernel left; a list that cannot hold the top-W sends the row to a rescan.
@@ -972,6 +972,7 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
             } else if (refresh) {
                 uint32_t evict;
                 if (P.fetch) {
+                    // (OTF Fetch comes here even when all f = W samples are fetched: it never writes the row.)
                     // The f - r cache picks play the part of the retained slots, the r fetched
                     // neighbours land in the r lowest other lanes; the other slots are blanked so that
                     // only the cache picks exclude candidates.  The row itself is not modified.

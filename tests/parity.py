@@ -33,6 +33,23 @@ class Pair:
         self.G = gs.gs_graph_create(self.g_dev.indptr, self.g_dev.indices, self.X)
         self.seed = seed
 
+    @classmethod
+    def from_csr(cls, indptr, indices, fanouts, cache_width, shared=False, seed=0x1234ABCD5678EF01):
+        """A hand-made graph (numpy CSR) instead of a named workload; no features, seeds = node order."""
+        self = cls.__new__(cls)
+        n = len(indptr) - 1
+        self.cfg = dict(name="custom", num_nodes=n, fanouts=list(fanouts), cache_width=cache_width, shared=shared, batch=n)
+        self.indptr, self.indices = np.asarray(indptr, dtype=np.int64), np.asarray(indices, dtype=np.int32)
+        self.deg = self.indptr[1:] - self.indptr[:-1]
+        from workloads.graphs import Graph
+        self.g_dev = Graph(n, len(self.indices), torch.from_numpy(self.indptr).cuda(), torch.from_numpy(self.indices).cuda())
+        self.X = None
+        self.perm = torch.arange(n, dtype=torch.int32)
+        self.L, self.W, self.shared = len(fanouts), cache_width, shared
+        self.G = gs.gs_graph_create(self.g_dev.indptr, self.g_dev.indices, None)
+        self.seed = seed
+        return self
+
     def samplers(self, max_seeds, tuning=None, theta=None):
         self.theta = theta
         if theta is None:

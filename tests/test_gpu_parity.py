@@ -181,6 +181,61 @@ def test_whole_graph_as_seeds(tiny):
     assert n[0] == n[-1] == tiny.cfg["num_nodes"]
 
 
+@pytest.mark.parametrize("fanouts,W", [([1], 1), ([32], 32), ([3], 32), ([2] * 8, 4), ([5, 5], 5), ([1, 32, 1], 32)])
+def test_extreme_shapes(fanouts, W):
+    """One hop and the maximum of eight, cache width 1 and the maximum 32, fan-out equal to the width."""
+    from parity import Pair
+    pair = Pair(get_config("tiny", fanouts=fanouts, cache_width=W), features=False)
+    for mode, gamma in (("otf", 0.3), ("fcr", 0.0), ("fetch", 0.5), ("fbl", 0.0)):
+        pair.run(mode, gamma, 2, batch_size=48, features=False)
+
+
+def test_otf_fetch_with_every_sample_fetched_and_fanout_equal_to_width():
+    """delta = 1 with f = W: as many neighbours are fetched as the row has slots, and the row must stay as it is."""
+    from parity import Pair
+    pair = Pair(get_config("tiny", fanouts=[10, 10], cache_width=10), features=False)
+    pair.run("fetch", 1.0, 3, features=False)
+    pair = Pair(get_config("mid", fanouts=[20, 20], cache_width=20), features=False)
+    pair.run("fetch", 1.0, 2, batch_size=256, features=False, rows=500)
+    pair.run("fetch", 1.0, 1, batch_size=256, features=False, rows=500, tuning=dict(lambda_full=1.0, hub_degree=64))
+    pair.run("fetch", 0.97, 1, batch_size=256, features=False, rows=500, tuning=dict(lambda_otf=1.0))
+
+
+def test_hand_made_graphs_hub_isolated_and_chain():
+    """A hub far above every chunking threshold next to isolated nodes; seeds without neighbours."""
+    from helpers import csr_from_rows
+    from parity import Pair
+    hub_deg = 150_000
+    n = hub_deg + 40
+    rows = [[] for _ in range(n)]
+    rows[0] = list(range(40, n))                    # the hub: every node from 40 on points to node 0
+    rows[1] = list(range(40, 40 + 9000))            # above the degree at which a row is split over warps
+    rows[2] = list(range(40, 40 + 129))             # just above the in-register limit
+    rows[3] = list(range(40, 40 + 128))             # at the in-register limit
+    rows[4] = list(range(40, 40 + 33))
+    rows[5] = list(range(40, 40 + 32))              # holds its whole adjacency
+    for v in range(40, 60):
+        rows[v] = [0, 1, 2, 3, 4, 5]                # so that later hops reach the hub rows again
+    indptr, indices = csr_from_rows(rows)
+    pair = Pair.from_csr(indptr, indices, [7, 10], 32)
+    C, ws, O = pair.samplers(64)
+    pair.check_rows(C, O, np.arange(64))
+    seeds = torch.arange(0, 64, dtype=torch.int32)                          # rows 6..39 are isolated
+    for step, (mode, gamma) in enumerate([("otf", 0.1), ("otf", 0.5), ("fcr", 0.0), ("fetch", 0.3), ("fbl", 0.0)], 1):
+        pair.check_batch(C, ws, O, seeds, mode, gamma, step, features=False)
+    # only isolated seeds: every block is empty and the frontier is the seeds
+    iso = torch.arange(6, 40, dtype=torch.int32)
+    n_, m_ = pair.check_batch(C, ws, O, iso, "otf", 0.3, 9, features=False)
+    assert n_ == [34, 34, 34] and m_ == [0, 0]
+    # the same graph with a split cache and a whole-cache refresh
+    C2, ws2, O2 = pair.samplers(64, theta=64)
+    pair.check_batch(C2, ws2, O2, seeds, "otf", 0.25, 1, features=False)
+    import paper_2406_17918_b200 as gs
+    gs.gs_cache_refresh_all(C2, gs.GS_MODE_OTF, 0.5, 2)
+    O2.refresh_all(oracle.MODE_OTF, 0.5, 2)
+    pair.check_rows(C2, O2, np.arange(64))
+
+
 def test_resume_from_export(tiny):
     import paper_2406_17918_b200 as gs
     B = tiny.cfg["batch"]
