@@ -427,7 +427,7 @@ def gs_shard_sample_rows(cache: Cache, nodes: torch.Tensor, layer: int, mode: in
     """Owner side of one hop: picks[n, fanout(layer)] (-1 padded) for n distinct nodes of this shard."""
     if nodes.dtype != torch.int32 or not nodes.is_cuda or not nodes.is_contiguous():
         raise TypeError("nodes must be a contiguous int32 CUDA tensor")
-    f = cache.fanouts[layer]
+    f = cache.fanouts[layer] if 0 <= layer < cache.num_hops else 1     # a bad layer is reported by the library
     if picks is None:
         picks = torch.empty((nodes.numel(), f), dtype=torch.int32, device=nodes.device)
     _check(_L.gs_shard_sample_rows(cache.handle, _ptr(nodes), nodes.numel(), int(layer), mode, float(rate), step,

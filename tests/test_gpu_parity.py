@@ -236,6 +236,33 @@ def test_hand_made_graphs_hub_isolated_and_chain():
     pair.check_rows(C2, O2, np.arange(64))
 
 
+@pytest.mark.parametrize("shared", [False, True])
+def test_degrees_at_every_internal_threshold(shared):
+    """Rows whose degree sits on and next to each switch inside the kernels (cache width, the in-register
+    limit, the candidate-pop switch, the scan chunk, the degree from which a row is split over warps), with the
+    default thresholds and with thresholds that make the first attempt fail."""
+    from helpers import csr_from_rows
+    from parity import Pair
+    degs = [0, 1, 31, 32, 33, 63, 64, 65, 127, 128, 129, 1023, 1024, 1025, 4095, 4096, 4097, 4100, 8191, 8192, 8193, 12289, 20000]
+    base = 64
+    n = base + max(degs)
+    rows = [[] for _ in range(n)]
+    for v, d in enumerate(degs):
+        rows[v] = list(range(base, base + d))
+    for v in range(base, base + 40):
+        rows[v] = list(range(0, len(degs)))          # the next hop comes back to the rows above
+    indptr, indices = csr_from_rows(rows)
+    pair = Pair.from_csr(indptr, indices, [9, 32], 32, shared=shared)
+    seeds = torch.arange(0, len(degs), dtype=torch.int32)
+    runs = [("otf", 0.1), ("otf", 0.5), ("fcr", 0.0), ("fetch", 0.3), ("fetch", 1.0), ("fbl", 0.0), ("otf", 0.97)]
+    for tuning in (None, dict(lambda_otf=1.0, lambda_full=4.0), dict(lambda_otf=60.0, lambda_full=200.0), dict(hub_degree=64)):
+        C, ws, O = pair.samplers(len(degs), tuning=tuning)
+        pair.check_rows(C, O, np.arange(len(degs)))
+        for i, (mode, gamma) in enumerate(runs):
+            step = 0xFFFFFFFF - i if tuning is None else i + 1           # the largest step numbers as well
+            pair.check_batch(C, ws, O, seeds, mode, gamma, step, features=False)
+
+
 def test_resume_from_export(tiny):
     import paper_2406_17918_b200 as gs
     B = tiny.cfg["batch"]

@@ -134,3 +134,47 @@ def test_bucket_and_gather_rows_primitives():
     assert torch.equal(out[ok], X[ids[ok].long()]) and bool((out[~ok] == 7).all())
     with pytest.raises(gs.GsError):
         gs.gs_gather_rows_peer([parts[0].data_ptr(), 0, parts[2].data_ptr()], 1000, torch.bfloat16, 24, 24, ids, out)
+
+
+def test_sharded_entry_points_reject_bad_arguments():
+    import paper_2406_17918_b200 as gs
+    s = Setup("tiny", 2, theta=12)
+    me = s.ranks[0]
+    nodes = torch.arange(0, 8, dtype=torch.int32, device="cuda")
+    picks_ws = me.ws_owner
+    for bad in [dict(layer=5), dict(layer=-1), dict(mode=9), dict(rate=1.5, mode=gs.GS_MODE_OTF), dict(step=0)]:
+        kw = dict(layer=0, mode=gs.GS_MODE_OTF, rate=0.25, step=1)
+        kw.update(bad)
+        with pytest.raises(gs.GsError):
+            gs.gs_shard_sample_rows(me.cache, nodes, kw["layer"], kw["mode"], kw["rate"], kw["step"], picks_ws)
+    with pytest.raises(gs.GsError) as e:
+        gs.gs_shard_sample_rows(me.cache, nodes, 0, gs.GS_MODE_OTF, 0.25, 1, picks_ws[:256])
+    assert e.value.status == 4                                           # GS_ERR_WORKSPACE
+    assert gs.gs_shard_sample_rows(me.cache, nodes[:0], 0, gs.GS_MODE_OTF, 0.25, 1, picks_ws).shape == (0, me.fanouts[0])
+    # a node id that is not a node: reported by the status call, nothing else breaks
+    bad_nodes = torch.tensor([1, 2, s.cfg["num_nodes"] + 7], dtype=torch.int32, device="cuda")
+    gs.gs_shard_sample_rows(me.cache, bad_nodes, 0, gs.GS_MODE_OTF, 0.25, 1, picks_ws)
+    with pytest.raises(gs.GsError) as e:
+        gs.gs_shard_status(me.cache)
+    assert e.value.status == 3                                           # GS_ERR_RANGE
+    gs.gs_shard_sample_rows(me.cache, nodes, 0, gs.GS_MODE_OTF, 0.25, 1, picks_ws)
+    gs.gs_shard_status(me.cache)                                         # the next call starts clean
+    # requester side: hops in order, starting at 0
+    reply = torch.full((8, me.fanouts[-1]), -1, dtype=torch.int32, device="cuda")
+    slot = torch.arange(8, dtype=torch.int32, device="cuda")
+    fresh = Setup("tiny", 1, theta=12).ranks[0]
+    with pytest.raises(gs.GsError):
+        gs.gs_shard_extend(fresh.cache, 1, None, reply, slot, fresh.ws)          # hop 1 before hop 0
+    with pytest.raises(gs.GsError):
+        gs.gs_shard_extend(fresh.cache, 0, None, reply, slot, fresh.ws)          # hop 0 without seeds
+    with pytest.raises(gs.GsError):
+        gs.gs_shard_extend(fresh.cache, 7, nodes, reply, slot, fresh.ws)
+    # all rows empty: every block is empty, the frontier is the seeds
+    block, frontier = gs.gs_shard_extend(fresh.cache, 0, nodes, reply, slot, fresh.ws)
+    n, m = gs.gs_batch_counts(fresh.cache)
+    assert n[:2] == [8, 8] and m[-1] == 0 and torch.equal(frontier[:8], nodes)
+    with pytest.raises(gs.GsError):
+        gs.gs_shard_bucket(nodes, 100, 65)
+    with pytest.raises(gs.GsError):
+        X = torch.zeros((4, 8), device="cuda")
+        gs.gs_gather_rows(X, nodes, torch.zeros((8, 4), device="cuda"))              # output rows narrower than the source rows
