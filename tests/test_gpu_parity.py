@@ -263,6 +263,58 @@ def test_degrees_at_every_internal_threshold(shared):
             pair.check_batch(C, ws, O, seeds, mode, gamma, step, features=False)
 
 
+def _random_graph(rng):
+    n = int(rng.integers(200, 2500)) if rng.random() < 0.75 else int(rng.integers(9000, 12000))
+    kind = rng.random(n)
+    deg = np.where(kind < 0.15, 0, np.where(kind < 0.75, rng.integers(1, 40, n), rng.integers(40, 400, n)))
+    for v in rng.choice(n, size=int(rng.integers(0, 4)), replace=False):      # a few rows far above the chunk sizes
+        deg[v] = int(rng.integers(1500, min(n - 1, 20000) + 1)) if n > 1501 else n - 1
+    deg = np.minimum(deg, n - 1)
+    indptr = np.zeros(n + 1, dtype=np.int64)
+    indptr[1:] = np.cumsum(deg)
+    indices = np.empty(int(indptr[-1]), dtype=np.int32)
+    for v in range(n):
+        if deg[v]:
+            nb = rng.choice(n - 1, size=int(deg[v]), replace=False)
+            nb = np.sort(np.where(nb >= v, nb + 1, nb))                        # no self loop, sorted, distinct
+            indices[indptr[v]:indptr[v + 1]] = nb
+    return indptr, indices
+
+
+@pytest.mark.parametrize("case", range(64))
+def test_randomised_configurations(case):
+    """Seeded random graphs, shapes, modes, rates, splits and thresholds: everything compared with the oracle."""
+    from parity import Pair
+    rng = np.random.default_rng(1000 + case)
+    indptr, indices = _random_graph(rng)
+    n = len(indptr) - 1
+    L = int(rng.integers(1, 5))
+    W = int(rng.choice([1, 2, 5, 8, 16, 20, 31, 32]))
+    fanouts = [int(rng.integers(1, W + 1)) for _ in range(L)]
+    shared = bool(rng.random() < 0.3)
+    theta = None if rng.random() < 0.6 else int(rng.integers(W, 129))
+    tuning = None
+    if rng.random() < 0.4:
+        tuning = dict(lambda_otf=float(rng.choice([1.0, 4.0, 40.0])), lambda_full=float(rng.choice([2.0, 30.0, 150.0])),
+                      hub_degree=int(rng.choice([64, 1000, 8192])))
+    pair = Pair.from_csr(indptr, indices, fanouts, W, shared=shared, seed=int(rng.integers(1, 2**63)))
+    B = int(rng.integers(1, min(n, 300) + 1))
+    C, ws, O = pair.samplers(B, tuning=tuning, theta=theta)
+    pair.check_rows(C, O, np.arange(n))
+    step = int(rng.integers(1, 2**32 - 10))
+    for b in range(4):
+        mode = str(rng.choice(["otf", "otf", "fcr", "fetch", "fbl"]))
+        rate = float(rng.choice([0.0, 0.1, 0.25, 0.5, 0.9, 1.0]))
+        seeds = torch.from_numpy(rng.choice(n, size=int(rng.integers(1, B + 1)), replace=False).astype(np.int32))
+        pair.check_batch(C, ws, O, seeds, mode, rate, step + b, features=False)
+        if rng.random() < 0.25:
+            import paper_2406_17918_b200 as gs
+            which = str(rng.choice(["otf", "fcr"]))
+            gs.gs_cache_refresh_all(C, {"otf": gs.GS_MODE_OTF, "fcr": gs.GS_MODE_FCR}[which], rate, step + b)
+            O.refresh_all({"otf": oracle.MODE_OTF, "fcr": oracle.MODE_FCR}[which], rate, step + b)
+    pair.check_rows(C, O, np.arange(n))
+
+
 def test_resume_from_export(tiny):
     import paper_2406_17918_b200 as gs
     B = tiny.cfg["batch"]
