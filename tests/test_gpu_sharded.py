@@ -178,3 +178,62 @@ def test_sharded_entry_points_reject_bad_arguments():
     with pytest.raises(gs.GsError):
         X = torch.zeros((4, 8), device="cuda")
         gs.gs_gather_rows(X, nodes, torch.zeros((8, 4), device="cuda"))              # output rows narrower than the source rows
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_randomised_sharded_runs(case):
+    """Seeded random graphs, world sizes, shapes, modes and rates; every rank's batch against one oracle sampler."""
+    import paper_2406_17918_b200 as gs
+    from paper_2406_17918_b200 import sharded
+    from test_gpu_parity import _random_graph
+
+    rng = np.random.default_rng(5000 + case)
+    indptr, indices = _random_graph(rng)
+    n = len(indptr) - 1
+    world = int(rng.integers(1, 6))
+    L = int(rng.integers(1, 4))
+    W = int(rng.choice([2, 8, 20, 32]))
+    fanouts = [int(rng.integers(1, W + 1)) for _ in range(L)]
+    shared = bool(rng.random() < 0.3)
+    theta = int(rng.integers(W, 129))
+    seed = int(rng.integers(1, 2**63))
+    ip_t, ix_t = torch.from_numpy(indptr), torch.from_numpy(indices)
+    X = torch.arange(n, dtype=torch.float32).reshape(n, 1).repeat(1, 4).contiguous()
+    B = int(rng.integers(1, min(n // world, 100) + 1))
+    ranks = []
+    for r in range(world):
+        ip, idx = sharded.shard_csr(ip_t, ix_t, r, world)
+        lo, hi = sharded.shard_range(n, r, world)
+        ranks.append(sharded.ShardRank(gs, r, world, ip.cuda(), idx.cuda(), X[lo:hi].cuda().contiguous(), fanouts, W, seed,
+                                       shared, theta, max_seeds=B, max_requests=n))
+    O = oracle.Sampler(indptr, indices, fanouts, W, seed, shared)
+    O.set_theta(theta)
+    step = int(rng.integers(1, 2**32 - 10))
+    for b in range(3):
+        mode = str(rng.choice(["otf", "otf", "fcr", "fetch", "fbl"]))
+        rate = float(rng.choice([0.0, 0.1, 0.25, 0.5, 1.0]))
+        gm, om = MODES[mode]
+        pool = rng.permutation(n)[: world * B].astype(np.int32)                 # the ranks' seeds may not overlap within a rank
+        seeds = [torch.from_numpy(pool[r * B:(r + 1) * B].copy()) for r in range(world)]
+        res = sharded.sample_batch_local(ranks, [s_.cuda() for s_ in seeds], gm, rate, step + b,
+                                         features="peer" if rng.random() < 0.5 else True)
+        for r in range(world):
+            blocks, frontier, nn, m, feats = res[r]
+            fr_o, n_o, blocks_o = O.sample_batch(seeds[r].numpy(), om, rate, step + b)
+            assert nn == n_o and np.array_equal(frontier[: nn[L]].cpu().numpy(), fr_o)
+            for layer in range(L):
+                k = L - 1 - layer
+                assert np.array_equal(blocks[layer].indptr(nn[k]).cpu().numpy(), blocks_o[layer].indptr)
+                assert np.array_equal(blocks[layer].indices(m[layer]).cpu().numpy(), blocks_o[layer].indices)
+            assert torch.equal(feats[:, 0].cpu(), torch.from_numpy(fr_o.astype(np.float32)))
+    # the owners' rows, dense part
+    deg = np.diff(indptr)
+    dense = np.nonzero(deg > theta)[0].astype(np.int32)
+    S = sharded.rows_per_shard(n, world)
+    for layer in range(1 if shared else L):
+        want = O.cache_rows(layer, dense)
+        for r in range(world):
+            sel = (dense // S) == r
+            if sel.any():
+                got = gs.gs_cache_read_rows(ranks[r].cache, layer, torch.from_numpy(dense[sel]).cuda()).cpu().numpy()
+                assert np.array_equal(got, want[sel])
