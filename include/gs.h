@@ -67,6 +67,14 @@ gs_status gs_graph_create(int64_t num_nodes, int64_t num_edges, const int64_t* d
                           int32_t feat_dim, int64_t feat_ld, gs_graph** out);
 void gs_graph_destroy(gs_graph*);
 
+/* Optional one-pass check of the graph contract on the device: row offsets start at 0, end at
+ * num_edges and never decrease; every neighbour id lies in [0, num_nodes); each row is strictly
+ * ascending (sorted, no duplicate neighbour) - the sampler relies on all of it and does not
+ * re-check it per batch.  Synchronises `stream`.  *h_first_bad_row = -1 and GS_OK if the graph
+ * is valid, else the lowest offending row and GS_ERR_ARG.  Uses an 8-byte device variable of the
+ * library: calls must not overlap. */
+gs_status gs_graph_validate(const gs_graph*, void* stream, int64_t* h_first_bad_row);
+
 /* Bytes of device memory the cache needs: a small state header, the relabel table (8 bytes per
  * node) and the slot rows (num_hops caches, or one if shared != 0). */
 gs_status gs_cache_bytes(const gs_graph*, int32_t num_hops, int32_t cache_width, int32_t shared, size_t* bytes);

@@ -67,6 +67,7 @@ def _load():
     psz = ctypes.POINTER(sz)
     sig = {
         "gs_graph_create": [i64, i64, vp, vp, vp, ctypes.c_int, i32, i64, pvp],
+        "gs_graph_validate": [vp, vp, ctypes.POINTER(i64)],
         "gs_cache_bytes": [vp, i32, i32, i32, psz],
         "gs_workspace_bytes": [vp, i32, vp, i32, psz],
         "gs_cache_init": [vp, i32, vp, i32, u64, i32, vp, sz, vp, pvp],
@@ -227,6 +228,13 @@ def gs_graph_create(indptr: torch.Tensor, indices: torch.Tensor, features, dtype
     _check(_L.gs_graph_create(indptr.numel() - 1, indices.numel(), _ptr(indptr), _ptr(indices), _ptr(features),
                               dtype, feat_dim, feat_ld, ctypes.byref(h)))
     return Graph(h, indptr, indices, features, dtype, feat_dim)
+
+
+def gs_graph_validate(graph: Graph, stream=None) -> int:
+    """Checks the CSR contract on the device; returns -1, or raises GsError naming the first bad row."""
+    bad = ctypes.c_int64(-1)
+    _check(_L.gs_graph_validate(graph.handle, _stream(stream), ctypes.byref(bad)))
+    return int(bad.value)
 
 
 def gs_cache_bytes(graph: Graph, num_hops: int, cache_width: int, shared: bool) -> int:

@@ -165,6 +165,16 @@ gs_status gs_graph_create(int64_t num_nodes, int64_t num_edges, const int64_t* d
 
 void gs_graph_destroy(gs_graph* g) { delete g; }
 
+gs_status gs_graph_validate(const gs_graph* g, void* stream, int64_t* h_first_bad_row) {
+    if (!g || !h_first_bad_row) return fail(GS_ERR_ARG, "NULL argument");
+    GS_CUDA(launch_validate_graph(GraphView{g->d_indptr, g->d_indices, g->num_nodes}, g->num_edges, h_first_bad_row,
+                                  (cudaStream_t)stream));
+    if (*h_first_bad_row >= 0)
+        return fail(GS_ERR_ARG, "CSR row %lld breaks the graph contract (offsets, id range, or ids not strictly ascending)",
+                    (long long)*h_first_bad_row);
+    return GS_OK;
+}
+
 gs_status gs_cache_bytes(const gs_graph* g, int32_t num_hops, int32_t cache_width, int32_t shared, size_t* bytes) {
     if (!bytes) return fail(GS_ERR_ARG, "bytes is NULL");
     gs_status st = check_shape(g, num_hops, cache_width);

@@ -296,6 +296,47 @@ cudaError_t launch_relabel(const RelabelParams& p, int64_t m_bound, cudaStream_t
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------- graph contract check
+// One warp per row: offsets non-decreasing, the row inside [0, num_edges], neighbour ids inside
+// [0, num_nodes) and strictly ascending (sorted, no duplicate).  The lowest offending row wins.
+__device__ unsigned long long g_first_bad_row;
+
+__global__ void __launch_bounds__(256) k_validate_graph(GraphView g, long long num_edges, unsigned long long* bad) {
+    const int lane = threadIdx.x & 31;
+    const long long warps = (long long)gridDim.x * (blockDim.x >> 5);
+    for (long long v = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); v < g.num_nodes; v += warps) {
+        const long long lo = g.indptr[v], hi = g.indptr[v + 1];
+        bool wrong = lo > hi || lo < 0 || hi > num_edges || (v == 0 && lo != 0) || (v == g.num_nodes - 1 && hi != num_edges);
+        if (!wrong)
+            for (long long e = lo + lane; e < hi; e += 32) {
+                const int32_t u = g.indices[e];
+                if (u < 0 || (long long)u >= g.num_nodes || (e > lo && g.indices[e - 1] >= u)) wrong = true;
+            }
+        if (__any_sync(FULL, wrong) && lane == 0) atomicMin(bad, (unsigned long long)v);
+    }
+}
+
+cudaError_t launch_validate_graph(const GraphView& g, int64_t num_edges, int64_t* h_first_bad_row, cudaStream_t s) {
+    unsigned long long* d_bad = nullptr;
+    cudaError_t e = cudaGetSymbolAddress((void**)&d_bad, g_first_bad_row);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(d_bad, 0xFF, sizeof(unsigned long long), s);
+    if (e != cudaSuccess) return e;
+    int64_t blocks = (g.num_nodes + 7) / 8;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    k_validate_graph<<<(int)blocks, 256, 0, s>>>(g, (long long)num_edges, d_bad);
+    count_launches(1);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    unsigned long long h = 0;
+    e = cudaMemcpyAsync(&h, d_bad, sizeof(h), cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return e;
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return e;
+    *h_first_bad_row = (h == ~0ull) ? -1 : (int64_t)h;
+    return cudaSuccess;
+}
+
 // ---------------------------------------------------------------- logical cache rows (parity / debug)
 __global__ void k_read_rows(const int32_t* slots, const int32_t* row_index, int pitch, int W, const int32_t* nodes,
                             int n, int32_t* out) {

@@ -315,6 +315,34 @@ def test_randomised_configurations(case):
     pair.check_rows(C, O, np.arange(n))
 
 
+def test_graph_contract_check(tiny):
+    import paper_2406_17918_b200 as gs
+    assert gs.gs_graph_validate(tiny.G) == -1
+    indptr, indices = torch.from_numpy(tiny.indptr), torch.from_numpy(tiny.indices)
+    v = int(np.nonzero(tiny.deg >= 3)[0][5])
+    a = int(tiny.indptr[v])
+
+    def first_bad(ip, ix):
+        G = gs.gs_graph_create(ip.cuda(), ix.cuda(), None)
+        with pytest.raises(gs.GsError) as e:
+            gs.gs_graph_validate(G)
+        assert e.value.status == 1
+        return int(str(e.value).split("CSR row ")[1].split(" ")[0])
+
+    ix = indices.clone(); ix[a], ix[a + 1] = indices[a + 1], indices[a]          # not ascending
+    assert first_bad(indptr, ix) == v
+    ix = indices.clone(); ix[a + 1] = ix[a]                                        # duplicate neighbour
+    assert first_bad(indptr, ix) == v
+    ix = indices.clone(); ix[a + 2] = tiny.cfg["num_nodes"]                        # id out of range
+    assert first_bad(indptr, ix) == v
+    ix = indices.clone(); ix[a] = -4
+    assert first_bad(indptr, ix) == v
+    ip = indptr.clone(); ip[v + 1] = ip[v] - 1                                     # offsets decrease
+    assert first_bad(ip, indices) == v
+    ip = indptr.clone(); ip[-1] += 1                                               # last offset is not num_edges
+    assert first_bad(ip, indices) == tiny.cfg["num_nodes"] - 1
+
+
 def test_resume_from_export(tiny):
     import paper_2406_17918_b200 as gs
     B = tiny.cfg["batch"]
