@@ -501,6 +501,7 @@ def main():
         "feature_gbs": feat_rows_all * cfg["feat_dim"] * esize / secs / 1e9,
         "hbm_frac_batch": (alg_all / secs / 1e9) / peak / max(1, world),
         "hbm_frac_batch_incl_scanned_csr": ((alg_all + 16.0 * philox_all) / secs / 1e9) / peak / max(1, world),
+        "hbm_frac_batch_incl_scanned_csr_of_nominal_8tbs": ((alg_all + 16.0 * philox_all) / secs / 1e9) / 8000.0 / max(1, world),
         "n_gpus": world,
         "steps": K,
         "warmup": Wm,
