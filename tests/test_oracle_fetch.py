@@ -91,3 +91,23 @@ def test_fetch_special_cases_on_a_batch():
                 assert set(row[:n_cache].tolist()) <= set(frozen[layer][dst[p]].tolist())
     for l in range(L):
         assert np.array_equal(a.cache_rows(l, range(N)), frozen[l])
+
+
+def test_fetch_of_every_sample_with_fanout_equal_to_width_leaves_the_cache_alone():
+    """f = W and delta = 1: as many neighbours are fetched as a row has slots; the row is still not written."""
+    cfg = get_config("tiny", fanouts=[10, 10], cache_width=10)
+    g = build_graph(cfg)
+    indptr, indices = g.indptr.numpy(), g.indices.numpy()
+    perm = seed_permutation(cfg)
+    N = cfg["num_nodes"]
+    a = oracle.Sampler(indptr, indices, cfg["fanouts"], 10, seed=8)
+    frozen = [a.cache_rows(l, range(N)) for l in range(2)]
+    fr, n, blocks = a.sample_batch(batch_seeds(perm, 0, cfg["batch"]).numpy(), oracle.MODE_OTF_FETCH, 1.0, 1)
+    b = oracle.Sampler(indptr, indices, cfg["fanouts"], 10, seed=8)
+    fb, nb, bb = b.sample_batch(batch_seeds(perm, 0, cfg["batch"]).numpy(), oracle.MODE_FBL, 0.0, 1)
+    for l in range(2):
+        assert np.array_equal(a.cache_rows(l, range(N)), frozen[l])
+        assert blocks[l].num_edges == bb[l].num_edges
+    # the same neighbours as Full Batch Load (only the order inside a row, and with it the order in which new
+    # nodes enter the frontier, differs: key order here, offset order there)
+    assert n == nb and set(fr.tolist()) == set(fb.tolist())
