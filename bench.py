@@ -209,6 +209,9 @@ def main():
     ap.add_argument("--no-overlap", action="store_true",
                     help="run the feature gather of a batch on the sampling stream instead of a second stream "
                          "(where it overlaps the first, latency-bound hops of the next batch)")
+    ap.add_argument("--gather-grid", type=int, default=None,
+                    help="blocks per SM in the gather's grid (default: 1024 short blocks when it overlaps the next "
+                         "batch, 16 long-lived ones when it runs on the sampling stream)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -290,6 +293,8 @@ def main():
     # Two workspaces / output buffers alternate; the batch's row count is copied out of the state header before the
     # next batch clears it.
     overlap = not args.no_overlap
+    gather_grid = args.gather_grid if args.gather_grid else (1024 if overlap else 16)
+    gs.gs_graph_set_gather_grid(G, gather_grid)
     nbuf = 2 if overlap else 1
     ws_list = [ws] + [torch.empty_like(ws) for _ in range(nbuf - 1)]
     out_list = [None] * nbuf
@@ -371,6 +376,7 @@ def main():
     # the gather alone (nothing else on the GPU), on the last batch's input nodes: the kernel's own rate
     jl = (Wm + K - 1) % nbuf
     iso = []
+    gs.gs_graph_set_gather_grid(G, 16)      # alone, a few long-lived blocks per SM are the fastest launch shape
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)    # larger than L2: no row survives between launches
     for _ in range(8):
         flush.zero_()
@@ -381,6 +387,7 @@ def main():
         iso.append((ia, ib))
     torch.cuda.synchronize()
     gather_alone_ms = sorted(a.elapsed_time(b) for a, b in iso[2:])[len(iso[2:]) // 2]
+    gs.gs_graph_set_gather_grid(G, gather_grid)
     del flush
     if clocks:
         time.sleep(0.1)
@@ -473,7 +480,9 @@ def main():
                    "ms_per_launch": gather_ms_per_launch, "traffic": gather_traffic,
                    "concurrent_with_next_batch": overlap,
                    "alone": {"achieved": alone_gbs, "frac": alone_gbs / peak, "ms_per_launch": gather_alone_ms,
-                             "what": "the same launch with nothing else running, L2 flushed before each, median of 6"},
+                             "what": "the same rows with nothing else running and 16 blocks per SM in the grid, L2 flushed before each "
+                                     "launch, median of 6"},
+                   "grid_blocks_per_sm": gather_grid,
                    "traffic_note": "bytes per launch; read bytes scaled by rows from the ncu capture of workload shared "
                                    "(same 256-byte rows), written bytes algorithmic" if gather_traffic else
                                    "no capture with this row size scales by rows; see profiles/"}

@@ -67,6 +67,12 @@ gs_status gs_graph_create(int64_t num_nodes, int64_t num_edges, const int64_t* d
                           int32_t feat_dim, int64_t feat_ld, gs_graph** out);
 void gs_graph_destroy(gs_graph*);
 
+/* Launch shape of gs_gather_features for this graph: the grid has at most 148 * blocks_per_sm blocks
+ * of 256 threads (8 are resident per SM; a block copies rows until the grid has covered them all).
+ * 0 restores the default (256).  Few long-lived blocks (16) are fastest when the gather runs alone;
+ * many short ones (256 - 1024) let kernels of a concurrent higher-priority stream start at once. */
+gs_status gs_graph_set_gather_grid(gs_graph*, int32_t blocks_per_sm);
+
 /* Optional one-pass check of the graph contract on the device: row offsets start at 0, end at
  * num_edges and never decrease; every neighbour id lies in [0, num_nodes); each row is strictly
  * ascending (sorted, no duplicate neighbour) - the sampler relies on all of it and does not

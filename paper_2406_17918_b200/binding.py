@@ -68,6 +68,7 @@ def _load():
     sig = {
         "gs_graph_create": [i64, i64, vp, vp, vp, ctypes.c_int, i32, i64, pvp],
         "gs_graph_validate": [vp, vp, ctypes.POINTER(i64)],
+        "gs_graph_set_gather_grid": [vp, i32],
         "gs_cache_bytes": [vp, i32, i32, i32, psz],
         "gs_workspace_bytes": [vp, i32, vp, i32, psz],
         "gs_cache_init": [vp, i32, vp, i32, u64, i32, vp, sz, vp, pvp],
@@ -228,6 +229,10 @@ def gs_graph_create(indptr: torch.Tensor, indices: torch.Tensor, features, dtype
     _check(_L.gs_graph_create(indptr.numel() - 1, indices.numel(), _ptr(indptr), _ptr(indices), _ptr(features),
                               dtype, feat_dim, feat_ld, ctypes.byref(h)))
     return Graph(h, indptr, indices, features, dtype, feat_dim)
+
+
+def gs_graph_set_gather_grid(graph: Graph, blocks_per_sm: int):
+    _check(_L.gs_graph_set_gather_grid(graph.handle, int(blocks_per_sm)))
 
 
 def gs_graph_validate(graph: Graph, stream=None) -> int:

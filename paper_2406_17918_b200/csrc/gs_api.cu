@@ -17,6 +17,7 @@ struct gs_graph {
     int32_t feat_dim;
     int64_t feat_ld;
     int32_t elem_bytes;
+    int32_t gather_blocks_per_sm;   // grid of gs_gather_features; 0 = the library's default
 };
 
 struct gs_cache {
@@ -157,13 +158,20 @@ gs_status gs_graph_create(int64_t num_nodes, int64_t num_edges, const int64_t* d
         if (feat_ld < feat_dim) return fail(GS_ERR_ARG, "feat_ld %lld < feat_dim %d", (long long)feat_ld, feat_dim);
         if (!aligned(d_features, (size_t)eb)) return fail(GS_ERR_ALIGN, "d_features must be aligned to its element size");
     }
-    gs_graph* g = new (std::nothrow) gs_graph{num_nodes, num_edges, d_indptr, d_indices, d_features, dtype, feat_dim, feat_ld, eb};
+    gs_graph* g = new (std::nothrow) gs_graph{num_nodes, num_edges, d_indptr, d_indices, d_features, dtype, feat_dim, feat_ld, eb, 0};
     if (!g) return fail(GS_ERR_ARG, "out of host memory");
     *out = g;
     return GS_OK;
 }
 
 void gs_graph_destroy(gs_graph* g) { delete g; }
+
+gs_status gs_graph_set_gather_grid(gs_graph* g, int32_t blocks_per_sm) {
+    if (!g) return fail(GS_ERR_ARG, "graph is NULL");
+    if (blocks_per_sm < 0 || blocks_per_sm > 4096) return fail(GS_ERR_ARG, "blocks_per_sm outside [0, 4096]");
+    g->gather_blocks_per_sm = blocks_per_sm;
+    return GS_OK;
+}
 
 gs_status gs_graph_validate(const gs_graph* g, void* stream, int64_t* h_first_bad_row) {
     if (!g || !h_first_bad_row) return fail(GS_ERR_ARG, "NULL argument");
@@ -814,7 +822,7 @@ gs_status gs_gather_rows(const void* d_src, gs_dtype dtype, int32_t row_elems, i
     // ids are global; the source holds rows first_row, first_row + 1, ...: address row 0 where it would be
     const uintptr_t base = (uintptr_t)d_src - (uintptr_t)(first_row * src_ld * eb);
     GS_CUDA(launch_gather((const void*)base, src_ld * eb, (int64_t)row_elems * eb, d_ids, d_count_or_null, count_bound, d_out,
-                          out_ld * eb, (cudaStream_t)stream));
+                          out_ld * eb, 0, (cudaStream_t)stream));
     return GS_OK;
 }
 
@@ -897,7 +905,8 @@ gs_status gs_gather_features(const gs_graph* g, const int32_t* d_ids, const int3
     if (!aligned(d_out, (size_t)g->elem_bytes)) return fail(GS_ERR_ALIGN, "d_out must be aligned to the element size");
     if (!aligned(d_ids, 4)) return fail(GS_ERR_ALIGN, "d_ids must be 4-byte aligned");
     GS_CUDA(launch_gather(g->d_features, g->feat_ld * g->elem_bytes, (int64_t)g->feat_dim * g->elem_bytes, d_ids,
-                          d_count_or_null, count_bound, d_out, out_ld * g->elem_bytes, (cudaStream_t)stream));
+                          d_count_or_null, count_bound, d_out, out_ld * g->elem_bytes, g->gather_blocks_per_sm,
+                          (cudaStream_t)stream));
     return GS_OK;
 }
 

@@ -17,9 +17,11 @@ namespace gs {
 #ifndef GS_GATHER_MIN_BLOCKS
 #define GS_GATHER_MIN_BLOCKS 8
 #endif
-// Blocks per SM in the grid: 8 are resident, the rest queue behind them.  Many short blocks cost
-// nothing when the gather runs alone (measured: 16 and 256 per SM give the same time) and let the
-// small kernels of a concurrent, higher-priority stream get SM slots within microseconds.
+// Blocks per SM in the grid (default; gs_graph_set_gather_grid overrides it per graph): 8 are
+// resident, the rest queue behind them.  A few long-lived blocks are best when the gather has the GPU
+// to itself (16 per SM: 0.193 ms for 2 M rows of 256 bytes; 256: 0.205; 1024: 0.248); many short
+// blocks let the small kernels of a concurrent, higher-priority stream get SM slots within
+// microseconds instead of after half the gather.
 #ifndef GS_GATHER_GRID_PER_SM
 #define GS_GATHER_GRID_PER_SM 256
 #endif
@@ -134,12 +136,12 @@ cudaError_t launch_gather_sharded(const void* const* bases, int32_t world, int64
 
 template <typename V>
 static void launch_t(const void* src, int64_t src_ld, int64_t row_bytes, const int32_t* ids, const int32_t* d_count,
-                     int32_t count_bound, void* dst, int64_t dst_ld, cudaStream_t s) {
+                     int32_t count_bound, void* dst, int64_t dst_ld, int32_t blocks_per_sm, cudaStream_t s) {
     const int units = (int)(row_bytes / (int64_t)sizeof(V));
     const int tpr = units < GT ? units : GT;
     const int rows_per_iter = GT / tpr;
     int64_t blocks = ((int64_t)count_bound + (int64_t)rows_per_iter * G_UNROLL - 1) / ((int64_t)rows_per_iter * G_UNROLL);
-    const int64_t cap = 148 * GS_GATHER_GRID_PER_SM;
+    const int64_t cap = 148 * (int64_t)(blocks_per_sm > 0 ? blocks_per_sm : GS_GATHER_GRID_PER_SM);
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     k_gather<V><<<(int)blocks, GT, 0, s>>>((const char*)src, src_ld, units, ids, d_count, count_bound, (char*)dst, dst_ld);
@@ -147,14 +149,14 @@ static void launch_t(const void* src, int64_t src_ld, int64_t row_bytes, const i
 
 cudaError_t launch_gather(const void* src, int64_t src_ld_bytes, int64_t row_bytes, const int32_t* ids,
                           const int32_t* d_count, int32_t count_bound, void* dst, int64_t dst_ld_bytes,
-                          cudaStream_t s) {
+                          int32_t blocks_per_sm, cudaStream_t s) {
     if (count_bound <= 0 || row_bytes <= 0) return cudaSuccess;
     const uint64_t all = (uint64_t)(uintptr_t)src | (uint64_t)(uintptr_t)dst | (uint64_t)src_ld_bytes |
                          (uint64_t)dst_ld_bytes | (uint64_t)row_bytes;
-    if ((all & 15) == 0) launch_t<uint4>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, s);
-    else if ((all & 7) == 0) launch_t<uint2>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, s);
-    else if ((all & 3) == 0) launch_t<uint32_t>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, s);
-    else launch_t<uint16_t>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, s);
+    if ((all & 15) == 0) launch_t<uint4>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, blocks_per_sm, s);
+    else if ((all & 7) == 0) launch_t<uint2>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, blocks_per_sm, s);
+    else if ((all & 3) == 0) launch_t<uint32_t>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, blocks_per_sm, s);
+    else launch_t<uint16_t>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, blocks_per_sm, s);
     count_launches(1);
     return cudaGetLastError();
 }
