@@ -1,4 +1,4 @@
-// S0 static pre-sample, S1 refresh (FCR / OTF) and S2 pick, fused per frontier node.
+// S0 static pre-sample, S1 refresh (FCR / OTF, and the FBL / OTF Fetch variants) and S2 pick.
 //
 // Every selection is "the k items first in (key, index) order" with Philox keys that depend on
 // (node, item index, step) only - not on the neighbour ids.  The scan over a node's deg edge
@@ -13,13 +13,19 @@
 // entries, after removing retained neighbours, of the top-W list of ALL edge offsets in FILL
 // order, because at most W - r retained neighbours can precede the r-th winner.
 //
-// Two kernels per step:
-//   k_refresh_pick      one warp per frontier node, software-pipelined: while the neighbour ids
-//                       of node i are in flight the warp already scans node i+1.  Nodes above the
-//                       hub degree are only registered, as a list of 4096-offset chunks.
-//   k_refresh_pick_hub  one warp per chunk; candidates go to a per-hub buffer in global memory,
-//                       and the warp that finishes a hub's last chunk completes the node.  No
-//                       warp ever waits for another one.
+// Kernels:
+//   k_scan + k_finish   every batch (see "split path" below): a pure Philox threshold scan over the
+//                       rows above SMALL_DEGREE, then one warp per frontier node for eviction,
+//                       refill, row update and pick.
+//   k_refresh_pick      refresh (+ optional pick) fused in one warp per node, software-pipelined:
+//                       while the neighbour ids of node i are in flight the warp already scans node
+//                       i+1.  Used where every node of a range is refreshed - the static pre-sample
+//                       and the whole-cache refresh.  Nodes above the hub degree are only
+//                       registered, as a list of 4096-offset chunks.
+//   k_refresh_pick_hub  one warp per chunk of a registered hub; candidates go to a per-hub buffer
+//                       in global memory, and the warp that finishes a hub's last chunk completes
+//                       the node.  Also redoes the long rows k_finish could not decide from their
+//                       candidate lists.  No warp ever waits for another one.
 #include "gs_device.cuh"
 #include "gs_internal.h"
 
