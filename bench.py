@@ -196,6 +196,9 @@ def main():
                     help="sampling mode (default: the config's OTF run); fbl = no cache, the paper's baseline "
                          "sampler; fetch = OTF Fetch")
     ap.add_argument("--rate", type=float, default=None, help="gamma (otf) or delta (fetch); default: the config's")
+    ap.add_argument("--fanouts", default=None, help="comma-separated fan-outs, input layer first (default: the workload's)")
+    ap.add_argument("--cache-width", type=int, default=None, help="cache width W (default: the workload's)")
+    ap.add_argument("--shared-cache", type=int, default=None, choices=[0, 1], help="one cache for all hops (default: the workload's)")
     ap.add_argument("--theta", type=int, default=None,
                     help="dense/sparse split: cache rows only for nodes with degree > theta (default: one row per node)")
     ap.add_argument("--period", type=int, default=None,
@@ -221,7 +224,14 @@ def main():
     from paper_2406_17918_b200 import replicas
 
     rank, local_rank, world = replicas.env_rank()
-    cfg = get_config(args.workload)
+    over = {}
+    if args.fanouts:
+        over["fanouts"] = [int(x) for x in args.fanouts.split(",")]
+    if args.cache_width:
+        over["cache_width"] = args.cache_width
+    if args.shared_cache is not None:
+        over["shared"] = bool(args.shared_cache)
+    cfg = get_config(args.workload, **over)
     mode, gamma = run_spec(cfg)
     if args.mode and args.mode != mode:
         mode, gamma = args.mode, {"fcr": 1.0, "fbl": 0.0, "fetch": 0.5, "otf": gamma}[args.mode]
