@@ -42,7 +42,7 @@ SAMPLER_SEED = 0x6A09E667F3BCC908
 #     rows mean fewer items per block, which makes the per-block scaling an upper estimate for the scale workload.
 #   k_gather with 256-byte bf16 rows, workload shared, batch 0: 13,165,824 B read for 50,620 rows (260 B per row: the
 #     row and its id); the 256 B written per row were still in L2 when that short launch ended, so the written bytes
-#     are counted as the algorithmic ones.  400-byte fp32 rows (workload large): 144,186,880 B read + 68,389,120 B
+#     are counted as the algorithmic ones.  400-byte fp32 rows (workload large): 144,179,968 B read + 67,727,104 B
 #     written (the rest still in L2) for 282 K rows: 1.28 x the algorithmic read (rows start on 16-byte boundaries).
 NCU_SCAN_BYTES_PER_BLOCK = (5653248 + 12544) / 16380004
 NCU_GATHER_READ_BYTES_PER_256B_ROW = 13165824 / 50620

@@ -244,7 +244,7 @@ gs_status gs_batch_counts(gs_cache*, void* stream, int32_t* h_num_nodes, int32_t
 
 /* Feature gather (the paper's "load embeddings", Section "System Components"):
  * out[p, :] = features[ids[p], :] for p < count, a bitwise copy.
- *   d_ids            int32 ids in [0, num_nodes)
+ *   d_ids            int32 ids in [0, num_nodes); any other id is skipped (its output row is left as it is)
  *   d_count_or_null  device scalar with the row count, or NULL to use count_bound
  *   count_bound      rows d_out has room for (and the count, when d_count_or_null is NULL)
  *   d_out            [count_bound][out_ld] elements of the graph's dtype, out_ld >= feat_dim
@@ -253,11 +253,11 @@ gs_status gs_gather_features(const gs_graph*, const int32_t* d_ids, const int32_
                              int32_t count_bound, void* d_out, int64_t out_ld, void* stream);
 
 /* out[i, :] = src[ids[i] - first_row, :] for any row-major matrix on the device (the copy kernel
- * of gs_gather_features).  `src` holds rows first_row, first_row + 1, ... of a larger matrix - a
- * feature shard - and ids are global; every id must lie inside the rows that `src` holds (not
- * checked); negative ids are skipped.  row_elems, src_ld, out_ld in elements of `dtype`. */
+ * of gs_gather_features).  `src` holds the src_rows rows first_row, first_row + 1, ... of a larger
+ * matrix - a feature shard - and ids are global; an id outside [first_row, first_row + src_rows)
+ * is skipped (its output row is left as it is).  row_elems, src_ld, out_ld in elements of `dtype`. */
 gs_status gs_gather_rows(const void* d_src, gs_dtype dtype, int32_t row_elems, int64_t src_ld, int64_t first_row,
-                         const int32_t* d_ids, const int32_t* d_count_or_null, int32_t count_bound, void* d_out,
+                         int64_t src_rows, const int32_t* d_ids, const int32_t* d_count_or_null, int32_t count_bound, void* d_out,
                          int64_t out_ld, void* stream);
 
 /* The feature step of a sharded run as ONE kernel over peer memory: out[i, :] = row ids[i] of a

@@ -85,7 +85,7 @@ def _load():
         "gs_cache_export": [vp, vp, sz, vp],
         "gs_cache_import": [vp, vp, sz, vp],
         "gs_sync_status": [vp, vp],
-        "gs_gather_rows": [vp, ctypes.c_int, i32, i64, i64, vp, vp, i32, vp, i64, vp],
+        "gs_gather_rows": [vp, ctypes.c_int, i32, i64, i64, i64, vp, vp, i32, vp, i64, vp],
         "gs_gather_rows_peer": [vp, i32, i64, ctypes.c_int, i32, i64, vp, vp, i32, vp, i64, vp],
         "gs_shard_bucket": [vp, i32, i64, i32, vp, vp, vp, vp],
         "gs_shard_workspace_bytes": [vp, i32, i32, psz],
@@ -395,7 +395,7 @@ def gs_gather_rows(src: torch.Tensor, ids: torch.Tensor, out: torch.Tensor, firs
         raise TypeError("ids must be an int32 CUDA tensor")
     dtype = {torch.float32: GS_F32, torch.bfloat16: GS_BF16}[src.dtype]
     bound = min(out.shape[0], ids.numel())
-    _check(_L.gs_gather_rows(_ptr(src), dtype, src.shape[1], src.stride(0), int(first_row), _ptr(ids), _ptr(count), bound,
+    _check(_L.gs_gather_rows(_ptr(src), dtype, src.shape[1], src.stride(0), int(first_row), src.shape[0], _ptr(ids), _ptr(count), bound,
                              _ptr(out), out.stride(0), _stream(stream)))
     return out
 

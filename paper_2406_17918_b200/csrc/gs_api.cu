@@ -809,7 +809,7 @@ gs_status gs_shard_extend(gs_cache* c, int32_t k, const int32_t* d_seeds, int32_
 }
 
 gs_status gs_gather_rows(const void* d_src, gs_dtype dtype, int32_t row_elems, int64_t src_ld, int64_t first_row,
-                         const int32_t* d_ids, const int32_t* d_count_or_null, int32_t count_bound, void* d_out,
+                         int64_t src_rows, const int32_t* d_ids, const int32_t* d_count_or_null, int32_t count_bound, void* d_out,
                          int64_t out_ld, void* stream) {
     if (dtype != GS_F32 && dtype != GS_BF16) return fail(GS_ERR_ARG, "unknown dtype %d", (int)dtype);
     const int64_t eb = dtype == GS_BF16 ? 2 : 4;
@@ -817,12 +817,12 @@ gs_status gs_gather_rows(const void* d_src, gs_dtype dtype, int32_t row_elems, i
     if (count_bound == 0) return GS_OK;
     if (!d_src || !d_ids || !d_out) return fail(GS_ERR_ARG, "NULL argument");
     if (row_elems < 1 || src_ld < row_elems || out_ld < row_elems) return fail(GS_ERR_ARG, "bad row size or pitch");
-    if (first_row < 0) return fail(GS_ERR_ARG, "first_row is negative");
+    if (first_row < 0 || src_rows < 1) return fail(GS_ERR_ARG, "first_row is negative or the source has no rows");
     if (!aligned(d_src, (size_t)eb) || !aligned(d_out, (size_t)eb) || !aligned(d_ids, 4)) return fail(GS_ERR_ALIGN, "misaligned argument");
     // ids are global; the source holds rows first_row, first_row + 1, ...: address row 0 where it would be
     const uintptr_t base = (uintptr_t)d_src - (uintptr_t)(first_row * src_ld * eb);
     GS_CUDA(launch_gather((const void*)base, src_ld * eb, (int64_t)row_elems * eb, d_ids, d_count_or_null, count_bound, d_out,
-                          out_ld * eb, 0, (cudaStream_t)stream));
+                          out_ld * eb, 0, first_row, first_row + src_rows, (cudaStream_t)stream));
     return GS_OK;
 }
 
@@ -905,8 +905,8 @@ gs_status gs_gather_features(const gs_graph* g, const int32_t* d_ids, const int3
     if (!aligned(d_out, (size_t)g->elem_bytes)) return fail(GS_ERR_ALIGN, "d_out must be aligned to the element size");
     if (!aligned(d_ids, 4)) return fail(GS_ERR_ALIGN, "d_ids must be 4-byte aligned");
     GS_CUDA(launch_gather(g->d_features, g->feat_ld * g->elem_bytes, (int64_t)g->feat_dim * g->elem_bytes, d_ids,
-                          d_count_or_null, count_bound, d_out, out_ld * g->elem_bytes, g->gather_blocks_per_sm,
-                          (cudaStream_t)stream));
+                          d_count_or_null, count_bound, d_out, out_ld * g->elem_bytes, g->gather_blocks_per_sm, 0,
+                          g->num_nodes, (cudaStream_t)stream));
     return GS_OK;
 }
 

@@ -34,7 +34,8 @@ template <typename V> __device__ __forceinline__ void st_stream(V* p, V v) { __s
 template <typename V>
 __global__ void __launch_bounds__(GT, GS_GATHER_MIN_BLOCKS) k_gather(const char* __restrict__ src, int64_t src_ld, int units,
                                                const int32_t* __restrict__ ids, const int32_t* __restrict__ d_count,
-                                               int count_bound, char* __restrict__ dst, int64_t dst_ld) {
+                                               int count_bound, char* __restrict__ dst, int64_t dst_ld, int id_lo,
+                                               int id_hi) {
     int n = d_count ? __ldg(d_count) : count_bound;
     if (n > count_bound) n = count_bound;
     // thread -> (row within group, first unit); tpr threads per row
@@ -51,7 +52,8 @@ __global__ void __launch_bounds__(GT, GS_GATHER_MIN_BLOCKS) k_gather(const char*
         for (int j = 0; j < G_UNROLL; ++j) {
             const int64_t rj = row + j * stride;
             const int32_t id = rj < n ? __ldg(ids + rj) : -1;
-            s[j] = id >= 0 ? reinterpret_cast<const V*>(src + (int64_t)id * src_ld) : nullptr;
+            // an id outside the rows the source holds is skipped: its output row is left as it is
+            s[j] = (id >= id_lo && id < id_hi) ? reinterpret_cast<const V*>(src + (int64_t)id * src_ld) : nullptr;
             d[j] = reinterpret_cast<V*>(dst + rj * dst_ld);
         }
         for (int u = u0; u < units; u += tpr) {
@@ -136,7 +138,8 @@ cudaError_t launch_gather_sharded(const void* const* bases, int32_t world, int64
 
 template <typename V>
 static void launch_t(const void* src, int64_t src_ld, int64_t row_bytes, const int32_t* ids, const int32_t* d_count,
-                     int32_t count_bound, void* dst, int64_t dst_ld, int32_t blocks_per_sm, cudaStream_t s) {
+                     int32_t count_bound, void* dst, int64_t dst_ld, int32_t blocks_per_sm, int id_lo, int id_hi,
+                     cudaStream_t s) {
     const int units = (int)(row_bytes / (int64_t)sizeof(V));
     const int tpr = units < GT ? units : GT;
     const int rows_per_iter = GT / tpr;
@@ -144,19 +147,22 @@ static void launch_t(const void* src, int64_t src_ld, int64_t row_bytes, const i
     const int64_t cap = 148 * (int64_t)(blocks_per_sm > 0 ? blocks_per_sm : GS_GATHER_GRID_PER_SM);
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    k_gather<V><<<(int)blocks, GT, 0, s>>>((const char*)src, src_ld, units, ids, d_count, count_bound, (char*)dst, dst_ld);
+    k_gather<V><<<(int)blocks, GT, 0, s>>>((const char*)src, src_ld, units, ids, d_count, count_bound, (char*)dst, dst_ld,
+                                           id_lo, id_hi);
 }
 
 cudaError_t launch_gather(const void* src, int64_t src_ld_bytes, int64_t row_bytes, const int32_t* ids,
                           const int32_t* d_count, int32_t count_bound, void* dst, int64_t dst_ld_bytes,
-                          int32_t blocks_per_sm, cudaStream_t s) {
+                          int32_t blocks_per_sm, int64_t id_lo, int64_t id_hi, cudaStream_t s) {
     if (count_bound <= 0 || row_bytes <= 0) return cudaSuccess;
+    if (id_lo < 0) id_lo = 0;
+    if (id_hi > 0x7FFFFFFFll) id_hi = 0x7FFFFFFFll;
     const uint64_t all = (uint64_t)(uintptr_t)src | (uint64_t)(uintptr_t)dst | (uint64_t)src_ld_bytes |
                          (uint64_t)dst_ld_bytes | (uint64_t)row_bytes;
-    if ((all & 15) == 0) launch_t<uint4>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, blocks_per_sm, s);
-    else if ((all & 7) == 0) launch_t<uint2>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, blocks_per_sm, s);
-    else if ((all & 3) == 0) launch_t<uint32_t>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, blocks_per_sm, s);
-    else launch_t<uint16_t>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, blocks_per_sm, s);
+    if ((all & 15) == 0) launch_t<uint4>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, blocks_per_sm, (int)id_lo, (int)id_hi, s);
+    else if ((all & 7) == 0) launch_t<uint2>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, blocks_per_sm, (int)id_lo, (int)id_hi, s);
+    else if ((all & 3) == 0) launch_t<uint32_t>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, blocks_per_sm, (int)id_lo, (int)id_hi, s);
+    else launch_t<uint16_t>(src, src_ld_bytes, row_bytes, ids, d_count, count_bound, dst, dst_ld_bytes, blocks_per_sm, (int)id_lo, (int)id_hi, s);
     count_launches(1);
     return cudaGetLastError();
 }

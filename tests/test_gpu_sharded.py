@@ -123,6 +123,14 @@ def test_bucket_and_gather_rows_primitives():
     out = torch.empty((333, 24), dtype=torch.bfloat16, device="cuda")
     gs.gs_gather_rows(X[400:700], ids, out, first_row=400)
     assert torch.equal(out, X[ids.long()])
+    # ids outside the rows the source holds are skipped
+    ids2 = ids.clone()
+    ids2[3], ids2[4], ids2[5] = 399, 700, -2
+    out2 = torch.full((333, 24), 9, dtype=torch.bfloat16, device="cuda")
+    gs.gs_gather_rows(X[400:700], ids2, out2, first_row=400)
+    keep = torch.ones(333, dtype=torch.bool, device="cuda")
+    keep[3:6] = False
+    assert torch.equal(out2[keep], X[ids2[keep].long()]) and bool((out2[~keep] == 9).all())
     # the same matrix as three shards of ceil(1000/3) rows, each at its own address
     parts = [X[0:334].clone(), X[334:668].clone(), X[668:1000].clone()]
     ids = torch.from_numpy(rng.integers(0, 1000, 4001).astype(np.int32)).cuda()
