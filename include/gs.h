@@ -313,7 +313,8 @@ gs_status gs_shard_status(gs_cache*, void* stream);
  * in d_sorted order; d_slot[n_k] as returned by gs_shard_bucket for frontier_k.  k = 0 starts a new
  * batch and takes the seeds (distinct, as for gs_sample_batch); later hops ignore d_seeds and
  * num_seeds.  The workspace is the one of gs_sample_batch (gs_workspace_bytes for num_seeds) and
- * must stay untouched between the hops of a batch.  Fills *block like gs_sample_batch fills
+ * must stay untouched between the hops of a batch.  A slot outside [0, n_k) or a pick outside
+ * [0, num_nodes) sets the device status GS_ERR_RANGE (see gs_batch_counts).  Fills *block like gs_sample_batch fills
  * blocks[L-1-k]; *d_frontier is the frontier array (frontier_{k+1} is its prefix of
  * *block->d_num_src ids).  Counts: gs_batch_counts, as after gs_sample_batch. */
 gs_status gs_shard_extend(gs_cache*, int32_t k, const int32_t* d_seeds, int32_t num_seeds, const int32_t* d_reply,

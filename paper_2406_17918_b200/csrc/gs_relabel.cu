@@ -65,8 +65,13 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
         }
         if (v >= 0 && P.reply) {
             // sharded run, requester side: the owners have sampled; a row's picks are the non-negative prefix
-            const int32_t* row = P.reply + (int64_t)(P.slot ? P.slot[p] : p) * P.f;
-            while (c < P.f && __ldg(row + c) >= 0) ++c;
+            const int sl = P.slot ? P.slot[p] : p;
+            if ((unsigned)sl >= (unsigned)n) {
+                raise_status(status, GS_ERR_RANGE);   // not a row of the reply: the node gets no picks
+            } else {
+                const int32_t* row = P.reply + (int64_t)sl * P.f;
+                while (c < P.f && __ldg(row + c) >= 0) ++c;
+            }
         } else if (v >= 0) {
             const int64_t deg = P.g.indptr[v + 1] - P.g.indptr[v];
             c = deg < (int64_t)P.f ? (int)deg : P.f;

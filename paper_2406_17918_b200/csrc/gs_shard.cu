@@ -111,7 +111,9 @@ __global__ void __launch_bounds__(SHARD_THREADS) k_import_picks(const int32_t* _
     const int64_t i = (int64_t)blockIdx.x * SHARD_THREADS + threadIdx.x;
     if (i >= (int64_t)n * f) return;
     const int p = (int)(i / f), t = (int)(i - (int64_t)p * f);
-    const int32_t u = __ldg(reply + (int64_t)(slot ? __ldg(slot + p) : p) * f + t);
+    const int sl = slot ? __ldg(slot + p) : p;
+    if ((unsigned)sl >= (unsigned)n) return;      // reported by the row-count kernel; the row has no picks
+    const int32_t u = __ldg(reply + (int64_t)sl * f + t);
     if (u < 0) return;
     if ((int64_t)u >= num_nodes) {
         atomicCAS(status, 0, GS_ERR_RANGE);

@@ -181,6 +181,18 @@ def test_sharded_entry_points_reject_bad_arguments():
     block, frontier = gs.gs_shard_extend(fresh.cache, 0, nodes, reply, slot, fresh.ws)
     n, m = gs.gs_batch_counts(fresh.cache)
     assert n[:2] == [8, 8] and m[-1] == 0 and torch.equal(frontier[:8], nodes)
+    # a slot that is not a row of the reply, a pick that is not a node: reported, nothing is read or written out of bounds
+    for bad_slot, bad_pick in ((True, False), (False, True)):
+        other = Setup("tiny", 1, theta=12).ranks[0]
+        sl, rp = slot.clone(), reply.clone()
+        if bad_slot:
+            sl[2] = 8
+        if bad_pick:
+            rp[3, 0] = s.cfg["num_nodes"]
+        gs.gs_shard_extend(other.cache, 0, nodes, rp, sl, other.ws)
+        with pytest.raises(gs.GsError) as e:
+            gs.gs_batch_counts(other.cache)
+        assert e.value.status == 3
     with pytest.raises(gs.GsError):
         gs.gs_shard_bucket(nodes, 100, 65)
     with pytest.raises(gs.GsError):
