@@ -1089,8 +1089,10 @@ cudaError_t launch_finish(const StepParams& p, int64_t n_bound, cudaStream_t s) 
     fb = fb > cap ? cap : (fb < 1 ? 1 : fb);
     k_finish<<<(int)fb, RP_THREADS, 0, s>>>(p);
     int launched = 1;
-    if (p.hub_cap > 0) {   // rows queued for a rescan (rare); exits at once when there are none
-        k_refresh_pick_hub<<<(int)cap, RP_THREADS, 0, s>>>(p);
+    if (p.hub_cap > 0) {   // rows queued for a rescan; exits at once when there are none
+        // a partial refresh queues a handful of rows per batch at most, a full one about 1 % of them
+        const int64_t hub_grid = (p.r >= p.W) ? cap : 148 * 2;
+        k_refresh_pick_hub<<<(int)hub_grid, RP_THREADS, 0, s>>>(p);
         launched = 2;
     }
     count_launches(launched);
