@@ -33,18 +33,21 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
     __shared__ int is_last;
     __shared__ int s_status;
     int32_t* status = P.hdr + HDR_STATUS;
-    if (threadIdx.x == 0) s_status = __ldcg(status);
+    if (threadIdx.x == 0) {
+        s_status = __ldcg(status);
+        is_last = 0;
+    }
     __syncthreads();
     if (s_status != 0) return;  // block-uniform: the barriers below stay convergent
     const int n = (P.k == 0) ? P.n_host : __ldcg(P.hdr + HDR_N + P.k);
-    // the grid is sized for the worst case; only the tiles that hold frontier nodes take part
+    // a capped grid walks the tiles that hold frontier nodes (the host only knows an upper bound of n)
     const int tiles = (n + SCAN_A_TILE - 1) / SCAN_A_TILE;
-    if ((int)blockIdx.x >= tiles) return;
-    const int p = blockIdx.x * SCAN_A_TILE + threadIdx.x;
+    const int refresh_from = P.d_refresh_from ? __ldcg(P.d_refresh_from) : 0;
+    for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    const int p = tile * SCAN_A_TILE + threadIdx.x;
     int c = 0;
     int nch = 0;   // scan work items of this node
     unsigned quads = 0, refreshed = 0;
-    const int refresh_from = P.d_refresh_from ? __ldcg(P.d_refresh_from) : 0;
     if (p < n) {
         int v;
         if (P.k == 0) {
@@ -97,13 +100,15 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
         if (p < n) P.item_start[p] = excl2;
     }
     if (threadIdx.x == 0) {
-        P.tile_sums2[blockIdx.x] = total2;
-        P.tile_sums[blockIdx.x] = total;
+        P.tile_sums2[tile] = total2;
+        P.tile_sums[tile] = total;
         __threadfence();
         const int ticket = atomicAdd(P.hdr + HDR_TICKET_A + P.k, 1);
         is_last = (ticket == tiles - 1);
     }
     __syncthreads();
+    if (is_last) break;   // every tile is done (this block's later ones included): finish below
+    }
     if (!is_last) return;
     __threadfence();
     const int m = scan_tiles_in_place<SCAN_A_TILE>(P.tile_sums, tiles, warp_sums);
@@ -118,7 +123,8 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
 __global__ void __launch_bounds__(1024) k_row_offsets(CountParams P) {
     if (__ldcg(P.hdr + HDR_STATUS) != 0) return;
     const int n = (P.k == 0) ? P.n_host : __ldcg(P.hdr + HDR_N + P.k);
-    const int p = blockIdx.x * SCAN_A_TILE + threadIdx.x;
+    for (int t = blockIdx.x; t <= n / SCAN_A_TILE; t += gridDim.x) {   // the tile of position n takes part too
+    const int p = t * SCAN_A_TILE + threadIdx.x;
     if (p < n) P.blk_indptr[p] += P.tile_sums[p / SCAN_A_TILE];
     else if (p == n) P.blk_indptr[n] = __ldcg(P.hdr + HDR_M + P.k);
     // scan work items: node p owns items [item_start[p], item_start[p+1]), one per chunk of its row
@@ -138,12 +144,15 @@ __global__ void __launch_bounds__(1024) k_row_offsets(CountParams P) {
     } else if (p == n) {
         P.item_start[n] = __ldcg(P.hdr + HDR_ITEMS + P.k);
     }
+    }
 }
 
 cudaError_t launch_row_counts(const CountParams& p, int64_t n_bound, cudaStream_t s) {
-    const int tiles = (int)((n_bound + SCAN_A_TILE - 1) / SCAN_A_TILE);
-    k_row_counts<<<tiles, SCAN_A_TILE, 0, s>>>(p);
-    k_row_offsets<<<(int)(n_bound / SCAN_A_TILE) + 1, SCAN_A_TILE, 0, s>>>(p);
+    // at most two resident blocks of 1,024 threads per SM; blocks walk the tiles that exist
+    int64_t tiles = n_bound / SCAN_A_TILE + 1;
+    if (tiles > 148 * 2) tiles = 148 * 2;
+    k_row_counts<<<(int)tiles, SCAN_A_TILE, 0, s>>>(p);
+    k_row_offsets<<<(int)tiles, SCAN_A_TILE, 0, s>>>(p);
     count_launches(2);
     return cudaGetLastError();
 }
@@ -164,16 +173,19 @@ __global__ void __launch_bounds__(FF_THREADS) k_first_flags(RelabelParams P) {
     __shared__ int s_wtot[FF_THREADS / 32];
     __shared__ int is_last;
     __shared__ int s_status;
-    if (threadIdx.x == 0) s_status = __ldcg(P.hdr + HDR_STATUS);
+    if (threadIdx.x == 0) {
+        s_status = __ldcg(P.hdr + HDR_STATUS);
+        is_last = 0;
+    }
     __syncthreads();
     if (s_status != 0) return;  // block-uniform
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int n = __ldcg(P.hdr + HDR_N + P.k);
     const int m = __ldcg(P.hdr + HDR_M + P.k);
-    // worst-case grid: tiles beyond the picks leave at once (at least one tile stays, to publish n_{k+1})
+    // a capped grid walks the tiles that hold picks (at least one, to publish n_{k+1})
     const int tiles = m > 0 ? (m + SCAN_E_TILE - 1) / SCAN_E_TILE : 1;
-    if ((int)blockIdx.x >= tiles) return;
-    const int wbase = blockIdx.x * SCAN_E_TILE + wid * 512;
+    for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    const int wbase = tile * SCAN_E_TILE + wid * 512;
     // 16 independent table probes per thread are in flight before anything is consumed
     int id[4][4];
     int pos[4][4];
@@ -234,12 +246,14 @@ __global__ void __launch_bounds__(FF_THREADS) k_first_flags(RelabelParams P) {
         }
     }
     if (threadIdx.x == 0) {
-        P.tile_sums[blockIdx.x] = total;
+        P.tile_sums[tile] = total;
         __threadfence();
         const int ticket = atomicAdd(P.hdr + HDR_TICKET_E + P.k, 1);
         is_last = (ticket == tiles - 1);
     }
-    __syncthreads();
+    __syncthreads();   // also keeps s_wtot of this tile intact until every warp has read it
+    if (is_last) break;
+    }
     if (!is_last) return;
     __threadfence();
     const int fresh = scan_tiles_in_place<FF_THREADS>(P.tile_sums, tiles, warp_sums);
@@ -292,8 +306,9 @@ __global__ void __launch_bounds__(256) k_relabel(RelabelParams P) {
 
 cudaError_t launch_relabel(const RelabelParams& p, int64_t m_bound, cudaStream_t s) {
     if (m_bound <= 0) m_bound = 1;
-    const int tiles = (int)((m_bound + SCAN_E_TILE - 1) / SCAN_E_TILE);
-    k_first_flags<<<tiles, FF_THREADS, 0, s>>>(p);
+    int64_t tiles = (m_bound + SCAN_E_TILE - 1) / SCAN_E_TILE;
+    if (tiles > 148 * 16) tiles = 148 * 16;    // blocks walk the tiles; enough of them that a usual batch has one tile each
+    k_first_flags<<<(int)tiles, FF_THREADS, 0, s>>>(p);
     int64_t blocks = (m_bound + 1023) / 1024;
     if (blocks > 148 * 32) blocks = 148 * 32;
     k_relabel<<<(int)blocks, 256, 0, s>>>(p);
