@@ -37,14 +37,14 @@ PHILOX_LANE_OPS = 60.0
 SAMPLER_SEED = 0x6A09E667F3BCC908
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one captured launch, from the ncu summaries under
 # profiles/ (captures on the small workloads; scaled to a launch of the benchmarked workload by the units processed).
-#   k_scan, workload large, sampling step 2 of batch 0: 5,653,248 B read + 12,544 B written for 16,380,004 Philox
+#   k_scan, workload large, sampling step 2 of batch 0: 5,650,944 B read + 12,288 B written for 16,380,004 Philox
 #     blocks in 45,281 work items.  The traffic is the items' descriptors, so it follows the number of items; larger
 #     rows mean fewer items per block, which makes the per-block scaling an upper estimate for the scale workload.
 #   k_gather with 256-byte bf16 rows, workload shared, batch 0: 13,165,824 B read for 50,620 rows (260 B per row: the
 #     row and its id); the 256 B written per row were still in L2 when that short launch ended, so the written bytes
-#     are counted as the algorithmic ones.  400-byte fp32 rows (workload large): 144,179,968 B read + 67,727,104 B
+#     are counted as the algorithmic ones.  400-byte fp32 rows (workload large): 144,189,696 B read + 67,959,552 B
 #     written (the rest still in L2) for 282 K rows: 1.28 x the algorithmic read (rows start on 16-byte boundaries).
-NCU_SCAN_BYTES_PER_BLOCK = (5653248 + 12544) / 16380004
+NCU_SCAN_BYTES_PER_BLOCK = (5650944 + 12288) / 16380004
 NCU_GATHER_READ_BYTES_PER_256B_ROW = 13165824 / 50620
 
 
