@@ -3,9 +3,14 @@
 
 One step = one mini-batch through the whole path: gs_sample_batch (refresh + pick + relabel +
 block CSR for every hop) followed by gs_gather_features for the input nodes, on fresh seeds and
-the next step number (the cache evolves as in training).
+the next step number (the cache evolves as in training).  By default a batch's gather runs on a
+second stream and overlaps the first hops of the next batch (--no-overlap: one stream).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload scale|large|shared|mid|tiny]
+                    [--mode otf|fcr|fbl|fetch] [--rate R] [--fanouts a,b,c] [--cache-width W] [--shared-cache 0|1]
+                    [--theta T]        dense/sparse split cache
+                    [--period T]       whole-cache refresh every T-th batch, pick-only batches
+                    [--sharded]        node-sharded run (one all-to-all round trip per hop)
     python bench.py --impl reference ...        # times the CPU oracle on a bounded sample
 
 Prints ONE JSON line on rank 0.
