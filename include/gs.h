@@ -20,7 +20,7 @@
  *   - Graph contract: CSR row v lists the in-neighbours of v in ascending order without
  *     duplicates; num_nodes < 2^31; indptr is int64, ids are int32.
  *   - Fan-outs are listed input-layer-first.  Sampling step k = 0..L-1 starts at the seeds and
- *     uses layer l = L-1-k (the paper's loop "for l = L to 1", Algorithm 2 SampleBlocks).
+ *     uses layer l = L-1-k (the layer loop of SampleBlocks in Algorithm 2 runs from the last layer down).
  *   - Randomness: every choice orders items by (key32(item), item) ascending where key32(i) is
  *     word (i & 3) of Philox4x32-10(counter = (i >> 2, node, step, (purpose << 8) | tag),
  *     key = (seed low word, seed high word)); purpose 1 = FILL over edge offsets of the node's
@@ -67,7 +67,7 @@ gs_status gs_graph_create(int64_t num_nodes, int64_t num_edges, const int64_t* d
                           int32_t feat_dim, int64_t feat_ld, gs_graph** out);
 void gs_graph_destroy(gs_graph*);
 
-/* Launch shape of gs_gather_features for this graph: the grid has at most 148 * blocks_per_sm blocks
+/* Launch shape of gs_gather_features for this graph: the grid has at most (SM count) * blocks_per_sm blocks
  * of 256 threads (8 are resident per SM; a block copies rows until the grid has covered them all).
  * 0 restores the default (256).  Few long-lived blocks (16) are fastest when the gather runs alone;
  * many short ones (256 - 1024) let kernels of a concurrent higher-priority stream start at once. */
@@ -89,8 +89,8 @@ gs_status gs_cache_bytes(const gs_graph*, int32_t num_hops, int32_t cache_width,
  * per-hop block arrays returned by gs_sample_batch live inside it. */
 gs_status gs_workspace_bytes(const gs_graph*, int32_t num_hops, const int32_t* fanouts, int32_t max_seeds, size_t* bytes);
 
-/* Static pre-sample (paper Algorithm 2, Initialize: "Pre-sample cache for each layer l"; Section
- * "Static and Dynamic Sampling").  For every node and every layer (one row per node if shared):
+/* Static pre-sample (paper Algorithm 2, Initialize step; Section "Static and Dynamic
+ * Sampling").  For every node and every layer (one row per node if shared):
  * degree <= cache_width -> the row is the adjacency in CSR order, remaining slots -1; otherwise
  * the row holds the cache_width neighbours first in FILL order at step 0, in that order.
  *   fanouts          h_ int32[num_hops], each in [1, cache_width]
@@ -122,8 +122,8 @@ gs_status gs_cache_init_split(const gs_graph*, int32_t num_hops, const int32_t* 
                               uint64_t seed, int32_t shared, int32_t theta, int64_t dense_rows,
                               void* d_cache_storage, size_t cache_bytes, void* stream, gs_cache** out);
 
-/* Whole-cache refresh: the refresh exactly as Algorithms 2 and 3 write it ("if t mod T = 0":
- * RefreshCache / CacheRefresh for l = 1..L) - every cached row of every layer's cache, not only the
+/* Whole-cache refresh: the refresh exactly as Algorithms 2 and 3 write it (their periodic-refresh
+ * condition on the batch counter t and the interval T: RefreshCache / CacheRefresh over all layers) - every cached row of every layer's cache, not only the
  * rows of a batch's frontier.  The caller owns the schedule: every T-th batch it calls this with
  * that batch's step, and samples all batches with gs_sample_batch(GS_MODE_OTF, gamma = 0), which is
  * SampleFromCache alone.
@@ -194,8 +194,9 @@ typedef struct {
     int64_t indices_capacity;
 } gs_block_buffers;
 
-/* Bytes of the scratch array built into the library for gs_sample_batch_noalloc.  Every GPU that
- * loads the library holds this much device memory from load until the process exits. */
+/* Bytes of the scratch array built into the library for gs_sample_batch_noalloc.  A GPU holds this
+ * much device memory from the first gs_cache_init / gs_cache_init_split on it (which looks the
+ * array up, the moment the CUDA runtime creates it there) until the process exits. */
 #define GS_NOALLOC_SCRATCH_BYTES (64u << 20)
 
 /* The same mini-batch as gs_sample_batch, for callers that cannot provide a scratch workspace
@@ -204,11 +205,15 @@ typedef struct {
  * has no counterpart to this call; it exists only for such deployments.  It allocates nothing
  * (no cudaMalloc / cudaFree, no allocating library routine): the scratch is a fixed array of
  * GS_NOALLOC_SCRATCH_BYTES inside the library, and the results go to buffers the caller passes:
- *   d_input_nodes   int32[input_nodes_capacity] receives the input-node list (the last frontier)
+ *   d_input_nodes   int32[input_nodes_capacity] receives the input-node list (the last frontier);
+ *                   4-byte aligned
  *   h_buffers       h_ array of num_hops entries, by layer: where each block's offsets and
  *                   block-local source ids go.  With n_0 = num_seeds, m_k = n_k * fanout of step k
  *                   and n_{k+1} = min(num_nodes, n_k + m_k), the block of step k needs n_k + 1
  *                   offsets and m_k indices, and the input-node list needs n_L ids.
+ *                   d_indptr must be 4-byte aligned and d_indices 16-BYTE aligned (the ids are
+ *                   stored four at a time); a caller that carves its arrays out of one buffer
+ *                   rounds each d_indices start up to 16 bytes.  GS_ERR_ALIGN otherwise.
  *   blocks          filled as by gs_sample_batch, pointing into the caller's buffers
  *   d_num_input_nodes  receives a device pointer to the count (may be NULL)
  * Everything else (seeds, mode, gamma, step, results, status reporting through gs_batch_counts) is
@@ -216,9 +221,13 @@ typedef struct {
  * Limits and rules
  *   - A batch needs as much scratch as gs_workspace_bytes reports for it; if that exceeds
  *     GS_NOALLOC_SCRATCH_BYTES the call returns GS_ERR_WORKSPACE (message with both sizes) and
- *     launches nothing.  Too-small output buffers are rejected the same way.
- *   - The first call on each device looks up the device address of the built-in array (with that
- *     device current).  Make that first call outside any stream capture.
+ *     launches nothing.  Too-small output buffers are rejected the same way, misaligned ones with
+ *     GS_ERR_ALIGN; every check runs on the host before the first launch.
+ *   - The device address of the built-in array is looked up once per device, with that device
+ *     current: by gs_cache_init / gs_cache_init_split, which is also when the array starts to
+ *     occupy memory there, so a deployment sees the full footprint at set-up.  Should the first
+ *     use on a device be this call itself (a cache created while another device was current), the
+ *     lookup happens here: make that first call outside any stream capture.
  *   - All calls on a device share the one array and it keeps the previous call's contents; the
  *     kernels initialise every part of it they read, so nothing has to be cleared between calls.
  *     Two calls whose kernels overlap on the GPU (different streams, different caches) race on
@@ -358,6 +367,12 @@ gs_status gs_sync_status(gs_cache*, void* stream);
  * refill, and the degree above which a whole thread block scans one node.  Values <= 0 keep the
  * defaults. */
 gs_status gs_cache_set_tuning(gs_cache*, double lambda_otf, double lambda_full, int32_t hub_degree);
+
+/* Test knob, process-wide: no kernel of the library is launched with more than max_blocks thread
+ * blocks (0 restores the designed grids).  Every kernel walks its work with a grid-stride or
+ * work-counter loop, so results never depend on the grid; tests use caps of 1-3 blocks to make
+ * each block walk many tiles, a path the designed grids only take on the largest batches. */
+gs_status gs_debug_set_grid_cap(int32_t max_blocks);
 
 /* Number of kernels this library has launched in the calling process (monotonic). */
 int64_t gs_kernel_launches(void);

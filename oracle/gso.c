@@ -310,8 +310,8 @@ int gso_refresh_node(gso_sampler* s, int32_t layer, int32_t v, uint32_t step, in
     return 0;
 }
 
-/* The refresh as Algorithms 2 and 3 state it ("if t mod T = 0": RefreshCache / CacheRefresh for
- * l = 1..L): every row of every layer's cache, not only the rows of the batch's frontier.
+/* The refresh as Algorithms 2 and 3 state it (their periodic branch: RefreshCache / CacheRefresh over
+ * all layers): every row of every layer's cache, not only the rows of the batch's frontier.
  * With a dense/sparse split only the dense part has rows. */
 int gso_refresh_all(gso_sampler* s, int mode, double gamma, uint32_t step) {
     if (!s || step == 0) return 1;

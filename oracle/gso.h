@@ -19,7 +19,7 @@
  * Conventions
  *   - CSR row v lists the in-neighbours of v, ascending, no duplicates; indptr int64, ids int32.
  *   - fan-outs are listed input-layer-first; sampling step k = 0..L-1 starts at the seeds and
- *     uses layer l = L-1-k (the paper's loop "for l = L to 1").
+ *     uses layer l = L-1-k (SampleBlocks in Algorithms 2 and 3 walks the layers from the last down).
  *   - item order: a precedes b  <=>  (key32(a), a) < (key32(b), b).
  *   - key32(i) = word (i & 3) of Philox4x32-10(counter = (i >> 2, v, step, (purpose << 8) | tag),
  *     key = (seed low word, seed high word)); purpose 1 = FILL over edge offsets,

@@ -96,6 +96,7 @@ def _load():
         "gs_cache_profile_begin": [vp, i32],
         "gs_cache_profile_end": [vp, vp, vp, vp],
         "gs_cache_set_tuning": [vp, dbl, dbl, i32],
+        "gs_debug_set_grid_cap": [i32],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -288,7 +289,7 @@ def gs_cache_init_split(graph: Graph, fanouts, cache_width: int, seed: int, shar
 
 
 def gs_cache_refresh_all(cache: Cache, mode: int, gamma: float, step: int, stream=None) -> None:
-    """Refresh every cached row of every layer (the 't mod T = 0' branch of Algorithms 2 and 3)."""
+    """Refresh every cached row of every layer (the periodic-refresh branch of Algorithms 2 and 3)."""
     _check(_L.gs_cache_refresh_all(cache.handle, mode, float(gamma), step, _stream(stream)))
 
 
@@ -505,6 +506,11 @@ def gs_cache_profile_end(cache: Cache, stream=None):
 
 def gs_sync_status(cache: Cache, stream=None):
     _check(_L.gs_sync_status(cache.handle, _stream(stream)))
+
+
+def gs_debug_set_grid_cap(max_blocks: int):
+    """Process-wide test knob: cap every kernel's grid at max_blocks blocks (0 = designed grids)."""
+    _check(_L.gs_debug_set_grid_cap(int(max_blocks)))
 
 
 def gs_cache_set_tuning(cache: Cache, lambda_otf=0.0, lambda_full=0.0, hub_degree=0):

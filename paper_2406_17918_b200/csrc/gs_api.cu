@@ -54,6 +54,26 @@ static std::atomic<long long> g_launches{0};
 
 void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+static std::atomic<int> g_sm_count[64];     // per device ordinal, 0 = not looked up yet
+static std::atomic<int> g_grid_cap{0};      // test knob: 0 = grids as designed
+
+int64_t sm_count() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    int n = g_sm_count[dev].load(std::memory_order_relaxed);
+    if (n <= 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        g_sm_count[dev].store(n, std::memory_order_relaxed);
+    }
+    return n;
+}
+
+int64_t limit_grid(int64_t blocks) {
+    const int cap = g_grid_cap.load(std::memory_order_relaxed);
+    if (cap > 0 && blocks > cap) blocks = cap;
+    return blocks < 1 ? 1 : blocks;
+}
+
 static gs_status fail(gs_status code, const char* fmt, ...) {
     va_list ap;
     va_start(ap, fmt);
@@ -140,6 +160,12 @@ extern "C" {
 const char* gs_last_error(void) { return g_err; }
 int32_t gs_stats_word_offset(void) { return HDR_STAT_SLOW; }
 int64_t gs_kernel_launches(void) { return (int64_t)g_launches.load(); }
+
+gs_status gs_debug_set_grid_cap(int32_t max_blocks) {
+    if (max_blocks < 0) return fail(GS_ERR_ARG, "max_blocks is negative");
+    g_grid_cap.store(max_blocks, std::memory_order_relaxed);
+    return GS_OK;
+}
 
 gs_status gs_graph_create(int64_t num_nodes, int64_t num_edges, const int64_t* d_indptr, const int32_t* d_indices,
                           const void* d_features, gs_dtype dtype, int32_t feat_dim, int64_t feat_ld, gs_graph** out) {
@@ -294,6 +320,10 @@ static gs_status cache_init_impl(const gs_graph* g, int32_t num_hops, const int3
     else st = gs_cache_bytes(g, num_hops, cache_width, shared, &need);
     if (st != GS_OK) return st;
     if (cache_bytes < need) return fail(GS_ERR_WORKSPACE, "cache storage has %zu bytes, %zu needed", cache_bytes, need);
+
+    // the built-in scratch array of gs_sample_batch_noalloc comes into being on this device now, not in a later batch
+    st = prepare_noalloc_scratch();
+    if (st != GS_OK) return st;
 
     gs_cache* c = new (std::nothrow) gs_cache{};
     if (!c) return fail(GS_ERR_ARG, "out of host memory");
@@ -641,6 +671,11 @@ static gs_status check_batch_args(gs_cache* c, const int32_t* seeds, int32_t num
 
 namespace gs {
 int32_t cache_num_hops(const gs_cache* c) { return c ? c->L : 0; }
+
+gs_status cache_workspace_bytes(const gs_cache* c, int32_t num_seeds, size_t* bytes) {
+    if (!c) return fail(GS_ERR_ARG, "cache is NULL");
+    return gs_workspace_bytes(c->graph, c->L, c->fanouts, num_seeds, bytes);
+}
 
 gs_status sample_batch_checked(gs_cache* c, const int32_t* d_seeds, int32_t num_seeds, gs_mode mode, double gamma,
                                uint32_t step, void* d_workspace, size_t workspace_bytes, cudaStream_t s,

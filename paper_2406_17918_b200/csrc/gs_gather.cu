@@ -109,7 +109,7 @@ static void launch_sharded_t(const ShardBases& sh, int num_rows, int rows_per_sh
     const int tpr = units < GT ? units : GT;
     const int rows_per_iter = GT / tpr;
     int64_t blocks = ((int64_t)count_bound + rows_per_iter - 1) / rows_per_iter;
-    const int64_t cap = 148 * GS_GATHER_GRID_PER_SM;
+    const int64_t cap = sm_count() * GS_GATHER_GRID_PER_SM;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     k_gather_sharded<V><<<(int)blocks, GT, 0, s>>>(sh, num_rows, rows_per_shard, src_ld, units, ids, d_count, count_bound,
@@ -144,9 +144,10 @@ static void launch_t(const void* src, int64_t src_ld, int64_t row_bytes, const i
     const int tpr = units < GT ? units : GT;
     const int rows_per_iter = GT / tpr;
     int64_t blocks = ((int64_t)count_bound + (int64_t)rows_per_iter * G_UNROLL - 1) / ((int64_t)rows_per_iter * G_UNROLL);
-    const int64_t cap = 148 * (int64_t)(blocks_per_sm > 0 ? blocks_per_sm : GS_GATHER_GRID_PER_SM);
+    const int64_t cap = sm_count() * (int64_t)(blocks_per_sm > 0 ? blocks_per_sm : GS_GATHER_GRID_PER_SM);
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
+    blocks = limit_grid(blocks);
     k_gather<V><<<(int)blocks, GT, 0, s>>>((const char*)src, src_ld, units, ids, d_count, count_bound, (char*)dst, dst_ld,
                                            id_lo, id_hi);
 }

@@ -207,6 +207,10 @@ struct RelabelParams {
 };
 
 void count_launches(int n);
+// Streaming multiprocessors of the current device (looked up once per device).
+int64_t sm_count();
+// Grid size after the test knob gs_debug_set_grid_cap (0 = no cap) has been applied.
+int64_t limit_grid(int64_t blocks);
 
 // Caller-owned output buffers that replace the output regions of the workspace (used by the
 // entry point whose scratch is a static device array).  Arrays are indexed by layer.
@@ -226,6 +230,10 @@ gs_status sample_batch_checked(gs_cache* c, const int32_t* d_seeds, int32_t num_
                                const OutputBuffers* out);
 gs_status set_error(gs_status code, const char* fmt, ...);
 int32_t cache_num_hops(const gs_cache* c);
+// Scratch bytes a batch of num_seeds seeds on this cache needs (what gs_workspace_bytes reports).
+gs_status cache_workspace_bytes(const gs_cache* c, int32_t num_seeds, size_t* bytes);
+// Looks up (and thereby materialises) the built-in scratch array of gs_sample_batch_noalloc on the current device.
+gs_status prepare_noalloc_scratch();
 
 cudaError_t launch_row_counts(const CountParams& p, int64_t n_bound, cudaStream_t s);
 cudaError_t launch_refresh_pick(const StepParams& p, int64_t n_bound, cudaStream_t s);

@@ -5,8 +5,10 @@
 // handed buffers by its host application and may not grow the process' footprint, or a service
 // with a fixed memory budget that is audited at start-up.  gs_sample_batch asks such a caller for
 // a scratch workspace it has no way to provide.  This variant keeps the scratch inside the
-// library instead, in a file-scope device array of fixed size that every GPU using the library
-// holds from load to exit; the caller passes only inputs and outputs.
+// library instead, in a file-scope device array of fixed size; the caller passes only inputs and
+// outputs.  The CUDA runtime materialises that array on a GPU the first time its address is
+// looked up there, which gs_cache_init does (prepare_noalloc_scratch below), so the memory is
+// taken at set-up, not in the middle of training, and is held until the process exits.
 #include <cstdio>
 #include <mutex>
 
@@ -40,6 +42,15 @@ static gs_status scratch_address(void** out) {
     return GS_OK;
 }
 
+// Called by gs_cache_init / gs_cache_init_split with the cache's device current: looks the address
+// up early, so that the array exists before the first batch and before any stream capture.
+gs_status prepare_noalloc_scratch() {
+    void* unused = nullptr;
+    return scratch_address(&unused);
+}
+
+static bool is_aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
 }  // namespace gs
 
 using namespace gs;
@@ -51,8 +62,25 @@ extern "C" gs_status gs_sample_batch_noalloc(gs_cache* cache, const int32_t* d_s
     if (!cache) return set_error(GS_ERR_ARG, "cache is NULL");
     if (!h_buffers) return set_error(GS_ERR_ARG, "h_buffers is NULL");
     if (!blocks) return set_error(GS_ERR_ARG, "blocks is NULL");
+    // The relabel kernel stores block-local ids four at a time: 16-byte stores into d_indices.
+    // Inside a workspace those arrays start on 256-byte boundaries; here they are the caller's, so
+    // the requirement is checked before anything is launched.
+    if (!is_aligned(d_input_nodes, 4)) return set_error(GS_ERR_ALIGN, "d_input_nodes must be 4-byte aligned");
+    const int32_t hops = cache_num_hops(cache);
+    for (int l = 0; l < hops; ++l) {
+        if (!is_aligned(h_buffers[l].d_indptr, 4))
+            return set_error(GS_ERR_ALIGN, "h_buffers[%d].d_indptr must be 4-byte aligned", l);
+        if (!is_aligned(h_buffers[l].d_indices, 16))
+            return set_error(GS_ERR_ALIGN, "h_buffers[%d].d_indices must be 16-byte aligned", l);
+    }
+    size_t need = 0;
+    gs_status st = cache_workspace_bytes(cache, num_seeds, &need);
+    if (st != GS_OK) return st;
+    if (need > (size_t)GS_NOALLOC_SCRATCH_BYTES)
+        return set_error(GS_ERR_WORKSPACE, "gs_sample_batch_noalloc: this batch needs %zu bytes of scratch, the built-in scratch "
+                         "array has %u", need, (unsigned)GS_NOALLOC_SCRATCH_BYTES);
     void* scratch = nullptr;
-    gs_status st = scratch_address(&scratch);
+    st = scratch_address(&scratch);
     if (st != GS_OK) return st;
     OutputBuffers out{};
     out.input_nodes = d_input_nodes;
@@ -62,7 +90,6 @@ extern "C" gs_status gs_sample_batch_noalloc(gs_cache* cache, const int32_t* d_s
         out.indptr[l] = nullptr;
         out.indices[l] = nullptr;
     }
-    const int32_t hops = cache_num_hops(cache);
     for (int l = 0; l < hops; ++l) {
         out.indptr[l] = h_buffers[l].d_indptr;
         out.indptr_capacity[l] = h_buffers[l].indptr_capacity;
@@ -70,16 +97,7 @@ extern "C" gs_status gs_sample_batch_noalloc(gs_cache* cache, const int32_t* d_s
         out.indices_capacity[l] = h_buffers[l].indices_capacity;
     }
     const int32_t* d_in = nullptr;
-    // A batch whose scratch does not fit the array fails here with GS_ERR_WORKSPACE and a message
-    // that names both sizes; nothing is launched in that case.
-    st = sample_batch_checked(cache, d_seeds, num_seeds, mode, gamma, step, scratch, (size_t)GS_NOALLOC_SCRATCH_BYTES,
-                              (cudaStream_t)stream, blocks, &d_in, d_num_input_nodes, &out);
-    if (st == GS_ERR_WORKSPACE) {
-        // keep the message of the size check, but say which buffer it is about
-        char msg[400];
-        snprintf(msg, sizeof(msg), "%s", gs_last_error());
-        return set_error(GS_ERR_WORKSPACE, "gs_sample_batch_noalloc (built-in scratch of %u bytes): %s",
-                         (unsigned)GS_NOALLOC_SCRATCH_BYTES, msg);
-    }
-    return st;
+    // Output buffers that are too small fail in here with GS_ERR_WORKSPACE, before any launch.
+    return sample_batch_checked(cache, d_seeds, num_seeds, mode, gamma, step, scratch, (size_t)GS_NOALLOC_SCRATCH_BYTES,
+                                (cudaStream_t)stream, blocks, &d_in, d_num_input_nodes, &out);
 }

@@ -1075,23 +1075,23 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
 }
 
 cudaError_t launch_scan(const StepParams& p, int64_t item_bound, cudaStream_t s) {
-    const int64_t cap = 148 * GS_SCAN_GRID_PER_SM;
+    const int64_t cap = sm_count() * GS_SCAN_GRID_PER_SM;
     int64_t sb = (item_bound + RP_WARPS - 1) / RP_WARPS;
-    sb = sb > cap ? cap : (sb < 1 ? 1 : sb);
+    sb = limit_grid(sb > cap ? cap : (sb < 1 ? 1 : sb));
     k_scan<<<(int)sb, RP_THREADS, 0, s>>>(p);
     count_launches(1);
     return cudaGetLastError();
 }
 
 cudaError_t launch_finish(const StepParams& p, int64_t n_bound, cudaStream_t s) {
-    const int64_t cap = 148 * 8;
+    const int64_t cap = sm_count() * 8;
     int64_t fb = (n_bound + RP_WARPS - 1) / RP_WARPS;
-    fb = fb > cap ? cap : (fb < 1 ? 1 : fb);
+    fb = limit_grid(fb > cap ? cap : (fb < 1 ? 1 : fb));
     k_finish<<<(int)fb, RP_THREADS, 0, s>>>(p);
     int launched = 1;
     if (p.hub_cap > 0) {   // rows queued for a rescan; exits at once when there are none
         // a partial refresh queues a handful of rows per batch at most, a full one about 1 % of them
-        const int64_t hub_grid = (p.r >= p.W) ? cap : 148 * 2;
+        const int64_t hub_grid = limit_grid((p.r >= p.W) ? cap : sm_count() * 2);
         k_refresh_pick_hub<<<(int)hub_grid, RP_THREADS, 0, s>>>(p);
         launched = 2;
     }
@@ -1117,20 +1117,21 @@ __global__ void __launch_bounds__(256) k_init_low_rows(GraphView g, int32_t* slo
 
 cudaError_t launch_init_low_rows(const GraphView& g, int32_t* slots, int32_t pitch, int32_t W, int32_t caches,
                                  cudaStream_t s) {
-    k_init_low_rows<<<148 * 16, 256, 0, s>>>(g, slots, pitch, W, caches);
+    k_init_low_rows<<<(int)(sm_count() * 16), 256, 0, s>>>(g, slots, pitch, W, caches);
     count_launches(1);
     return cudaGetLastError();
 }
 
 cudaError_t launch_refresh_pick(const StepParams& p, int64_t n_bound, cudaStream_t s) {
     int64_t blocks = (n_bound + RP_WARPS - 1) / RP_WARPS;
-    const int64_t cap = 148 * 8;
+    const int64_t cap = sm_count() * 8;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
+    blocks = limit_grid(blocks);
     k_refresh_pick<<<(int)blocks, RP_THREADS, 0, s>>>(p);
     int launched = 1;
     if (p.hub_cap > 0) {
-        k_refresh_pick_hub<<<(int)cap, RP_THREADS, 0, s>>>(p);
+        k_refresh_pick_hub<<<(int)limit_grid(cap), RP_THREADS, 0, s>>>(p);
         launched = 2;
     }
     count_launches(launched);

@@ -150,7 +150,8 @@ __global__ void __launch_bounds__(1024) k_row_offsets(CountParams P) {
 cudaError_t launch_row_counts(const CountParams& p, int64_t n_bound, cudaStream_t s) {
     // at most two resident blocks of 1,024 threads per SM; blocks walk the tiles that exist
     int64_t tiles = n_bound / SCAN_A_TILE + 1;
-    if (tiles > 148 * 2) tiles = 148 * 2;
+    if (tiles > sm_count() * 2) tiles = sm_count() * 2;
+    tiles = limit_grid(tiles);
     k_row_counts<<<(int)tiles, SCAN_A_TILE, 0, s>>>(p);
     k_row_offsets<<<(int)tiles, SCAN_A_TILE, 0, s>>>(p);
     count_launches(2);
@@ -307,10 +308,12 @@ __global__ void __launch_bounds__(256) k_relabel(RelabelParams P) {
 cudaError_t launch_relabel(const RelabelParams& p, int64_t m_bound, cudaStream_t s) {
     if (m_bound <= 0) m_bound = 1;
     int64_t tiles = (m_bound + SCAN_E_TILE - 1) / SCAN_E_TILE;
-    if (tiles > 148 * 16) tiles = 148 * 16;    // blocks walk the tiles; enough of them that a usual batch has one tile each
+    if (tiles > sm_count() * 16) tiles = sm_count() * 16;    // blocks walk the tiles; enough of them that a usual batch has one tile each
+    tiles = limit_grid(tiles);
     k_first_flags<<<(int)tiles, FF_THREADS, 0, s>>>(p);
     int64_t blocks = (m_bound + 1023) / 1024;
-    if (blocks > 148 * 32) blocks = 148 * 32;
+    if (blocks > sm_count() * 32) blocks = sm_count() * 32;
+    blocks = limit_grid(blocks);
     k_relabel<<<(int)blocks, 256, 0, s>>>(p);
     count_launches(2);
     return cudaGetLastError();
@@ -343,7 +346,7 @@ cudaError_t launch_validate_graph(const GraphView& g, int64_t num_edges, int64_t
     e = cudaMemsetAsync(d_bad, 0xFF, sizeof(unsigned long long), s);
     if (e != cudaSuccess) return e;
     int64_t blocks = (g.num_nodes + 7) / 8;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks > sm_count() * 16) blocks = sm_count() * 16;
     k_validate_graph<<<(int)blocks, 256, 0, s>>>(g, (long long)num_edges, d_bad);
     count_launches(1);
     e = cudaGetLastError();

@@ -1,4 +1,4 @@
-"""Pins of the oracle's whole-cache periodic refresh (Algorithms 2 and 3: 'if t mod T = 0')."""
+"""Pins of the oracle's whole-cache periodic refresh (the periodic branch of Algorithms 2 and 3, taken every T-th batch)."""
 import numpy as np
 import pytest
 

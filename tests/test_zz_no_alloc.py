@@ -96,3 +96,64 @@ def test_noalloc_rejects_what_does_not_fit():
     gs.gs_sample_batch_noalloc(C, perm[:1024].cuda(), gs.GS_MODE_OTF, 0.3, 1, inp, ip, ix)
     n, m = gs.gs_batch_counts(C)
     assert n[0] == 1024 and n[L] <= nb[L] and all(x > 0 for x in m)
+
+
+def test_noalloc_refuses_misaligned_output_buffers_before_any_launch():
+    """A caller that packs its int32 arrays back to back can end up with a d_indices that is only
+    4-byte aligned; the ids are stored 16 bytes at a time, so the call must refuse such a buffer
+    on the host (GS_ERR_ALIGN) and launch nothing.  Only the refusal is exercised here."""
+    import paper_2406_17918_b200 as gs
+
+    cfg = get_config("tiny")
+    g = build_graph(cfg).to("cuda")
+    perm = seed_permutation(cfg)
+    G = gs.gs_graph_create(g.indptr, g.indices, None)
+    fan, W, B, L = cfg["fanouts"], cfg["cache_width"], cfg["batch"], len(cfg["fanouts"])
+    C = gs.gs_cache_init(G, fan, W, 5, False)
+    gs.gs_sync_status(C)
+    nb, mb = _bounds(cfg["num_nodes"], fan, B)
+    inp = torch.zeros(nb[L], dtype=torch.int32, device="cuda")
+    ip = [torch.zeros(nb[L - 1 - l] + 1, dtype=torch.int32, device="cuda") for l in range(L)]
+    ix_big = [torch.zeros(mb[L - 1 - l] + 4, dtype=torch.int32, device="cuda") for l in range(L)]
+    seeds = batch_seeds(perm, 0, B).cuda()
+    launches = gs.gs_kernel_launches()
+    for shift in (1, 2, 3):
+        ix = [t[shift:] for t in ix_big]            # 4-, 8- and 12-byte offsets from a 16-byte boundary
+        assert ix[0].data_ptr() % 16 != 0
+        with pytest.raises(gs.GsError) as e:
+            gs.gs_sample_batch_noalloc(C, seeds, gs.GS_MODE_OTF, 0.25, 1, inp, ip, ix)
+        assert e.value.status == 2 and "16-byte" in str(e.value)
+    assert gs.gs_kernel_launches() == launches      # refused on the host: nothing ran
+    # the same buffers at an aligned offset are accepted
+    gs.gs_sample_batch_noalloc(C, seeds, gs.GS_MODE_OTF, 0.25, 1, inp, ip, [t[4:] for t in ix_big])
+    n, m = gs.gs_batch_counts(C)
+    assert n[0] == B
+
+
+def test_noalloc_call_leaves_device_memory_unchanged():
+    """The built-in scratch array is materialised when the cache is created (gs_cache_init looks its
+    address up), so a batch through the no-allocation call must not change the free device memory."""
+    import paper_2406_17918_b200 as gs
+
+    cfg = get_config("tiny")
+    g = build_graph(cfg).to("cuda")
+    perm = seed_permutation(cfg)
+    G = gs.gs_graph_create(g.indptr, g.indices, None)
+    fan, W, B, L = cfg["fanouts"], cfg["cache_width"], cfg["batch"], len(cfg["fanouts"])
+    C = gs.gs_cache_init(G, fan, W, 9, False)
+    nb, mb = _bounds(cfg["num_nodes"], fan, B)
+    inp = torch.zeros(nb[L], dtype=torch.int32, device="cuda")
+    ip = [torch.zeros(nb[L - 1 - l] + 1, dtype=torch.int32, device="cuda") for l in range(L)]
+    ix = [torch.zeros(mb[L - 1 - l], dtype=torch.int32, device="cuda") for l in range(L)]
+    seeds = [batch_seeds(perm, b, B).cuda() for b in range(3)]
+    # first batch: the CUDA runtime loads the kernels' code on first use, which is not the call's doing
+    gs.gs_sample_batch_noalloc(C, seeds[2], gs.GS_MODE_OTF, 0.25, 1, inp, ip, ix)
+    gs.gs_sync_status(C)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for b in range(2):
+        gs.gs_sample_batch_noalloc(C, seeds[b], gs.GS_MODE_OTF, 0.25, b + 2, inp, ip, ix)
+    gs.gs_sync_status(C)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
