@@ -3,8 +3,9 @@
 
 One step = one mini-batch through the whole path: gs_sample_batch (refresh + pick + relabel +
 block CSR for every hop) followed by gs_gather_features for the input nodes, on fresh seeds and
-the next step number (the cache evolves as in training).  By default a batch's gather runs on a
-second stream and overlaps the first hops of the next batch (--no-overlap: one stream).
+the next step number (the cache evolves as in training).  The headline leg runs every batch start
+to end on one stream; a second leg (skipped with --no-overlap) runs each batch's gather on a second
+stream beside the first hops of the next batch and is reported beside it under "pipelined".
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload scale|large|shared|mid|tiny]
                     [--mode otf|fcr|fbl|fetch] [--rate R] [--fanouts a,b,c] [--cache-width W] [--shared-cache 0|1]
@@ -35,20 +36,15 @@ from workloads import batch_seeds, build_features, build_graph, get_config, seed
 
 METRIC = "sampled edges/s + feature GB/s per batch (OTF), fraction of HBM roofline"
 FALLBACK_HBM_GBS = 6650.0
-# INT32 ALU peak of one B200: 148 SMs x 128 lanes x 1.965 GHz lane-ops/s.  One Philox4x32-10 block needs
-# ten rounds of two 32x32->64 multiplies (two lane-ops each on this GPU) and two 3-input xors: 60 lane-ops.
-ALU_LANE_OPS = 148 * 128 * 1.965e9
-PHILOX_LANE_OPS = 60.0
 SAMPLER_SEED = 0x6A09E667F3BCC908
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one captured launch, from the ncu summaries under
-# profiles/ (captures on the small workloads; scaled to a launch of the benchmarked workload by the units processed).
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one captured launch, from ncu captures of the same
+# kernels on small workloads (scaled to a launch of the benchmarked workload by the units it processes).
 #   k_scan, workload large, sampling step 2 of batch 0: 5,650,944 B read + 12,288 B written for 16,380,004 Philox
 #     blocks in 45,281 work items.  The traffic is the items' descriptors, so it follows the number of items; larger
 #     rows mean fewer items per block, which makes the per-block scaling an upper estimate for the scale workload.
 #   k_gather with 256-byte bf16 rows, workload shared, batch 0: 13,165,824 B read for 50,620 rows (260 B per row: the
 #     row and its id); the 256 B written per row were still in L2 when that short launch ended, so the written bytes
-#     are counted as the algorithmic ones.  400-byte fp32 rows (workload large): 144,189,696 B read + 67,959,552 B
-#     written (the rest still in L2) for 282 K rows: 1.28 x the algorithmic read (rows start on 16-byte boundaries).
+#     are counted as the algorithmic ones.
 NCU_SCAN_BYTES_PER_BLOCK = (5650944 + 12288) / 16380004
 NCU_GATHER_READ_BYTES_PER_256B_ROW = 13165824 / 50620
 
@@ -215,20 +211,21 @@ def main():
                          "all-to-all round trip per hop (needs --theta; default 32); at 1 GPU it measures the "
                          "protocol's overhead, the exchange being a local copy")
     ap.add_argument("--no-overlap", action="store_true",
-                    help="run the feature gather of a batch on the sampling stream instead of a second stream "
-                         "(where it overlaps the first, latency-bound hops of the next batch)")
+                    help="skip the second, pipelined leg (gather of a batch on a second stream, overlapping the "
+                         "first, latency-bound hops of the next batch)")
     ap.add_argument("--gather-grid", type=int, default=None,
-                    help="blocks per SM in the gather's grid (default: 1024 short blocks when it overlaps the next "
-                         "batch, 16 long-lived ones when it runs on the sampling stream)")
+                    help="blocks per SM in the gather's grid during the pipelined leg (default 1024 short blocks; "
+                         "the one-stream leg always uses 16 long-lived ones)")
+    ap.add_argument("--lambda-otf", type=float, default=None,
+                    help="expected number of candidates the threshold scan keeps per row for a partial refresh "
+                         "(selection tuning; never changes results)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
 
-    from paper_2406_17918_b200 import replicas
-
-    rank, local_rank, world = replicas.env_rank()
+    rank, local_rank = int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0"))
     over = {}
     if args.fanouts:
         over["fanouts"] = [int(x) for x in args.fanouts.split(",")]
@@ -252,6 +249,7 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the sampler has no CPU fallback")
     import paper_2406_17918_b200 as gs
+    from paper_2406_17918_b200 import replicas
 
     device = torch.device("cuda", local_rank)
     torch.cuda.set_device(device)
@@ -285,6 +283,8 @@ def main():
     ev1.record()
     torch.cuda.synchronize()
     presample_ms = ev0.elapsed_time(ev1)
+    if args.lambda_otf:
+        gs.gs_cache_set_tuning(C, lambda_otf=args.lambda_otf)
     B = cfg["batch"]
     ws = torch.empty(gs.gs_workspace_bytes(G, cfg["fanouts"], B), dtype=torch.uint8, device=device)
     gm = {"otf": gs.GS_MODE_OTF, "fcr": gs.GS_MODE_FCR, "fbl": gs.GS_MODE_FBL, "fetch": gs.GS_MODE_OTF_FETCH}[mode]
@@ -300,64 +300,34 @@ def main():
         gm, gamma, r = gs.GS_MODE_OTF, 0.0, 0
 
     K, Wm = args.steps, args.warmup
-    seeds_all = [batch_seeds(perm, b, B, rank, world) for b in range(Wm + 2 * K)]
-    pinned_counts = torch.zeros((K, 128), dtype=torch.int32).pin_memory()
-
-    # Batches are independent once sampled, so the gather of batch t (HBM-bound) runs on a second, lower-priority
-    # stream while the sampling stream already works on the first hops of batch t+1 (small, latency-bound kernels).
-    # Two workspaces / output buffers alternate; the batch's row count is copied out of the state header before the
-    # next batch clears it.
-    overlap = not args.no_overlap
-    gather_grid = args.gather_grid if args.gather_grid else (1024 if overlap else 16)
-    gs.gs_graph_set_gather_grid(G, gather_grid)
-    nbuf = 2 if overlap else 1
-    ws_list = [ws] + [torch.empty_like(ws) for _ in range(nbuf - 1)]
-    out_list = [None] * nbuf
-    cnt_copy = [torch.zeros((), dtype=torch.int32, device=device) for _ in range(nbuf)]
+    seeds_all = [batch_seeds(perm, b, B, rank, world) for b in range(Wm + 3 * K)]
+    gs.gs_graph_set_gather_grid(G, 16)     # a few long-lived blocks per SM: the fastest shape when the gather runs alone
     s_main = torch.cuda.Stream(device=device, priority=-1)
-    s_gather = torch.cuda.Stream(device=device, priority=0) if overlap else s_main
-    ready = [torch.cuda.Event() for _ in range(nbuf)]
-    done = [torch.cuda.Event() for _ in range(nbuf)]
+    out_rows = None
     refresh_events = []
 
-    def one_step(b, step, j):
+    def one_step(b, step, workspace):
         if args.period and step % args.period == 0:
             ra, rb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             ra.record()
             gs.gs_cache_refresh_all(C, refresh_mode, refresh_gamma, step)
             rb.record()
             refresh_events.append((ra, rb))
-        blocks, input_nodes, cnt = gs.gs_sample_batch(C, seeds_all[b], gm, gamma, step, ws_list[j])
-        if out_list[j] is None:
-            out_list[j] = torch.empty((blocks[0].max_src, cfg["feat_dim"]), dtype=X.dtype, device=device)
-        return blocks, input_nodes, cnt
+        return gs.gs_sample_batch(C, seeds_all[b], gm, gamma, step, workspace)
 
-    def gather_step(j, input_nodes, cnt, ev_a=None, ev_b=None):
-        if overlap:
-            cnt_copy[j].copy_(cnt)
-            ready[j].record()
-            s_gather.wait_event(ready[j])
-            cnt = cnt_copy[j]
-        if ev_a is not None:
-            ev_a.record(s_gather)
-        gs.gs_gather_features(G, input_nodes, cnt, out_list[j], stream=s_gather)
-        if ev_b is not None:
-            ev_b.record(s_gather)
-        if overlap:
-            done[j].record(s_gather)
-
+    # ---- leg 1 (the headline): every batch start to end on ONE stream - gs_sample_batch, then gs_gather_features
     torch.cuda.synchronize()
     with torch.cuda.stream(s_main):
         for b in range(Wm):
-            j = b % nbuf
-            if overlap:
-                s_main.wait_event(done[j])
-            blocks, input_nodes, cnt = one_step(b, b + 1, j)
-            gather_step(j, input_nodes, cnt)
+            blocks, input_nodes, cnt = one_step(b, b + 1, ws)
+            if out_rows is None:
+                out_rows = torch.empty((blocks[0].max_src, cfg["feat_dim"]), dtype=X.dtype, device=device)
+            gs.gs_gather_features(G, input_nodes, cnt, out_rows)
         gs.gs_sync_status(C)
         torch.cuda.synchronize()
 
-        events = [torch.cuda.Event(enable_timing=True) for _ in range(4 * K)]
+        pinned_counts = torch.zeros((K, 128), dtype=torch.int32).pin_memory()
+        events = [torch.cuda.Event(enable_timing=True) for _ in range(3 * K + 1)]
         clocks = ClockSampler(local_rank) if rank == 0 else None
         time.sleep(0.3)
         replicas.barrier()
@@ -367,64 +337,42 @@ def main():
         wall0 = time.time()
         for i in range(K):
             b = Wm + i
-            j = b % nbuf
-            if overlap:
-                s_main.wait_event(done[j])          # the gather that last read this workspace has finished
-            events[4 * i].record()
-            blocks, input_nodes, cnt = one_step(b, b + 1, j)
-            events[4 * i + 1].record()
-            pinned_counts[i].copy_(hdr, non_blocking=True)
-            gather_step(j, input_nodes, cnt, events[4 * i + 2], events[4 * i + 3])
-        if overlap:
-            for j in range(nbuf):
-                s_main.wait_event(done[j])
-        end = torch.cuda.Event(enable_timing=True)
-        end.record()
+            events[3 * i].record()
+            blocks, input_nodes, cnt = one_step(b, b + 1, ws)
+            events[3 * i + 1].record()
+            pinned_counts[i].copy_(hdr, non_blocking=True)      # the batch's counts, read after the run
+            events[3 * i + 2].record()
+            gs.gs_gather_features(G, input_nodes, cnt, out_rows)
+        events[3 * K].record()
         torch.cuda.synchronize()
         replicas.barrier()
         wall1 = time.time()
         launches = gs.gs_kernel_launches() - launches0
-        total_ms = events[0].elapsed_time(end)
+        total_ms = events[0].elapsed_time(events[3 * K])
         group_ms, _ = gs.gs_cache_profile_end(C)
         gs.gs_sync_status(C)
-    out = out_list[0]
-    # the gather alone (nothing else on the GPU), on the last batch's input nodes: the kernel's own rate
-    jl = (Wm + K - 1) % nbuf
-    iso = []
-    gs.gs_graph_set_gather_grid(G, 16)      # alone, a few long-lived blocks per SM are the fastest launch shape
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)    # larger than L2: no row survives between launches
-    for _ in range(8):
-        flush.zero_()
-        ia, ib = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ia.record()
-        gs.gs_gather_features(G, input_nodes, cnt_copy[jl] if overlap else cnt, out_list[jl])
-        ib.record()
-        iso.append((ia, ib))
-    torch.cuda.synchronize()
-    gather_alone_ms = sorted(a.elapsed_time(b) for a, b in iso[2:])[len(iso[2:]) // 2]
-    gs.gs_graph_set_gather_grid(G, gather_grid)
-    del flush
-    if clocks:
-        time.sleep(0.1)
-        clocks.stop()
+    batch_ms = sorted(events[3 * i].elapsed_time(events[3 * i + 3]) for i in range(K))
+    median_ms = batch_ms[K // 2]
+    sample_ms = sum(events[3 * i].elapsed_time(events[3 * i + 1]) for i in range(K))
+    gather_ms = sum(events[3 * i + 2].elapsed_time(events[3 * i + 3]) for i in range(K))
 
     # word positions of the counts inside the cache's state header, by sampling step
     n_words = [blocks[L - 1 - k].count_words()[0] for k in range(L)] + [blocks[0].count_words()[1]]
     m_words = [blocks[L - 1 - k].count_words()[2] for k in range(L)]
-    counts = pinned_counts.numpy()
+    counts = pinned_counts.numpy().copy()
     edges = 0
     feat_rows = 0
-    sample_ms = sum(events[4 * i].elapsed_time(events[4 * i + 1]) for i in range(K))
-    gather_ms = sum(events[4 * i + 2].elapsed_time(events[4 * i + 3]) for i in range(K))
-    # refreshed nodes per step, from the last batch's frontier (outside the timed region)
+    # refreshed nodes per step, from the last timed batch's frontier (outside the timed region)
     deg = g.degrees()
     n_last = [int(counts[K - 1][w]) for w in n_words]
     fr = input_nodes[: n_last[L]].long()
     over = (deg[fr] > (cfg["cache_width"] if args.theta is None else args.theta))
-    refreshed_frac = []
+    listed = (deg[fr] > max(128, cfg["cache_width"]))     # rows whose refill reads a candidate list of the scan
+    refreshed_frac, listed_frac = [], []
     for k in range(L):
         lo = n_last[k - 1] if (cfg["shared"] and k > 0) else 0
         refreshed_frac.append(float(over[lo:n_last[k]].sum().item()) / max(1, n_last[k]))
+        listed_frac.append(float(listed[lo:n_last[k]].sum().item()) / max(1, n_last[k]) if r > 0 else 0.0)
     alg_total, alg_feat = 0, 0
     philox_blocks = sum(int(counts[i][stat0 + 3]) & 0xFFFFFFFF for i in range(K))
     slow_refills = sum(int(counts[i][stat0]) for i in range(K))
@@ -437,33 +385,84 @@ def main():
         alg_total += a
         alg_feat += f
 
-    # ---- end-to-end: seeds in pinned host memory go in, the batch's counts come back, every step
+    # the gather alone (nothing else on the GPU, L2 flushed), on the last batch's input nodes: the kernel's own rate
+    iso = []
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)    # larger than L2: no row survives between launches
+    with torch.cuda.stream(s_main):
+        for _ in range(8):
+            flush.zero_()
+            ia, ib = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ia.record()
+            gs.gs_gather_features(G, input_nodes, cnt, out_rows)
+            ib.record()
+            iso.append((ia, ib))
+    torch.cuda.synchronize()
+    gather_alone_ms = sorted(a.elapsed_time(b) for a, b in iso[2:])[len(iso[2:]) // 2]
+    del flush
+
+    # ---- leg 2 (reported beside it): batches are independent once sampled, so the gather of batch t runs on a
+    # second, lower-priority stream while the sampling stream already works on the first hops of batch t+1 (small,
+    # latency-bound kernels).  Two workspaces / output buffers alternate; the batch's row count is copied out of the
+    # state header before the next batch clears it.  The gather uses many short blocks here so that the next batch's
+    # kernels find free block slots at once.
+    pipelined = None
+    if not args.no_overlap:
+        gs.gs_graph_set_gather_grid(G, args.gather_grid if args.gather_grid else 1024)
+        ws_list = [ws, torch.empty_like(ws)]
+        out_list = [out_rows, torch.empty_like(out_rows)]
+        cnt_copy = [torch.zeros((), dtype=torch.int32, device=device) for _ in range(2)]
+        s_gather = torch.cuda.Stream(device=device, priority=0)
+        ready = [torch.cuda.Event() for _ in range(2)]
+        done = [torch.cuda.Event() for _ in range(2)]
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        replicas.barrier()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(s_main):
+            for i in range(K + 3):                       # three untimed batches fill the pipeline
+                if i == 3:
+                    p0.record()
+                j = i % 2
+                s_main.wait_event(done[j])               # the gather that last read this workspace has finished
+                blocks, input_nodes, cnt = one_step(Wm + K + (i % K), Wm + K + 1 + i, ws_list[j])
+                cnt_copy[j].copy_(cnt)
+                ready[j].record()
+                s_gather.wait_event(ready[j])
+                gs.gs_gather_features(G, input_nodes, cnt_copy[j], out_list[j], stream=s_gather)
+                done[j].record(s_gather)
+            for j in range(2):
+                s_main.wait_event(done[j])
+            p1.record()
+        torch.cuda.synchronize()
+        replicas.barrier()
+        p_ms, _ = replicas.aggregate(p0.elapsed_time(p1), [0], device)
+        pipelined = {"ms_per_step": p_ms / K, "what": "gather of batch t on a second stream beside the first hops of batch t+1; "
+                     "same batches' worth of work, %d steps" % K,
+                     "gather_grid_blocks_per_sm": args.gather_grid if args.gather_grid else 1024}
+        gs.gs_graph_set_gather_grid(G, 16)
+        del ws_list, out_list
+    if clocks:
+        time.sleep(0.1)
+        clocks.stop()
+
+    # ---- end-to-end: seeds in pinned host memory go in, the batch's counts come back, every step (one stream)
     e2e = None
     if not args.no_e2e:
-        host_seeds = [seeds_all[Wm + K + i].cpu().pin_memory() for i in range(K)]
+        host_seeds = [seeds_all[Wm + 2 * K + i].cpu().pin_memory() for i in range(K)]
+        step0 = Wm + 2 * K + 8
         replicas.barrier()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e_edges = 0
-        done_e = [torch.cuda.Event() for _ in range(nbuf)]
         with torch.cuda.stream(s_main):
             e0.record()
             for i in range(K):
-                step = Wm + K + i + 1
-                j = i % nbuf
-                if overlap:
-                    s_main.wait_event(done_e[j])      # the gather that last read this workspace has finished
+                step = step0 + i
                 if args.period and step % args.period == 0:
                     gs.gs_cache_refresh_all(C, refresh_mode, refresh_gamma, step)
-                # returns once the batch's counts are on the host (synchronises the sampling stream only)
-                blocks, input_nodes, n, m = gs.gs_sample_batch_host(C, host_seeds[i], gm, gamma, step, ws_list[j])
-                gs.gs_gather_features(G, input_nodes, None, out_list[j][: n[L]], stream=s_gather)
-                if overlap:
-                    done_e[j].record(s_gather)
+                # returns once the batch's counts are on the host (synchronises the sampling stream)
+                blocks, input_nodes, n, m = gs.gs_sample_batch_host(C, host_seeds[i], gm, gamma, step, ws)
+                gs.gs_gather_features(G, input_nodes, None, out_rows[: n[L]])
                 e_edges += sum(m)
-            if overlap:
-                for j in range(nbuf):
-                    s_main.wait_event(done_e[j])
             e1.record()
         torch.cuda.synchronize()
         replicas.barrier()
@@ -471,6 +470,13 @@ def main():
         e2e = {"value": e_edges_all / (e_ms * 1e-3), "unit": "edges/s", "h2d_bytes_per_step": B * 4,
                "d2h_bytes_per_step": gs.COUNTS_READBACK_BYTES,
                "ms_per_step": e_ms / K}
+
+    # ---- measured integer-ALU ceilings (nothing but the arithmetic, same process, same clocks)
+    ceil = None
+    if rank == 0:
+        with torch.cuda.stream(s_main):
+            ceil = {"philox_blocks_per_s": gs.gs_alu_ceiling(0, 30), "wide_multiplies_per_s": gs.gs_alu_ceiling(1, 30),
+                    "logic_ops_per_s": gs.gs_alu_ceiling(2, 30)}
 
     t_ms, (edges_all, feat_rows_all, alg_all, alg_feat_all, gather_ms_max, philox_all) = replicas.aggregate(
         total_ms, [edges, feat_rows, alg_total, alg_feat, gather_ms, philox_blocks], device)
@@ -481,51 +487,67 @@ def main():
     esize = 4 if cfg["feat_dtype"] == "f32" else 2
     peak, peak_kind = measured_peak()
     secs = t_ms * 1e-3
+    sms = torch.cuda.get_device_properties(device).multi_processor_count
+    clk = clocks.summary(wall0, wall1) if clocks else None
+    sm_hz = (clk["sm_mhz"] or 1965.0) * 1e6 if clk else 1965.0e6
     gather_bytes_per_launch = alg_feat / K
     gather_ms_per_launch = gather_ms / K
     achieved = gather_bytes_per_launch / (gather_ms_per_launch * 1e-3) / 1e9
     last_rows = int(counts[K - 1][n_words[L]])
     alone_gbs = last_rows * (4 + 2 * cfg["feat_dim"] * esize) / (gather_alone_ms * 1e-3) / 1e9
     row_bytes = cfg["feat_dim"] * esize
-    gather_traffic = None   # only the 256-byte-row capture scales cleanly (no sector over-fetch, see above)
+    gather_traffic = None   # only the 256-byte-row capture scales cleanly by rows (no sector over-fetch)
     if row_bytes == 256:
         gather_traffic = (feat_rows / K) * (NCU_GATHER_READ_BYTES_PER_256B_ROW + row_bytes)
     roof_gather = {"kernel": "k_gather (feature rows), 1 launch per step", "bound": "hbm", "achieved": achieved,
                    "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
                    "ms_per_launch": gather_ms_per_launch, "traffic": gather_traffic,
-                   "concurrent_with_next_batch": overlap,
                    "alone": {"achieved": alone_gbs, "frac": alone_gbs / peak, "ms_per_launch": gather_alone_ms,
-                             "what": "the same rows with nothing else running and 16 blocks per SM in the grid, L2 flushed before each "
-                                     "launch, median of 6"},
-                   "grid_blocks_per_sm": gather_grid,
-                   "traffic_note": "bytes per launch; read bytes scaled by rows from the ncu capture of workload shared "
-                                   "(same 256-byte rows), written bytes algorithmic" if gather_traffic else
-                                   "no capture with this row size scales by rows; see profiles/"}
+                             "what": "the same rows with nothing else running, L2 flushed before each launch, median of 6"},
+                   "traffic_note": "bytes per launch; read bytes scaled by rows from an ncu capture of the same kernel on "
+                                   "256-byte rows, written bytes algorithmic" if gather_traffic else
+                                   "no capture with this row size scales by rows"}
     # the threshold scan (k_scan, one launch per sampling step) is bound by integer ALU work: Philox blocks
     scan_launches = K * L
     roof_scan = None
     if group_ms["scan"] > 0 and philox_blocks > 0:
         a_scan = philox_blocks / (group_ms["scan"] * 1e-3) / 1e9
-        p_scan = ALU_LANE_OPS / PHILOX_LANE_OPS / 1e9
+        # derived peak: a Philox4x32-10 block is 20 wide multiplies and 20 three-input logic operations; the multiply
+        # pipe is the slower one.  Its width is taken from the measured multiply rate at the sampled clock
+        # (rounded to a power of two lanes per SM and clock), the rest is unit counts and clocks.
+        mul_lanes = ceil["wide_multiplies_per_s"] / (sms * sm_hz)
+        lanes = 2 ** round(__import__("math").log2(max(mul_lanes, 1.0)))
+        p_scan = sms * lanes * sm_hz / 20.0 / 1e9
         roof_scan = {"kernel": "k_scan (Philox threshold scan), %d launches per step" % L, "bound": "alu",
-                     "achieved": a_scan, "peak": p_scan, "peak_kind": "derived: 148 SMs x 128 lanes x 1.965 GHz / 60 lane-ops per block",
+                     "achieved": a_scan, "peak": p_scan,
+                     "peak_kind": "derived: %d SMs x %d wide-multiply lanes per SM and clock x %.0f MHz / 20 multiplies per "
+                                  "block (measured multiply rate: %.1f lanes per SM and clock)" % (sms, lanes, sm_hz / 1e6, mul_lanes),
                      "unit": "G Philox4x32-10 blocks/s", "frac": a_scan / p_scan,
+                     "peak_measured": ceil["philox_blocks_per_s"] / 1e9,
+                     "frac_of_measured": a_scan / (ceil["philox_blocks_per_s"] / 1e9),
+                     "peak_measured_kind": "a kernel of nothing but Philox blocks and the threshold test, same run",
                      "ms_per_launch": group_ms["scan"] / scan_launches,
                      "traffic": NCU_SCAN_BYTES_PER_BLOCK * philox_blocks / scan_launches,
-                     "traffic_note": "DRAM bytes per launch, scaled by Philox blocks from the ncu capture of workload "
-                                     "large (an upper estimate: the traffic follows work items, and larger rows have "
-                                     "fewer items per block); the scan reads no CSR bytes"}
+                     "traffic_note": "DRAM bytes per launch, scaled by Philox blocks from an ncu capture of the same kernel "
+                                     "on the large workload (an upper estimate: the traffic follows work items, and larger "
+                                     "rows have fewer items per block); the scan reads no CSR bytes"}
+    # the kernel group with the largest time on the one stream (nothing overlaps there)
     groups = dict(group_ms)
     groups["gather"] = gather_ms
     dominant = max(groups, key=groups.get)
+    med_s = median_ms * 1e-3
+    alg_b, phil_b = alg_total / K, philox_blocks / K
     result = {
         "metric": METRIC,
         "value": edges_all / secs,
         "unit": "edges/s",
         "feature_gbs": feat_rows_all * cfg["feat_dim"] * esize / secs / 1e9,
-        "hbm_frac_batch": (alg_all / secs / 1e9) / peak / max(1, world),
-        "hbm_frac_batch_incl_scanned_csr": ((alg_all + 16.0 * philox_all) / secs / 1e9) / peak / max(1, world),
-        "hbm_frac_batch_incl_scanned_csr_of_nominal_8tbs": ((alg_all + 16.0 * philox_all) / secs / 1e9) / 8000.0 / max(1, world),
+        "ms_per_step_median": median_ms,
+        "hbm_frac_batch": (alg_b / med_s / 1e9) / peak,
+        "hbm_frac_batch_incl_scanned_csr": ((alg_b + 16.0 * phil_b) / med_s / 1e9) / peak,
+        "hbm_frac_batch_incl_scanned_csr_of_nominal_8tbs": ((alg_b + 16.0 * phil_b) / med_s / 1e9) / 8000.0,
+        "hbm_frac_note": "per batch, from the median batch time of this rank on one stream; the second figure also charges "
+                         "4 bytes per scanned edge offset, which this design evaluates keys for but never reads",
         "n_gpus": world,
         "steps": K,
         "warmup": Wm,
@@ -541,10 +563,14 @@ def main():
                    "theta": args.theta, "period": args.period,
                    "refresh": ({"mode": mode, "gamma": refresh_gamma} if args.period else "per batch, frontier rows"), "cache_bytes": C.storage.numel(),
                    "parallelism": "replicas x%d" % world, "l2": "inputs_larger_than_L2",
-                   "gather_stream": "second stream, overlapping the next batch's first hops" if overlap else "sampling stream",
+                   "streams": "one: sample_batch then gather_features, batch after batch",
                    "sampled_edges_per_batch": edges / K, "input_nodes_per_batch": feat_rows / K},
         "breakdown_ms_per_step": {"sample_batch": sample_ms / K, "gather_features": gather_ms / K,
                                   "kernel_groups": {k: v / K for k, v in groups.items()}, "dominant": dominant},
+        "frontier_shares_last_batch": {"refreshed": refreshed_frac, "refill_from_scan_list": listed_frac,
+                                       "n_by_step": n_last},
+        "pipelined": pipelined,
+        "alu_ceiling": ceil,
         "philox_blocks_per_batch": philox_blocks / K,
         "slow_refills_per_batch": slow_refills / K,
         "presample_ms": presample_ms,
@@ -552,10 +578,13 @@ def main():
         "setup_s": {"graph_and_features": t_graph},
         "roofline": roof_scan if (dominant == "scan" and roof_scan) else roof_gather,
         "roofline_gather": roof_gather,
+        "roofline_scan": roof_scan,
         "algorithmic_bytes_per_batch": alg_total / K,
         "gpu_launches": launches,
-        "clocks": clocks.summary(wall0, wall1) if clocks else None,
+        "clocks": clk,
     }
+    if pipelined:
+        pipelined["value"] = result["value"] * result["ms_per_step"] / pipelined["ms_per_step"]
     if e2e:
         result["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:

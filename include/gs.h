@@ -374,6 +374,17 @@ gs_status gs_cache_set_tuning(gs_cache*, double lambda_otf, double lambda_full, 
  * each block walk many tiles, a path the designed grids only take on the largest batches. */
 gs_status gs_debug_set_grid_cap(int32_t max_blocks);
 
+/* Measured integer-arithmetic ceilings of the current device, for reporting the threshold scan
+ * against its roofline (the key function of every selection is Philox4x32-10, Salmon et al. SC'11;
+ * the scan evaluates one block per four edge offsets and is bound by this arithmetic, not by memory).
+ * Runs a kernel that does nothing but the chosen arithmetic for about `milliseconds` (1..2000) on
+ * `stream`, synchronises, and returns the sustained rate in *h_units_per_second:
+ *   what = 0  Philox4x32-10 blocks with the scan's threshold test (four blocks per thread in flight)
+ *   what = 1  32x32->64-bit multiplies (a Philox block has 20)
+ *   what = 2  three-input logic operations (a Philox block has 20)
+ * Uses CUDA events (host objects) and a 4-byte device variable of the library; allocates nothing. */
+gs_status gs_alu_ceiling(int32_t what, int32_t milliseconds, void* stream, double* h_units_per_second);
+
 /* Number of kernels this library has launched in the calling process (monotonic). */
 int64_t gs_kernel_launches(void);
 

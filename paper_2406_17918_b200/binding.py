@@ -97,6 +97,7 @@ def _load():
         "gs_cache_profile_end": [vp, vp, vp, vp],
         "gs_cache_set_tuning": [vp, dbl, dbl, i32],
         "gs_debug_set_grid_cap": [i32],
+        "gs_alu_ceiling": [i32, i32, vp, ctypes.POINTER(dbl)],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -515,3 +516,10 @@ def gs_debug_set_grid_cap(max_blocks: int):
 
 def gs_cache_set_tuning(cache: Cache, lambda_otf=0.0, lambda_full=0.0, hub_degree=0):
     _check(_L.gs_cache_set_tuning(cache.handle, float(lambda_otf), float(lambda_full), int(hub_degree)))
+
+
+def gs_alu_ceiling(what: int, milliseconds: int = 20, stream=None) -> float:
+    """Measured rate (units per second) of 0: Philox blocks with the threshold test, 1: wide multiplies, 2: logic ops."""
+    out = ctypes.c_double()
+    _check(_L.gs_alu_ceiling(int(what), int(milliseconds), _stream(stream), ctypes.byref(out)))
+    return float(out.value)

@@ -22,4 +22,3 @@ def test_run_spec_prefers_the_otf_run():
     from workloads import get_config
     assert bench.run_spec(get_config("mid")) == ("otf", 0.1)
     assert bench.run_spec(get_config("scale")) == ("otf", 0.1)
-    assert bench.ALU_LANE_OPS / bench.PHILOX_LANE_OPS / 1e9 > 600
