@@ -186,6 +186,60 @@ def cpu_oracle_baseline(cfg, indptr_h, indices_h, perm, mode, gamma, budget_s=32
     return best[0], best[1], desc, best[3]
 
 
+def verify_first_batch(gs, cfg, g, G, C, X, seeds, gm, mode, gamma, ws, theta, row_samples=4000):
+    """One whole batch (step 1 on a fresh cache) on the GPU and through the CPU oracle, compared element by
+    element.  Raises on the first difference; returns a summary for the result line."""
+    import numpy as np
+
+    import oracle
+    from workloads import feature_rows
+
+    L, W = len(cfg["fanouts"]), cfg["cache_width"]
+    blocks, input_nodes, cnt = gs.gs_sample_batch(C, seeds, gm, gamma, 1, ws)
+    n, m = gs.gs_batch_counts(C)
+    got_frontier = input_nodes[: n[L]].cpu().numpy()
+    got_blocks = [(blocks[l].indptr(n[L - 1 - l]).cpu().numpy(), blocks[l].indices(m[l]).cpu().numpy()) for l in range(L)]
+    out = torch.empty((n[L], cfg["feat_dim"]), dtype=X.dtype, device=X.device)
+    gs.gs_gather_features(G, input_nodes, cnt, out)
+    got_feat = out.cpu().view(torch.int32 if X.dtype == torch.float32 else torch.int16).numpy()
+    del out
+    O = oracle.Sampler(g.indptr.cpu().numpy(), g.indices.cpu().numpy(), cfg["fanouts"], W, SAMPLER_SEED, cfg["shared"])
+    if theta is not None:
+        O.set_theta(theta)
+    om = {"otf": oracle.MODE_OTF, "fcr": oracle.MODE_FCR, "fbl": oracle.MODE_FBL, "fetch": oracle.MODE_OTF_FETCH}[mode]
+    t0 = time.perf_counter()
+    frontier, n_o, blocks_o = O.sample_batch(seeds.cpu().numpy(), om, gamma, 1)
+    t_oracle = time.perf_counter() - t0
+
+    def same(a, b, what):
+        if a.shape != b.shape or not np.array_equal(a, b):
+            raise SystemExit("verify: %s differs from the oracle" % what)
+
+    if list(n) != list(n_o):
+        raise SystemExit("verify: frontier sizes %s differ from the oracle's %s" % (n, n_o))
+    same(got_frontier, frontier, "the input-node list")
+    for l in range(L):
+        same(got_blocks[l][0], blocks_o[l].indptr, "block %d offsets" % l)
+        same(got_blocks[l][1], blocks_o[l].indices, "block %d indices" % l)
+    rng = np.random.default_rng(1)
+    nodes = frontier[rng.choice(len(frontier), min(row_samples, len(frontier)), replace=False)]
+    if theta is not None:
+        deg = (g.indptr[1:] - g.indptr[:-1]).cpu().numpy()
+        nodes = nodes[deg[nodes] > theta]
+    for layer in range(1 if cfg["shared"] else L):
+        rows = gs.gs_cache_read_rows(C, layer, torch.from_numpy(nodes).to(X.device)).cpu().numpy()
+        same(rows, O.cache_rows(layer, nodes), "cache rows of layer %d" % layer)
+    ids = torch.from_numpy(frontier.astype("int64"))
+    Xs = feature_rows(cfg, ids) if cfg["feat_kind"] == "hash" else X.cpu()[ids]
+    want = Xs.view(torch.int32 if X.dtype == torch.float32 else torch.int16).numpy()
+    same(got_feat, oracle.gather(want, np.arange(len(frontier), dtype=np.int32)), "the gathered feature rows")
+    O.close()
+    return {"workload": cfg["name"], "batches": 1, "seeds": int(seeds.numel()), "input_nodes": int(n[L]),
+            "edges": int(sum(m)), "cache_rows_compared": int(len(nodes)) * (1 if cfg["shared"] else L),
+            "compared": "input nodes, block offsets and indices of every hop, sampled cache rows, all gathered feature rows: identical",
+            "oracle_seconds": t_oracle}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -219,6 +273,11 @@ def main():
     ap.add_argument("--lambda-otf", type=float, default=None,
                     help="expected number of candidates the threshold scan keeps per row for a partial refresh "
                          "(selection tuning; never changes results)")
+    ap.add_argument("--verify", action="store_true",
+                    help="before anything is timed, run the first batch (full size, step 1) on the GPU and through "
+                         "the CPU oracle and compare every output element by element: input nodes, every block's "
+                         "offsets and indices, cache rows of sampled frontier nodes, gathered feature rows "
+                         "(the oracle needs minutes on the largest workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -301,6 +360,11 @@ def main():
 
     K, Wm = args.steps, args.warmup
     seeds_all = [batch_seeds(perm, b, B, rank, world) for b in range(Wm + 3 * K)]
+    verified = None
+    if args.verify and args.period:
+        raise SystemExit("--verify checks a batch with its own refresh; it does not combine with --period")
+    if args.verify and rank == 0:
+        verified = verify_first_batch(gs, cfg, g, G, C, X, seeds_all[0], gm, mode, gamma, ws, args.theta)
     gs.gs_graph_set_gather_grid(G, 16)     # a few long-lived blocks per SM: the fastest shape when the gather runs alone
     s_main = torch.cuda.Stream(device=device, priority=-1)
     out_rows = None
@@ -570,6 +634,7 @@ def main():
         "frontier_shares_last_batch": {"refreshed": refreshed_frac, "refill_from_scan_list": listed_frac,
                                        "n_by_step": n_last},
         "pipelined": pipelined,
+        "verified": verified,
         "alu_ceiling": ceil,
         "philox_blocks_per_batch": philox_blocks / K,
         "slow_refills_per_batch": slow_refills / K,

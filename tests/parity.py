@@ -85,6 +85,7 @@ class Pair:
         else:
             blocks, input_nodes, cnt = gs.gs_sample_batch(C, seeds.cuda(), gm, gamma, step, ws)
             n, m = gs.gs_batch_counts(C)
+        self.last_input_nodes = input_nodes      # aliases the workspace: valid until the next batch on it
         frontier, n_o, blocks_o = O.sample_batch(seeds.cpu().numpy(), om, gamma, step)
         assert n == n_o, (n, n_o)
         got_frontier = input_nodes[: n[self.L]].cpu().numpy()

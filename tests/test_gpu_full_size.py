@@ -184,3 +184,36 @@ def test_scale_sampled_nodes_and_properties():
     got = out[sel].cpu()
     assert np.array_equal(got.view(torch.int16).numpy(), oracle.gather(want.view(torch.int16).numpy(), np.arange(5000, dtype=np.int32)))
     assert torch.equal(out.view(torch.int16), X[fl].view(torch.int16))
+
+
+def test_scale_whole_batch_against_the_oracle():
+    """A whole batch of the benchmarked configuration (8,192 seeds, OTF gamma = 0.1; the oracle needs about
+    three minutes on one core), every output array element by element: the 2.0 M input nodes, block offsets
+    and the 5.1 M block indices of all hops, the cache rows of 3,000 sampled frontier nodes at every layer,
+    and the gathered feature rows of all input nodes."""
+    import paper_2406_17918_b200 as gs
+    from parity import Pair
+
+    cfg = get_config("scale")
+    g = build_graph(cfg, device="cuda")
+    X = build_features(cfg, device="cuda")
+    perm = seed_permutation(cfg, device="cuda")
+    fan, W, L = cfg["fanouts"], cfg["cache_width"], len(cfg["fanouts"])
+    B = cfg["batch"]
+    seed = 0x6A09E667F3BCC908
+    pair = Pair.__new__(Pair)
+    pair.cfg, pair.L, pair.W, pair.shared, pair.X, pair.theta = cfg, L, W, False, None, None
+    pair.G = gs.gs_graph_create(g.indptr, g.indices, X)
+    C = gs.gs_cache_init(pair.G, fan, W, seed, False)
+    ws = torch.empty(gs.gs_workspace_bytes(pair.G, fan, B), dtype=torch.uint8, device="cuda")
+    O = oracle.Sampler(g.indptr.cpu().numpy(), g.indices.cpu().numpy(), fan, W, seed, False)
+    seeds = batch_seeds(perm, 5, cfg["batch"])[:B]
+    n, m = pair.check_batch(C, ws, O, seeds, "otf", 0.1, 1, features=False, rows=3000)
+    assert n[L] > 1000000 and sum(m) > 4000000 and int(g.degrees().max()) > 500000
+    # S5: every input node's row against the feature function, copied by the oracle's gather
+    input_nodes = pair.last_input_nodes
+    out = torch.empty((n[L], cfg["feat_dim"]), dtype=X.dtype, device="cuda")
+    gs.gs_gather_features(pair.G, input_nodes, None, out)
+    ids = input_nodes[: n[L]].cpu()
+    want = feature_rows(cfg, ids.long()).view(torch.int16).numpy()
+    assert np.array_equal(out.cpu().view(torch.int16).numpy(), oracle.gather(want, np.arange(n[L], dtype=np.int32)))
