@@ -270,6 +270,8 @@ def main():
     ap.add_argument("--gather-grid", type=int, default=None,
                     help="blocks per SM in the gather's grid during the pipelined leg (default 1024 short blocks; "
                          "the one-stream leg always uses 16 long-lived ones)")
+    ap.add_argument("--dedup", default=None, choices=["direct", "hash", "sort", "auto"],
+                    help="how first occurrences are found for dedup + relabel (default: the library's choice)")
     ap.add_argument("--lambda-otf", type=float, default=None,
                     help="expected number of candidates the threshold scan keeps per row for a partial refresh "
                          "(selection tuning; never changes results)")
@@ -344,6 +346,8 @@ def main():
     presample_ms = ev0.elapsed_time(ev1)
     if args.lambda_otf:
         gs.gs_cache_set_tuning(C, lambda_otf=args.lambda_otf)
+    if args.dedup:
+        gs.gs_cache_set_dedup(C, {"direct": gs.GS_DEDUP_DIRECT, "hash": gs.GS_DEDUP_HASH, "sort": gs.GS_DEDUP_SORT, "auto": gs.GS_DEDUP_AUTO}[args.dedup])
     B = cfg["batch"]
     ws = torch.empty(gs.gs_workspace_bytes(G, cfg["fanouts"], B), dtype=torch.uint8, device=device)
     gm = {"otf": gs.GS_MODE_OTF, "fcr": gs.GS_MODE_FCR, "fbl": gs.GS_MODE_FBL, "fetch": gs.GS_MODE_OTF_FETCH}[mode]
@@ -624,7 +628,7 @@ def main():
         "config": {"workload": cfg["name"], "num_nodes": g.num_nodes, "num_edges": g.num_edges,
                    "fanouts": cfg["fanouts"], "cache_width": cfg["cache_width"], "mode": mode, "gamma": gamma,
                    "batch": B, "shared_cache": cfg["shared"], "feat_dim": cfg["feat_dim"],
-                   "theta": args.theta, "period": args.period,
+                   "theta": args.theta, "period": args.period, "dedup": args.dedup or "default",
                    "refresh": ({"mode": mode, "gamma": refresh_gamma} if args.period else "per batch, frontier rows"), "cache_bytes": C.storage.numel(),
                    "parallelism": "replicas x%d" % world, "l2": "inputs_larger_than_L2",
                    "streams": "one: sample_batch then gather_features, batch after batch",

@@ -368,6 +368,25 @@ gs_status gs_sync_status(gs_cache*, void* stream);
  * defaults. */
 gs_status gs_cache_set_tuning(gs_cache*, double lambda_otf, double lambda_full, int32_t hub_degree);
 
+/* How gs_sample_batch finds each id's first occurrence for the dedup + relabel of a step (the paper's
+ * Algorithms 2 and 3 only say that the sampled neighbours become the next frontier and that blocks are
+ * returned; the three methods give identical blocks and differ in speed only):
+ *   GS_DEDUP_DIRECT            direct-address table of 8 bytes per graph node inside the cache storage;
+ *                              every pick claims its position with one atomicMin.
+ *   GS_DEDUP_HASH              open-addressing hash table of 1.5 x (frontier + picks) entries, rebuilt at
+ *                              every sampling step inside the workspace: follows the batch, not the graph.
+ *   GS_DEDUP_SORT              stable radix sort of (id, position) pairs; run heads are first occurrences.
+ *   GS_DEDUP_AUTO (default)    per sampling step, by measurement on B200: the hash table when the direct
+ *                              table is larger than 64 MiB (it then falls out of L2) and the step can hold
+ *                              half a million keys or more, the direct table otherwise.
+ * Applies to the following gs_sample_batch / gs_sample_batch_host / gs_sample_batch_noalloc calls on this
+ * cache; the node-sharded calls always use the direct table. */
+#define GS_DEDUP_DIRECT 0
+#define GS_DEDUP_HASH 1
+#define GS_DEDUP_SORT 2
+#define GS_DEDUP_AUTO 3
+gs_status gs_cache_set_dedup(gs_cache*, int32_t method);
+
 /* Test knob, process-wide: no kernel of the library is launched with more than max_blocks thread
  * blocks (0 restores the designed grids).  Every kernel walks its work with a grid-stride or
  * work-counter loop, so results never depend on the grid; tests use caps of 1-3 blocks to make

@@ -18,6 +18,7 @@ _HEADER = os.path.join(os.path.dirname(_HERE), "include", "gs.h")
 
 GS_MODE_FCR, GS_MODE_OTF, GS_MODE_FBL, GS_MODE_OTF_FETCH = 0, 1, 2, 3
 GS_F32, GS_BF16 = 0, 1
+GS_DEDUP_DIRECT, GS_DEDUP_HASH, GS_DEDUP_SORT, GS_DEDUP_AUTO = 0, 1, 2, 3
 GS_MAX_HOPS = 8
 COUNTS_READBACK_BYTES = 4 * (1 + (GS_MAX_HOPS + 1) + GS_MAX_HOPS)  # status + n_k + m_k, what gs_batch_counts copies
 
@@ -98,6 +99,7 @@ def _load():
         "gs_cache_set_tuning": [vp, dbl, dbl, i32],
         "gs_debug_set_grid_cap": [i32],
         "gs_alu_ceiling": [i32, i32, vp, ctypes.POINTER(dbl)],
+        "gs_cache_set_dedup": [vp, i32],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -523,3 +525,8 @@ def gs_alu_ceiling(what: int, milliseconds: int = 20, stream=None) -> float:
     out = ctypes.c_double()
     _check(_L.gs_alu_ceiling(int(what), int(milliseconds), _stream(stream), ctypes.byref(out)))
     return float(out.value)
+
+
+def gs_cache_set_dedup(cache: Cache, method: int):
+    """GS_DEDUP_DIRECT / GS_DEDUP_HASH / GS_DEDUP_SORT for the following batches on this cache."""
+    _check(_L.gs_cache_set_dedup(cache.handle, int(method)))

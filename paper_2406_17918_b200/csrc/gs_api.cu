@@ -38,6 +38,7 @@ struct gs_cache {
     int32_t theta;            // split cache: nodes with degree <= theta have no row (-1: every node has one)
     int64_t rows;             // cache rows per cache (num_nodes, or the dense nodes of a split cache)
     int32_t* d_row_index;     // split cache only
+    int32_t dedup;            // DedupMethod of gs_sample_batch
     int32_t* h_pinned;        // pinned staging for counts
     // optional device timing of the kernel groups (gs_cache_profile_begin / _end)
     cudaEvent_t* prof_events;
@@ -344,6 +345,7 @@ static gs_status cache_init_impl(const gs_graph* g, int32_t num_hops, const int3
     c->d_slots = (int32_t*)(c->d_storage + HDR_BYTES + table_bytes(g) + (split_cache ? row_index_bytes(g) : 0));
     c->slot_bytes = (size_t)c->num_caches * (size_t)c->rows * (size_t)c->pitch * 4;
     c->serial = 0;
+    c->dedup = DEDUP_AUTO;
     c->lambda_otf = 18.0f;
     c->lambda_full = 72.0f;
     c->hub_degree = 8192;
@@ -446,6 +448,13 @@ gs_status gs_cache_profile_end(gs_cache* c, void* stream, double* h_ms, int64_t*
     return GS_OK;
 }
 
+gs_status gs_cache_set_dedup(gs_cache* c, int32_t method) {
+    if (!c) return fail(GS_ERR_ARG, "cache is NULL");
+    if (method != DEDUP_DIRECT && method != DEDUP_HASH && method != DEDUP_SORT && method != DEDUP_AUTO) return fail(GS_ERR_ARG, "unknown dedup method %d", method);
+    c->dedup = method;
+    return GS_OK;
+}
+
 gs_status gs_cache_set_tuning(gs_cache* c, double lambda_otf, double lambda_full, int32_t hub_degree) {
     if (!c) return fail(GS_ERR_ARG, "cache is NULL");
     if (lambda_otf > 0) c->lambda_otf = (float)lambda_otf;
@@ -520,6 +529,11 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
     const bool prof = !hop && c->prof_events && c->prof_used < c->prof_cap;
     for (int k = 0; k < L; ++k) {
         const int layer = hop ? hop->layer : L - 1 - k;
+        // how this step finds first occurrences; key bounds grow with k, so AUTO never returns from the hash
+        // table to the direct one inside a batch (the direct table is not maintained by the other methods)
+        int32_t dedup = c->dedup;
+        if (dedup == DEDUP_AUTO)
+            dedup = (g->num_nodes * 8 > DEDUP_AUTO_TABLE_BYTES && b.nb[k] + b.mb[k] >= DEDUP_AUTO_MIN_KEYS) ? DEDUP_HASH : DEDUP_DIRECT;
         cudaEvent_t* ev = prof ? c->prof_events + ((size_t)c->prof_used * L + k) * PROF_EVENTS_PER_STEP : nullptr;
         if (ev) GS_CUDA(cudaEventRecord(ev[0], s));
         int32_t* blk_indptr = out ? out->indptr[layer] : (int32_t*)(ws + w.blk_indptr[k]);
@@ -537,7 +551,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         C.tile_sums = tiles_a;
         C.table = c->d_table;
         C.stamp = stamp;
-        C.no_stamp = hop ? 1 : 0;
+        C.no_stamp = hop ? 1 : 0;   // the seeds are stamped in the direct table with every dedup method: duplicates are caught before anything is refreshed
         // a partial refresh runs as scan + finish kernels; FCR (and r = 0) use the fused kernels
         int32_t n_fetch = 0;
         if (mode == GS_MODE_OTF_FETCH) {
@@ -580,6 +594,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         P.work_counter_scan = hdr + HDR_WORK3 + k;
         P.do_pick = 1;
         P.init_rows = 0;
+        if (dedup != DEDUP_DIRECT) P.table = nullptr;   // positions are claimed after the step, from the picked array
         if (hop) {   // a shared cache refreshes every requested node: the same keys give the same row again
             P.table = nullptr;
             P.status = hdr + HDR_STATUS;
@@ -631,7 +646,12 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         R.table = c->d_table;
         R.stamp = stamp;
         R.n_cap = b.nb[k + 1];
-        GS_CUDA(launch_relabel(R, b.mb[k], s));
+        R.method = dedup;
+        R.scratch = (unsigned long long*)(ws + w.dedup);
+        R.scratch_entries = w.dedup_entries;
+        R.id_bits = 1;
+        while (R.id_bits < 32 && ((int64_t)1 << R.id_bits) < g->num_nodes) R.id_bits += 1;
+        GS_CUDA(launch_relabel(R, b.nb[k], b.mb[k], s));
         if (ev) GS_CUDA(cudaEventRecord(ev[4], s));
 
         gs_block& B = blocks[layer];
@@ -828,7 +848,8 @@ gs_status gs_shard_extend(gs_cache* c, int32_t k, const int32_t* d_seeds, int32_
     R.table = c->d_table;
     R.stamp = c->shard_stamp;
     R.n_cap = b.nb[k + 1];
-    GS_CUDA(launch_relabel(R, b.mb[k], s));
+    R.method = DEDUP_DIRECT;
+    GS_CUDA(launch_relabel(R, b.nb[k], b.mb[k], s));
 
     gs_block& B = *block;
     B.max_dst = (int32_t)b.nb[k];

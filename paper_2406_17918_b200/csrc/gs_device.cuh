@@ -114,4 +114,21 @@ __device__ __forceinline__ int block_exclusive_scan(int x, int* warp_sums, int* 
     return warp_sums[wid] + incl - x;
 }
 
+// In-place exclusive scan of tile_sums[0..T) by one block of BT threads; returns the total.
+template <int BT>
+__device__ __forceinline__ int scan_tiles_in_place(int32_t* tile_sums, int T, int* warp_sums) {
+    int carry = 0;
+    for (int base = 0; base < T; base += BT) {
+        const int i = base + (int)threadIdx.x;
+        const int x = (i < T) ? __ldcg(tile_sums + i) : 0;
+        int total;
+        const int excl = block_exclusive_scan<BT>(x, warp_sums, &total);
+        if (i < T) tile_sums[i] = carry + excl;
+        carry += total;
+    }
+    return carry;
+}
+
+__device__ __forceinline__ void raise_status(int32_t* status, int code) { atomicCAS(status, 0, code); }
+
 }  // namespace gs

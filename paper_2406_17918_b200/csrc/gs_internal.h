@@ -46,6 +46,17 @@ constexpr int SCAN_E_TILE = 4096;  // picked edges per tile of the first-occurre
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Entries of the batch-sized hash table for n + m keys (load factor at most 2/3).
+__host__ __device__ inline int64_t dedup_hash_capacity(int64_t keys) {
+    return (keys + keys / 2 + 64) & ~(int64_t)1;
+}
+// 8-byte scratch entries the sort needs for `keys` pairs: two key buffers, the digit counters of every
+// 4096-key tile, one run-head word per 1024 keys, a ticket and the 256 digit totals.
+__host__ __device__ inline int64_t dedup_sort_entries(int64_t keys) {
+    const int64_t tiles = (keys + 4095) / 4096 + 1, tiles1k = (keys + 1023) / 1024 + 1;
+    return 2 * keys + 64 + (256 * tiles + tiles1k + 1024) / 2 + 8;
+}
+
 struct Bounds {
     int32_t L;
     int64_t nb[GS_MAX_HOPS + 1];  // upper bound of n_k
@@ -72,6 +83,8 @@ struct WorkspaceLayout {
     size_t hub_entry, hub_state, hub_items, hub_cand;
     int64_t hub_cap, item_cap;
     size_t tiles_a2, item_start, items, cand_count, cand;   // split OTF path
+    size_t dedup;
+    int64_t dedup_entries;
     int64_t scan_item_cap;
     size_t total;
 };
@@ -112,6 +125,18 @@ inline WorkspaceLayout make_layout(const Bounds& b, int64_t num_edges) {
     w.items = take((size_t)w.scan_item_cap * 4);
     w.cand_count = take((size_t)max_n * 4);
     w.cand = take((size_t)max_n * SPLIT_CAND_CAP * 8);
+    w.dedup = w.cand;   // free once the step's picks are written: scratch of the alternative dedup methods
+    {
+        int64_t need = 0;
+        for (int k = 0; k < b.L; ++k) {
+            const int64_t keys = b.nb[k] + b.mb[k];
+            const int64_t e = dedup_sort_entries(keys) > dedup_hash_capacity(keys) ? dedup_sort_entries(keys) : dedup_hash_capacity(keys);
+            if (e > need) need = e;
+        }
+        w.dedup_entries = need;
+        const size_t have = off - w.cand;
+        if ((size_t)need * 8 > have) off = align_up(w.cand + (size_t)need * 8, 256);
+    }
     w.total = off;
     return w;
 }
@@ -193,6 +218,19 @@ struct CountParams {
     const int32_t* slot;     // requester side: row of `reply` that belongs to frontier position p
 };
 
+// How the position of an id's first occurrence in "frontier ++ picked" is found (S3).
+enum DedupMethod : int32_t {
+    DEDUP_DIRECT = 0,   // direct-address table uint64[num_nodes]; the pick kernels claim positions with atomicMin
+    DEDUP_HASH = 1,     // open-addressing hash table sized to the batch (1.5 x (n_k + m_k) entries), rebuilt per step
+    DEDUP_SORT = 2,     // stable radix sort of (id, position) pairs; the head of each run of equal ids is the first occurrence
+    DEDUP_AUTO = 3      // per sampling step: the hash table where the direct table is far larger than L2 and the step is large
+};
+// DEDUP_AUTO takes the hash table for a step when the direct table (8 bytes per node) exceeds this many bytes
+// - it no longer stays in the 126 MB L2 - and the step may hold at least this many keys (frontier + picks bound);
+// measured on B200: below either limit the direct table wins.
+constexpr int64_t DEDUP_AUTO_TABLE_BYTES = (int64_t)64 << 20;
+constexpr int64_t DEDUP_AUTO_MIN_KEYS = (int64_t)1 << 19;
+
 struct RelabelParams {
     int32_t* hdr;
     int32_t k;
@@ -201,9 +239,13 @@ struct RelabelParams {
     int32_t* tile_sums;
     int32_t* frontier;
     int32_t* local;
-    unsigned long long* table;
+    unsigned long long* table;       // DEDUP_DIRECT only
     uint32_t stamp;
     int64_t n_cap;
+    int32_t method;
+    unsigned long long* scratch;     // hash table, or the two key buffers and counters of the sort
+    int64_t scratch_entries;         // 8-byte entries available there
+    int32_t id_bits;                 // bits of a node id (sort passes)
 };
 
 void count_launches(int n);
@@ -241,7 +283,11 @@ cudaError_t launch_init_low_rows(const GraphView& g, int32_t* slots, int32_t pit
                                  cudaStream_t s);
 cudaError_t launch_scan(const StepParams& p, int64_t item_bound, cudaStream_t s);
 cudaError_t launch_finish(const StepParams& p, int64_t n_bound, cudaStream_t s);
-cudaError_t launch_relabel(const RelabelParams& p, int64_t m_bound, cudaStream_t s);
+cudaError_t launch_relabel(const RelabelParams& p, int64_t n_bound, int64_t m_bound, cudaStream_t s);
+// Pre-passes of the alternative dedup methods: both leave in aux[e] what the first-occurrence kernel needs
+// (DEDUP_HASH: the table slot of the pick's id; DEDUP_SORT: the first position of the pick's id).
+cudaError_t launch_dedup_hash(const RelabelParams& p, int64_t n_bound, int64_t m_bound, cudaStream_t s);
+cudaError_t launch_dedup_sort(const RelabelParams& p, int64_t n_bound, int64_t m_bound, cudaStream_t s);
 cudaError_t launch_gather(const void* src, int64_t src_ld_bytes, int64_t row_bytes, const int32_t* ids,
                           const int32_t* d_count, int32_t count_bound, void* dst, int64_t dst_ld_bytes,
                           int32_t blocks_per_sm /* 0: the default */, int64_t id_lo, int64_t id_hi /* ids outside

@@ -7,23 +7,6 @@
 
 namespace gs {
 
-__device__ __forceinline__ void raise_status(int32_t* status, int code) { atomicCAS(status, 0, code); }
-
-// In-place exclusive scan of tile_sums[0..T) by one block of BT threads; returns the total.
-template <int BT>
-__device__ int scan_tiles_in_place(int32_t* tile_sums, int T, int* warp_sums) {
-    int carry = 0;
-    for (int base = 0; base < T; base += BT) {
-        const int i = base + (int)threadIdx.x;
-        const int x = (i < T) ? __ldcg(tile_sums + i) : 0;
-        int total;
-        const int excl = block_exclusive_scan<BT>(x, warp_sums, &total);
-        if (i < T) tile_sums[i] = carry + excl;
-        carry += total;
-    }
-    return carry;
-}
-
 // ---------------------------------------------------------------- row counts
 // Per frontier node p: count(p) = min(f, deg(frontier[p])) - the number of picks is known from the
 // degree alone, so the block CSR offsets exist before anything is sampled.  Step 0 also copies
@@ -169,6 +152,9 @@ cudaError_t launch_row_counts(const CountParams& p, int64_t n_bound, cudaStream_
 constexpr int FF_THREADS = 256;                 // 8 warps, each owns 512 consecutive picks of the tile
 static_assert(SCAN_E_TILE == FF_THREADS * 16, "tile = 16 picks per thread");
 
+// METHOD says where the first position of a pick's id comes from: the direct-address table (read with the
+// id), the batch-sized hash table (aux[e] holds the id's slot), or aux[e] itself (the sort left it there).
+template <int METHOD>
 __global__ void __launch_bounds__(FF_THREADS) k_first_flags(RelabelParams P) {
     __shared__ int warp_sums[33];
     __shared__ int s_wtot[FF_THREADS / 32];
@@ -194,14 +180,18 @@ __global__ void __launch_bounds__(FF_THREADS) k_first_flags(RelabelParams P) {
     for (int j = 0; j < 4; ++j) {
         const int e0 = wbase + j * 128 + lane * 4;
         int4 v = make_int4(0, 0, 0, 0);
-        if (e0 < m) v = *reinterpret_cast<const int4*>(P.picked + e0);  // buffer is padded to 4
+        if (e0 < m) v = *reinterpret_cast<const int4*>((METHOD == DEDUP_DIRECT ? P.picked : P.aux) + e0);  // buffers are padded to 4
         id[j][0] = v.x; id[j][1] = v.y; id[j][2] = v.z; id[j][3] = v.w;
     }
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const int e0 = wbase + j * 128 + lane * 4;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) pos[j][i] = (e0 + i < m) ? (int)(uint32_t)__ldcg(P.table + id[j][i]) : -1;
+        for (int i = 0; i < 4; ++i) {
+            if (METHOD == DEDUP_DIRECT) pos[j][i] = (e0 + i < m) ? (int)(uint32_t)__ldcg(P.table + id[j][i]) : -1;
+            else if (METHOD == DEDUP_HASH) pos[j][i] = (e0 + i < m) ? (int)(uint32_t)__ldcg(P.scratch + id[j][i]) : -1;
+            else pos[j][i] = (e0 + i < m) ? id[j][i] : -1;
+        }
     }
     int cnt[4], incl[4], before[4];
     int wtotal = 0;
@@ -290,7 +280,7 @@ __global__ void __launch_bounds__(256) k_relabel(RelabelParams P) {
                 if (val[i] < 0 && (int64_t)loc < P.n_cap) {
                     const int id = P.picked[e0 + i];
                     P.frontier[loc] = id;
-                    P.table[id] = ((unsigned long long)P.stamp << 32) | (unsigned)loc;
+                    if (P.table) P.table[id] = ((unsigned long long)P.stamp << 32) | (unsigned)loc;
                 }
             }
             out[i] = loc;
@@ -305,16 +295,27 @@ __global__ void __launch_bounds__(256) k_relabel(RelabelParams P) {
     }
 }
 
-cudaError_t launch_relabel(const RelabelParams& p, int64_t m_bound, cudaStream_t s) {
+cudaError_t launch_relabel(const RelabelParams& p, int64_t n_bound, int64_t m_bound, cudaStream_t s) {
     if (m_bound <= 0) m_bound = 1;
+    if (p.method == DEDUP_HASH) {
+        cudaError_t e = launch_dedup_hash(p, n_bound, m_bound, s);
+        if (e != cudaSuccess) return e;
+    } else if (p.method == DEDUP_SORT) {
+        cudaError_t e = launch_dedup_sort(p, n_bound, m_bound, s);
+        if (e != cudaSuccess) return e;
+    }
     int64_t tiles = (m_bound + SCAN_E_TILE - 1) / SCAN_E_TILE;
     if (tiles > sm_count() * 16) tiles = sm_count() * 16;    // blocks walk the tiles; enough of them that a usual batch has one tile each
     tiles = limit_grid(tiles);
-    k_first_flags<<<(int)tiles, FF_THREADS, 0, s>>>(p);
+    if (p.method == DEDUP_HASH) k_first_flags<DEDUP_HASH><<<(int)tiles, FF_THREADS, 0, s>>>(p);
+    else if (p.method == DEDUP_SORT) k_first_flags<DEDUP_SORT><<<(int)tiles, FF_THREADS, 0, s>>>(p);
+    else k_first_flags<DEDUP_DIRECT><<<(int)tiles, FF_THREADS, 0, s>>>(p);
     int64_t blocks = (m_bound + 1023) / 1024;
     if (blocks > sm_count() * 32) blocks = sm_count() * 32;
     blocks = limit_grid(blocks);
-    k_relabel<<<(int)blocks, 256, 0, s>>>(p);
+    RelabelParams q = p;
+    if (p.method != DEDUP_DIRECT) q.table = nullptr;
+    k_relabel<<<(int)blocks, 256, 0, s>>>(q);
     count_launches(2);
     return cudaGetLastError();
 }

@@ -58,6 +58,8 @@ class Pair:
             C = gs.gs_cache_init_split(self.G, self.cfg["fanouts"], self.W, self.seed, self.shared, theta)
         if tuning:
             gs.gs_cache_set_tuning(C, **tuning)
+        if getattr(self, "dedup", 0):
+            gs.gs_cache_set_dedup(C, self.dedup)
         ws = torch.empty(gs.gs_workspace_bytes(self.G, self.cfg["fanouts"], max_seeds), dtype=torch.uint8, device="cuda")
         O = oracle.Sampler(self.indptr, self.indices, self.cfg["fanouts"], self.W, self.seed, self.shared)
         if theta is not None:
