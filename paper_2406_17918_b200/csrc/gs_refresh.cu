@@ -32,16 +32,13 @@
 namespace gs {
 
 #ifndef GS_SCAN_BATCH_DIV
-#define GS_SCAN_BATCH_DIV 4
+#define GS_SCAN_BATCH_DIV 16
 #endif
 #ifndef GS_SCAN_MIN_BLOCKS
-#define GS_SCAN_MIN_BLOCKS 1
+#define GS_SCAN_MIN_BLOCKS 3
 #endif
 #ifndef GS_FINISH_MIN_BLOCKS
 #define GS_FINISH_MIN_BLOCKS 4
-#endif
-#ifndef GS_SCAN_GRID_PER_SM
-#define GS_SCAN_GRID_PER_SM 8
 #endif
 constexpr int RP_THREADS = 256;
 constexpr int RP_WARPS = RP_THREADS / 32;
@@ -677,17 +674,12 @@ __global__ void __launch_bounds__(RP_THREADS, GS_SCAN_MIN_BLOCKS) k_scan(const _
     batch = batch < 1 ? 1 : (batch > 32 ? 32 : batch);
     const uint32_t lt = lanemask_lt();
     const int warp_gid = blockIdx.x * RP_WARPS + (threadIdx.x >> 5);
-    bool first_grab = true;
-    while (true) {
-        int base = 0;
-        if (first_grab) {
-            base = warp_gid * batch;
-            first_grab = false;
-        } else {
-            if (lane == 0) base = atomicAdd(P.work_counter_scan, batch) + total_warps * batch;
-            base = __shfl_sync(FULL, base, 0);
-        }
-        if (base >= total) break;
+    // every warp owns one batch up front; the next one is asked for while the current one is scanned, so the
+    // round trip of the atomic is never waited for
+    int base = warp_gid * batch;
+    while (base < total) {
+        int next_base = 0;
+        if (lane == 0) next_base = atomicAdd(P.work_counter_scan, batch) + total_warps * batch;
         const int cnt = (base + batch < total ? base + batch : total) - base;
         int p_l = 0, chunk_l = 0;
         int32_t v_l = 0;
@@ -754,16 +746,20 @@ __global__ void __launch_bounds__(RP_THREADS, GS_SCAN_MIN_BLOCKS) k_scan(const _
                     const uint4 o0 = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
                     const uint4 o1 = philox4x32_10_rk(q + 32, (uint32_t)v, P.step, P.word_fill, P.rk);
                     const uint4 o2 = philox4x32_10_rk(q + 64, (uint32_t)v, P.step, P.word_fill, P.rk);
-                    const uint4 o3 = philox4x32_10_rk(q + 96, (uint32_t)v, P.step, P.word_fill, P.rk);
                     take_hits(q, o0, q < qe);
                     take_hits(q + 32, o1, q + 32 < qe);
                     take_hits(q + 64, o2, q + 64 < qe);
-                    take_hits(q + 96, o3, q + 96 < qe);
+                    if (groups > 3) {
+                        const uint4 o3 = philox4x32_10_rk(q + 96, (uint32_t)v, P.step, P.word_fill, P.rk);
+                        take_hits(q + 96, o3, q + 96 < qe);
+                    }
                 } else {
                     const uint4 o0 = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
-                    const uint4 o1 = philox4x32_10_rk(q + 32, (uint32_t)v, P.step, P.word_fill, P.rk);
                     take_hits(q, o0, q < qe);
-                    take_hits(q + 32, o1, q + 32 < qe);
+                    if (groups > 1) {
+                        const uint4 o1 = philox4x32_10_rk(q + 32, (uint32_t)v, P.step, P.word_fill, P.rk);
+                        take_hits(q + 32, o1, q + 32 < qe);
+                    }
                 }
             }
             __syncwarp();
@@ -782,6 +778,7 @@ __global__ void __launch_bounds__(RP_THREADS, GS_SCAN_MIN_BLOCKS) k_scan(const _
                 if (dst + t < SPLIT_CAND_CAP) P.cand[(size_t)p * SPLIT_CAND_CAP + dst + t] = stage[t];
             __syncwarp();
         }
+        base = __shfl_sync(FULL, next_base, 0);
     }
 }
 
@@ -1075,7 +1072,15 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
 }
 
 cudaError_t launch_scan(const StepParams& p, int64_t item_bound, cudaStream_t s) {
-    const int64_t cap = sm_count() * GS_SCAN_GRID_PER_SM;
+    // the blocks that are resident together walk all the work: a block that only starts when another one has
+    // left would find its up-front batch late, at the tail of the launch
+    static int resident = 0;   // same kernel, same block size on every device of a process
+    if (resident <= 0) {
+        int r = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, k_scan, RP_THREADS, 0) != cudaSuccess || r < 1) r = 2;
+        resident = r;
+    }
+    const int64_t cap = sm_count() * resident;
     int64_t sb = (item_bound + RP_WARPS - 1) / RP_WARPS;
     sb = limit_grid(sb > cap ? cap : (sb < 1 ? 1 : sb));
     k_scan<<<(int)sb, RP_THREADS, 0, s>>>(p);

@@ -174,35 +174,67 @@ def _all_to_all_v(send, send_counts, width, group):
     return recv, recv_counts
 
 
+class ShardedBatchError(RuntimeError):
+    """Raised by EVERY rank of a sharded batch when any rank met an error inside a hop."""
+
+    def __init__(self, code, local_message):
+        what = {1: "a rank could not build its requests (a node id outside the graph)",
+                2: "an owner could not serve a request list (longer than max_requests, or a device-detected error)"}
+        super().__init__("sharded batch abandoned: %s%s" % (what.get(code, "error %d" % code),
+                                                            "; on this rank: " + local_message if local_message else ""))
+        self.code = code
+
+
 def sample_batch(rank_state: ShardRank, seeds, mode, rate, step, features=True, group=None, feature_bases=None):
     """This rank's part of a sharded batch (every rank of `group` calls it with the same mode, rate
     and step).  Returns (blocks by layer, frontier tensor, n list, m list, feature rows or None).
     `feature_bases`: device addresses of every rank's feature rows as mapped into this process (CUDA
     IPC, symmetric memory, ...); when given, the feature step is one kernel of peer loads instead of an
-    all-to-all round trip."""
+    all-to-all round trip.
+
+    Failures are collective: a rank that cannot build its requests or serve a list still takes part in
+    both exchanges of the hop (with no requests / placeholder rows), an error word is reduced over the
+    group after the reply exchange, and then every rank raises :class:`ShardedBatchError` - no rank is
+    left waiting inside a collective for one that has gone."""
     me = rank_state
     L = me.L
     me.begin(seeds)
+    dev = seeds.device
 
-    def round_trip(ids, counts, serve, width, dtype):
+    def round_trip(make_requests, serve, width, dtype):
+        err, msg = 0, ""
+        try:
+            ids, counts = make_requests()
+        except (ValueError, RuntimeError) as e:
+            err, msg = 1, str(e)
+            ids, counts = torch.empty(0, dtype=torch.int32, device=dev), [0] * me.world
         recv, recv_counts = _all_to_all_v(ids, counts, (), group)
-        served = serve(_split(recv, recv_counts))
-        back = torch.cat(served) if served else torch.empty((0,) + width, dtype=dtype, device=ids.device)
-        reply = torch.empty((ids.numel(),) + width, dtype=dtype, device=ids.device)
+        back = None
+        try:
+            served = serve(_split(recv, recv_counts))
+            back = torch.cat(served) if served else torch.empty((0,) + width, dtype=dtype, device=dev)
+        except (ValueError, RuntimeError) as e:
+            err, msg = 2, str(e)
+        if back is None or back.shape[0] != sum(recv_counts):
+            back = torch.zeros((sum(recv_counts),) + width, dtype=dtype, device=dev)   # placeholder rows keep the exchange whole
+        reply = torch.empty((ids.numel(),) + width, dtype=dtype, device=dev)
         dist.all_to_all_single(reply, back.contiguous(), counts, recv_counts, group=group)
+        word = torch.tensor([err], dtype=torch.int32, device=dev)
+        dist.all_reduce(word, op=dist.ReduceOp.MAX, group=group)
+        code = int(word.item())
+        if code:
+            raise ShardedBatchError(code, msg)
         return reply
 
     for k in range(L):
         layer = L - 1 - k
-        ids, counts = me.hop_requests(k)
-        reply = round_trip(ids, counts, lambda lists: me.hop_serve(layer, lists, mode, rate, step),
+        reply = round_trip(lambda: me.hop_requests(k), lambda lists: me.hop_serve(layer, lists, mode, rate, step),
                            (me.fanouts[layer],), torch.int32)
         me.hop_finish(k, reply)
     feats = None
     if features and feature_bases is not None:
         feats = me.feature_pull(feature_bases)
     elif features:
-        ids, counts = me.feature_requests()
-        rows = round_trip(ids, counts, me.feature_serve, (me.features.shape[1],), me.features.dtype)
+        rows = round_trip(me.feature_requests, me.feature_serve, (me.features.shape[1],), me.features.dtype)
         feats = me.feature_finish(rows)
     return me.blocks, me.frontier, me.n, me.m, feats

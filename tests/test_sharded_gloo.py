@@ -1,4 +1,4 @@
-"""The node-sharded driver (one process per rank, all_to_all_single) on CPU with gloo, world size 2,
+"""The node-sharded driver (one process per rank, all_to_all_single) on CPU with gloo, world sizes 2 and 3,
 with the oracle's per-node primitives standing in for the kernels; plus the oracle-level facts the
 sharded design rests on."""
 import os
@@ -56,8 +56,9 @@ def _worker(rank, world, port, out_dir):
     dist.destroy_process_group()
 
 
-def test_two_ranks_equal_one_sampler_taking_the_batches_in_turn(tmp_path):
-    world = 2
+@pytest.mark.parametrize("world", [2, 3])
+def test_ranks_equal_one_sampler_taking_the_batches_in_turn(tmp_path, world):
+    """World size 3 gives uneven shards (2,708 nodes: 903 + 903 + 902)."""
     mp.spawn(_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
     res = [torch.load(os.path.join(tmp_path, "r%d.pt" % r)) for r in range(world)]
     cfg = get_config("tiny")
@@ -79,6 +80,43 @@ def test_two_ranks_equal_one_sampler_taking_the_batches_in_turn(tmp_path):
                 assert np.array_equal(got["indptr"][l].numpy(), blocks[l].indptr)
                 assert np.array_equal(got["indices"][l].numpy(), blocks[l].indices)
             assert torch.equal(got["feats"], X[torch.from_numpy(fr.astype(np.int64))])
+
+
+def _failing_worker(rank, world, port, out_dir):
+    import torch.distributed as dist
+
+    import fake_shard_ops as ops
+    from paper_2406_17918_b200 import sharded
+
+    dist.init_process_group("gloo", rank=rank, world_size=world, init_method="tcp://127.0.0.1:%d" % port)
+    cfg = get_config("tiny")
+    g = build_graph(cfg)
+    perm = seed_permutation(cfg)
+    X = _features(cfg["num_nodes"])
+    ip, idx = sharded.shard_csr(g.indptr, g.indices, rank, world)
+    lo, hi = sharded.shard_range(cfg["num_nodes"], rank, world)
+    # the last rank can serve three nodes per list only: its first hop fails on the owner side
+    cap = 3 if rank == world - 1 else cfg["num_nodes"]
+    me = sharded.ShardRank(ops, rank, world, ip, idx, X[lo:hi].contiguous(), cfg["fanouts"], cfg["cache_width"], SEED,
+                           cfg["shared"], THETA, max_seeds=cfg["batch"], max_requests=cap)
+    seeds = batch_seeds(perm, 1, cfg["batch"], rank, world)
+    outcome = "returned"
+    try:
+        sharded.sample_batch(me, seeds, ops.GS_MODE_OTF, 0.25, 1)
+    except sharded.ShardedBatchError as e:
+        outcome = "raised %d" % e.code
+    with open(os.path.join(out_dir, "f%d.txt" % rank), "w") as fh:
+        fh.write(outcome)
+    dist.barrier()            # every rank is still alive and in step
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_a_failure_on_one_rank_ends_the_batch_on_every_rank(tmp_path, world):
+    """An owner that cannot serve a list must not leave the others inside a collective: all ranks raise."""
+    mp.spawn(_failing_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    for r in range(world):
+        assert open(os.path.join(tmp_path, "f%d.txt" % r)).read() == "raised 2"
 
 
 def test_refreshing_a_row_twice_in_one_step_equals_once():
