@@ -42,11 +42,12 @@ SAMPLER_SEED = 0x6A09E667F3BCC908
 #   k_scan, workload large, sampling step 2 of batch 0: 5,650,944 B read + 12,288 B written for 16,380,004 Philox
 #     blocks in 45,281 work items.  The traffic is the items' descriptors, so it follows the number of items; larger
 #     rows mean fewer items per block, which makes the per-block scaling an upper estimate for the scale workload.
-#   k_gather with 256-byte bf16 rows, workload shared, batch 0: 13,165,824 B read for 50,620 rows (260 B per row: the
-#     row and its id); the 256 B written per row were still in L2 when that short launch ended, so the written bytes
-#     are counted as the algorithmic ones.
+#   k_gather with 256-byte bf16 rows, all 736,389 rows of workload shared once each in random order (--gather-only):
+#     191,470,592 B read (260 B per row: the row and its id, no over-fetch); 137 MB of the 188.5 MB written reached
+#     DRAM inside the launch, the rest was still in L2 when it ended, so the written bytes are counted as the
+#     algorithmic 256 B per row.
 NCU_SCAN_BYTES_PER_BLOCK = (5650944 + 12288) / 16380004
-NCU_GATHER_READ_BYTES_PER_256B_ROW = 13165824 / 50620
+NCU_GATHER_READ_BYTES_PER_256B_ROW = 191470592 / 736389
 
 
 def measured_peak():
@@ -280,6 +281,9 @@ def main():
                          "the CPU oracle and compare every output element by element: input nodes, every block's "
                          "offsets and indices, cache rows of sampled frontier nodes, gathered feature rows "
                          "(the oracle needs minutes on the largest workload)")
+    ap.add_argument("--gather-only", type=int, default=None, metavar="ROWS",
+                    help="time gs_gather_features alone on ROWS distinct, randomly ordered rows of the workload's feature matrix "
+                         "(a small, self-contained launch for profiler captures of the gather kernel); prints its own line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -319,6 +323,8 @@ def main():
         print("warning: --gpus %d but WORLD_SIZE=%d" % (args.gpus, world), file=sys.stderr)
     if args.sharded:
         return sharded_arm(args, cfg, mode, gamma, rank, local_rank, world, device)
+    if args.gather_only:
+        return gather_arm(args, cfg, device)
 
     # ---- inputs, resident in HBM before anything is timed
     t_setup = time.time()
@@ -665,6 +671,44 @@ def main():
                                   "host_cores": os.cpu_count(), "kind": "oracle", "sample": desc}
     print(json.dumps(result))
     replicas.shutdown()
+    return 0
+
+
+def gather_arm(args, cfg, device):
+    """gs_gather_features alone: ROWS distinct rows of the workload's feature matrix in a seeded random order."""
+    import paper_2406_17918_b200 as gs
+    from workloads.hashing import splitmix64
+
+    N, rows = cfg["num_nodes"], args.gather_only
+    X = build_features(cfg, device=device if cfg["feat_kind"] == "hash" else "cpu").to(device)
+    rows = min(rows, N)
+    # distinct rows in a seeded random order: every row is read from DRAM once, none is served twice from L2
+    ids = torch.argsort(splitmix64(torch.arange(N, dtype=torch.int64, device=device) + 0x5EED))[:rows].to(torch.int32)
+    indptr = torch.zeros(N + 1, dtype=torch.int64, device=device)
+    G = gs.gs_graph_create(indptr, torch.zeros(1, dtype=torch.int32, device=device), X)
+    gs.gs_graph_set_gather_grid(G, 16)
+    out = torch.empty((rows, cfg["feat_dim"]), dtype=X.dtype, device=device)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    times = []
+    for i in range(args.warmup + args.steps):
+        flush.zero_()                       # larger than L2: no row survives between launches
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        gs.gs_gather_features(G, ids, None, out)
+        b.record()
+        torch.cuda.synchronize()
+        if i >= args.warmup:
+            times.append(a.elapsed_time(b))
+    times.sort()
+    ms = times[len(times) // 2]
+    esize = 4 if cfg["feat_dtype"] == "f32" else 2
+    nbytes = rows * (4 + 2 * cfg["feat_dim"] * esize)
+    peak, peak_kind = measured_peak()
+    assert torch.equal(out.view(torch.int16 if esize == 2 else torch.int32), X[ids.long()].view(torch.int16 if esize == 2 else torch.int32))
+    print(json.dumps({"gather_only": {"workload": cfg["name"], "rows": rows, "row_bytes": cfg["feat_dim"] * esize,
+                                      "ms_per_launch_median": ms, "algorithmic_bytes": nbytes,
+                                      "achieved_gbs": nbytes / (ms * 1e-3) / 1e9, "peak_gbs": peak, "peak_kind": "of " + peak_kind,
+                                      "frac": nbytes / (ms * 1e-3) / 1e9 / peak, "gpu_launches": args.warmup + args.steps}}))
     return 0
 
 

@@ -281,7 +281,7 @@ gs_status gs_gather_rows_peer(const void* const* h_shard_bases, int32_t world, i
                               int32_t count_bound, void* d_out, int64_t out_ld, void* stream);
 
 /* ---- Node-sharded sampling over several GPUs (the paper's Section "Shared Cache Mode" speaks of a
- * cache that serves multiple computation processes; the partition and the exchange are this
+ * cache shared by several trainer processes; the partition and the exchange are this
  * library's).  Nodes are partitioned by id range: shard o of `world` owns the nodes
  * [o*S, (o+1)*S), S = ceil(num_nodes / world), with their CSR rows, cache rows and feature rows.
  * A shard's gs_graph has the full num_nodes and an indptr in which only the owned rows are
