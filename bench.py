@@ -341,7 +341,7 @@ def main():
         ev0.record()
         C = gs.gs_cache_init(G, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED, cfg["shared"], storage=storage)
     else:
-        dense_rows = int((g.degrees() > args.theta).sum().item())
+        dense_rows = gs.gs_graph_count_dense(G, args.theta)
         storage = torch.empty(gs.gs_cache_bytes_split(G, L_hops, cfg["cache_width"], cfg["shared"], dense_rows),
                               dtype=torch.uint8, device=device)
         ev0.record()

@@ -118,6 +118,9 @@ void gs_cache_destroy(gs_cache*);
  * gs_cache_init_split synchronises `stream` once (to verify dense_rows). */
 gs_status gs_cache_bytes_split(const gs_graph*, int32_t num_hops, int32_t cache_width, int32_t shared,
                                int64_t dense_rows, size_t* bytes);
+/* Counts the nodes with degree > theta on the device (the dense_rows argument above and below) and
+ * synchronises `stream`.  Uses an 8-byte device variable of the library: calls must not overlap. */
+gs_status gs_graph_count_dense(const gs_graph*, int32_t theta, void* stream, int64_t* h_dense_rows);
 gs_status gs_cache_init_split(const gs_graph*, int32_t num_hops, const int32_t* fanouts, int32_t cache_width,
                               uint64_t seed, int32_t shared, int32_t theta, int64_t dense_rows,
                               void* d_cache_storage, size_t cache_bytes, void* stream, gs_cache** out);

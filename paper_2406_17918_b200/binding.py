@@ -100,6 +100,7 @@ def _load():
         "gs_debug_set_grid_cap": [i32],
         "gs_alu_ceiling": [i32, i32, vp, ctypes.POINTER(dbl)],
         "gs_cache_set_dedup": [vp, i32],
+        "gs_graph_count_dense": [vp, i32, vp, ctypes.POINTER(i64)],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -275,12 +276,18 @@ def gs_cache_bytes_split(graph: Graph, num_hops: int, cache_width: int, shared: 
     return out.value
 
 
+def gs_graph_count_dense(graph: Graph, theta: int, stream=None) -> int:
+    """Nodes with degree > theta, counted by the library (synchronises)."""
+    out = ctypes.c_int64()
+    _check(_L.gs_graph_count_dense(graph.handle, int(theta), _stream(stream), ctypes.byref(out)))
+    return int(out.value)
+
+
 def gs_cache_init_split(graph: Graph, fanouts, cache_width: int, seed: int, shared: bool, theta: int,
                         dense_rows: int = None, storage: torch.Tensor = None, stream=None) -> Cache:
     """Cache rows only for nodes with degree > theta; the others are sampled from the graph."""
     if dense_rows is None:
-        deg = graph.indptr[1:] - graph.indptr[:-1]
-        dense_rows = int((deg > theta).sum().item())
+        dense_rows = gs_graph_count_dense(graph, theta, stream)
     if storage is None:
         storage = torch.empty(gs_cache_bytes_split(graph, len(fanouts), cache_width, shared, dense_rows),
                               dtype=torch.uint8, device=graph.indptr.device)

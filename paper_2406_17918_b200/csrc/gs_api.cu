@@ -210,6 +210,13 @@ gs_status gs_graph_validate(const gs_graph* g, void* stream, int64_t* h_first_ba
     return GS_OK;
 }
 
+gs_status gs_graph_count_dense(const gs_graph* g, int32_t theta, void* stream, int64_t* h_dense_rows) {
+    if (!g || !h_dense_rows) return fail(GS_ERR_ARG, "NULL argument");
+    if (theta < 0) return fail(GS_ERR_ARG, "theta must be >= 0");
+    GS_CUDA(launch_count_dense(GraphView{g->d_indptr, g->d_indices, g->num_nodes}, theta, h_dense_rows, (cudaStream_t)stream));
+    return GS_OK;
+}
+
 gs_status gs_cache_bytes(const gs_graph* g, int32_t num_hops, int32_t cache_width, int32_t shared, size_t* bytes) {
     if (!bytes) return fail(GS_ERR_ARG, "bytes is NULL");
     gs_status st = check_shape(g, num_hops, cache_width);

@@ -297,6 +297,7 @@ cudaError_t launch_gather_sharded(const void* const* bases, int32_t world, int64
                                   int64_t row_bytes, const int32_t* ids, const int32_t* d_count, int32_t count_bound,
                                   void* dst, int64_t dst_ld_bytes, cudaStream_t s);
 cudaError_t launch_validate_graph(const GraphView& g, int64_t num_edges, int64_t* h_first_bad_row, cudaStream_t s);
+cudaError_t launch_count_dense(const GraphView& g, int32_t theta, int64_t* h_count, cudaStream_t s);
 cudaError_t launch_read_rows(const int32_t* slots, const int32_t* row_index, int32_t pitch, int32_t W,
                              const int32_t* nodes, int32_t n, int32_t* out, cudaStream_t s);
 cudaError_t launch_shard_bucket(const int32_t* nodes, int32_t n, int32_t rows_per_shard, int32_t world, int32_t* sorted,

@@ -361,6 +361,39 @@ cudaError_t launch_validate_graph(const GraphView& g, int64_t num_edges, int64_t
     return cudaSuccess;
 }
 
+// ---------------------------------------------------------------- dense part of a split cache
+// Number of nodes with degree > theta (what gs_cache_bytes_split and gs_cache_init_split are sized from).
+__device__ unsigned long long g_dense_count;
+
+__global__ void __launch_bounds__(256) k_count_dense(GraphView g, long long theta, unsigned long long* out) {
+    unsigned mine = 0;
+    for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < g.num_nodes; v += (long long)gridDim.x * blockDim.x)
+        mine += (g.indptr[v + 1] - g.indptr[v] > theta) ? 1u : 0u;
+    mine = __reduce_add_sync(FULL, mine);
+    if ((threadIdx.x & 31) == 0 && mine) atomicAdd(out, (unsigned long long)mine);
+}
+
+cudaError_t launch_count_dense(const GraphView& g, int32_t theta, int64_t* h_count, cudaStream_t s) {
+    unsigned long long* d = nullptr;
+    cudaError_t e = cudaGetSymbolAddress((void**)&d, g_dense_count);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(d, 0, sizeof(unsigned long long), s);
+    if (e != cudaSuccess) return e;
+    int64_t blocks = (g.num_nodes + 255) / 256;
+    if (blocks > sm_count() * 16) blocks = sm_count() * 16;
+    k_count_dense<<<(int)blocks, 256, 0, s>>>(g, (long long)theta, d);
+    count_launches(1);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    unsigned long long h = 0;
+    e = cudaMemcpyAsync(&h, d, sizeof(h), cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return e;
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return e;
+    *h_count = (int64_t)h;
+    return cudaSuccess;
+}
+
 // ---------------------------------------------------------------- logical cache rows (parity / debug)
 __global__ void k_read_rows(const int32_t* slots, const int32_t* row_index, int pitch, int W, const int32_t* nodes,
                             int n, int32_t* out) {
