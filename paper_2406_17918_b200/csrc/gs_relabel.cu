@@ -251,46 +251,58 @@ __global__ void __launch_bounds__(FF_THREADS) k_first_flags(RelabelParams P) {
     if (threadIdx.x == 0) P.hdr[HDR_N + P.k + 1] = n + fresh;
 }
 
-// Four consecutive picks per thread, so that the dependent probes of four items overlap.
+// Eight consecutive picks per thread, so that the dependent probes of eight items overlap.
+constexpr int RL_PICKS = 8;
+
 __global__ void __launch_bounds__(256) k_relabel(RelabelParams P) {
     if (__ldcg(P.hdr + HDR_STATUS) != 0) return;
     const int n = __ldcg(P.hdr + HDR_N + P.k);
     const int m = __ldcg(P.hdr + HDR_M + P.k);
-    for (int e0 = 4 * (blockIdx.x * blockDim.x + threadIdx.x); e0 < m; e0 += 4 * gridDim.x * blockDim.x) {
-        const int4 a = *reinterpret_cast<const int4*>(P.aux + e0);   // padded to 4
-        const int val[4] = {a.x, a.y, a.z, a.w};
-        int ref[4], tile[4];
+    for (int e0 = RL_PICKS * (blockIdx.x * blockDim.x + threadIdx.x); e0 < m; e0 += RL_PICKS * gridDim.x * blockDim.x) {
+        int val[RL_PICKS];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int q = 0; q < RL_PICKS / 4; ++q) {
+            int4 a = make_int4(0, 0, 0, 0);
+            if (e0 + 4 * q < m) a = *reinterpret_cast<const int4*>(P.aux + e0 + 4 * q);   // padded to 4
+            val[4 * q] = a.x; val[4 * q + 1] = a.y; val[4 * q + 2] = a.z; val[4 * q + 3] = a.w;
+        }
+        int ref[RL_PICKS], tile[RL_PICKS], id[RL_PICKS];
+#pragma unroll
+        for (int i = 0; i < RL_PICKS; ++i) {
             // first occurrence: own mark; later occurrence of a new id: the mark of its first occurrence
             const int src = (val[i] < 0) ? e0 + i : (val[i] >= n ? val[i] - n : -1);
             ref[i] = val[i];
             tile[i] = 0;
+            id[i] = 0;
             if (e0 + i < m && src >= 0) {
                 if (val[i] >= 0) ref[i] = P.aux[src];
+                else id[i] = P.picked[e0 + i];
                 tile[i] = P.tile_sums[src / SCAN_E_TILE];
             }
         }
-        int out[4];
+        int out[RL_PICKS];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < RL_PICKS; ++i) {
             int loc = val[i];
             if (e0 + i < m && (val[i] < 0 || val[i] >= n)) {
                 loc = n + (-ref[i] - 1) + tile[i];
                 if (val[i] < 0 && (int64_t)loc < P.n_cap) {
-                    const int id = P.picked[e0 + i];
-                    P.frontier[loc] = id;
-                    if (P.table) P.table[id] = ((unsigned long long)P.stamp << 32) | (unsigned)loc;
+                    P.frontier[loc] = id[i];
+                    if (P.table) P.table[id[i]] = ((unsigned long long)P.stamp << 32) | (unsigned)loc;
                 }
             }
             out[i] = loc;
         }
-        if (e0 + 3 < m) {
-            *reinterpret_cast<int4*>(P.local + e0) = make_int4(out[0], out[1], out[2], out[3]);
-        } else {
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (e0 + i < m) P.local[e0 + i] = out[i];
+        for (int q = 0; q < RL_PICKS / 4; ++q) {
+            const int e = e0 + 4 * q;
+            if (e + 3 < m) {
+                *reinterpret_cast<int4*>(P.local + e) = make_int4(out[4 * q], out[4 * q + 1], out[4 * q + 2], out[4 * q + 3]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (e + i < m) P.local[e + i] = out[4 * q + i];
+            }
         }
     }
 }
@@ -310,8 +322,8 @@ cudaError_t launch_relabel(const RelabelParams& p, int64_t n_bound, int64_t m_bo
     if (p.method == DEDUP_HASH) k_first_flags<DEDUP_HASH><<<(int)tiles, FF_THREADS, 0, s>>>(p);
     else if (p.method == DEDUP_SORT) k_first_flags<DEDUP_SORT><<<(int)tiles, FF_THREADS, 0, s>>>(p);
     else k_first_flags<DEDUP_DIRECT><<<(int)tiles, FF_THREADS, 0, s>>>(p);
-    int64_t blocks = (m_bound + 1023) / 1024;
-    if (blocks > sm_count() * 32) blocks = sm_count() * 32;
+    int64_t blocks = (m_bound + 256 * RL_PICKS - 1) / (256 * RL_PICKS);
+    if (blocks > sm_count() * 16) blocks = sm_count() * 16;
     blocks = limit_grid(blocks);
     RelabelParams q = p;
     if (p.method != DEDUP_DIRECT) q.table = nullptr;
