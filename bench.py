@@ -39,14 +39,14 @@ FALLBACK_HBM_GBS = 6650.0
 SAMPLER_SEED = 0x6A09E667F3BCC908
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one captured launch, from ncu captures of the same
 # kernels on small workloads (scaled to a launch of the benchmarked workload by the units it processes).
-#   k_scan, workload large, sampling step 2 of batch 0: 5,650,944 B read + 12,288 B written for 16,380,004 Philox
-#     blocks in 45,281 work items.  The traffic is the items' descriptors, so it follows the number of items; larger
+#   k_scan, workload large, sampling step 2 of a batch: 5,612,800 B read + 12,544 B written for 16.38 M Philox
+#     blocks in 45 K work items.  The traffic is the items' descriptors, so it follows the number of items; larger
 #     rows mean fewer items per block, which makes the per-block scaling an upper estimate for the scale workload.
 #   k_gather with 256-byte bf16 rows, all 736,389 rows of workload shared once each in random order (--gather-only):
 #     191,470,592 B read (260 B per row: the row and its id, no over-fetch); 137 MB of the 188.5 MB written reached
 #     DRAM inside the launch, the rest was still in L2 when it ended, so the written bytes are counted as the
 #     algorithmic 256 B per row.
-NCU_SCAN_BYTES_PER_BLOCK = (5650944 + 12288) / 16380004
+NCU_SCAN_BYTES_PER_BLOCK = (5612800 + 12544) / 16380004
 NCU_GATHER_READ_BYTES_PER_256B_ROW = 191470592 / 736389
 
 
