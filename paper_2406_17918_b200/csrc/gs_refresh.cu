@@ -67,7 +67,7 @@ __device__ __forceinline__ int warp_collect(const StepParams& P, int32_t v, uint
     const uint32_t lt = lanemask_lt();
     for (uint32_t qb = q_begin; qb < q_end; qb += 32) {
         const uint32_t q = qb + lane;
-        const uint4 o = philox4x32_10(q, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
+        const uint4 o = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
         const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
         const bool inq = q < q_end;
         const bool any = inq && (min(min(kk[0], kk[1]), min(kk[2], kk[3])) <= tinc);
@@ -99,7 +99,7 @@ __device__ __noinline__ void warp_exact_top(const StepParams& P, int32_t v, uint
     const uint32_t nq = (deg + 3u) >> 2;
     for (uint32_t qb = 0; qb < nq; qb += 32) {
         const uint32_t q = qb + lane;
-        const uint4 o = philox4x32_10(q, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
+        const uint4 o = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
         const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
@@ -355,7 +355,7 @@ struct Quick {
 __device__ __forceinline__ uint32_t evict_mask_for(const StepParams& P, int32_t v, int lane) {
     const uint32_t wmask = P.W >= 32 ? FULL : ((1u << P.W) - 1u);
     if (P.r >= P.W) return wmask;
-    const uint4 o = philox4x32_10((uint32_t)lane >> 2, (uint32_t)v, P.step, P.word_evict, P.key0, P.key1);
+    const uint4 o = philox4x32_10_rk((uint32_t)lane >> 2, (uint32_t)v, P.step, P.word_evict, P.rk);
     return warp_smallest_k(word_of(o, lane & 3), wmask, P.r, lane);
 }
 
@@ -371,7 +371,7 @@ __device__ __forceinline__ void warp_pick(const StepParams& P, int32_t v, uint32
     const uint32_t cmask = cnt >= 32 ? FULL : ((1u << cnt) - 1u);
     uint32_t pm = cmask;
     if (cnt > P.f) {
-        const uint4 o = philox4x32_10((uint32_t)lane >> 2, (uint32_t)v, P.step, P.word_pick, P.key0, P.key1);
+        const uint4 o = philox4x32_10_rk((uint32_t)lane >> 2, (uint32_t)v, P.step, P.word_pick, P.rk);
         pm = warp_smallest_k(word_of(o, lane & 3), cmask, P.f, lane);
     }
     if ((pm >> lane) & 1u) {
@@ -599,7 +599,7 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick_hub(const __grid
         int* cand_count = &P.hub_state[h].x;
         for (uint32_t qb = qa; qb < qe; qb += 32) {
             const uint32_t q = qb + lane;
-            const uint4 o = philox4x32_10(q, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
+            const uint4 o = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
             const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
             const bool inq = q < qe;
             const bool any = inq && (min(min(kk[0], kk[1]), min(kk[2], kk[3])) <= tinc);
@@ -786,8 +786,7 @@ __global__ void __launch_bounds__(RP_THREADS, GS_SCAN_MIN_BLOCKS) k_scan(const _
 __device__ __forceinline__ void evict_pick_keys(const StepParams& P, int32_t v, int lane, uint32_t& ekey,
                                                 uint32_t& pkey) {
     const bool second = (lane >> 3) & 1;
-    const uint4 o = philox4x32_10((uint32_t)lane & 7u, (uint32_t)v, P.step, second ? P.word_pick : P.word_evict,
-                                  P.key0, P.key1);
+    const uint4 o = philox4x32_10_rk((uint32_t)lane & 7u, (uint32_t)v, P.step, second ? P.word_pick : P.word_evict, P.rk);
     const int src = lane >> 2, w = lane & 3;
     const uint32_t e0 = __shfl_sync(FULL, o.x, src), e1 = __shfl_sync(FULL, o.y, src);
     const uint32_t e2 = __shfl_sync(FULL, o.z, src), e3 = __shfl_sync(FULL, o.w, src);
@@ -802,7 +801,7 @@ __device__ __forceinline__ void evict_pick_keys(const StepParams& P, int32_t v, 
 // and the r smallest remaining (key, offset) pairs go to the evicted slots in ascending order.
 __device__ __forceinline__ void small_refill(const StepParams& P, int32_t v, int64_t row_start, uint32_t deg,
                                              uint32_t evict, int32_t& slot, int lane) {
-    const uint4 o = philox4x32_10((uint32_t)lane, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
+    const uint4 o = philox4x32_10_rk((uint32_t)lane, (uint32_t)v, P.step, P.word_fill, P.rk);
     const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
     int32_t nb[4];
     bool ok[4];
@@ -912,7 +911,7 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
                 if ((int)deg <= f) {
                     if (lane < (int)deg) id = __ldg(P.g.indices + rs + lane);
                 } else {
-                    const uint4 o = philox4x32_10((uint32_t)lane, (uint32_t)v, P.step, P.word_fetch, P.key0, P.key1);
+                    const uint4 o = philox4x32_10_rk((uint32_t)lane, (uint32_t)v, P.step, P.word_fetch, P.rk);
                     const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
@@ -945,7 +944,7 @@ __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(con
                 int c = -1;
                 uint32_t tinc = 0xFFFFFFFFu;
                 if (deg <= (uint32_t)SMALL_DEGREE) {
-                    const uint4 o = philox4x32_10((uint32_t)lane, (uint32_t)v, P.step, P.word_fill, P.key0, P.key1);
+                    const uint4 o = philox4x32_10_rk((uint32_t)lane, (uint32_t)v, P.step, P.word_fill, P.rk);
                     const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
