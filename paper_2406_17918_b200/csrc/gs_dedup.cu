@@ -32,6 +32,7 @@ __device__ __forceinline__ uint32_t mix32(uint32_t x) {
 }
 
 __global__ void __launch_bounds__(DD_THREADS) k_hash_clear(RelabelParams P) {
+    chain_wait();
     if (__ldcg(P.hdr + HDR_STATUS) != 0) return;
     const long long keys = (long long)__ldcg(P.hdr + HDR_N + P.k) + __ldcg(P.hdr + HDR_M + P.k);
     long long cap = dedup_hash_capacity(keys);
@@ -44,6 +45,7 @@ __global__ void __launch_bounds__(DD_THREADS) k_hash_clear(RelabelParams P) {
 }
 
 __global__ void __launch_bounds__(DD_THREADS) k_hash_insert(RelabelParams P) {
+    chain_wait();
     int32_t* status = P.hdr + HDR_STATUS;
     if (__ldcg(status) != 0) return;
     const int n = __ldcg(P.hdr + HDR_N + P.k);
@@ -82,10 +84,10 @@ cudaError_t launch_dedup_hash(const RelabelParams& p, int64_t n_bound, int64_t m
     const int64_t keys = n_bound + m_bound;
     int64_t blocks = (dedup_hash_capacity(keys) / 2 + DD_THREADS - 1) / DD_THREADS;
     if (blocks > sm_count() * 8) blocks = sm_count() * 8;
-    k_hash_clear<<<(int)limit_grid(blocks), DD_THREADS, 0, s>>>(p);
+    launch_chained(k_hash_clear, limit_grid(blocks), DD_THREADS, s, p);
     blocks = (keys + DD_THREADS - 1) / DD_THREADS;
     if (blocks > sm_count() * 32) blocks = sm_count() * 32;
-    k_hash_insert<<<(int)limit_grid(blocks), DD_THREADS, 0, s>>>(p);
+    launch_chained(k_hash_insert, limit_grid(blocks), DD_THREADS, s, p);
     count_launches(2);
     return cudaGetLastError();
 }

@@ -41,6 +41,13 @@ __device__ __forceinline__ uint4 philox4x32_10_rk(uint32_t c0, uint32_t c1, uint
     return make_uint4(c0, c1, c2, c3);
 }
 
+// Kernels of a batch are launched with programmatic stream serialization: a kernel may be set up on the GPU
+// while its predecessor in the stream is still draining, and must call this before it reads anything the
+// predecessor wrote (it returns once the predecessor has completed and its writes are visible).
+__device__ __forceinline__ void chain_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ uint32_t word_of(const uint4& o, uint32_t w) {
     return w == 0 ? o.x : (w == 1 ? o.y : (w == 2 ? o.z : o.w));
 }

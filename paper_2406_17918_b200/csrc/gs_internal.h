@@ -248,6 +248,22 @@ struct RelabelParams {
     int32_t id_bits;                 // bits of a node id (sort passes)
 };
 
+// Launch with programmatic stream serialization (the kernel starts with chain_wait()).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), int64_t grid, int block, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 void count_launches(int n);
 // Streaming multiprocessors of the current device (looked up once per device).
 int64_t sm_count();

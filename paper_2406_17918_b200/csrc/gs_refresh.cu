@@ -461,6 +461,7 @@ struct NodeState {
 };
 
 __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick(const __grid_constant__ StepParams P) {
+    chain_wait();
     __shared__ unsigned long long s_buf[RP_WARPS][CAND_CAP];
     if (__ldcg(P.status) != 0) return;   // set only by earlier kernels of the batch: uniform
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -564,6 +565,7 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick(const __grid_con
 
 // ---------------------------------------------------------------- warp-per-chunk kernel (hubs)
 __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick_hub(const __grid_constant__ StepParams P) {
+    chain_wait();
     __shared__ unsigned long long s_buf[RP_WARPS][CAND_CAP];
     if (__ldcg(P.status) != 0) return;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -660,6 +662,7 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick_hub(const __grid
 // neighbours among the first ones) take the retry ladder of the fused path.
 
 __global__ void __launch_bounds__(RP_THREADS, GS_SCAN_MIN_BLOCKS) k_scan(const __grid_constant__ StepParams P) {
+    chain_wait();
     __shared__ unsigned long long s_stage[RP_WARPS][SPLIT_CAND_CAP];
     __shared__ int s_hits[RP_WARPS];
     if (__ldcg(P.status) != 0) return;
@@ -842,6 +845,7 @@ __device__ __forceinline__ void small_refill(const StepParams& P, int32_t v, int
 }
 
 __global__ void __launch_bounds__(RP_THREADS, GS_FINISH_MIN_BLOCKS) k_finish(const __grid_constant__ StepParams P) {
+    chain_wait();
     __shared__ unsigned long long s_buf[RP_WARPS][CAND_CAP];
     if (__ldcg(P.status) != 0) return;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -1082,7 +1086,7 @@ cudaError_t launch_scan(const StepParams& p, int64_t item_bound, cudaStream_t s)
     const int64_t cap = sm_count() * resident;
     int64_t sb = (item_bound + RP_WARPS - 1) / RP_WARPS;
     sb = limit_grid(sb > cap ? cap : (sb < 1 ? 1 : sb));
-    k_scan<<<(int)sb, RP_THREADS, 0, s>>>(p);
+    launch_chained(k_scan, sb, RP_THREADS, s, p);
     count_launches(1);
     return cudaGetLastError();
 }
@@ -1091,12 +1095,12 @@ cudaError_t launch_finish(const StepParams& p, int64_t n_bound, cudaStream_t s) 
     const int64_t cap = sm_count() * 8;
     int64_t fb = (n_bound + RP_WARPS - 1) / RP_WARPS;
     fb = limit_grid(fb > cap ? cap : (fb < 1 ? 1 : fb));
-    k_finish<<<(int)fb, RP_THREADS, 0, s>>>(p);
+    launch_chained(k_finish, fb, RP_THREADS, s, p);
     int launched = 1;
     if (p.hub_cap > 0) {   // rows queued for a rescan; exits at once when there are none
         // a partial refresh queues a handful of rows per batch at most, a full one about 1 % of them
         const int64_t hub_grid = limit_grid((p.r >= p.W) ? cap : sm_count() * 2);
-        k_refresh_pick_hub<<<(int)hub_grid, RP_THREADS, 0, s>>>(p);
+        launch_chained(k_refresh_pick_hub, hub_grid, RP_THREADS, s, p);
         launched = 2;
     }
     count_launches(launched);
@@ -1132,10 +1136,10 @@ cudaError_t launch_refresh_pick(const StepParams& p, int64_t n_bound, cudaStream
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     blocks = limit_grid(blocks);
-    k_refresh_pick<<<(int)blocks, RP_THREADS, 0, s>>>(p);
+    launch_chained(k_refresh_pick, blocks, RP_THREADS, s, p);
     int launched = 1;
     if (p.hub_cap > 0) {
-        k_refresh_pick_hub<<<(int)limit_grid(cap), RP_THREADS, 0, s>>>(p);
+        launch_chained(k_refresh_pick_hub, limit_grid(cap), RP_THREADS, s, p);
         launched = 2;
     }
     count_launches(launched);

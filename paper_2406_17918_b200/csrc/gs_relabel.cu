@@ -12,6 +12,7 @@ namespace gs {
 // degree alone, so the block CSR offsets exist before anything is sampled.  Step 0 also copies
 // the seeds into the frontier, validates them and preloads the relabel table with their positions.
 __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
+    chain_wait();
     __shared__ int warp_sums[33];
     __shared__ int is_last;
     __shared__ int s_status;
@@ -104,6 +105,7 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
 }
 
 __global__ void __launch_bounds__(1024) k_row_offsets(CountParams P) {
+    chain_wait();
     if (__ldcg(P.hdr + HDR_STATUS) != 0) return;
     const int n = (P.k == 0) ? P.n_host : __ldcg(P.hdr + HDR_N + P.k);
     for (int t = blockIdx.x; t <= n / SCAN_A_TILE; t += gridDim.x) {   // the tile of position n takes part too
@@ -135,8 +137,8 @@ cudaError_t launch_row_counts(const CountParams& p, int64_t n_bound, cudaStream_
     int64_t tiles = n_bound / SCAN_A_TILE + 1;
     if (tiles > sm_count() * 2) tiles = sm_count() * 2;
     tiles = limit_grid(tiles);
-    k_row_counts<<<(int)tiles, SCAN_A_TILE, 0, s>>>(p);
-    k_row_offsets<<<(int)tiles, SCAN_A_TILE, 0, s>>>(p);
+    launch_chained(k_row_counts, tiles, SCAN_A_TILE, s, p);
+    launch_chained(k_row_offsets, tiles, SCAN_A_TILE, s, p);
     count_launches(2);
     return cudaGetLastError();
 }
@@ -156,6 +158,7 @@ static_assert(SCAN_E_TILE == FF_THREADS * 16, "tile = 16 picks per thread");
 // id), the batch-sized hash table (aux[e] holds the id's slot), or aux[e] itself (the sort left it there).
 template <int METHOD>
 __global__ void __launch_bounds__(FF_THREADS) k_first_flags(RelabelParams P) {
+    chain_wait();
     __shared__ int warp_sums[33];
     __shared__ int s_wtot[FF_THREADS / 32];
     __shared__ int is_last;
@@ -255,6 +258,7 @@ __global__ void __launch_bounds__(FF_THREADS) k_first_flags(RelabelParams P) {
 constexpr int RL_PICKS = 8;
 
 __global__ void __launch_bounds__(256) k_relabel(RelabelParams P) {
+    chain_wait();
     if (__ldcg(P.hdr + HDR_STATUS) != 0) return;
     const int n = __ldcg(P.hdr + HDR_N + P.k);
     const int m = __ldcg(P.hdr + HDR_M + P.k);
@@ -319,15 +323,15 @@ cudaError_t launch_relabel(const RelabelParams& p, int64_t n_bound, int64_t m_bo
     int64_t tiles = (m_bound + SCAN_E_TILE - 1) / SCAN_E_TILE;
     if (tiles > sm_count() * 16) tiles = sm_count() * 16;    // blocks walk the tiles; enough of them that a usual batch has one tile each
     tiles = limit_grid(tiles);
-    if (p.method == DEDUP_HASH) k_first_flags<DEDUP_HASH><<<(int)tiles, FF_THREADS, 0, s>>>(p);
-    else if (p.method == DEDUP_SORT) k_first_flags<DEDUP_SORT><<<(int)tiles, FF_THREADS, 0, s>>>(p);
-    else k_first_flags<DEDUP_DIRECT><<<(int)tiles, FF_THREADS, 0, s>>>(p);
+    if (p.method == DEDUP_HASH) launch_chained(k_first_flags<DEDUP_HASH>, tiles, FF_THREADS, s, p);
+    else if (p.method == DEDUP_SORT) launch_chained(k_first_flags<DEDUP_SORT>, tiles, FF_THREADS, s, p);
+    else launch_chained(k_first_flags<DEDUP_DIRECT>, tiles, FF_THREADS, s, p);
     int64_t blocks = (m_bound + 256 * RL_PICKS - 1) / (256 * RL_PICKS);
     if (blocks > sm_count() * 16) blocks = sm_count() * 16;
     blocks = limit_grid(blocks);
     RelabelParams q = p;
     if (p.method != DEDUP_DIRECT) q.table = nullptr;
-    k_relabel<<<(int)blocks, 256, 0, s>>>(q);
+    launch_chained(k_relabel, blocks, 256, s, q);
     count_launches(2);
     return cudaGetLastError();
 }
