@@ -17,6 +17,9 @@
  *     kernels of that batch then write nothing further.
  *   - All work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default stream)
  *     and is asynchronous unless a call says it synchronises.
+ *     The kernels of a batch are launched with programmatic stream serialization (a kernel is set
+ *     up on the GPU while its predecessor drains and waits for it before it reads anything); towards
+ *     other work on `stream` the usual stream order holds.
  *   - Graph contract: CSR row v lists the in-neighbours of v in ascending order without
  *     duplicates; num_nodes < 2^31; indptr is int64, ids are int32.
  *   - Fan-outs are listed input-layer-first.  Sampling step k = 0..L-1 starts at the seeds and
