@@ -455,7 +455,9 @@ def main():
         m = [int(counts[i][w]) for w in m_words]
         edges += sum(m)
         feat_rows += n[L]
-        a, f = algorithmic_bytes(cfg, n, m, [refreshed_frac[k] * n[k] for k in range(L)], r)
+        # rows refreshed in this batch, all steps together (counted on the device by the row-count kernel)
+        refreshed_rows = int(counts[i][stat0 + 2]) & 0xFFFFFFFF
+        a, f = algorithmic_bytes(cfg, n, m, [refreshed_rows] + [0] * (L - 1), r)
         alg_total += a
         alg_feat += f
 
