@@ -311,6 +311,11 @@ gs_status gs_gather_rows_peer(const void* const* h_shard_bases, int32_t world, i
  * [0, num_nodes)); the words between are scratch.  world <= 64.  Asynchronous on `stream`. */
 gs_status gs_shard_bucket(const int32_t* d_nodes, int32_t n, int64_t num_nodes, int32_t world, int32_t* d_sorted,
                           int32_t* d_slot, int32_t* d_counts, void* stream);
+/* The same for a list whose length is a device scalar (the frontier of the previous hop: *d_n, e.g.
+ * gs_block.d_num_src), of at most n_bound ids: the requester needs no host copy of the frontier's size
+ * before it buckets; the group sizes it reads back for the exchange add up to the length. */
+gs_status gs_shard_bucket_counted(const int32_t* d_nodes, const int32_t* d_n, int32_t n_bound, int64_t num_nodes,
+                                  int32_t world, int32_t* d_sorted, int32_t* d_slot, int32_t* d_counts, void* stream);
 
 /* Owner side.  For n distinct nodes of this shard: refresh (per mode / rate, exactly as
  * gs_sample_batch does for a frontier at `layer`) and pick; d_picks[n][fanout(layer)] receives the

@@ -89,6 +89,7 @@ def _load():
         "gs_gather_rows": [vp, ctypes.c_int, i32, i64, i64, i64, vp, vp, i32, vp, i64, vp],
         "gs_gather_rows_peer": [vp, i32, i64, ctypes.c_int, i32, i64, vp, vp, i32, vp, i64, vp],
         "gs_shard_bucket": [vp, i32, i64, i32, vp, vp, vp, vp],
+        "gs_shard_bucket_counted": [vp, vp, i32, i64, i32, vp, vp, vp, vp],
         "gs_shard_workspace_bytes": [vp, i32, i32, psz],
         "gs_shard_sample_rows": [vp, vp, i32, i32, ctypes.c_int, dbl, u32, vp, sz, vp, vp],
         "gs_shard_status": [vp, vp],
@@ -428,15 +429,20 @@ def gs_gather_rows_peer(shard_bases, num_rows: int, dtype: torch.dtype, row_elem
     return out
 
 
-def gs_shard_bucket(nodes: torch.Tensor, num_nodes: int, world: int, stream=None):
-    """Group node ids by owner.  Returns (sorted ids, slot of every input id, int32[2*world+1] device counts)."""
+def gs_shard_bucket(nodes: torch.Tensor, num_nodes: int, world: int, stream=None, count=None):
+    """Group node ids by owner.  Returns (sorted ids, slot of every input id, int32[2*world+1] device counts).
+    `count`: a 0-d int32 CUDA tensor with the list's length when only the device knows it (`nodes` is then the bound)."""
     if nodes.dtype != torch.int32 or not nodes.is_cuda or not nodes.is_contiguous():
         raise TypeError("nodes must be a contiguous int32 CUDA tensor")
     sorted_ids = torch.empty_like(nodes)
     slot = torch.empty_like(nodes)
     counts = torch.empty(2 * world + 1, dtype=torch.int32, device=nodes.device)
-    _check(_L.gs_shard_bucket(_ptr(nodes), nodes.numel(), int(num_nodes), int(world), _ptr(sorted_ids), _ptr(slot),
-                              _ptr(counts), _stream(stream)))
+    if count is None:
+        _check(_L.gs_shard_bucket(_ptr(nodes), nodes.numel(), int(num_nodes), int(world), _ptr(sorted_ids), _ptr(slot),
+                                  _ptr(counts), _stream(stream)))
+    else:
+        _check(_L.gs_shard_bucket_counted(_ptr(nodes), _ptr(count), nodes.numel(), int(num_nodes), int(world),
+                                          _ptr(sorted_ids), _ptr(slot), _ptr(counts), _stream(stream)))
     return sorted_ids, slot, counts
 
 

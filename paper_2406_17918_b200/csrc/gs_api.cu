@@ -748,16 +748,27 @@ gs_status gs_cache_refresh_all(gs_cache* c, gs_mode mode, double gamma, uint32_t
 
 /* ---------------------------------------------------------------- node-sharded sampling */
 
-gs_status gs_shard_bucket(const int32_t* d_nodes, int32_t n, int64_t num_nodes, int32_t world, int32_t* d_sorted,
-                          int32_t* d_slot, int32_t* d_counts, void* stream) {
+static gs_status shard_bucket_impl(const int32_t* d_nodes, int32_t n, const int32_t* d_n, int64_t num_nodes, int32_t world,
+                                   int32_t* d_sorted, int32_t* d_slot, int32_t* d_counts, void* stream) {
     if (world < 1 || world > 64) return fail(GS_ERR_ARG, "world %d outside [1, 64]", world);
     if (num_nodes < 1 || num_nodes >= ((int64_t)1 << 31)) return fail(GS_ERR_ARG, "num_nodes outside [1, 2^31)");
     if (n < 0) return fail(GS_ERR_ARG, "n is negative");
     if (!d_counts || (n > 0 && (!d_nodes || !d_sorted || !d_slot))) return fail(GS_ERR_ARG, "NULL argument");
     const int32_t rows_per_shard = (int32_t)((num_nodes + world - 1) / world);
-    GS_CUDA(launch_shard_bucket(d_nodes, n, rows_per_shard, world, d_sorted, d_slot, d_counts, d_counts + 2 * world,
+    GS_CUDA(launch_shard_bucket(d_nodes, n, d_n, rows_per_shard, world, d_sorted, d_slot, d_counts, d_counts + 2 * world,
                                 (cudaStream_t)stream));
     return GS_OK;
+}
+
+gs_status gs_shard_bucket(const int32_t* d_nodes, int32_t n, int64_t num_nodes, int32_t world, int32_t* d_sorted,
+                          int32_t* d_slot, int32_t* d_counts, void* stream) {
+    return shard_bucket_impl(d_nodes, n, nullptr, num_nodes, world, d_sorted, d_slot, d_counts, stream);
+}
+
+gs_status gs_shard_bucket_counted(const int32_t* d_nodes, const int32_t* d_n, int32_t n_bound, int64_t num_nodes,
+                                  int32_t world, int32_t* d_sorted, int32_t* d_slot, int32_t* d_counts, void* stream) {
+    if (!d_n) return fail(GS_ERR_ARG, "d_n is NULL");
+    return shard_bucket_impl(d_nodes, n_bound, d_n, num_nodes, world, d_sorted, d_slot, d_counts, stream);
 }
 
 gs_status gs_shard_workspace_bytes(const gs_graph* g, int32_t fanout, int32_t max_nodes, size_t* bytes) {

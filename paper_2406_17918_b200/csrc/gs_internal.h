@@ -316,7 +316,7 @@ cudaError_t launch_validate_graph(const GraphView& g, int64_t num_edges, int64_t
 cudaError_t launch_count_dense(const GraphView& g, int32_t theta, int64_t* h_count, cudaStream_t s);
 cudaError_t launch_read_rows(const int32_t* slots, const int32_t* row_index, int32_t pitch, int32_t W,
                              const int32_t* nodes, int32_t n, int32_t* out, cudaStream_t s);
-cudaError_t launch_shard_bucket(const int32_t* nodes, int32_t n, int32_t rows_per_shard, int32_t world, int32_t* sorted,
+cudaError_t launch_shard_bucket(const int32_t* nodes, int32_t n, const int32_t* d_n, int32_t rows_per_shard, int32_t world, int32_t* sorted,
                                 int32_t* slot, int32_t* counts_and_scratch, int32_t* status, cudaStream_t s);
 cudaError_t launch_export_picks(const int32_t* blk_indptr, const int32_t* picked, int32_t n, int32_t f, int32_t* out,
                                 cudaStream_t s);

@@ -17,9 +17,11 @@ constexpr int SHARD_MAX_WORLD = 64;
 
 // Pass 1: how many of the n nodes belong to each owner (block-local histogram, one global atomic
 // per owner and block).
-__global__ void __launch_bounds__(SHARD_THREADS) k_bucket_count(const int32_t* __restrict__ nodes, int n, int rows_per_shard,
+__global__ void __launch_bounds__(SHARD_THREADS) k_bucket_count(const int32_t* __restrict__ nodes, int n, const int32_t* __restrict__ d_n,
+                                                                int rows_per_shard,
                                                                 int world, int32_t* __restrict__ counts, int32_t* status) {
     __shared__ int hist[SHARD_MAX_WORLD];
+    if (d_n) n = min(n, max(0, __ldcg(d_n)));   // the list's length may live on the device; n is its bound then
     if (threadIdx.x < SHARD_MAX_WORLD) hist[threadIdx.x] = 0;
     __syncthreads();
     const int i = blockIdx.x * SHARD_THREADS + threadIdx.x;
@@ -35,12 +37,14 @@ __global__ void __launch_bounds__(SHARD_THREADS) k_bucket_count(const int32_t* _
 
 // Pass 2: place every node in its owner's segment of `sorted` and remember where it went.  The
 // order inside a segment is whatever the atomics give; `slot` is what ties a reply to its node.
-__global__ void __launch_bounds__(SHARD_THREADS) k_bucket_place(const int32_t* __restrict__ nodes, int n, int rows_per_shard,
+__global__ void __launch_bounds__(SHARD_THREADS) k_bucket_place(const int32_t* __restrict__ nodes, int n, const int32_t* __restrict__ d_n,
+                                                                int rows_per_shard,
                                                                 int world, const int32_t* __restrict__ counts,
                                                                 int32_t* __restrict__ cursor, int32_t* __restrict__ sorted,
                                                                 int32_t* __restrict__ slot) {
     __shared__ int hist[SHARD_MAX_WORLD];
     __shared__ int base[SHARD_MAX_WORLD];
+    if (d_n) n = min(n, max(0, __ldcg(d_n)));
     if (threadIdx.x < SHARD_MAX_WORLD) hist[threadIdx.x] = 0;
     __syncthreads();
     const int i = blockIdx.x * SHARD_THREADS + threadIdx.x;
@@ -66,13 +70,13 @@ __global__ void __launch_bounds__(SHARD_THREADS) k_bucket_place(const int32_t* _
     }
 }
 
-cudaError_t launch_shard_bucket(const int32_t* nodes, int32_t n, int32_t rows_per_shard, int32_t world, int32_t* sorted,
+cudaError_t launch_shard_bucket(const int32_t* nodes, int32_t n, const int32_t* d_n, int32_t rows_per_shard, int32_t world, int32_t* sorted,
                                 int32_t* slot, int32_t* counts_and_scratch, int32_t* status, cudaStream_t s) {
     cudaError_t e = cudaMemsetAsync(counts_and_scratch, 0, (size_t)(2 * world + 1) * sizeof(int32_t), s);
     if (e != cudaSuccess || n <= 0) return e;
     const int blocks = (n + SHARD_THREADS - 1) / SHARD_THREADS;
-    k_bucket_count<<<blocks, SHARD_THREADS, 0, s>>>(nodes, n, rows_per_shard, world, counts_and_scratch, status);
-    k_bucket_place<<<blocks, SHARD_THREADS, 0, s>>>(nodes, n, rows_per_shard, world, counts_and_scratch,
+    k_bucket_count<<<blocks, SHARD_THREADS, 0, s>>>(nodes, n, d_n, rows_per_shard, world, counts_and_scratch, status);
+    k_bucket_place<<<blocks, SHARD_THREADS, 0, s>>>(nodes, n, d_n, rows_per_shard, world, counts_and_scratch,
                                                     counts_and_scratch + world, sorted, slot);
     count_launches(2);
     return cudaGetLastError();

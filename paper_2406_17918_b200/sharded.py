@@ -69,44 +69,72 @@ class ShardRank:
         self.n = []
 
     # ---- requester side
+    # The host learns the size of a frontier only from the group sizes it has to read back for the exchange
+    # anyway (one host sync per hop): the bucket kernel takes the frontier's length from the device, the
+    # batch's counts and device status are read once, at the end of the batch.
     def begin(self, seeds):
         self.seeds = seeds
         self.frontier, self.n = seeds, [seeds.numel()]
+        self.count_dev = None                      # device scalar with the current frontier's length
         self.blocks = [None] * self.L
+        self.m = [0] * self.L
 
-    def requests(self, nodes):
-        """Bucket `nodes` by owner -> (ids grouped by owner, group sizes as a list); remembers the slots."""
-        sorted_ids, self.slot, counts = self.ops.gs_shard_bucket(nodes, self.num_nodes, self.world)
+    def requests(self, nodes, count=None):
+        """Bucket `nodes` (all of it, or its first *count ids) by owner -> (ids grouped by owner, group sizes
+        as a list); remembers the slots."""
+        if count is None:
+            sorted_ids, self.slot, counts = self.ops.gs_shard_bucket(nodes, self.num_nodes, self.world)
+        else:
+            sorted_ids, self.slot, counts = self.ops.gs_shard_bucket(nodes, self.num_nodes, self.world, count=count)
         c = counts.cpu().tolist()                      # the all-to-all needs the sizes on the host
         if c[2 * self.world] != 0:
             raise ValueError("a node id is outside [0, num_nodes)")
-        return sorted_ids, c[: self.world]
+        total = sum(c[: self.world])
+        return sorted_ids[:total], c[: self.world]
+
+    def _frontier_bound(self, k):
+        """Upper bound of n_k from the last size the host knows."""
+        if k == 0:
+            return self.n[0]
+        layer_before = self.L - k              # fan-out of sampling step k - 1
+        return min(self.num_nodes, self.n[k - 1] * (1 + self.fanouts[layer_before]))
 
     def hop_requests(self, k):
-        return self.requests(self.frontier[: self.n[k]])
+        bound = self._frontier_bound(k)
+        ids, counts = self.requests(self.frontier[:bound], self.count_dev)
+        if k > 0:
+            self.n.append(sum(counts))             # n_k
+        return ids, counts
 
     def hop_finish(self, k, reply):
         """`reply`: [n_k, f] rows of picks in the order the requests were sent."""
         block, frontier = self.ops.gs_shard_extend(self.cache, k, self.seeds if k == 0 else None, reply, self.slot, self.ws)
-        n, m = self.ops.gs_batch_counts(self.cache)   # n_{k+1} sizes the next hop's exchange
         self.blocks[self.L - 1 - k] = block
-        self.frontier, self.n, self.m = frontier, n[: k + 2], m
-        return n[k + 1]
+        self.frontier = frontier
+        self.count_dev = block.counts_device()[1]  # n_{k+1}, on the device
 
     def feature_requests(self):
-        return self.requests(self.frontier[: self.n[self.L]])
+        ids, counts = self.requests(self.frontier[: self._frontier_bound(self.L)], self.count_dev)
+        self.n.append(sum(counts))                 # n_L
+        return ids, counts
+
+    def finish_batch(self):
+        """Counts and device status of the batch, read once (synchronises)."""
+        n, m = self.ops.gs_batch_counts(self.cache)
+        self.n, self.m = list(n), list(m)
+        self.ops.gs_shard_status(self.cache)       # the lists this rank served
 
     def feature_pull(self, shard_bases):
         """The feature step as one kernel: every input node's row is read straight from its owner's
         memory (`shard_bases[o]`: device address of rank o's feature rows, peer-mapped where o is another GPU)."""
-        n = self.n[self.L]
-        out = torch.empty((n, self.features.shape[1]), dtype=self.features.dtype, device=self.features.device)
+        bound = self._frontier_bound(self.L)
+        out = torch.empty((bound, self.features.shape[1]), dtype=self.features.dtype, device=self.features.device)
         return self.ops.gs_gather_rows_peer(shard_bases, self.num_nodes, self.features.dtype, self.features.shape[1],
-                                            self.features.stride(0), self.frontier[:n], out)
+                                            self.features.stride(0), self.frontier[:bound], out, count=self.count_dev)
 
     def feature_finish(self, rows):
         out = torch.empty((self.n[self.L], rows.shape[1]), dtype=rows.dtype, device=rows.device)
-        return self.ops.gs_gather_rows(rows, self.slot, out)
+        return self.ops.gs_gather_rows(rows, self.slot[: self.n[self.L]], out)
 
     # ---- owner side
     def hop_serve(self, layer, lists, mode, rate, step):
@@ -116,8 +144,7 @@ class ShardRank:
             if nodes.numel() > self.max_requests:
                 raise ValueError("a request list of %d nodes exceeds max_requests %d" % (nodes.numel(), self.max_requests))
             out.append(self.ops.gs_shard_sample_rows(self.cache, nodes.contiguous(), layer, mode, rate, step, self.ws_owner))
-        self.ops.gs_shard_status(self.cache)
-        return out
+        return out                                 # device-detected problems are read once, in finish_batch
 
     def feature_serve(self, lists):
         out = []
@@ -158,6 +185,9 @@ def sample_batch_local(ranks, seeds_per_rank, mode, rate, step, features=True):
     elif features:
         rows = round_trip([r.feature_requests() for r in ranks], lambda owner, lists: owner.feature_serve(lists))
         feats = [r.feature_finish(x.contiguous()) for r, x in zip(ranks, rows)]
+    for r in ranks:
+        r.finish_batch()
+    feats = [f if f is None else f[: r.n[L]] for r, f in zip(ranks, feats)]
     return [(r.blocks, r.frontier, r.n, r.m, f) for r, f in zip(ranks, feats)]
 
 
@@ -193,48 +223,64 @@ def sample_batch(rank_state: ShardRank, seeds, mode, rate, step, features=True, 
     all-to-all round trip.
 
     Failures are collective: a rank that cannot build its requests or serve a list still takes part in
-    both exchanges of the hop (with no requests / placeholder rows), an error word is reduced over the
-    group after the reply exchange, and then every rank raises :class:`ShardedBatchError` - no rank is
+    every exchange of the batch (with no requests / placeholder rows), an error word is reduced over the
+    group after the last exchange, and then every rank raises :class:`ShardedBatchError` - no rank is
     left waiting inside a collective for one that has gone."""
     me = rank_state
     L = me.L
     me.begin(seeds)
     dev = seeds.device
+    state = {"err": 0, "msg": ""}
+
+    def fail(code, e):
+        if not state["err"]:
+            state["err"], state["msg"] = code, str(e)
 
     def round_trip(make_requests, serve, width, dtype):
-        err, msg = 0, ""
-        try:
-            ids, counts = make_requests()
-        except (ValueError, RuntimeError) as e:
-            err, msg = 1, str(e)
-            ids, counts = torch.empty(0, dtype=torch.int32, device=dev), [0] * me.world
+        ids, counts = torch.empty(0, dtype=torch.int32, device=dev), [0] * me.world
+        if state["err"] != 1:                      # a rank whose own batch is broken asks for nothing more
+            try:
+                ids, counts = make_requests()
+            except (ValueError, RuntimeError) as e:
+                fail(1, e)
+                ids, counts = torch.empty(0, dtype=torch.int32, device=dev), [0] * me.world
         recv, recv_counts = _all_to_all_v(ids, counts, (), group)
         back = None
         try:
             served = serve(_split(recv, recv_counts))
             back = torch.cat(served) if served else torch.empty((0,) + width, dtype=dtype, device=dev)
         except (ValueError, RuntimeError) as e:
-            err, msg = 2, str(e)
+            fail(2, e)
         if back is None or back.shape[0] != sum(recv_counts):
             back = torch.zeros((sum(recv_counts),) + width, dtype=dtype, device=dev)   # placeholder rows keep the exchange whole
         reply = torch.empty((ids.numel(),) + width, dtype=dtype, device=dev)
         dist.all_to_all_single(reply, back.contiguous(), counts, recv_counts, group=group)
-        word = torch.tensor([err], dtype=torch.int32, device=dev)
-        dist.all_reduce(word, op=dist.ReduceOp.MAX, group=group)
-        code = int(word.item())
-        if code:
-            raise ShardedBatchError(code, msg)
         return reply
 
     for k in range(L):
         layer = L - 1 - k
         reply = round_trip(lambda: me.hop_requests(k), lambda lists: me.hop_serve(layer, lists, mode, rate, step),
                            (me.fanouts[layer],), torch.int32)
-        me.hop_finish(k, reply)
+        if state["err"] != 1:
+            me.hop_finish(k, reply)
     feats = None
     if features and feature_bases is not None:
-        feats = me.feature_pull(feature_bases)
+        if state["err"] != 1:
+            feats = me.feature_pull(feature_bases)
     elif features:
         rows = round_trip(me.feature_requests, me.feature_serve, (me.features.shape[1],), me.features.dtype)
-        feats = me.feature_finish(rows)
+        if state["err"] != 1:
+            feats = me.feature_finish(rows)
+    if state["err"] != 1:
+        try:
+            me.finish_batch()
+        except (ValueError, RuntimeError) as e:
+            fail(2, e)
+    word = torch.tensor([state["err"]], dtype=torch.int32, device=dev)
+    dist.all_reduce(word, op=dist.ReduceOp.MAX, group=group)
+    code = int(word.item())
+    if code:
+        raise ShardedBatchError(code, state["msg"])
+    if feats is not None:
+        feats = feats[: me.n[L]]
     return me.blocks, me.frontier, me.n, me.m, feats

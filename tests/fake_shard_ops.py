@@ -17,8 +17,12 @@ class _Graph:
 
 
 class _Block:
-    def __init__(self, indptr, indices):
+    def __init__(self, indptr, indices, num_src=0):
         self._indptr, self._indices = indptr, indices
+        self._counts = (len(indptr) - 1, num_src, len(indices))
+
+    def counts_device(self):
+        return tuple(torch.tensor(c, dtype=torch.int32) for c in self._counts)
 
     def indptr(self, n):
         return torch.from_numpy(self._indptr[: n + 1])
@@ -51,16 +55,18 @@ def gs_shard_workspace_bytes(graph, fanout, max_nodes):
     return 256
 
 
-def gs_shard_bucket(nodes, num_nodes, world):
-    v = nodes.numpy()
+def gs_shard_bucket(nodes, num_nodes, world, count=None):
+    v = nodes.numpy() if count is None else nodes.numpy()[: int(count)]
     S = (num_nodes + world - 1) // world
     owner = v // S
     order = np.argsort(owner, kind="stable")
-    slot = np.empty(len(v), dtype=np.int32)
+    slot = np.zeros(nodes.numel(), dtype=np.int32)
     slot[order] = np.arange(len(v), dtype=np.int32)
     counts = np.zeros(2 * world + 1, dtype=np.int32)
     counts[:world] = np.bincount(owner, minlength=world)
-    return torch.from_numpy(v[order].copy()), torch.from_numpy(slot), torch.from_numpy(counts)
+    sorted_ids = np.zeros(nodes.numel(), dtype=np.int32)
+    sorted_ids[: len(v)] = v[order]
+    return torch.from_numpy(sorted_ids), torch.from_numpy(slot), torch.from_numpy(counts)
 
 
 def gs_shard_sample_rows(cache, nodes, layer, mode, rate, step, ws):
@@ -103,7 +109,7 @@ def gs_shard_extend(cache, k, seeds, reply, slot, ws):
         indptr.append(len(local))
     cache.n.append(len(cache.frontier))
     cache.m[L - 1 - k] = len(local)
-    return _Block(np.array(indptr, dtype=np.int32), np.array(local, dtype=np.int32)), \
+    return _Block(np.array(indptr, dtype=np.int32), np.array(local, dtype=np.int32), len(cache.frontier)), \
         torch.tensor(cache.frontier, dtype=torch.int32)
 
 
