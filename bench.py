@@ -265,6 +265,10 @@ def main():
                     help="node-sharded run: rank o owns the CSR, cache and feature rows of an id range, one "
                          "all-to-all round trip per hop (needs --theta; default 32); at 1 GPU it measures the "
                          "protocol's overhead, the exchange being a local copy")
+    ap.add_argument("--feature-exchange", default=None, choices=["peer", "roundtrip"],
+                    help="with --sharded: how feature rows reach the requester (default: peer with one rank, roundtrip otherwise)")
+    ap.add_argument("--exact-sizes", action="store_true",
+                    help="with --sharded: keep the exact-size exchanges (host reads the group sizes) for the timed batches")
     ap.add_argument("--no-overlap", action="store_true",
                     help="skip the second, pipelined leg (gather of a batch on a second stream, overlapping the "
                          "first, latency-bound hops of the next batch)")
@@ -738,14 +742,41 @@ def sharded_arm(args, cfg, mode, gamma, rank, local_rank, world, device):
     gm = {"otf": gs.GS_MODE_OTF, "fcr": gs.GS_MODE_FCR, "fbl": gs.GS_MODE_FBL, "fetch": gs.GS_MODE_OTF_FETCH}[mode]
     K, Wm = args.steps, args.warmup
 
+    # The feature step: a round trip like a hop (ids out, rows back, reordered), or one kernel that loads every
+    # row straight from its owner's memory.  The latter needs the peers' feature shards mapped into this
+    # process; with one rank the only "peer" is this GPU.
+    feat = args.feature_exchange or ("peer" if world == 1 else "roundtrip")
+    if feat == "peer" and world > 1:
+        raise SystemExit("--feature-exchange peer needs the peers' feature shards mapped into every process: not set up by this script")
+
     def one(step):
         seeds = batch_seeds(perm, step, B, rank, world)
         if world > 1:
             return sharded.sample_batch(me, seeds, gm, gamma, step)
-        return sharded.sample_batch_local([me], [seeds], gm, gamma, step)[0]
+        return sharded.sample_batch_local([me], [seeds], gm, gamma, step, features="peer" if feat == "peer" else True)[0]
 
+    # Warm-up with exact-size exchanges (the host reads the group sizes of every exchange): the largest group
+    # seen sizes the segments of the fixed-capacity exchanges the timed batches use (+25 %, the same on every rank).
+    seen = [0] * (L + 1)
     for t in range(1, Wm + 1):
         one(t)
+        seen = [max(a, b) for a, b in zip(seen, me.seen)]
+    exact_ms = None
+    if not args.exact_sizes:
+        torch.cuda.synchronize()
+        x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        x0.record()
+        for t in range(Wm + 1, Wm + 1 + max(3, K // 4)):
+            one(t)
+            seen = [max(a, b) for a, b in zip(seen, me.seen)]
+        x1.record()
+        torch.cuda.synchronize()
+        exact_ms = replicas.aggregate(x0.elapsed_time(x1) / max(3, K // 4), [0], device)[0]
+        _, seen = replicas.aggregate(0.0, seen, device, reduce="max")
+        caps = [(int(c * 1.25) + 255) // 256 * 256 for c in seen]
+        me.set_capacities(caps)
+        for t in range(1, 4):
+            one(Wm + K + t)
     clocks = ClockSampler(local_rank) if rank == 0 else None
     time.sleep(0.3)
     replicas.barrier()
@@ -755,7 +786,7 @@ def sharded_arm(args, cfg, mode, gamma, rank, local_rank, world, device):
     wall0 = time.time()
     edges = rows = 0
     e0.record()
-    for t in range(Wm + 1, Wm + K + 1):
+    for t in range(2 * Wm + K + 4, 2 * Wm + 2 * K + 4):
         blocks, frontier, n, m, feats = one(t)
         edges += sum(m)
         rows += n[L]
@@ -780,6 +811,11 @@ def sharded_arm(args, cfg, mode, gamma, rank, local_rank, world, device):
                        "shared_cache": cfg["shared"], "feat_dim": cfg["feat_dim"],
                        "parallelism": "node-sharded x%d (one all-to-all round trip per hop%s)"
                                       % (world, "" if world > 1 else "; 1 rank: local copy"),
+                       "exchange": "exact sizes (one host read per exchange)" if me.caps is None else
+                                   "fixed capacity per pair of ranks %s, no host read inside a batch" % me.caps,
+                       "ms_per_step_exact_sizes": exact_ms,
+                       "feature_step": "one kernel of loads from the owners' memory" if feat == "peer" else
+                                       "all-to-all round trip (ids out, rows back, reorder)",
                        "l2": "inputs_larger_than_L2", "cache_bytes_per_rank": me.cache.storage.numel()},
             "roofline": None, "e2e": None, "gpu_launches": launches,
             "clocks": clocks.summary(wall0, wall1) if clocks else None}))

@@ -313,9 +313,20 @@ gs_status gs_shard_bucket(const int32_t* d_nodes, int32_t n, int64_t num_nodes, 
                           int32_t* d_slot, int32_t* d_counts, void* stream);
 /* The same for a list whose length is a device scalar (the frontier of the previous hop: *d_n, e.g.
  * gs_block.d_num_src), of at most n_bound ids: the requester needs no host copy of the frontier's size
- * before it buckets; the group sizes it reads back for the exchange add up to the length. */
+ * before it buckets; the group sizes it reads back for the exchange add up to the length.  *d_n > n_bound
+ * sets word 2*world to GS_ERR_WORKSPACE (only the first n_bound ids are grouped). */
 gs_status gs_shard_bucket_counted(const int32_t* d_nodes, const int32_t* d_n, int32_t n_bound, int64_t num_nodes,
                                   int32_t world, int32_t* d_sorted, int32_t* d_slot, int32_t* d_counts, void* stream);
+
+/* The same with every owner's group at a fixed pitch: owner o's ids are d_sorted[o*capacity ..
+ * o*capacity + counts[o]) (d_sorted holds world*capacity ids, the rest of a segment is left as it is), so the
+ * groups can be exchanged in equal splits without the host ever reading a size; the counts travel as a
+ * device array beside them.  d_n_or_null as for gs_shard_bucket_counted (NULL: all n_bound ids).  A group
+ * larger than `capacity` sets word 2*world to GS_ERR_WORKSPACE; its surplus nodes get slot -1 and are dropped
+ * (gs_shard_extend_fixed then reports them too). */
+gs_status gs_shard_bucket_fixed(const int32_t* d_nodes, const int32_t* d_n_or_null, int32_t n_bound, int64_t num_nodes,
+                                int32_t world, int32_t capacity, int32_t* d_sorted, int32_t* d_slot, int32_t* d_counts,
+                                void* stream);
 
 /* Owner side.  For n distinct nodes of this shard: refresh (per mode / rate, exactly as
  * gs_sample_batch does for a frontier at `layer`) and pick; d_picks[n][fanout(layer)] receives the
@@ -323,10 +334,16 @@ gs_status gs_shard_bucket_counted(const int32_t* d_nodes, const int32_t* d_n, in
  * its own (a second header) and does not touch the relabel table, so it may run between the hops
  * of this rank's own batch.  Lists of different requesters go in separate calls (a node may
  * appear in several of them).  Workspace: gs_shard_workspace_bytes(graph, fanout(layer), n).
- * gs_shard_status synchronises `stream` and reports a bad node id met by the last call. */
+ * gs_shard_sample_rows_counted takes the list's length from the device (*d_n, at most n_bound; e.g. a word of
+ * the exchanged counts of gs_shard_bucket_fixed) and writes only that many rows of d_picks[n_bound][fanout].
+ * gs_shard_status synchronises `stream`, reports a bad node id met by any list served since its last call
+ * (after such an id the later lists are not served) and clears that state. */
 gs_status gs_shard_workspace_bytes(const gs_graph*, int32_t fanout, int32_t max_nodes, size_t* bytes);
 gs_status gs_shard_sample_rows(gs_cache*, const int32_t* d_nodes, int32_t n, int32_t layer, gs_mode mode, double rate,
                                uint32_t step, void* d_workspace, size_t workspace_bytes, void* stream, int32_t* d_picks);
+gs_status gs_shard_sample_rows_counted(gs_cache*, const int32_t* d_nodes, const int32_t* d_n, int32_t n_bound, int32_t layer,
+                                       gs_mode mode, double rate, uint32_t step, void* d_workspace, size_t workspace_bytes,
+                                       void* stream, int32_t* d_picks);
 gs_status gs_shard_status(gs_cache*, void* stream);
 
 /* Requester side, hop k = 0 .. num_hops-1 in order.  d_reply[n_k][fanout(L-1-k)]: the owners' rows
@@ -340,6 +357,12 @@ gs_status gs_shard_status(gs_cache*, void* stream);
 gs_status gs_shard_extend(gs_cache*, int32_t k, const int32_t* d_seeds, int32_t num_seeds, const int32_t* d_reply,
                           const int32_t* d_slot, void* d_workspace, size_t workspace_bytes, void* stream, gs_block* block,
                           const int32_t** d_frontier);
+/* The same for replies at a fixed pitch (gs_shard_bucket_fixed): d_reply[reply_rows][fanout] with
+ * reply_rows = world * capacity, d_slot the positions that call returned (required).  A slot outside
+ * [0, reply_rows) sets GS_ERR_RANGE. */
+gs_status gs_shard_extend_fixed(gs_cache*, int32_t k, const int32_t* d_seeds, int32_t num_seeds, const int32_t* d_reply,
+                                int32_t reply_rows, const int32_t* d_slot, void* d_workspace, size_t workspace_bytes,
+                                void* stream, gs_block* block, const int32_t** d_frontier);
 
 /* Copy n logical cache rows (cache_width slots each, -1 = empty) of `layer` into d_out[n][cache_width]. */
 gs_status gs_cache_read_rows(const gs_cache*, int32_t layer, const int32_t* d_nodes, int32_t n,

@@ -91,9 +91,12 @@ def _load():
         "gs_shard_bucket": [vp, i32, i64, i32, vp, vp, vp, vp],
         "gs_shard_bucket_counted": [vp, vp, i32, i64, i32, vp, vp, vp, vp],
         "gs_shard_workspace_bytes": [vp, i32, i32, psz],
+        "gs_shard_bucket_fixed": [vp, vp, i32, i64, i32, i32, vp, vp, vp, vp],
         "gs_shard_sample_rows": [vp, vp, i32, i32, ctypes.c_int, dbl, u32, vp, sz, vp, vp],
+        "gs_shard_sample_rows_counted": [vp, vp, vp, i32, i32, ctypes.c_int, dbl, u32, vp, sz, vp, vp],
         "gs_shard_status": [vp, vp],
         "gs_shard_extend": [vp, i32, vp, i32, vp, vp, vp, sz, vp, vp, pvp],
+        "gs_shard_extend_fixed": [vp, i32, vp, i32, vp, i32, vp, vp, sz, vp, vp, pvp],
         "gs_batch_stats": [vp, vp, vp],
         "gs_cache_profile_begin": [vp, i32],
         "gs_cache_profile_end": [vp, vp, vp, vp],
@@ -429,15 +432,29 @@ def gs_gather_rows_peer(shard_bases, num_rows: int, dtype: torch.dtype, row_elem
     return out
 
 
-def gs_shard_bucket(nodes: torch.Tensor, num_nodes: int, world: int, stream=None, count=None):
+def gs_shard_bucket(nodes: torch.Tensor, num_nodes: int, world: int, stream=None, count=None, capacity=None, out=None):
     """Group node ids by owner.  Returns (sorted ids, slot of every input id, int32[2*world+1] device counts).
-    `count`: a 0-d int32 CUDA tensor with the list's length when only the device knows it (`nodes` is then the bound)."""
+    `count`: a 0-d int32 CUDA tensor with the list's length when only the device knows it (`nodes` is then the bound).
+    `capacity`: every owner's group gets a segment of that many ids (sorted ids: world*capacity entries) instead of
+    the groups being packed.  `out`: (sorted, slot, counts) tensors to write into instead of new ones."""
     if nodes.dtype != torch.int32 or not nodes.is_cuda or not nodes.is_contiguous():
         raise TypeError("nodes must be a contiguous int32 CUDA tensor")
-    sorted_ids = torch.empty_like(nodes)
-    slot = torch.empty_like(nodes)
-    counts = torch.empty(2 * world + 1, dtype=torch.int32, device=nodes.device)
-    if count is None:
+    if out is not None:
+        sorted_ids, slot, counts = out
+        need = nodes.numel() if capacity is None else world * int(capacity)
+        if sorted_ids.numel() < need or slot.numel() < nodes.numel() or counts.numel() < 2 * world + 1:
+            raise ValueError("an output tensor is too small")
+        for t in out:
+            if t.dtype != torch.int32 or not t.is_cuda or not t.is_contiguous():
+                raise TypeError("outputs must be contiguous int32 CUDA tensors")
+    else:
+        sorted_ids = torch.empty_like(nodes) if capacity is None else torch.empty(world * int(capacity), dtype=torch.int32, device=nodes.device)
+        slot = torch.empty_like(nodes)
+        counts = torch.empty(2 * world + 1, dtype=torch.int32, device=nodes.device)
+    if capacity is not None:
+        _check(_L.gs_shard_bucket_fixed(_ptr(nodes), _ptr(count), nodes.numel(), int(num_nodes), int(world), int(capacity),
+                                        _ptr(sorted_ids), _ptr(slot), _ptr(counts), _stream(stream)))
+    elif count is None:
         _check(_L.gs_shard_bucket(_ptr(nodes), nodes.numel(), int(num_nodes), int(world), _ptr(sorted_ids), _ptr(slot),
                                   _ptr(counts), _stream(stream)))
     else:
@@ -453,15 +470,24 @@ def gs_shard_workspace_bytes(graph: Graph, fanout: int, max_nodes: int) -> int:
 
 
 def gs_shard_sample_rows(cache: Cache, nodes: torch.Tensor, layer: int, mode: int, rate: float, step: int,
-                         workspace: torch.Tensor, picks: torch.Tensor = None, stream=None) -> torch.Tensor:
-    """Owner side of one hop: picks[n, fanout(layer)] (-1 padded) for n distinct nodes of this shard."""
+                         workspace: torch.Tensor, picks: torch.Tensor = None, stream=None, count=None) -> torch.Tensor:
+    """Owner side of one hop: picks[n, fanout(layer)] (-1 padded) for n distinct nodes of this shard.
+    `count`: a 0-d / 1-element int32 CUDA tensor with the list's length (`nodes` is then the bound; only that
+    many rows of `picks` are written)."""
     if nodes.dtype != torch.int32 or not nodes.is_cuda or not nodes.is_contiguous():
         raise TypeError("nodes must be a contiguous int32 CUDA tensor")
     f = cache.fanouts[layer] if 0 <= layer < cache.num_hops else 1     # a bad layer is reported by the library
     if picks is None:
         picks = torch.empty((nodes.numel(), f), dtype=torch.int32, device=nodes.device)
-    _check(_L.gs_shard_sample_rows(cache.handle, _ptr(nodes), nodes.numel(), int(layer), mode, float(rate), step,
-                                   _ptr(workspace), workspace.numel(), _stream(stream), _ptr(picks)))
+    elif picks.dtype != torch.int32 or not picks.is_contiguous() or picks.numel() < nodes.numel() * f:
+        raise TypeError("picks must be a contiguous int32 tensor of at least [len(nodes), fanout]")
+    if count is None:
+        _check(_L.gs_shard_sample_rows(cache.handle, _ptr(nodes), nodes.numel(), int(layer), mode, float(rate), step,
+                                       _ptr(workspace), workspace.numel(), _stream(stream), _ptr(picks)))
+    else:
+        _check(_L.gs_shard_sample_rows_counted(cache.handle, _ptr(nodes), _ptr(count), nodes.numel(), int(layer), mode,
+                                               float(rate), step, _ptr(workspace), workspace.numel(), _stream(stream),
+                                               _ptr(picks)))
     return picks
 
 
@@ -470,13 +496,21 @@ def gs_shard_status(cache: Cache, stream=None):
 
 
 def gs_shard_extend(cache: Cache, k: int, seeds, reply: torch.Tensor, slot: torch.Tensor, workspace: torch.Tensor,
-                    stream=None):
-    """Requester side of hop k.  Returns (block of layer L-1-k, frontier array aliasing the workspace)."""
+                    stream=None, reply_rows=None):
+    """Requester side of hop k.  Returns (block of layer L-1-k, frontier array aliasing the workspace).
+    `reply_rows`: rows of a fixed-pitch reply (world * capacity, see gs_shard_bucket)."""
     cb = _CBlock()
     d_fr = ctypes.c_void_p()
-    _check(_L.gs_shard_extend(cache.handle, int(k), _ptr(seeds), 0 if seeds is None else seeds.numel(), _ptr(reply),
-                              _ptr(slot), _ptr(workspace), workspace.numel(), _stream(stream), ctypes.byref(cb),
-                              ctypes.byref(d_fr)))
+    if reply_rows is None:
+        _check(_L.gs_shard_extend(cache.handle, int(k), _ptr(seeds), 0 if seeds is None else seeds.numel(), _ptr(reply),
+                                  _ptr(slot), _ptr(workspace), workspace.numel(), _stream(stream), ctypes.byref(cb),
+                                  ctypes.byref(d_fr)))
+    else:
+        if 0 <= k < cache.num_hops and reply.numel() < int(reply_rows) * cache.fanouts[cache.num_hops - 1 - k]:
+            raise ValueError("reply holds fewer than reply_rows rows")
+        _check(_L.gs_shard_extend_fixed(cache.handle, int(k), _ptr(seeds), 0 if seeds is None else seeds.numel(), _ptr(reply),
+                                        int(reply_rows), _ptr(slot), _ptr(workspace), workspace.numel(), _stream(stream),
+                                        ctypes.byref(cb), ctypes.byref(d_fr)))
     block = Block(cb, workspace, cache.storage)
     off = d_fr.value - workspace.data_ptr()
     return block, workspace[off:off + 4 * block.max_src].view(torch.int32)

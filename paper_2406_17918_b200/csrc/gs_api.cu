@@ -486,6 +486,7 @@ static uint32_t next_stamp(gs_cache* c, cudaStream_t s) {
 struct HopArgs {
     int32_t layer;
     int32_t* d_picks;   // [n][f], -1 padded
+    const int32_t* d_n; // length of the list on the device (num_seeds is its bound then), or NULL
 };
 
 static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_seeds, gs_mode mode, double gamma,
@@ -531,7 +532,10 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         stamp = next_stamp(c, s);
         if (!stamp) return cuda_fail(cudaGetLastError(), "cudaMemsetAsync");
     }
-    GS_CUDA(cudaMemsetAsync(hdr, 0, HDR_ONE, s));
+    // the owner-side status word outlives the call: gs_shard_status reports (and clears) what any list
+    // served since its last call has met
+    if (hop) GS_CUDA(cudaMemsetAsync(hdr + HDR_STATUS + 1, 0, HDR_ONE - sizeof(int32_t), s));
+    else GS_CUDA(cudaMemsetAsync(hdr, 0, HDR_ONE, s));
 
     const bool prof = !hop && c->prof_events && c->prof_used < c->prof_cap;
     for (int k = 0; k < L; ++k) {
@@ -554,6 +558,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         C.k = k;
         C.f = c->fanouts[layer];
         C.n_host = num_seeds;
+        C.d_n0 = hop ? hop->d_n : nullptr;
         C.blk_indptr = blk_indptr;
         C.tile_sums = tiles_a;
         C.table = c->d_table;
@@ -638,7 +643,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         GS_CUDA(launch_finish(P, b.nb[k], s));
         if (ev) GS_CUDA(cudaEventRecord(ev[3], s));
         if (hop) {
-            GS_CUDA(launch_export_picks(blk_indptr, picked, num_seeds, c->fanouts[layer], hop->d_picks, s));
+            GS_CUDA(launch_export_picks(blk_indptr, picked, num_seeds, hdr + HDR_N, c->fanouts[layer], hop->d_picks, s));
             break;
         }
 
@@ -749,34 +754,43 @@ gs_status gs_cache_refresh_all(gs_cache* c, gs_mode mode, double gamma, uint32_t
 /* ---------------------------------------------------------------- node-sharded sampling */
 
 static gs_status shard_bucket_impl(const int32_t* d_nodes, int32_t n, const int32_t* d_n, int64_t num_nodes, int32_t world,
-                                   int32_t* d_sorted, int32_t* d_slot, int32_t* d_counts, void* stream) {
+                                   int32_t capacity, int32_t* d_sorted, int32_t* d_slot, int32_t* d_counts, void* stream) {
     if (world < 1 || world > 64) return fail(GS_ERR_ARG, "world %d outside [1, 64]", world);
     if (num_nodes < 1 || num_nodes >= ((int64_t)1 << 31)) return fail(GS_ERR_ARG, "num_nodes outside [1, 2^31)");
     if (n < 0) return fail(GS_ERR_ARG, "n is negative");
+    if (capacity < 0 || (int64_t)capacity * world >= ((int64_t)1 << 31)) return fail(GS_ERR_ARG, "capacity outside [0, 2^31 / world)");
     if (!d_counts || (n > 0 && (!d_nodes || !d_sorted || !d_slot))) return fail(GS_ERR_ARG, "NULL argument");
     const int32_t rows_per_shard = (int32_t)((num_nodes + world - 1) / world);
-    GS_CUDA(launch_shard_bucket(d_nodes, n, d_n, rows_per_shard, world, d_sorted, d_slot, d_counts, d_counts + 2 * world,
-                                (cudaStream_t)stream));
+    GS_CUDA(launch_shard_bucket(d_nodes, n, d_n, rows_per_shard, world, capacity, d_sorted, d_slot, d_counts,
+                                d_counts + 2 * world, (cudaStream_t)stream));
     return GS_OK;
 }
 
 gs_status gs_shard_bucket(const int32_t* d_nodes, int32_t n, int64_t num_nodes, int32_t world, int32_t* d_sorted,
                           int32_t* d_slot, int32_t* d_counts, void* stream) {
-    return shard_bucket_impl(d_nodes, n, nullptr, num_nodes, world, d_sorted, d_slot, d_counts, stream);
+    return shard_bucket_impl(d_nodes, n, nullptr, num_nodes, world, 0, d_sorted, d_slot, d_counts, stream);
 }
 
 gs_status gs_shard_bucket_counted(const int32_t* d_nodes, const int32_t* d_n, int32_t n_bound, int64_t num_nodes,
                                   int32_t world, int32_t* d_sorted, int32_t* d_slot, int32_t* d_counts, void* stream) {
     if (!d_n) return fail(GS_ERR_ARG, "d_n is NULL");
-    return shard_bucket_impl(d_nodes, n_bound, d_n, num_nodes, world, d_sorted, d_slot, d_counts, stream);
+    return shard_bucket_impl(d_nodes, n_bound, d_n, num_nodes, world, 0, d_sorted, d_slot, d_counts, stream);
+}
+
+gs_status gs_shard_bucket_fixed(const int32_t* d_nodes, const int32_t* d_n_or_null, int32_t n_bound, int64_t num_nodes,
+                                int32_t world, int32_t capacity, int32_t* d_sorted, int32_t* d_slot, int32_t* d_counts,
+                                void* stream) {
+    if (capacity < 1) return fail(GS_ERR_ARG, "capacity must be >= 1");
+    return shard_bucket_impl(d_nodes, n_bound, d_n_or_null, num_nodes, world, capacity, d_sorted, d_slot, d_counts, stream);
 }
 
 gs_status gs_shard_workspace_bytes(const gs_graph* g, int32_t fanout, int32_t max_nodes, size_t* bytes) {
     return gs_workspace_bytes(g, 1, &fanout, max_nodes, bytes);
 }
 
-gs_status gs_shard_sample_rows(gs_cache* c, const int32_t* d_nodes, int32_t n, int32_t layer, gs_mode mode, double rate,
-                               uint32_t step, void* d_workspace, size_t workspace_bytes, void* stream, int32_t* d_picks) {
+static gs_status shard_sample_rows_impl(gs_cache* c, const int32_t* d_nodes, const int32_t* d_n, int32_t n, int32_t layer,
+                                        gs_mode mode, double rate, uint32_t step, void* d_workspace, size_t workspace_bytes,
+                                        void* stream, int32_t* d_picks) {
     if (!c) return fail(GS_ERR_ARG, "cache is NULL");
     if (layer < 0 || layer >= c->L) return fail(GS_ERR_ARG, "layer %d outside [0, %d)", layer, c->L);
     if (n == 0) return GS_OK;
@@ -785,9 +799,22 @@ gs_status gs_shard_sample_rows(gs_cache* c, const int32_t* d_nodes, int32_t n, i
     gs_status st = check_batch_args(c, d_nodes, n, mode, rate, step, d_workspace, unused);
     if (st != GS_OK) return st;
     if (!aligned(d_nodes, 4) || !aligned(d_picks, 4)) return fail(GS_ERR_ALIGN, "node and pick arrays must be 4-byte aligned");
-    HopArgs hop{layer, d_picks};
+    HopArgs hop{layer, d_picks, d_n};
     return sample_impl(c, d_nodes, n, mode, rate, step, d_workspace, workspace_bytes, (cudaStream_t)stream, unused, nullptr,
                        nullptr, nullptr, &hop);
+}
+
+gs_status gs_shard_sample_rows(gs_cache* c, const int32_t* d_nodes, int32_t n, int32_t layer, gs_mode mode, double rate,
+                               uint32_t step, void* d_workspace, size_t workspace_bytes, void* stream, int32_t* d_picks) {
+    return shard_sample_rows_impl(c, d_nodes, nullptr, n, layer, mode, rate, step, d_workspace, workspace_bytes, stream, d_picks);
+}
+
+gs_status gs_shard_sample_rows_counted(gs_cache* c, const int32_t* d_nodes, const int32_t* d_n, int32_t n_bound, int32_t layer,
+                                       gs_mode mode, double rate, uint32_t step, void* d_workspace, size_t workspace_bytes,
+                                       void* stream, int32_t* d_picks) {
+    if (!d_n) return fail(GS_ERR_ARG, "d_n is NULL");
+    if (c && n_bound > 0 && (int64_t)n_bound > c->graph->num_nodes) n_bound = (int32_t)c->graph->num_nodes;   // a list of distinct nodes
+    return shard_sample_rows_impl(c, d_nodes, d_n, n_bound, layer, mode, rate, step, d_workspace, workspace_bytes, stream, d_picks);
 }
 
 gs_status gs_shard_status(gs_cache* c, void* stream) {
@@ -796,14 +823,15 @@ gs_status gs_shard_status(gs_cache* c, void* stream) {
     GS_CUDA(cudaMemcpyAsync(c->h_pinned, c->d_hdr + HDR_OWNER + HDR_STATUS, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
     GS_CUDA(cudaStreamSynchronize(s));
     const int status = c->h_pinned[0];
+    if (status != 0) GS_CUDA(cudaMemsetAsync(c->d_hdr + HDR_OWNER + HDR_STATUS, 0, sizeof(int32_t), s));
     if (status == GS_ERR_RANGE) return fail(GS_ERR_RANGE, "a requested node id is outside [0, num_nodes)");
     if (status != 0) return fail(GS_ERR_CUDA, "unexpected device status %d", status);
     return GS_OK;
 }
 
-gs_status gs_shard_extend(gs_cache* c, int32_t k, const int32_t* d_seeds, int32_t num_seeds, const int32_t* d_reply,
-                          const int32_t* d_slot, void* d_workspace, size_t workspace_bytes, void* stream, gs_block* block,
-                          const int32_t** d_frontier) {
+static gs_status shard_extend_impl(gs_cache* c, int32_t k, const int32_t* d_seeds, int32_t num_seeds, const int32_t* d_reply,
+                                   int32_t reply_rows, const int32_t* d_slot, void* d_workspace, size_t workspace_bytes,
+                                   void* stream, gs_block* block, const int32_t** d_frontier) {
     if (!c) return fail(GS_ERR_ARG, "cache is NULL");
     if (k < 0 || k >= c->L) return fail(GS_ERR_ARG, "hop %d outside [0, %d)", k, c->L);
     if (!d_reply || !block) return fail(GS_ERR_ARG, "NULL argument");
@@ -851,10 +879,17 @@ gs_status gs_shard_extend(gs_cache* c, int32_t k, const int32_t* d_seeds, int32_
     C.cand_count = (int32_t*)(ws + w.cand_count);
     C.scan_item_cap = w.scan_item_cap;
     C.reply = d_reply;
+    C.reply_rows = reply_rows;
     C.slot = d_slot;
     GS_CUDA(launch_row_counts(C, b.nb[k], s));
-    GS_CUDA(launch_import_picks(c->d_hdr, k, (int32_t)b.nb[k], C.f, d_reply, d_slot, blk_indptr, picked, c->d_table,
-                                c->shard_stamp, g->num_nodes, c->d_hdr + HDR_STATUS, s));
+    // first occurrences are found as in gs_sample_batch: the direct table takes its claims while the picks are
+    // imported, the other methods work from the picked array afterwards
+    int32_t dedup = c->dedup;
+    if (dedup == DEDUP_AUTO)
+        dedup = (g->num_nodes * 8 > DEDUP_AUTO_TABLE_BYTES && b.nb[k] + b.mb[k] >= DEDUP_AUTO_MIN_KEYS) ? DEDUP_HASH : DEDUP_DIRECT;
+    GS_CUDA(launch_import_picks(c->d_hdr, k, (int32_t)b.nb[k], C.f, d_reply, reply_rows, d_slot, blk_indptr, picked,
+                                dedup == DEDUP_DIRECT ? c->d_table : nullptr, c->shard_stamp, g->num_nodes,
+                                c->d_hdr + HDR_STATUS, s));
     RelabelParams R{};
     R.hdr = c->d_hdr;
     R.k = k;
@@ -866,7 +901,11 @@ gs_status gs_shard_extend(gs_cache* c, int32_t k, const int32_t* d_seeds, int32_
     R.table = c->d_table;
     R.stamp = c->shard_stamp;
     R.n_cap = b.nb[k + 1];
-    R.method = DEDUP_DIRECT;
+    R.method = dedup;
+    R.scratch = (unsigned long long*)(ws + w.dedup);
+    R.scratch_entries = w.dedup_entries;
+    R.id_bits = 1;
+    while (R.id_bits < 32 && ((int64_t)1 << R.id_bits) < g->num_nodes) R.id_bits += 1;
     GS_CUDA(launch_relabel(R, b.nb[k], b.mb[k], s));
 
     gs_block& B = *block;
@@ -880,6 +919,21 @@ gs_status gs_shard_extend(gs_cache* c, int32_t k, const int32_t* d_seeds, int32_
     B.d_indices = blk_indices;
     if (d_frontier) *d_frontier = frontier;
     return GS_OK;
+}
+
+gs_status gs_shard_extend(gs_cache* c, int32_t k, const int32_t* d_seeds, int32_t num_seeds, const int32_t* d_reply,
+                          const int32_t* d_slot, void* d_workspace, size_t workspace_bytes, void* stream, gs_block* block,
+                          const int32_t** d_frontier) {
+    return shard_extend_impl(c, k, d_seeds, num_seeds, d_reply, 0, d_slot, d_workspace, workspace_bytes, stream, block, d_frontier);
+}
+
+gs_status gs_shard_extend_fixed(gs_cache* c, int32_t k, const int32_t* d_seeds, int32_t num_seeds, const int32_t* d_reply,
+                                int32_t reply_rows, const int32_t* d_slot, void* d_workspace, size_t workspace_bytes,
+                                void* stream, gs_block* block, const int32_t** d_frontier) {
+    if (reply_rows < 1) return fail(GS_ERR_ARG, "reply_rows must be >= 1");
+    if (!d_slot) return fail(GS_ERR_ARG, "d_slot is NULL");
+    return shard_extend_impl(c, k, d_seeds, num_seeds, d_reply, reply_rows, d_slot, d_workspace, workspace_bytes, stream, block,
+                             d_frontier);
 }
 
 gs_status gs_gather_rows(const void* d_src, gs_dtype dtype, int32_t row_elems, int64_t src_ld, int64_t first_row,

@@ -216,6 +216,8 @@ struct CountParams {
     int32_t no_stamp;        // owner side: step 0 neither checks duplicates nor touches the relabel table
     const int32_t* reply;    // requester side: picks by row [rows][f], -1 padded; row lengths come from here, not from degrees
     const int32_t* slot;     // requester side: row of `reply` that belongs to frontier position p
+    int32_t reply_rows;      // rows `reply` holds when its segments have a fixed pitch; 0: exactly n_k rows
+    const int32_t* d_n0;     // step 0: the list's length on the device (n_host is its bound then), or NULL
 };
 
 // How the position of an id's first occurrence in "frontier ++ picked" is found (S3).
@@ -316,12 +318,13 @@ cudaError_t launch_validate_graph(const GraphView& g, int64_t num_edges, int64_t
 cudaError_t launch_count_dense(const GraphView& g, int32_t theta, int64_t* h_count, cudaStream_t s);
 cudaError_t launch_read_rows(const int32_t* slots, const int32_t* row_index, int32_t pitch, int32_t W,
                              const int32_t* nodes, int32_t n, int32_t* out, cudaStream_t s);
-cudaError_t launch_shard_bucket(const int32_t* nodes, int32_t n, const int32_t* d_n, int32_t rows_per_shard, int32_t world, int32_t* sorted,
-                                int32_t* slot, int32_t* counts_and_scratch, int32_t* status, cudaStream_t s);
-cudaError_t launch_export_picks(const int32_t* blk_indptr, const int32_t* picked, int32_t n, int32_t f, int32_t* out,
+cudaError_t launch_shard_bucket(const int32_t* nodes, int32_t n, const int32_t* d_n, int32_t rows_per_shard, int32_t world,
+                                int32_t capacity, int32_t* sorted, int32_t* slot, int32_t* counts_and_scratch, int32_t* status,
                                 cudaStream_t s);
+cudaError_t launch_export_picks(const int32_t* blk_indptr, const int32_t* picked, int32_t n, const int32_t* d_n, int32_t f,
+                                int32_t* out, cudaStream_t s);
 cudaError_t launch_import_picks(const int32_t* hdr, int32_t k, int32_t n_bound, int32_t f, const int32_t* reply,
-                                const int32_t* slot, const int32_t* blk_indptr, int32_t* picked, unsigned long long* table,
+                                int32_t reply_rows, const int32_t* slot, const int32_t* blk_indptr, int32_t* picked, unsigned long long* table,
                                 uint32_t stamp, int64_t num_nodes, int32_t* status, cudaStream_t s);
 cudaError_t launch_build_row_index(const GraphView& g, int32_t theta, int32_t* row_index, int32_t* tile_sums,
                                    int32_t* d_dense_rows, cudaStream_t s);

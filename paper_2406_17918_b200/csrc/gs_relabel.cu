@@ -23,7 +23,8 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
     }
     __syncthreads();
     if (s_status != 0) return;  // block-uniform: the barriers below stay convergent
-    const int n = (P.k == 0) ? P.n_host : __ldcg(P.hdr + HDR_N + P.k);
+    int n = (P.k == 0) ? P.n_host : __ldcg(P.hdr + HDR_N + P.k);
+    if (P.k == 0 && P.d_n0) n = min(n, max(0, __ldcg(P.d_n0)));
     // a capped grid walks the tiles that hold frontier nodes (the host only knows an upper bound of n)
     const int tiles = (n + SCAN_A_TILE - 1) / SCAN_A_TILE;
     const int refresh_from = P.d_refresh_from ? __ldcg(P.d_refresh_from) : 0;
@@ -53,7 +54,7 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
         if (v >= 0 && P.reply) {
             // sharded run, requester side: the owners have sampled; a row's picks are the non-negative prefix
             const int sl = P.slot ? P.slot[p] : p;
-            if ((unsigned)sl >= (unsigned)n) {
+            if ((unsigned)sl >= (unsigned)(P.reply_rows > 0 ? P.reply_rows : n)) {
                 raise_status(status, GS_ERR_RANGE);   // not a row of the reply: the node gets no picks
             } else {
                 const int32_t* row = P.reply + (int64_t)sl * P.f;
@@ -107,7 +108,8 @@ __global__ void __launch_bounds__(1024) k_row_counts(CountParams P) {
 __global__ void __launch_bounds__(1024) k_row_offsets(CountParams P) {
     chain_wait();
     if (__ldcg(P.hdr + HDR_STATUS) != 0) return;
-    const int n = (P.k == 0) ? P.n_host : __ldcg(P.hdr + HDR_N + P.k);
+    int n = (P.k == 0) ? P.n_host : __ldcg(P.hdr + HDR_N + P.k);
+    if (P.k == 0 && P.d_n0) n = min(n, max(0, __ldcg(P.d_n0)));
     for (int t = blockIdx.x; t <= n / SCAN_A_TILE; t += gridDim.x) {   // the tile of position n takes part too
     const int p = t * SCAN_A_TILE + threadIdx.x;
     if (p < n) P.blk_indptr[p] += P.tile_sums[p / SCAN_A_TILE];

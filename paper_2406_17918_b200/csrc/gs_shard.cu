@@ -21,7 +21,11 @@ __global__ void __launch_bounds__(SHARD_THREADS) k_bucket_count(const int32_t* _
                                                                 int rows_per_shard,
                                                                 int world, int32_t* __restrict__ counts, int32_t* status) {
     __shared__ int hist[SHARD_MAX_WORLD];
-    if (d_n) n = min(n, max(0, __ldcg(d_n)));   // the list's length may live on the device; n is its bound then
+    if (d_n) {   // the list's length may live on the device; n is its bound then, and a longer list is an error
+        const int len = __ldcg(d_n);
+        if (len > n && blockIdx.x == 0 && threadIdx.x == 0) atomicCAS(status, 0, GS_ERR_WORKSPACE);
+        n = min(n, max(0, len));
+    }
     if (threadIdx.x < SHARD_MAX_WORLD) hist[threadIdx.x] = 0;
     __syncthreads();
     const int i = blockIdx.x * SHARD_THREADS + threadIdx.x;
@@ -39,9 +43,9 @@ __global__ void __launch_bounds__(SHARD_THREADS) k_bucket_count(const int32_t* _
 // order inside a segment is whatever the atomics give; `slot` is what ties a reply to its node.
 __global__ void __launch_bounds__(SHARD_THREADS) k_bucket_place(const int32_t* __restrict__ nodes, int n, const int32_t* __restrict__ d_n,
                                                                 int rows_per_shard,
-                                                                int world, const int32_t* __restrict__ counts,
+                                                                int world, int capacity, const int32_t* __restrict__ counts,
                                                                 int32_t* __restrict__ cursor, int32_t* __restrict__ sorted,
-                                                                int32_t* __restrict__ slot) {
+                                                                int32_t* __restrict__ slot, int32_t* status) {
     __shared__ int hist[SHARD_MAX_WORLD];
     __shared__ int base[SHARD_MAX_WORLD];
     if (d_n) n = min(n, max(0, __ldcg(d_n)));
@@ -57,85 +61,117 @@ __global__ void __launch_bounds__(SHARD_THREADS) k_bucket_place(const int32_t* _
         else rank = atomicAdd(&hist[o], 1);
     }
     __syncthreads();
+    // packed: owner o's segment starts where the smaller owners' end; fixed pitch: at o * capacity, and a
+    // node beyond the segment's capacity is dropped and reported
     if (threadIdx.x < world) {
         int start = 0;
-        for (int j = 0; j < (int)threadIdx.x; ++j) start += __ldg(counts + j);
-        base[threadIdx.x] = start + (hist[threadIdx.x] ? atomicAdd(cursor + threadIdx.x, hist[threadIdx.x]) : 0);
+        if (capacity > 0) start = (int)threadIdx.x * capacity;
+        else
+            for (int j = 0; j < (int)threadIdx.x; ++j) start += __ldg(counts + j);
+        base[threadIdx.x] = (hist[threadIdx.x] ? atomicAdd(cursor + threadIdx.x, hist[threadIdx.x]) : 0);
+        hist[threadIdx.x] = start;   // every rank of this block was taken before the barrier above
     }
     __syncthreads();
     if (i < n) {
-        const int pos = o >= 0 ? base[o] + rank : -1;
+        int pos = -1;
+        if (o >= 0) {
+            const int in_segment = base[o] + rank;
+            if (capacity > 0 && in_segment >= capacity) atomicCAS(status, 0, GS_ERR_WORKSPACE);
+            else pos = hist[o] + in_segment;
+        }
         slot[i] = pos;
         if (pos >= 0) sorted[pos] = v;
     }
 }
 
-cudaError_t launch_shard_bucket(const int32_t* nodes, int32_t n, const int32_t* d_n, int32_t rows_per_shard, int32_t world, int32_t* sorted,
-                                int32_t* slot, int32_t* counts_and_scratch, int32_t* status, cudaStream_t s) {
+cudaError_t launch_shard_bucket(const int32_t* nodes, int32_t n, const int32_t* d_n, int32_t rows_per_shard, int32_t world,
+                                int32_t capacity, int32_t* sorted, int32_t* slot, int32_t* counts_and_scratch, int32_t* status,
+                                cudaStream_t s) {
     cudaError_t e = cudaMemsetAsync(counts_and_scratch, 0, (size_t)(2 * world + 1) * sizeof(int32_t), s);
     if (e != cudaSuccess || n <= 0) return e;
     const int blocks = (n + SHARD_THREADS - 1) / SHARD_THREADS;
     k_bucket_count<<<blocks, SHARD_THREADS, 0, s>>>(nodes, n, d_n, rows_per_shard, world, counts_and_scratch, status);
-    k_bucket_place<<<blocks, SHARD_THREADS, 0, s>>>(nodes, n, d_n, rows_per_shard, world, counts_and_scratch,
-                                                    counts_and_scratch + world, sorted, slot);
+    k_bucket_place<<<blocks, SHARD_THREADS, 0, s>>>(nodes, n, d_n, rows_per_shard, world, capacity, counts_and_scratch,
+                                                    counts_and_scratch + world, sorted, slot, status);
     count_launches(2);
     return cudaGetLastError();
 }
 
-// Owner side: the picks of node p, picked[blk_indptr[p] .. blk_indptr[p+1]), as a fixed row of f ids.
-__global__ void __launch_bounds__(SHARD_THREADS) k_export_picks(const int32_t* __restrict__ blk_indptr,
-                                                                const int32_t* __restrict__ picked, int n, int f,
-                                                                int32_t* __restrict__ out) {
-    const int64_t i = (int64_t)blockIdx.x * SHARD_THREADS + threadIdx.x;
-    if (i >= (int64_t)n * f) return;
-    const int p = (int)(i / f), t = (int)(i - (int64_t)p * f);
-    const int lo = __ldg(blk_indptr + p), hi = __ldg(blk_indptr + p + 1);
-    out[i] = (lo + t < hi) ? __ldg(picked + lo + t) : -1;
+// Both pick-row kernels walk (node, item) pairs with a capped grid: the host only knows an upper bound of the
+// list's length, often several times the real one, and a block per 256 pairs of the bound costs more than the copy.
+__device__ __forceinline__ void split_pair(unsigned long long i, unsigned f, unsigned& p, unsigned& t) {
+    p = (i >> 32) ? (unsigned)(i / f) : (unsigned)i / f;
+    t = (unsigned)(i - (unsigned long long)p * f);
 }
 
-cudaError_t launch_export_picks(const int32_t* blk_indptr, const int32_t* picked, int32_t n, int32_t f, int32_t* out,
-                                cudaStream_t s) {
+// Owner side: the picks of node p, picked[blk_indptr[p] .. blk_indptr[p+1]), as a fixed row of f ids.
+__global__ void __launch_bounds__(SHARD_THREADS) k_export_picks(const int32_t* __restrict__ blk_indptr,
+                                                                const int32_t* __restrict__ picked, int n,
+                                                                const int32_t* __restrict__ d_n, int f,
+                                                                int32_t* __restrict__ out) {
+    n = min(n, max(0, __ldcg(d_n)));   // rows of the list that were sampled (none after a device-detected error)
+    const unsigned long long total = (unsigned long long)n * (unsigned)f;
+    for (unsigned long long i = (unsigned long long)blockIdx.x * SHARD_THREADS + threadIdx.x; i < total;
+         i += (unsigned long long)gridDim.x * SHARD_THREADS) {
+        unsigned p, t;
+        split_pair(i, (unsigned)f, p, t);
+        const int lo = __ldg(blk_indptr + p), hi = __ldg(blk_indptr + p + 1);
+        out[i] = (lo + (int)t < hi) ? __ldg(picked + lo + t) : -1;
+    }
+}
+
+static unsigned pair_grid(int64_t n_bound, int32_t f) {
+    int64_t blocks = (n_bound * f + SHARD_THREADS - 1) / SHARD_THREADS;
+    const int64_t cap = sm_count() * 16;
+    return (unsigned)limit_grid(blocks < cap ? (blocks < 1 ? 1 : blocks) : cap);
+}
+
+cudaError_t launch_export_picks(const int32_t* blk_indptr, const int32_t* picked, int32_t n, const int32_t* d_n, int32_t f,
+                                int32_t* out, cudaStream_t s) {
     if (n <= 0) return cudaSuccess;
-    const int64_t blocks = ((int64_t)n * f + SHARD_THREADS - 1) / SHARD_THREADS;
-    k_export_picks<<<(unsigned)blocks, SHARD_THREADS, 0, s>>>(blk_indptr, picked, n, f, out);
+    k_export_picks<<<pair_grid(n, f), SHARD_THREADS, 0, s>>>(blk_indptr, picked, n, d_n, f, out);
     count_launches(1);
     return cudaGetLastError();
 }
 
-// Requester side: the returned rows become the step's picked-edge array, and every pick claims its
-// id in the relabel table with its edge position - what the pick kernels do when they run locally.
+// Requester side: the returned rows become the step's picked-edge array, and (with the direct-address
+// table; `table` is NULL otherwise) every pick claims its id in the relabel table with its edge
+// position - what the pick kernels do when they run locally.
 __global__ void __launch_bounds__(SHARD_THREADS) k_import_picks(const int32_t* __restrict__ hdr, int k, int f,
-                                                                const int32_t* __restrict__ reply,
+                                                                const int32_t* __restrict__ reply, int reply_rows,
                                                                 const int32_t* __restrict__ slot,
                                                                 const int32_t* __restrict__ blk_indptr,
                                                                 int32_t* __restrict__ picked, unsigned long long* table,
                                                                 uint32_t stamp, int64_t num_nodes, int32_t* status) {
     if (__ldcg(hdr + HDR_STATUS) != 0) return;
     const int n = __ldcg(hdr + HDR_N + k);
-    const int64_t i = (int64_t)blockIdx.x * SHARD_THREADS + threadIdx.x;
-    if (i >= (int64_t)n * f) return;
-    const int p = (int)(i / f), t = (int)(i - (int64_t)p * f);
-    const int sl = slot ? __ldg(slot + p) : p;
-    if ((unsigned)sl >= (unsigned)n) return;      // reported by the row-count kernel; the row has no picks
-    const int32_t u = __ldg(reply + (int64_t)sl * f + t);
-    if (u < 0) return;
-    if ((int64_t)u >= num_nodes) {
-        atomicCAS(status, 0, GS_ERR_RANGE);
-        return;
+    const unsigned rows = (unsigned)(reply_rows > 0 ? reply_rows : n);
+    const unsigned long long total = (unsigned long long)max(n, 0) * (unsigned)f;
+    for (unsigned long long i = (unsigned long long)blockIdx.x * SHARD_THREADS + threadIdx.x; i < total;
+         i += (unsigned long long)gridDim.x * SHARD_THREADS) {
+        unsigned p, t;
+        split_pair(i, (unsigned)f, p, t);
+        const int sl = slot ? __ldg(slot + p) : (int)p;
+        if ((unsigned)sl >= rows) continue;           // reported by the row-count kernel; the row has no picks
+        const int32_t u = __ldg(reply + (int64_t)sl * f + t);
+        if (u < 0) continue;
+        if ((int64_t)u >= num_nodes) {
+            atomicCAS(status, 0, GS_ERR_RANGE);
+            continue;
+        }
+        const int e = __ldg(blk_indptr + p) + (int)t;
+        if (e >= __ldg(blk_indptr + p + 1)) continue;   // beyond the row's non-negative prefix: not a pick
+        picked[e] = u;
+        if (table) atomicMin(table + u, ((unsigned long long)stamp << 32) | ((uint32_t)n + (uint32_t)e));
     }
-    const int e = __ldg(blk_indptr + p) + t;
-    if (e >= __ldg(blk_indptr + p + 1)) return;   // beyond the row's non-negative prefix: not a pick
-    picked[e] = u;
-    atomicMin(table + u, ((unsigned long long)stamp << 32) | ((uint32_t)n + (uint32_t)e));
 }
 
 cudaError_t launch_import_picks(const int32_t* hdr, int32_t k, int32_t n_bound, int32_t f, const int32_t* reply,
-                                const int32_t* slot, const int32_t* blk_indptr, int32_t* picked, unsigned long long* table,
+                                int32_t reply_rows, const int32_t* slot, const int32_t* blk_indptr, int32_t* picked, unsigned long long* table,
                                 uint32_t stamp, int64_t num_nodes, int32_t* status, cudaStream_t s) {
     if (n_bound <= 0) return cudaSuccess;
-    const int64_t blocks = ((int64_t)n_bound * f + SHARD_THREADS - 1) / SHARD_THREADS;
-    k_import_picks<<<(unsigned)blocks, SHARD_THREADS, 0, s>>>(hdr, k, f, reply, slot, blk_indptr, picked, table, stamp,
-                                                              num_nodes, status);
+    k_import_picks<<<pair_grid(n_bound, f), SHARD_THREADS, 0, s>>>(hdr, k, f, reply, reply_rows, slot, blk_indptr, picked, table,
+                                                                   stamp, num_nodes, status);
     count_launches(1);
     return cudaGetLastError();
 }

@@ -37,15 +37,15 @@ def barrier():
         dist.barrier()
 
 
-def aggregate(ms_local: float, units_local, device="cpu"):
-    """(max over ranks of ms, elementwise sum over ranks of units)."""
+def aggregate(ms_local: float, units_local, device="cpu", reduce="sum"):
+    """(max over ranks of ms, elementwise sum - or, with reduce="max", maximum - over ranks of units)."""
     units = [float(u) for u in units_local]
     if not dist.is_initialized():
         return float(ms_local), units
     t = torch.tensor([ms_local], dtype=torch.float64, device=device)
     u = torch.tensor(units, dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    dist.all_reduce(u, op=dist.ReduceOp.MAX if reduce == "max" else dist.ReduceOp.SUM)
     return float(t.item()), [float(x) for x in u.tolist()]
 
 

@@ -67,6 +67,7 @@ class ShardRank:
                                     dtype=torch.uint8, device=dev)
         self.blocks = [None] * self.L
         self.n = []
+        self.caps = None                           # fixed-capacity exchanges: see set_capacities
 
     # ---- requester side
     # The host learns the size of a frontier only from the group sizes it has to read back for the exchange
@@ -78,6 +79,8 @@ class ShardRank:
         self.count_dev = None                      # device scalar with the current frontier's length
         self.blocks = [None] * self.L
         self.m = [0] * self.L
+        self.seen = []                             # exact-size mode: the largest group of every exchange so far
+        self.feat_bound = None
 
     def requests(self, nodes, count=None):
         """Bucket `nodes` (all of it, or its first *count ids) by owner -> (ids grouped by owner, group sizes
@@ -88,8 +91,10 @@ class ShardRank:
             sorted_ids, self.slot, counts = self.ops.gs_shard_bucket(nodes, self.num_nodes, self.world, count=count)
         c = counts.cpu().tolist()                      # the all-to-all needs the sizes on the host
         if c[2 * self.world] != 0:
-            raise ValueError("a node id is outside [0, num_nodes)")
+            raise ValueError("a node id is outside [0, num_nodes)" if c[2 * self.world] == 3 else
+                             "the frontier is longer than the bound it was bucketed with")
         total = sum(c[: self.world])
+        self.seen.append(max(c[: self.world]))     # largest group of this exchange: what a fixed capacity has to hold
         return sorted_ids[:total], c[: self.world]
 
     def _frontier_bound(self, k):
@@ -124,17 +129,123 @@ class ShardRank:
         self.n, self.m = list(n), list(m)
         self.ops.gs_shard_status(self.cache)       # the lists this rank served
 
-    def feature_pull(self, shard_bases):
+    def feature_pull(self, shard_bases, bound=None):
         """The feature step as one kernel: every input node's row is read straight from its owner's
-        memory (`shard_bases[o]`: device address of rank o's feature rows, peer-mapped where o is another GPU)."""
-        bound = self._frontier_bound(self.L)
+        memory (`shard_bases[o]`: device address of rank o's feature rows, peer-mapped where o is another GPU).
+        `bound`: rows to allocate for when the host does not know the last hop's size."""
+        if bound is None:
+            bound = self._frontier_bound(self.L) if self.caps is None else self._product_bound(self.L)
         out = torch.empty((bound, self.features.shape[1]), dtype=self.features.dtype, device=self.features.device)
+        self.feat_bound = bound
         return self.ops.gs_gather_rows_peer(shard_bases, self.num_nodes, self.features.dtype, self.features.shape[1],
                                             self.features.stride(0), self.frontier[:bound], out, count=self.count_dev)
 
     def feature_finish(self, rows):
         out = torch.empty((self.n[self.L], rows.shape[1]), dtype=rows.dtype, device=rows.device)
         return self.ops.gs_gather_rows(rows, self.slot[: self.n[self.L]], out)
+
+    # ---- the same phases with fixed-capacity exchanges: no size ever goes through the host
+    # Every (requester, owner) pair gets a segment of caps[k] ids at hop k (caps[L]: the feature request), the
+    # group sizes travel as a device array beside the ids, owners take each list's length from there, and the
+    # replies come back at the same pitch.  The exchanges are equal-split all-to-alls of pre-allocated buffers,
+    # so a batch has no host synchronisation before finish_batch.  A group that outgrows its segment is a
+    # device-detected error of the batch (reported by finish_batch), never an overrun.
+    def set_capacities(self, caps):
+        """caps[0..L-1]: ids per (requester, owner) pair at each hop; caps[L]: at the feature request (omit or 0
+        when features are pulled from peer memory).  Every rank must use the same values."""
+        caps = [int(c) for c in caps] + [0] * (self.L + 1 - len(caps))
+        if len(caps) != self.L + 1 or min(caps[: self.L]) < 1:
+            raise ValueError("one positive capacity per hop (and optionally one for the features) expected")
+        R, dev = self.world, self.features.device
+        self.caps = caps
+        need = min(self.num_nodes, max(caps[: self.L]))
+        if need > self.max_requests:
+            self.max_requests = need
+            self.ws_owner = torch.empty(self.ops.gs_shard_workspace_bytes(self.graph, max(self.fanouts), need),
+                                        dtype=torch.uint8, device=dev)
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.counts_all = torch.zeros((self.L + 1, 2 * R + 1), **i32)
+        self.counts_host = torch.zeros((self.L + 1, 2 * R + 1), dtype=torch.int32, pin_memory=dev.type == "cuda")
+        self.fx = []
+        for k in range(self.L + 1):
+            C = caps[k]
+            b = {"sorted": torch.empty(R * C, **i32), "recv": torch.empty(R * C, **i32), "recv_counts": torch.empty(R, **i32)}
+            if k < self.L:
+                f = self.fanouts[self.L - 1 - k]
+                b["out"], b["reply"] = torch.empty((R * C, f), **i32), torch.empty((R * C, f), **i32)
+            else:
+                D = self.features.shape[1]
+                b["out"] = torch.empty((R * C, D), dtype=self.features.dtype, device=dev)
+                b["reply"] = torch.empty((R * C, D), dtype=self.features.dtype, device=dev)
+            self.fx.append(b)
+        self.fx_slot = None
+
+    def _product_bound(self, k):
+        bound = self.n[0]
+        for j in range(k):
+            bound = min(self.num_nodes, bound * (1 + self.fanouts[self.L - 1 - j]))
+        return bound
+
+    def _bound_fixed(self, k):
+        """Upper bound of n_k that needs no host knowledge of the batch: the fan-out product, the node count, and
+        what the segments can hold at all."""
+        bound = self._product_bound(k)
+        # the slots of a hop are read for every frontier node, so they cover the whole bound; the feature
+        # request needs no more than the segments can hold (a longer frontier is reported by the bucket call)
+        return min(bound, self.world * self.caps[k]) if k == self.L and self.caps[k] > 0 else bound
+
+    def requests_fixed(self, k):
+        """-> (ids [world * caps[k]] at fixed pitch, group sizes as a device tensor [world])."""
+        bound = self._bound_fixed(k)
+        if self.fx_slot is None or self.fx_slot.numel() < bound:
+            self.fx_slot = torch.empty(max(bound, 1), dtype=torch.int32, device=self.features.device)
+        b = self.fx[k]
+        _, self.slot, counts = self.ops.gs_shard_bucket(self.frontier[:bound], self.num_nodes, self.world,
+                                                        count=self.count_dev, capacity=self.caps[k],
+                                                        out=(b["sorted"], self.fx_slot[:bound], self.counts_all[k]))
+        return b["sorted"], counts[: self.world]
+
+    def hop_finish_fixed(self, k, reply):
+        block, frontier = self.ops.gs_shard_extend(self.cache, k, self.seeds if k == 0 else None, reply, self.slot, self.ws,
+                                                   reply_rows=self.world * self.caps[k])
+        self.blocks[self.L - 1 - k] = block
+        self.frontier = frontier
+        self.count_dev = block.counts_device()[1]
+
+    def hop_serve_fixed(self, layer, recv, recv_counts, mode, rate, step, out):
+        """recv [world * C] ids, requester r's list in segment r, its length recv_counts[r] -> out [world * C, f]."""
+        C = recv.numel() // self.world
+        for r in range(self.world):
+            self.ops.gs_shard_sample_rows(self.cache, recv[r * C:(r + 1) * C], layer, mode, rate, step, self.ws_owner,
+                                          picks=out[r * C:(r + 1) * C], count=recv_counts[r:r + 1])
+        return out
+
+    def feature_serve_fixed(self, recv, recv_counts, out):
+        C = recv.numel() // self.world
+        for r in range(self.world):
+            self.ops.gs_gather_rows(self.features, recv[r * C:(r + 1) * C], out[r * C:(r + 1) * C], first_row=self.first_row,
+                                    count=recv_counts[r:r + 1])
+        return out
+
+    def feature_finish_fixed(self, rows):
+        bound = self._bound_fixed(self.L)
+        out = torch.empty((bound, rows.shape[1]), dtype=rows.dtype, device=rows.device)
+        return self.ops.gs_gather_rows(rows, self.slot[:bound], out, count=self.count_dev)
+
+    def finish_batch_fixed(self):
+        """Counts, device status and the bucket calls' error words of the batch, read once (synchronises)."""
+        self.counts_host.copy_(self.counts_all, non_blocking=True)
+        self.finish_batch()                        # synchronises the stream the copy above is on
+        if self.feat_bound is not None and self.n[self.L] > self.feat_bound:
+            raise RuntimeError("%d input nodes, feature rows were allocated for %d" % (self.n[self.L], self.feat_bound))
+        words = self.counts_host[:, 2 * self.world].tolist()
+        if any(w == 3 for w in words):             # GS_ERR_RANGE
+            raise ValueError("a node id is outside [0, num_nodes)")
+        if any(words):
+            k = [i for i, w in enumerate(words) if w][0]
+            raise RuntimeError("the requests of %s outgrew their segment of %d ids (groups: %s)"
+                               % ("hop %d" % k if k < self.L else "the feature step", self.caps[k],
+                                  self.counts_host[k, : self.world].tolist()))
 
     # ---- owner side
     def hop_serve(self, layer, lists, mode, rate, step):
@@ -166,6 +277,8 @@ def sample_batch_local(ranks, seeds_per_rank, mode, rate, step, features=True):
     L = ranks[0].L
     for r, seeds in zip(ranks, seeds_per_rank):
         r.begin(seeds)
+    if ranks[0].caps is not None:
+        return _sample_batch_local_fixed(ranks, mode, rate, step, features)
 
     def round_trip(req, serve):
         sent = [_split(ids, counts) for ids, counts in req]                 # sent[r][o]
@@ -187,6 +300,44 @@ def sample_batch_local(ranks, seeds_per_rank, mode, rate, step, features=True):
         feats = [r.feature_finish(x.contiguous()) for r, x in zip(ranks, rows)]
     for r in ranks:
         r.finish_batch()
+    feats = [f if f is None else f[: r.n[L]] for r, f in zip(ranks, feats)]
+    return [(r.blocks, r.frontier, r.n, r.m, f) for r, f in zip(ranks, feats)]
+
+
+def _sample_batch_local_fixed(ranks, mode, rate, step, features):
+    """sample_batch_local with fixed-capacity exchanges (ShardRank.set_capacities): the copies below stand for the
+    equal-split all-to-alls; the host reads nothing before the end of the batch."""
+    R, L = len(ranks), ranks[0].L
+
+    def round_trip(k, req, serve):
+        C = ranks[0].caps[k]
+        replies = [r.fx[k]["reply"] for r in ranks]
+        for o, owner in enumerate(ranks):
+            b = owner.fx[k]
+            for r in range(R):                                   # what rank r sends to owner o
+                b["recv"][r * C:(r + 1) * C].copy_(req[r][0][o * C:(o + 1) * C])
+                b["recv_counts"][r:r + 1].copy_(req[r][1][o:o + 1])
+            serve(owner, b["recv"], b["recv_counts"], b["out"])
+            for r in range(R):                                   # and what comes back
+                replies[r][o * C:(o + 1) * C].copy_(b["out"][r * C:(r + 1) * C])
+        return replies
+
+    for k in range(L):
+        layer = L - 1 - k
+        replies = round_trip(k, [r.requests_fixed(k) for r in ranks],
+                             lambda owner, recv, rc, out: owner.hop_serve_fixed(layer, recv, rc, mode, rate, step, out))
+        for r, reply in zip(ranks, replies):
+            r.hop_finish_fixed(k, reply)
+    feats = [None] * R
+    if features == "peer":
+        bases = [r.features.data_ptr() for r in ranks]
+        feats = [r.feature_pull(bases, bound=r._bound_fixed(L) if r.caps[L] else None) for r in ranks]
+    elif features:
+        rows = round_trip(L, [r.requests_fixed(L) for r in ranks],
+                          lambda owner, recv, rc, out: owner.feature_serve_fixed(recv, rc, out))
+        feats = [r.feature_finish_fixed(x) for r, x in zip(ranks, rows)]
+    for r in ranks:
+        r.finish_batch_fixed()
     feats = [f if f is None else f[: r.n[L]] for r, f in zip(ranks, feats)]
     return [(r.blocks, r.frontier, r.n, r.m, f) for r, f in zip(ranks, feats)]
 
@@ -236,6 +387,9 @@ def sample_batch(rank_state: ShardRank, seeds, mode, rate, step, features=True, 
         if not state["err"]:
             state["err"], state["msg"] = code, str(e)
 
+    if me.caps is not None:
+        return _sample_batch_fixed(me, mode, rate, step, features, group, feature_bases, state, fail)
+
     def round_trip(make_requests, serve, width, dtype):
         ids, counts = torch.empty(0, dtype=torch.int32, device=dev), [0] * me.world
         if state["err"] != 1:                      # a rank whose own batch is broken asks for nothing more
@@ -276,6 +430,63 @@ def sample_batch(rank_state: ShardRank, seeds, mode, rate, step, features=True, 
             me.finish_batch()
         except (ValueError, RuntimeError) as e:
             fail(2, e)
+    word = torch.tensor([state["err"]], dtype=torch.int32, device=dev)
+    dist.all_reduce(word, op=dist.ReduceOp.MAX, group=group)
+    code = int(word.item())
+    if code:
+        raise ShardedBatchError(code, state["msg"])
+    if feats is not None:
+        feats = feats[: me.n[L]]
+    return me.blocks, me.frontier, me.n, me.m, feats
+
+
+def _sample_batch_fixed(me, mode, rate, step, features, group, feature_bases, state, fail):
+    """sample_batch with fixed-capacity exchanges (ShardRank.set_capacities): three equal-split all-to-alls per hop
+    (group sizes, ids, rows) on pre-allocated buffers, no host synchronisation before the end of the batch.  Every
+    rank always takes part in every exchange, whatever it has met; errors (host- or device-detected, a group that
+    outgrew its segment included) are reduced once, after the last exchange."""
+    L, dev = me.L, me.features.device
+
+    def round_trip(k, serve):
+        b = me.fx[k]
+        ids, counts = b["sorted"], me.counts_all[k, : me.world]
+        if state["err"] != 1:
+            try:
+                ids, counts = me.requests_fixed(k)
+            except (ValueError, RuntimeError) as e:
+                fail(1, e)
+        if state["err"] == 1:
+            counts = torch.zeros(me.world, dtype=torch.int32, device=dev)      # this rank asks for nothing more
+        dist.all_to_all_single(b["recv_counts"], counts, group=group)
+        dist.all_to_all_single(b["recv"], ids, group=group)
+        try:
+            serve(b["recv"], b["recv_counts"], b["out"])
+        except (ValueError, RuntimeError) as e:
+            fail(2, e)
+        dist.all_to_all_single(b["reply"], b["out"], group=group)
+        return b["reply"]
+
+    for k in range(L):
+        layer = L - 1 - k
+        reply = round_trip(k, lambda recv, rc, out: me.hop_serve_fixed(layer, recv, rc, mode, rate, step, out))
+        if state["err"] != 1:
+            try:
+                me.hop_finish_fixed(k, reply)
+            except (ValueError, RuntimeError) as e:
+                fail(1, e)
+    feats = None
+    if features and feature_bases is not None:
+        if state["err"] != 1:
+            feats = me.feature_pull(feature_bases, bound=me._bound_fixed(L) if me.caps[L] else None)
+    elif features:
+        rows = round_trip(L, me.feature_serve_fixed)
+        if state["err"] != 1:
+            feats = me.feature_finish_fixed(rows)
+    if state["err"] != 1:
+        try:
+            me.finish_batch_fixed()
+        except (ValueError, RuntimeError) as e:
+            fail(2 if "requested node" in str(e) else 1, e)
     word = torch.tensor([state["err"]], dtype=torch.int32, device=dev)
     dist.all_reduce(word, op=dist.ReduceOp.MAX, group=group)
     code = int(word.item())

@@ -55,25 +55,41 @@ def gs_shard_workspace_bytes(graph, fanout, max_nodes):
     return 256
 
 
-def gs_shard_bucket(nodes, num_nodes, world, count=None):
+def gs_shard_bucket(nodes, num_nodes, world, count=None, capacity=None, out=None):
     v = nodes.numpy() if count is None else nodes.numpy()[: int(count)]
     S = (num_nodes + world - 1) // world
     owner = v // S
     order = np.argsort(owner, kind="stable")
-    slot = np.zeros(nodes.numel(), dtype=np.int32)
-    slot[order] = np.arange(len(v), dtype=np.int32)
     counts = np.zeros(2 * world + 1, dtype=np.int32)
     counts[:world] = np.bincount(owner, minlength=world)
-    sorted_ids = np.zeros(nodes.numel(), dtype=np.int32)
-    sorted_ids[: len(v)] = v[order]
-    return torch.from_numpy(sorted_ids), torch.from_numpy(slot), torch.from_numpy(counts)
+    slot = np.zeros(nodes.numel(), dtype=np.int32)
+    if capacity is None:
+        slot[order] = np.arange(len(v), dtype=np.int32)
+        sorted_ids = np.zeros(nodes.numel(), dtype=np.int32)
+        sorted_ids[: len(v)] = v[order]
+    else:                                   # every owner's group in a segment of `capacity` ids; the surplus is dropped
+        sorted_ids = np.full(world * capacity, -7, dtype=np.int32)
+        starts = np.concatenate([[0], np.cumsum(counts[:world])])
+        rank_in_group = np.arange(len(v)) - starts[owner[order]]
+        pos = np.where(rank_in_group < capacity, owner[order] * capacity + rank_in_group, -1).astype(np.int32)
+        slot[order] = pos
+        sorted_ids[pos[pos >= 0]] = v[order][pos >= 0]
+        if (pos < 0).any():
+            counts[2 * world] = 4          # GS_ERR_WORKSPACE
+    res = (torch.from_numpy(sorted_ids), torch.from_numpy(slot), torch.from_numpy(counts))
+    if out is not None:
+        for dst, src in zip(out, res):
+            dst[: src.numel()].copy_(src)
+        return out
+    return res
 
 
-def gs_shard_sample_rows(cache, nodes, layer, mode, rate, step, ws):
+def gs_shard_sample_rows(cache, nodes, layer, mode, rate, step, ws, picks=None, count=None):
     f = cache.fanouts[layer]
-    out = np.full((nodes.numel(), f), -1, dtype=np.int32)
+    ids = nodes.numpy() if count is None else nodes.numpy()[: int(count)]
+    out = np.full((len(ids), f), -1, dtype=np.int32)
     O, om = cache.O, _OM[mode]
-    for i, v in enumerate(nodes.numpy().tolist()):
+    for i, v in enumerate(ids.tolist()):
         if om == oracle.MODE_FBL or cache.graph.deg[v] <= cache.theta:
             row = O.fbl_node(layer, v, step)
         elif om == oracle.MODE_OTF_FETCH:
@@ -82,6 +98,9 @@ def gs_shard_sample_rows(cache, nodes, layer, mode, rate, step, ws):
             O.refresh_node(layer, v, step, oracle.refresh_count(om, rate, cache.W))
             row = O.pick_node(layer, v, step)
         out[i, : len(row)] = row
+    if picks is not None:                   # only the list's rows are written
+        picks[: len(ids)].copy_(torch.from_numpy(out))
+        return picks
     return torch.from_numpy(out)
 
 
@@ -89,7 +108,7 @@ def gs_shard_status(cache):
     pass
 
 
-def gs_shard_extend(cache, k, seeds, reply, slot, ws):
+def gs_shard_extend(cache, k, seeds, reply, slot, ws, reply_rows=None):
     L = len(cache.fanouts)
     if k == 0:
         cache.frontier = seeds.numpy().tolist()
@@ -99,6 +118,9 @@ def gs_shard_extend(cache, k, seeds, reply, slot, ws):
     n_k = cache.n[k]
     indptr, local = [0], []
     for p in range(n_k):
+        if sl[p] < 0:                       # dropped by a full segment: no picks (the batch is reported as failed)
+            indptr.append(len(local))
+            continue
         for u in rows[sl[p]]:
             if u < 0:
                 break
@@ -117,6 +139,9 @@ def gs_batch_counts(cache):
     return list(cache.n), list(cache.m)
 
 
-def gs_gather_rows(src, ids, out, first_row=0):
-    out.copy_(src[ids.long() - first_row])
+def gs_gather_rows(src, ids, out, first_row=0, count=None):
+    n = min(out.shape[0], ids.numel()) if count is None else min(int(count), out.shape[0], ids.numel())
+    idx = ids[:n].long() - first_row
+    ok = (idx >= 0) & (idx < src.shape[0])  # an id outside the source leaves its output row as it is
+    out[:n][ok] = src[idx[ok]]
     return out

@@ -16,7 +16,7 @@ MODES = {"fcr": (0, oracle.MODE_FCR), "otf": (1, oracle.MODE_OTF), "fbl": (2, or
 
 
 class Setup:
-    def __init__(self, name, world, theta, seed=5, B=None):
+    def __init__(self, name, world, theta, seed=5, B=None, fixed=False):
         import paper_2406_17918_b200 as gs
         from paper_2406_17918_b200 import sharded
         self.gs, self.sharded = gs, sharded
@@ -36,6 +36,9 @@ class Setup:
             self.ranks.append(sharded.ShardRank(gs, r, world, ip.cuda(), idx.cuda(), self.X[lo:hi].cuda().contiguous(),
                                                 cfg["fanouts"], cfg["cache_width"], seed, cfg["shared"], theta,
                                                 max_seeds=self.B, max_requests=min(N, self.B * 400)))
+        if fixed:   # fixed-capacity exchanges; a group holds distinct nodes of one owner, so a shard's size always suffices
+            for r in self.ranks:
+                r.set_capacities([sharded.rows_per_shard(N, world)] * (len(cfg["fanouts"]) + 1))
         self.O = oracle.Sampler(self.indptr, self.indices, cfg["fanouts"], cfg["cache_width"], seed, cfg["shared"])
         self.O.set_theta(theta)
 
@@ -77,9 +80,10 @@ class Setup:
                 assert np.array_equal(got, want[(nodes // S) == r]), (layer, r)
 
 
+@pytest.mark.parametrize("fixed", [False, True])
 @pytest.mark.parametrize("world", [1, 2, 3])
-def test_sharded_tiny_all_modes(world):
-    s = Setup("tiny", world, theta=12)
+def test_sharded_tiny_all_modes(world, fixed):
+    s = Setup("tiny", world, theta=12, fixed=fixed)
     t = 1
     for mode, rate in [("otf", 0.25), ("otf", 0.25), ("fcr", 0.0), ("fetch", 0.5), ("fbl", 0.0), ("otf", 0.0), ("otf", 1.0)]:
         s.step(mode, rate, t)
@@ -98,6 +102,79 @@ def test_sharded_mid_and_shared_cache():
     for t in (1, 2):
         s.step("otf", 0.3, t)
     s.check_rows(sample=4000)
+
+
+def test_sharded_mid_fixed_capacity_exchanges():
+    """Segments sized from an exact-size batch (the largest group seen, plus a margin), as a deployment would do."""
+    s = Setup("mid", 3, theta=24, B=512)
+    s.step("otf", 0.3, 1)
+    seen = np.max([r.seen for r in s.ranks], axis=0)                  # one entry per exchange: L hops + features
+    caps = [int(c * 1.3) + 8 for c in seen]
+    for r in s.ranks:
+        r.set_capacities(caps)
+    for t in (2, 3):
+        s.step("otf", 0.3, t, features="peer" if t == 3 else True)
+    s.step("fetch", 0.5, 4)
+    s.check_rows(sample=4000)
+    # segments that cannot hold the groups: the batch is reported as failed and nothing overruns
+    for r in s.ranks:
+        r.set_capacities([64] * len(caps))
+    seeds = [batch_seeds(s.perm, 5, s.B, r, s.world).cuda() for r in range(s.world)]
+    with pytest.raises(RuntimeError):
+        s.sharded.sample_batch_local(s.ranks, seeds, 1, 0.3, 5)
+    torch.cuda.synchronize()
+
+
+def test_fixed_pitch_primitives():
+    import paper_2406_17918_b200 as gs
+    rng = np.random.default_rng(11)
+    N, world, cap = 100003, 5, 13000
+    S = (N + world - 1) // world
+    full = torch.from_numpy(rng.choice(N, 60000, replace=False).astype(np.int32)).cuda()
+    count = torch.tensor(41234, dtype=torch.int32, device="cuda")
+    for cnt in (None, count):
+        n = full.numel() if cnt is None else int(cnt.item())
+        sorted_ids, slot, counts = gs.gs_shard_bucket(full, N, world, count=cnt, capacity=cap)
+        v = full.cpu().numpy()[:n]
+        c, so, sl = counts.cpu().numpy(), sorted_ids.cpu().numpy(), slot.cpu().numpy()[:n]
+        owner = v // S
+        assert sorted_ids.numel() == world * cap and c[2 * world] == 0
+        assert np.array_equal(c[:world], np.bincount(owner, minlength=world))
+        assert np.array_equal(sl // cap, owner) and (sl % cap < c[owner]).all()        # each id inside its owner's segment
+        assert np.array_equal(so[sl], v) and len(np.unique(sl)) == n
+    # a group larger than its segment: flagged, the surplus gets slot -1, nothing is written beyond the segment
+    small = 7000
+    out = (torch.full((world * small + 64,), -5, dtype=torch.int32, device="cuda"), torch.empty_like(full),
+           torch.empty(2 * world + 1, dtype=torch.int32, device="cuda"))
+    sorted_ids, slot, counts = gs.gs_shard_bucket(full, N, world, capacity=small, out=out)
+    c, sl = counts.cpu().numpy(), slot.cpu().numpy()
+    owner = full.cpu().numpy() // S
+    assert c[2 * world] == 4 and (c[:world] > small).any()                                 # GS_ERR_WORKSPACE
+    assert bool((sorted_ids[world * small:] == -5).all())
+    for o in range(world):
+        mine = sl[owner == o]
+        assert (mine >= 0).sum() == min(small, c[o]) and ((mine < 0) | (mine // small == o)).all()
+    # a device length above the bound: flagged as well
+    long = torch.tensor(full.numel() + 1, dtype=torch.int32, device="cuda")
+    assert gs.gs_shard_bucket(full, N, world, count=long, capacity=cap)[2].cpu().numpy()[2 * world] == 4
+    assert gs.gs_shard_bucket(full, N, world, count=long)[2].cpu().numpy()[2 * world] == 4
+    with pytest.raises(gs.GsError):
+        gs.gs_shard_bucket(full, N, world, capacity=0)
+    # owner side with the list's length on the device: the first *count rows equal the exact-size call, the rest is untouched
+    s = Setup("tiny", 1, theta=12)
+    me = s.ranks[0]
+    nodes = torch.from_numpy(np.random.default_rng(2).choice(s.cfg["num_nodes"], 300, replace=False).astype(np.int32)).cuda()
+    f = me.fanouts[0]
+    want = gs.gs_shard_sample_rows(me.cache, nodes[:211].contiguous(), 0, gs.GS_MODE_FBL, 0.0, 3, me.ws_owner)
+    got = torch.full((300, f), -9, dtype=torch.int32, device="cuda")
+    gs.gs_shard_sample_rows(me.cache, nodes, 0, gs.GS_MODE_FBL, 0.0, 3, me.ws_owner, picks=got,
+                            count=torch.tensor([211], dtype=torch.int32, device="cuda"))
+    gs.gs_shard_status(me.cache)
+    assert torch.equal(got[:211], want) and bool((got[211:] == -9).all())
+    gs.gs_shard_sample_rows(me.cache, nodes, 0, gs.GS_MODE_FBL, 0.0, 3, me.ws_owner, picks=got,
+                            count=torch.tensor([0], dtype=torch.int32, device="cuda"))       # an empty list
+    gs.gs_shard_status(me.cache)
+    assert torch.equal(got[:211], want)
 
 
 def test_bucket_and_gather_rows_primitives():
@@ -226,6 +303,10 @@ def test_randomised_sharded_runs(case):
         lo, hi = sharded.shard_range(n, r, world)
         ranks.append(sharded.ShardRank(gs, r, world, ip.cuda(), idx.cuda(), X[lo:hi].cuda().contiguous(), fanouts, W, seed,
                                        shared, theta, max_seeds=B, max_requests=n))
+        if case % 2:            # odd cases: fixed-capacity exchanges (a shard's size always holds a group)
+            ranks[-1].set_capacities([sharded.rows_per_shard(n, world)] * (L + 1))
+        # the requester's dedup + relabel with each way of finding first occurrences
+        gs.gs_cache_set_dedup(ranks[-1].cache, [gs.GS_DEDUP_AUTO, gs.GS_DEDUP_HASH, gs.GS_DEDUP_SORT, gs.GS_DEDUP_DIRECT][(case // 2) % 4])
     O = oracle.Sampler(indptr, indices, fanouts, W, seed, shared)
     O.set_theta(theta)
     step = int(rng.integers(1, 2**32 - 10))

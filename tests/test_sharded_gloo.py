@@ -25,7 +25,7 @@ def _features(n, d=6):
     return (torch.arange(n * d, dtype=torch.float32).reshape(n, d) * 0.5).contiguous()
 
 
-def _worker(rank, world, port, out_dir):
+def _worker(rank, world, port, out_dir, capacity=None):
     import torch.distributed as dist
 
     import fake_shard_ops as ops
@@ -40,6 +40,8 @@ def _worker(rank, world, port, out_dir):
     lo, hi = sharded.shard_range(cfg["num_nodes"], rank, world)
     me = sharded.ShardRank(ops, rank, world, ip, idx, X[lo:hi].contiguous(), cfg["fanouts"], cfg["cache_width"], SEED,
                            cfg["shared"], THETA, max_seeds=cfg["batch"], max_requests=cfg["num_nodes"])
+    if capacity:            # fixed-capacity exchanges: no size is read on the host inside a batch
+        me.set_capacities([capacity] * (len(cfg["fanouts"]) + 1))
     out = []
     t = 1
     for mode, rate in [(ops.GS_MODE_OTF, 0.25), (ops.GS_MODE_OTF, 0.25), (ops.GS_MODE_FCR, 0.0), (ops.GS_MODE_OTF_FETCH, 0.5),
@@ -56,10 +58,11 @@ def _worker(rank, world, port, out_dir):
     dist.destroy_process_group()
 
 
-@pytest.mark.parametrize("world", [2, 3])
-def test_ranks_equal_one_sampler_taking_the_batches_in_turn(tmp_path, world):
-    """World size 3 gives uneven shards (2,708 nodes: 903 + 903 + 902)."""
-    mp.spawn(_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+@pytest.mark.parametrize("world,capacity", [(2, None), (3, None), (2, 1500), (3, 920)])
+def test_ranks_equal_one_sampler_taking_the_batches_in_turn(tmp_path, world, capacity):
+    """World size 3 gives uneven shards (2,708 nodes: 903 + 903 + 902).  With a capacity the exchanges have a
+    fixed pitch (segments of that many ids per pair of ranks) and the driver reads no size inside a batch."""
+    mp.spawn(_worker, args=(world, _free_port(), str(tmp_path), capacity), nprocs=world, join=True)
     res = [torch.load(os.path.join(tmp_path, "r%d.pt" % r)) for r in range(world)]
     cfg = get_config("tiny")
     g = build_graph(cfg)
@@ -82,7 +85,7 @@ def test_ranks_equal_one_sampler_taking_the_batches_in_turn(tmp_path, world):
             assert torch.equal(got["feats"], X[torch.from_numpy(fr.astype(np.int64))])
 
 
-def _failing_worker(rank, world, port, out_dir):
+def _failing_worker(rank, world, port, out_dir, capacity=None):
     import torch.distributed as dist
 
     import fake_shard_ops as ops
@@ -96,9 +99,11 @@ def _failing_worker(rank, world, port, out_dir):
     ip, idx = sharded.shard_csr(g.indptr, g.indices, rank, world)
     lo, hi = sharded.shard_range(cfg["num_nodes"], rank, world)
     # the last rank can serve three nodes per list only: its first hop fails on the owner side
-    cap = 3 if rank == world - 1 else cfg["num_nodes"]
+    cap = 3 if rank == world - 1 and not capacity else cfg["num_nodes"]
     me = sharded.ShardRank(ops, rank, world, ip, idx, X[lo:hi].contiguous(), cfg["fanouts"], cfg["cache_width"], SEED,
                            cfg["shared"], THETA, max_seeds=cfg["batch"], max_requests=cap)
+    if capacity:
+        me.set_capacities([capacity] * (len(cfg["fanouts"]) + 1))
     seeds = batch_seeds(perm, 1, cfg["batch"], rank, world)
     outcome = "returned"
     try:
@@ -117,6 +122,15 @@ def test_a_failure_on_one_rank_ends_the_batch_on_every_rank(tmp_path, world):
     mp.spawn(_failing_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
     for r in range(world):
         assert open(os.path.join(tmp_path, "f%d.txt" % r)).read() == "raised 2"
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_a_group_that_outgrows_its_segment_ends_the_batch_on_every_rank(tmp_path, world):
+    """Fixed-capacity exchanges: segments of 40 ids cannot hold the second hop's groups; nothing overruns, every
+    exchange of the batch still takes place, and all ranks raise (a requester-side error: code 1)."""
+    mp.spawn(_failing_worker, args=(world, _free_port(), str(tmp_path), 40), nprocs=world, join=True)
+    for r in range(world):
+        assert open(os.path.join(tmp_path, "f%d.txt" % r)).read() == "raised 1"
 
 
 def test_refreshing_a_row_twice_in_one_step_equals_once():
