@@ -267,6 +267,10 @@ def main():
                          "protocol's overhead, the exchange being a local copy")
     ap.add_argument("--feature-exchange", default=None, choices=["peer", "roundtrip"],
                     help="with --sharded: how feature rows reach the requester (default: peer with one rank, roundtrip otherwise)")
+    ap.add_argument("--local-ranks", type=int, default=1,
+                    help="with --sharded on one GPU: run this many ranks of the sharded job in this process, phase by phase")
+    ap.add_argument("--no-merge", action="store_true",
+                    help="with --sharded: owners serve the requesters' lists one by one instead of merging them")
     ap.add_argument("--exact-sizes", action="store_true",
                     help="with --sharded: keep the exact-size exchanges (host reads the group sizes) for the timed batches")
     ap.add_argument("--no-overlap", action="store_true",
@@ -725,42 +729,60 @@ def sharded_arm(args, cfg, mode, gamma, rank, local_rank, world, device):
     from paper_2406_17918_b200 import replicas, sharded
 
     theta = 32 if args.theta is None else args.theta
+    # With one process, --local-ranks R runs R ranks of a sharded job on this GPU, phase by phase (nothing waits
+    # on anything): what the protocol and the owners' merged serving cost and save can be measured without R GPUs.
+    R = max(1, args.local_ranks) if world == 1 else 1
+    vworld = world * R
     g = build_graph(cfg, device=device)
     N = cfg["num_nodes"]
-    lo, hi = sharded.shard_range(N, rank, world)
-    ip, idx = sharded.shard_csr(g.indptr, g.indices, rank, world)
     num_edges = g.num_edges
-    del g
-    X = build_features(cfg, device=device, row_range=(lo, hi))
     perm = seed_permutation(cfg, device=device)
     B, L = cfg["batch"], len(cfg["fanouts"])
     bound = B
     for k in range(L - 1):
         bound = min(N, bound * (1 + cfg["fanouts"][L - 1 - k]))
-    me = sharded.ShardRank(gs, rank, world, ip, idx, X, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED, cfg["shared"],
-                           theta, max_seeds=B, max_requests=bound)
+    shards = [sharded.shard_csr(g.indptr, g.indices, rank * R + j, vworld) for j in range(R)]
+    del g
+    mine = []
+    for j, (ip, idx) in enumerate(shards):
+        X = build_features(cfg, device=device, row_range=sharded.shard_range(N, rank * R + j, vworld))
+        mine.append(sharded.ShardRank(gs, rank * R + j, vworld, ip, idx, X, cfg["fanouts"], cfg["cache_width"], SAMPLER_SEED,
+                                      cfg["shared"], theta, max_seeds=B, max_requests=bound))
+    del shards
+    me = mine[0]
     gm = {"otf": gs.GS_MODE_OTF, "fcr": gs.GS_MODE_FCR, "fbl": gs.GS_MODE_FBL, "fetch": gs.GS_MODE_OTF_FETCH}[mode]
     K, Wm = args.steps, args.warmup
 
     # The feature step: a round trip like a hop (ids out, rows back, reordered), or one kernel that loads every
     # row straight from its owner's memory.  The latter needs the peers' feature shards mapped into this
-    # process; with one rank the only "peer" is this GPU.
+    # process; with one process every "peer" is this GPU.
     feat = args.feature_exchange or ("peer" if world == 1 else "roundtrip")
     if feat == "peer" and world > 1:
         raise SystemExit("--feature-exchange peer needs the peers' feature shards mapped into every process: not set up by this script")
 
     def one(step):
-        seeds = batch_seeds(perm, step, B, rank, world)
+        """-> (edges, input rows) of this process's batches of the step"""
         if world > 1:
-            return sharded.sample_batch(me, seeds, gm, gamma, step)
-        return sharded.sample_batch_local([me], [seeds], gm, gamma, step, features="peer" if feat == "peer" else True)[0]
+            blocks, frontier, n, m, feats = sharded.sample_batch(me, batch_seeds(perm, step, B, rank, world), gm, gamma, step)
+            return sum(m), n[L]
+        res = sharded.sample_batch_local(mine, [batch_seeds(perm, step, B, j, R) for j in range(R)], gm, gamma, step,
+                                         features="peer" if feat == "peer" else True)
+        return sum(sum(r[3]) for r in res), sum(r[2][L] for r in res)
+
+    def largest_groups(seen):
+        for r in mine:
+            got = list(r.seen)
+            if len(got) == L:                      # no feature request was bucketed (rows are pulled): size the output instead
+                got.append((r.n[L] + vworld - 1) // vworld)
+            seen = [max(a, b) for a, b in zip(seen, got)]
+        return seen
 
     # Warm-up with exact-size exchanges (the host reads the group sizes of every exchange): the largest group
     # seen sizes the segments of the fixed-capacity exchanges the timed batches use (+25 %, the same on every rank).
     seen = [0] * (L + 1)
     for t in range(1, Wm + 1):
         one(t)
-        seen = [max(a, b) for a, b in zip(seen, me.seen)]
+        seen = largest_groups(seen)
     exact_ms = None
     if not args.exact_sizes:
         torch.cuda.synchronize()
@@ -768,13 +790,14 @@ def sharded_arm(args, cfg, mode, gamma, rank, local_rank, world, device):
         x0.record()
         for t in range(Wm + 1, Wm + 1 + max(3, K // 4)):
             one(t)
-            seen = [max(a, b) for a, b in zip(seen, me.seen)]
+            seen = largest_groups(seen)
         x1.record()
         torch.cuda.synchronize()
         exact_ms = replicas.aggregate(x0.elapsed_time(x1) / max(3, K // 4), [0], device)[0]
         _, seen = replicas.aggregate(0.0, seen, device, reduce="max")
         caps = [(int(c * 1.25) + 255) // 256 * 256 for c in seen]
-        me.set_capacities(caps)
+        for r in mine:
+            r.set_capacities(caps, merge=False if args.no_merge else None)
         for t in range(1, 4):
             one(Wm + K + t)
     clocks = ClockSampler(local_rank) if rank == 0 else None
@@ -787,9 +810,9 @@ def sharded_arm(args, cfg, mode, gamma, rank, local_rank, world, device):
     edges = rows = 0
     e0.record()
     for t in range(2 * Wm + K + 4, 2 * Wm + 2 * K + 4):
-        blocks, frontier, n, m, feats = one(t)
-        edges += sum(m)
-        rows += n[L]
+        em, rn = one(t)
+        edges += em
+        rows += rn
     e1.record()
     torch.cuda.synchronize()
     replicas.barrier()
@@ -810,7 +833,11 @@ def sharded_arm(args, cfg, mode, gamma, rank, local_rank, world, device):
                        "cache_width": cfg["cache_width"], "mode": mode, "gamma": gamma, "batch": B, "theta": theta,
                        "shared_cache": cfg["shared"], "feat_dim": cfg["feat_dim"],
                        "parallelism": "node-sharded x%d (one all-to-all round trip per hop%s)"
-                                      % (world, "" if world > 1 else "; 1 rank: local copy"),
+                                      % (vworld, "" if world > 1 else "; %d rank(s) in one process on one GPU, phase by phase: "
+                                                                        "the exchange is a local copy" % R),
+                       "ms_per_batch": t_ms / K / R,
+                       "owner_serving": None if me.caps is None else
+                                        ("requesters' lists merged, distinct nodes sampled once" if me.merge else "list by list"),
                        "exchange": "exact sizes (one host read per exchange)" if me.caps is None else
                                    "fixed capacity per pair of ranks %s, no host read inside a batch" % me.caps,
                        "ms_per_step_exact_sizes": exact_ms,

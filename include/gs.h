@@ -346,6 +346,22 @@ gs_status gs_shard_sample_rows_counted(gs_cache*, const int32_t* d_nodes, const 
                                        void* stream, int32_t* d_picks);
 gs_status gs_shard_status(gs_cache*, void* stream);
 
+/* Owner side, all requesters' fixed-pitch lists at once (d_lists[world][capacity], lengths d_counts[world], as
+ * they arrive from the exchange): a node that several requesters ask for - every hub - is sampled once.
+ * gs_shard_merge gives every requested node one place in d_distinct (at most min(world*capacity, rows_owned)
+ * ids, in no particular order); d_num_distinct: int32[2] on the device, [0] = how many, [1] = 0 or GS_ERR_RANGE
+ * (an id outside the rows this shard owns, [first_row, first_row + rows_owned); such entries are skipped).
+ * d_index: int32[rows_owned], owned by the caller, all -1 before the first call; it holds the nodes' places
+ * until gs_shard_fan_out has run.  Then gs_shard_sample_rows_counted(d_distinct, d_num_distinct, ...) samples the
+ * distinct nodes into d_rows[..][fanout], and gs_shard_fan_out copies every list entry's row to
+ * d_out[world*capacity][fanout] (the reply at the lists' pitch) and puts d_index back to all -1.  The rows are
+ * the ones the per-list calls give: picks are keyed by (node, step), not by who asks. */
+gs_status gs_shard_merge(const int32_t* d_lists, const int32_t* d_counts, int32_t world, int32_t capacity, int64_t first_row,
+                         int64_t rows_owned, int32_t* d_index, int32_t* d_distinct, int32_t* d_num_distinct, void* stream);
+gs_status gs_shard_fan_out(const int32_t* d_lists, const int32_t* d_counts, int32_t world, int32_t capacity, int64_t first_row,
+                           int64_t rows_owned, int32_t* d_index, const int32_t* d_distinct, const int32_t* d_num_distinct,
+                           const int32_t* d_rows, int32_t fanout, int32_t* d_out, void* stream);
+
 /* Requester side, hop k = 0 .. num_hops-1 in order.  d_reply[n_k][fanout(L-1-k)]: the owners' rows
  * in d_sorted order; d_slot[n_k] as returned by gs_shard_bucket for frontier_k.  k = 0 starts a new
  * batch and takes the seeds (distinct, as for gs_sample_batch); later hops ignore d_seeds and

@@ -95,6 +95,8 @@ def _load():
         "gs_shard_sample_rows": [vp, vp, i32, i32, ctypes.c_int, dbl, u32, vp, sz, vp, vp],
         "gs_shard_sample_rows_counted": [vp, vp, vp, i32, i32, ctypes.c_int, dbl, u32, vp, sz, vp, vp],
         "gs_shard_status": [vp, vp],
+        "gs_shard_merge": [vp, vp, i32, i32, i64, i64, vp, vp, vp, vp],
+        "gs_shard_fan_out": [vp, vp, i32, i32, i64, i64, vp, vp, vp, vp, i32, vp, vp],
         "gs_shard_extend": [vp, i32, vp, i32, vp, vp, vp, sz, vp, vp, pvp],
         "gs_shard_extend_fixed": [vp, i32, vp, i32, vp, i32, vp, vp, sz, vp, vp, pvp],
         "gs_batch_stats": [vp, vp, vp],
@@ -489,6 +491,39 @@ def gs_shard_sample_rows(cache: Cache, nodes: torch.Tensor, layer: int, mode: in
                                                float(rate), step, _ptr(workspace), workspace.numel(), _stream(stream),
                                                _ptr(picks)))
     return picks
+
+
+def _i32_cuda(*tensors):
+    for t in tensors:
+        if t.dtype != torch.int32 or not t.is_cuda or not t.is_contiguous():
+            raise TypeError("contiguous int32 CUDA tensors expected")
+
+
+def gs_shard_merge(lists: torch.Tensor, counts: torch.Tensor, world: int, first_row: int, index: torch.Tensor,
+                   distinct: torch.Tensor, num_distinct: torch.Tensor, stream=None):
+    """Owner side: one place in `distinct` for every node any of the `world` fixed-pitch lists asks for.
+    index: int32[rows owned], all -1 between batches; num_distinct: int32[2] (count, status word)."""
+    _i32_cuda(lists, counts, index, distinct, num_distinct)
+    capacity = lists.numel() // int(world)
+    if lists.numel() != capacity * world or counts.numel() < world or num_distinct.numel() < 2 or \
+            distinct.numel() < min(lists.numel(), index.numel()):
+        raise ValueError("bad tensor sizes")
+    _check(_L.gs_shard_merge(_ptr(lists), _ptr(counts), int(world), capacity, int(first_row), index.numel(), _ptr(index),
+                             _ptr(distinct), _ptr(num_distinct), _stream(stream)))
+    return distinct, num_distinct
+
+
+def gs_shard_fan_out(lists: torch.Tensor, counts: torch.Tensor, world: int, first_row: int, index: torch.Tensor,
+                     distinct: torch.Tensor, num_distinct: torch.Tensor, rows: torch.Tensor, out: torch.Tensor, stream=None):
+    """out[e] = rows[place of lists[e]] for every entry of every list; puts `index` back to all -1."""
+    _i32_cuda(lists, counts, index, distinct, num_distinct, rows, out)
+    capacity = lists.numel() // int(world)
+    f = rows.shape[1]
+    if out.numel() < lists.numel() * f or rows.shape[0] < min(lists.numel(), index.numel()) or distinct.numel() < min(lists.numel(), index.numel()):
+        raise ValueError("bad tensor sizes")
+    _check(_L.gs_shard_fan_out(_ptr(lists), _ptr(counts), int(world), capacity, int(first_row), index.numel(), _ptr(index),
+                               _ptr(distinct), _ptr(num_distinct), _ptr(rows), int(f), _ptr(out), _stream(stream)))
+    return out
 
 
 def gs_shard_status(cache: Cache, stream=None):

@@ -817,6 +817,39 @@ gs_status gs_shard_sample_rows_counted(gs_cache* c, const int32_t* d_nodes, cons
     return shard_sample_rows_impl(c, d_nodes, d_n, n_bound, layer, mode, rate, step, d_workspace, workspace_bytes, stream, d_picks);
 }
 
+static gs_status check_merge_args(const int32_t* d_lists, const int32_t* d_counts, int32_t world, int32_t capacity,
+                                  int64_t first_row, int64_t rows_owned, const int32_t* d_index, const int32_t* d_distinct) {
+    if (world < 1 || world > 64) return fail(GS_ERR_ARG, "world %d outside [1, 64]", world);
+    if (capacity < 1 || (int64_t)capacity * world >= ((int64_t)1 << 31)) return fail(GS_ERR_ARG, "capacity outside [1, 2^31 / world)");
+    if (first_row < 0 || rows_owned < 1 || first_row + rows_owned > ((int64_t)1 << 31)) return fail(GS_ERR_ARG, "bad row range");
+    if (!d_lists || !d_counts || !d_index || !d_distinct) return fail(GS_ERR_ARG, "NULL argument");
+    return GS_OK;
+}
+
+gs_status gs_shard_merge(const int32_t* d_lists, const int32_t* d_counts, int32_t world, int32_t capacity, int64_t first_row,
+                         int64_t rows_owned, int32_t* d_index, int32_t* d_distinct, int32_t* d_num_distinct, void* stream) {
+    gs_status st = check_merge_args(d_lists, d_counts, world, capacity, first_row, rows_owned, d_index, d_distinct);
+    if (st != GS_OK) return st;
+    if (!d_num_distinct) return fail(GS_ERR_ARG, "d_num_distinct is NULL");
+    GS_CUDA(launch_shard_merge(d_lists, d_counts, world, capacity, first_row, rows_owned, d_index, d_distinct, d_num_distinct,
+                               (cudaStream_t)stream));
+    return GS_OK;
+}
+
+gs_status gs_shard_fan_out(const int32_t* d_lists, const int32_t* d_counts, int32_t world, int32_t capacity, int64_t first_row,
+                           int64_t rows_owned, int32_t* d_index, const int32_t* d_distinct, const int32_t* d_num_distinct,
+                           const int32_t* d_rows, int32_t fanout, int32_t* d_out, void* stream) {
+    gs_status st = check_merge_args(d_lists, d_counts, world, capacity, first_row, rows_owned, d_index, d_distinct);
+    if (st != GS_OK) return st;
+    if (!d_num_distinct || !d_rows || !d_out) return fail(GS_ERR_ARG, "NULL argument");
+    if (fanout < 1 || fanout > GS_MAX_CACHE_WIDTH) return fail(GS_ERR_ARG, "fanout %d outside [1, %d]", fanout, GS_MAX_CACHE_WIDTH);
+    int64_t bound = (int64_t)world * capacity;
+    if (bound > rows_owned) bound = rows_owned;
+    GS_CUDA(launch_shard_fan_out(d_lists, d_counts, world, capacity, first_row, rows_owned, d_index, d_distinct, (int32_t)bound,
+                                 d_rows, d_num_distinct, fanout, d_out, (cudaStream_t)stream));
+    return GS_OK;
+}
+
 gs_status gs_shard_status(gs_cache* c, void* stream) {
     if (!c) return fail(GS_ERR_ARG, "cache is NULL");
     cudaStream_t s = (cudaStream_t)stream;

@@ -326,6 +326,11 @@ cudaError_t launch_export_picks(const int32_t* blk_indptr, const int32_t* picked
 cudaError_t launch_import_picks(const int32_t* hdr, int32_t k, int32_t n_bound, int32_t f, const int32_t* reply,
                                 int32_t reply_rows, const int32_t* slot, const int32_t* blk_indptr, int32_t* picked, unsigned long long* table,
                                 uint32_t stamp, int64_t num_nodes, int32_t* status, cudaStream_t s);
+cudaError_t launch_shard_merge(const int32_t* lists, const int32_t* counts, int32_t world, int32_t capacity, int64_t first_row,
+                               int64_t rows_owned, int32_t* index, int32_t* distinct, int32_t* out_words, cudaStream_t s);
+cudaError_t launch_shard_fan_out(const int32_t* lists, const int32_t* counts, int32_t world, int32_t capacity, int64_t first_row,
+                                 int64_t rows_owned, int32_t* index, const int32_t* distinct, int32_t distinct_bound,
+                                 const int32_t* rows, const int32_t* d_num_rows, int32_t f, int32_t* out, cudaStream_t s);
 cudaError_t launch_build_row_index(const GraphView& g, int32_t theta, int32_t* row_index, int32_t* tile_sums,
                                    int32_t* d_dense_rows, cudaStream_t s);
 

@@ -176,4 +176,105 @@ cudaError_t launch_import_picks(const int32_t* hdr, int32_t k, int32_t n_bound, 
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------- owner side: all requesters' lists at once
+// A hub sits in every requester's frontier, and serving the lists one by one scans its row once per requester.
+// The lists (fixed pitch, lengths on the device) are merged instead: every owned node that anyone asks for
+// gets one position in a list of distinct nodes (`index`, one word per owned row, -1 = not asked for), that
+// list is sampled once, and the rows are fanned out to the requesters' segments.  Same rows either way:
+// picks are keyed by (node, step), not by who asks.
+__global__ void __launch_bounds__(SHARD_THREADS) k_merge_claim(const int32_t* __restrict__ lists,
+                                                               const int32_t* __restrict__ counts, int world, int capacity,
+                                                               int64_t first_row, int64_t rows_owned, int32_t* index,
+                                                               int32_t* __restrict__ distinct, int32_t* out_words) {
+    __shared__ int s_new, s_base;
+    const int64_t total = (int64_t)world * capacity;
+    for (int64_t e0 = (int64_t)blockIdx.x * SHARD_THREADS; e0 < total; e0 += (int64_t)gridDim.x * SHARD_THREADS) {
+        if (threadIdx.x == 0) s_new = 0;
+        __syncthreads();
+        const int64_t e = e0 + threadIdx.x;
+        int32_t v = -1;
+        int64_t loc = -1;
+        int rank = -1;
+        if (e < total) {
+            const int r = (int)(e / capacity), i = (int)(e - (int64_t)r * capacity);
+            if (i < min(max(__ldg(counts + r), 0), capacity)) {
+                v = __ldg(lists + e);
+                loc = (int64_t)v - first_row;
+                if (loc < 0 || loc >= rows_owned) {
+                    atomicCAS(out_words + 1, 0, GS_ERR_RANGE);
+                    loc = -1;
+                } else if (atomicCAS(index + loc, -1, -2) == -1) {
+                    rank = atomicAdd(&s_new, 1);          // the first to ask for this node places it
+                }
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) s_base = s_new ? atomicAdd(out_words, s_new) : 0;
+        __syncthreads();
+        if (rank >= 0) {
+            distinct[s_base + rank] = v;
+            index[loc] = s_base + rank;
+        }
+        __syncthreads();   // s_new and s_base are reused by the next round
+    }
+}
+
+// out[e][:] = rows[index[node of entry e]][:] for every entry of every requester's list.
+__global__ void __launch_bounds__(SHARD_THREADS) k_fan_out(const int32_t* __restrict__ lists, const int32_t* __restrict__ counts,
+                                                           int world, int capacity, int64_t first_row, int64_t rows_owned,
+                                                           const int32_t* __restrict__ index, const int32_t* __restrict__ rows,
+                                                           const int32_t* __restrict__ d_num_rows, int f,
+                                                           int32_t* __restrict__ out) {
+    const int num_rows = __ldcg(d_num_rows);
+    const unsigned long long total = (unsigned long long)world * capacity * (unsigned)f;
+    for (unsigned long long i = (unsigned long long)blockIdx.x * SHARD_THREADS + threadIdx.x; i < total;
+         i += (unsigned long long)gridDim.x * SHARD_THREADS) {
+        unsigned e, t;
+        split_pair(i, (unsigned)f, e, t);
+        const unsigned r = e / (unsigned)capacity, j = e - r * (unsigned)capacity;
+        if ((int)j >= min(max(__ldg(counts + r), 0), capacity)) continue;
+        const int64_t loc = (int64_t)__ldg(lists + e) - first_row;
+        if (loc < 0 || loc >= rows_owned) continue;        // reported by the merge
+        const int pos = __ldcg(index + loc);
+        out[i] = ((unsigned)pos < (unsigned)num_rows) ? __ldg(rows + (int64_t)pos * f + t) : -1;
+    }
+}
+
+// The index goes back to "nobody asks" for exactly the nodes that were placed.
+__global__ void __launch_bounds__(SHARD_THREADS) k_merge_reset(const int32_t* __restrict__ distinct,
+                                                               const int32_t* __restrict__ d_num, int bound, int64_t first_row,
+                                                               int64_t rows_owned, int32_t* index) {
+    const int n = min(bound, max(0, __ldcg(d_num)));
+    for (int j = blockIdx.x * SHARD_THREADS + threadIdx.x; j < n; j += gridDim.x * SHARD_THREADS) {
+        const int64_t loc = (int64_t)__ldg(distinct + j) - first_row;
+        if (loc >= 0 && loc < rows_owned) index[loc] = -1;
+    }
+}
+
+cudaError_t launch_shard_merge(const int32_t* lists, const int32_t* counts, int32_t world, int32_t capacity, int64_t first_row,
+                               int64_t rows_owned, int32_t* index, int32_t* distinct, int32_t* out_words, cudaStream_t s) {
+    cudaError_t e = cudaMemsetAsync(out_words, 0, 2 * sizeof(int32_t), s);
+    if (e != cudaSuccess) return e;
+    int64_t blocks = ((int64_t)world * capacity + SHARD_THREADS - 1) / SHARD_THREADS;
+    const int64_t cap = sm_count() * 16;
+    blocks = limit_grid(blocks < cap ? (blocks < 1 ? 1 : blocks) : cap);
+    k_merge_claim<<<(unsigned)blocks, SHARD_THREADS, 0, s>>>(lists, counts, world, capacity, first_row, rows_owned, index,
+                                                             distinct, out_words);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_shard_fan_out(const int32_t* lists, const int32_t* counts, int32_t world, int32_t capacity, int64_t first_row,
+                                 int64_t rows_owned, int32_t* index, const int32_t* distinct, int32_t distinct_bound,
+                                 const int32_t* rows, const int32_t* d_num_rows, int32_t f, int32_t* out, cudaStream_t s) {
+    k_fan_out<<<pair_grid((int64_t)world * capacity, f), SHARD_THREADS, 0, s>>>(lists, counts, world, capacity, first_row,
+                                                                               rows_owned, index, rows, d_num_rows, f, out);
+    int64_t blocks = ((int64_t)distinct_bound + SHARD_THREADS - 1) / SHARD_THREADS;
+    const int64_t cap = sm_count() * 16;
+    blocks = limit_grid(blocks < cap ? (blocks < 1 ? 1 : blocks) : cap);
+    k_merge_reset<<<(unsigned)blocks, SHARD_THREADS, 0, s>>>(distinct, d_num_rows, distinct_bound, first_row, rows_owned, index);
+    count_launches(2);
+    return cudaGetLastError();
+}
+
 }  // namespace gs

@@ -150,9 +150,14 @@ class ShardRank:
     # replies come back at the same pitch.  The exchanges are equal-split all-to-alls of pre-allocated buffers,
     # so a batch has no host synchronisation before finish_batch.  A group that outgrows its segment is a
     # device-detected error of the batch (reported by finish_batch), never an overrun.
-    def set_capacities(self, caps):
+    def set_capacities(self, caps, merge=None):
         """caps[0..L-1]: ids per (requester, owner) pair at each hop; caps[L]: at the feature request (omit or 0
-        when features are pulled from peer memory).  Every rank must use the same values."""
+        when features are pulled from peer memory).  Every rank must use the same values.
+        merge: the owner merges the requesters' lists of a hop and samples every distinct node once (a hub sits
+        in every requester's frontier) instead of serving the lists one by one; same rows either way.  Default: with
+        more than one rank (with one there is nothing to merge, only the cost of doing it)."""
+        if merge is None:
+            merge = self.world > 1
         caps = [int(c) for c in caps] + [0] * (self.L + 1 - len(caps))
         if len(caps) != self.L + 1 or min(caps[: self.L]) < 1:
             raise ValueError("one positive capacity per hop (and optionally one for the features) expected")
@@ -164,6 +169,19 @@ class ShardRank:
             self.ws_owner = torch.empty(self.ops.gs_shard_workspace_bytes(self.graph, max(self.fanouts), need),
                                         dtype=torch.uint8, device=dev)
         i32 = dict(dtype=torch.int32, device=dev)
+        lo, hi = shard_range(self.num_nodes, self.rank, self.world)
+        self.merge = bool(merge) and hi > lo
+        if self.merge:
+            D = min(R * max(caps[: self.L]), hi - lo)          # distinct nodes a hop can ask this owner for
+            if D > self.max_requests:
+                self.max_requests = D
+                self.ws_owner = torch.empty(self.ops.gs_shard_workspace_bytes(self.graph, max(self.fanouts), D),
+                                            dtype=torch.uint8, device=dev)
+            self.merge_index = torch.full((hi - lo,), -1, **i32)
+            self.merge_distinct = torch.empty(D, **i32)
+            self.merge_rows = torch.empty(D * max(self.fanouts), **i32)
+            self.merge_num = torch.zeros((self.L, 2), **i32)   # per hop: distinct nodes, status word
+            self.merge_host = torch.zeros((self.L, 2), dtype=torch.int32, pin_memory=dev.type == "cuda")
         self.counts_all = torch.zeros((self.L + 1, 2 * R + 1), **i32)
         self.counts_host = torch.zeros((self.L + 1, 2 * R + 1), dtype=torch.int32, pin_memory=dev.type == "cuda")
         self.fx = []
@@ -215,6 +233,15 @@ class ShardRank:
     def hop_serve_fixed(self, layer, recv, recv_counts, mode, rate, step, out):
         """recv [world * C] ids, requester r's list in segment r, its length recv_counts[r] -> out [world * C, f]."""
         C = recv.numel() // self.world
+        if self.merge:
+            f = self.fanouts[layer]
+            D = min(recv.numel(), self.merge_index.numel())
+            distinct, num = self.merge_distinct[:D], self.merge_num[self.L - 1 - layer]
+            rows = self.merge_rows[: D * f].view(D, f)
+            self.ops.gs_shard_merge(recv, recv_counts, self.world, self.first_row, self.merge_index, distinct, num)
+            self.ops.gs_shard_sample_rows(self.cache, distinct, layer, mode, rate, step, self.ws_owner, picks=rows, count=num[0:1])
+            self.ops.gs_shard_fan_out(recv, recv_counts, self.world, self.first_row, self.merge_index, distinct, num, rows, out)
+            return out
         for r in range(self.world):
             self.ops.gs_shard_sample_rows(self.cache, recv[r * C:(r + 1) * C], layer, mode, rate, step, self.ws_owner,
                                           picks=out[r * C:(r + 1) * C], count=recv_counts[r:r + 1])
@@ -235,7 +262,11 @@ class ShardRank:
     def finish_batch_fixed(self):
         """Counts, device status and the bucket calls' error words of the batch, read once (synchronises)."""
         self.counts_host.copy_(self.counts_all, non_blocking=True)
-        self.finish_batch()                        # synchronises the stream the copy above is on
+        if self.merge:
+            self.merge_host.copy_(self.merge_num, non_blocking=True)
+        self.finish_batch()                        # synchronises the stream the copies above are on
+        if self.merge and any(self.merge_host[:, 1].tolist()):
+            raise ValueError("a requested node id is not a row of this shard")
         if self.feat_bound is not None and self.n[self.L] > self.feat_bound:
             raise RuntimeError("%d input nodes, feature rows were allocated for %d" % (self.n[self.L], self.feat_bound))
         words = self.counts_host[:, 2 * self.world].tolist()

@@ -104,6 +104,37 @@ def gs_shard_sample_rows(cache, nodes, layer, mode, rate, step, ws, picks=None, 
     return torch.from_numpy(out)
 
 
+def gs_shard_merge(lists, counts, world, first_row, index, distinct, num_distinct):
+    C = lists.numel() // world
+    L, cnt, idx = lists.numpy(), counts.numpy(), index.numpy()
+    assert (idx == -1).all()
+    n, bad = 0, 0
+    for r in range(world):
+        for v in L[r * C: r * C + min(int(cnt[r]), C)].tolist():
+            loc = v - first_row
+            if loc < 0 or loc >= len(idx):
+                bad = 3
+            elif idx[loc] < 0:
+                idx[loc] = n
+                distinct[n] = v
+                n += 1
+    num_distinct[0], num_distinct[1] = n, bad
+    return distinct, num_distinct
+
+
+def gs_shard_fan_out(lists, counts, world, first_row, index, distinct, num_distinct, rows, out):
+    C = lists.numel() // world
+    L, cnt, idx = lists.numpy(), counts.numpy(), index.numpy()
+    for r in range(world):
+        for i in range(min(int(cnt[r]), C)):
+            loc = L[r * C + i] - first_row
+            if 0 <= loc < len(idx):
+                out[r * C + i] = rows[idx[loc]]
+    for v in distinct[: int(num_distinct[0])].tolist():
+        idx[v - first_row] = -1
+    return out
+
+
 def gs_shard_status(cache):
     pass
 

@@ -37,8 +37,8 @@ class Setup:
                                                 cfg["fanouts"], cfg["cache_width"], seed, cfg["shared"], theta,
                                                 max_seeds=self.B, max_requests=min(N, self.B * 400)))
         if fixed:   # fixed-capacity exchanges; a group holds distinct nodes of one owner, so a shard's size always suffices
-            for r in self.ranks:
-                r.set_capacities([sharded.rows_per_shard(N, world)] * (len(cfg["fanouts"]) + 1))
+            for r in self.ranks:    # owners merge the requesters' lists unless fixed == "lists"
+                r.set_capacities([sharded.rows_per_shard(N, world)] * (len(cfg["fanouts"]) + 1), merge=fixed != "lists")   # merged serving also with one rank, for coverage
         self.O = oracle.Sampler(self.indptr, self.indices, cfg["fanouts"], cfg["cache_width"], seed, cfg["shared"])
         self.O.set_theta(theta)
 
@@ -80,7 +80,7 @@ class Setup:
                 assert np.array_equal(got, want[(nodes // S) == r]), (layer, r)
 
 
-@pytest.mark.parametrize("fixed", [False, True])
+@pytest.mark.parametrize("fixed", [False, True, "lists"])
 @pytest.mark.parametrize("world", [1, 2, 3])
 def test_sharded_tiny_all_modes(world, fixed):
     s = Setup("tiny", world, theta=12, fixed=fixed)
@@ -221,6 +221,51 @@ def test_bucket_and_gather_rows_primitives():
         gs.gs_gather_rows_peer([parts[0].data_ptr(), 0, parts[2].data_ptr()], 1000, torch.bfloat16, 24, 24, ids, out)
 
 
+def test_merge_and_fan_out_primitives():
+    import paper_2406_17918_b200 as gs
+    rng = np.random.default_rng(21)
+    world, C, first, owned, f = 4, 5000, 70000, 30011, 7
+    lists = torch.full((world * C,), -3, dtype=torch.int32)
+    cnt = [4100, 0, 5000, 777]
+    hot = rng.choice(owned, 600, replace=False) + first                       # nodes every requester asks for
+    for r in range(world):
+        rest = rng.choice(owned, cnt[r], replace=False) + first
+        v = np.unique(np.concatenate([hot[: min(600, cnt[r])], rest]))[: cnt[r]] if cnt[r] else rest
+        lists[r * C: r * C + cnt[r]] = torch.from_numpy(rng.permutation(v).astype(np.int32))
+    lists_d, counts = lists.cuda(), torch.tensor(cnt, dtype=torch.int32, device="cuda")
+    index = torch.full((owned,), -1, dtype=torch.int32, device="cuda")
+    D = min(world * C, owned)
+    distinct = torch.empty(D, dtype=torch.int32, device="cuda")
+    num = torch.zeros(2, dtype=torch.int32, device="cuda")
+    gs.gs_shard_merge(lists_d, counts, world, first, index, distinct, num)
+    asked = np.unique(np.concatenate([lists.numpy()[r * C: r * C + cnt[r]] for r in range(world)]))
+    n = int(num[0].item())
+    got = distinct[:n].cpu().numpy()
+    assert int(num[1].item()) == 0 and n == len(asked) and np.array_equal(np.sort(got), asked)
+    idx = index.cpu().numpy()
+    assert np.array_equal(idx[got - first], np.arange(n)) and (np.delete(idx, asked - first) == -1).all()
+    rows = torch.from_numpy(rng.integers(0, 1 << 30, (D, f)).astype(np.int32)).cuda()
+    out = torch.full((world * C, f), -8, dtype=torch.int32, device="cuda")
+    gs.gs_shard_fan_out(lists_d, counts, world, first, index, distinct, num, rows, out)
+    want = np.full((world * C, f), -8, dtype=np.int32)
+    rows_h = rows.cpu().numpy()
+    for r in range(world):
+        ids = lists.numpy()[r * C: r * C + cnt[r]]
+        want[r * C: r * C + cnt[r]] = rows_h[idx[ids - first]]
+    assert np.array_equal(out.cpu().numpy(), want)
+    assert bool((index == -1).all())                                            # ready for the next hop
+    # an id this shard does not own: reported, skipped, the others are placed
+    bad = lists_d.clone()
+    bad[3] = first + owned
+    gs.gs_shard_merge(bad, counts, world, first, index, distinct, num)
+    assert num.cpu().tolist() == [len(asked) - 1 if lists[3].item() not in np.concatenate(
+        [lists.numpy()[r * C: r * C + cnt[r]] for r in range(1, world)] + [lists.numpy()[:3], lists.numpy()[4:cnt[0]]]) else len(asked), 3]
+    gs.gs_shard_fan_out(bad, counts, world, first, index, distinct, num, rows, out)
+    assert bool((index == -1).all())
+    with pytest.raises(gs.GsError):
+        gs.gs_shard_merge(lists_d[: 65 * 300], torch.zeros(65, dtype=torch.int32, device="cuda"), 65, first, index, distinct, num)
+
+
 def test_sharded_entry_points_reject_bad_arguments():
     import paper_2406_17918_b200 as gs
     s = Setup("tiny", 2, theta=12)
@@ -304,7 +349,7 @@ def test_randomised_sharded_runs(case):
         ranks.append(sharded.ShardRank(gs, r, world, ip.cuda(), idx.cuda(), X[lo:hi].cuda().contiguous(), fanouts, W, seed,
                                        shared, theta, max_seeds=B, max_requests=n))
         if case % 2:            # odd cases: fixed-capacity exchanges (a shard's size always holds a group)
-            ranks[-1].set_capacities([sharded.rows_per_shard(n, world)] * (L + 1))
+            ranks[-1].set_capacities([sharded.rows_per_shard(n, world)] * (L + 1), merge=case % 4 == 1)
         # the requester's dedup + relabel with each way of finding first occurrences
         gs.gs_cache_set_dedup(ranks[-1].cache, [gs.GS_DEDUP_AUTO, gs.GS_DEDUP_HASH, gs.GS_DEDUP_SORT, gs.GS_DEDUP_DIRECT][(case // 2) % 4])
     O = oracle.Sampler(indptr, indices, fanouts, W, seed, shared)

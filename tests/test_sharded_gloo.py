@@ -41,7 +41,7 @@ def _worker(rank, world, port, out_dir, capacity=None):
     me = sharded.ShardRank(ops, rank, world, ip, idx, X[lo:hi].contiguous(), cfg["fanouts"], cfg["cache_width"], SEED,
                            cfg["shared"], THETA, max_seeds=cfg["batch"], max_requests=cfg["num_nodes"])
     if capacity:            # fixed-capacity exchanges: no size is read on the host inside a batch
-        me.set_capacities([capacity] * (len(cfg["fanouts"]) + 1))
+        me.set_capacities([abs(capacity)] * (len(cfg["fanouts"]) + 1), merge=capacity > 0)
     out = []
     t = 1
     for mode, rate in [(ops.GS_MODE_OTF, 0.25), (ops.GS_MODE_OTF, 0.25), (ops.GS_MODE_FCR, 0.0), (ops.GS_MODE_OTF_FETCH, 0.5),
@@ -58,10 +58,11 @@ def _worker(rank, world, port, out_dir, capacity=None):
     dist.destroy_process_group()
 
 
-@pytest.mark.parametrize("world,capacity", [(2, None), (3, None), (2, 1500), (3, 920)])
+@pytest.mark.parametrize("world,capacity", [(2, None), (3, None), (2, 1500), (3, 920), (3, -920)])
 def test_ranks_equal_one_sampler_taking_the_batches_in_turn(tmp_path, world, capacity):
     """World size 3 gives uneven shards (2,708 nodes: 903 + 903 + 902).  With a capacity the exchanges have a
-    fixed pitch (segments of that many ids per pair of ranks) and the driver reads no size inside a batch."""
+    fixed pitch (segments of that many ids per pair of ranks) and the driver reads no size inside a batch; the owners
+    merge the requesters' lists and sample every distinct node once (negative: they serve the lists one by one)."""
     mp.spawn(_worker, args=(world, _free_port(), str(tmp_path), capacity), nprocs=world, join=True)
     res = [torch.load(os.path.join(tmp_path, "r%d.pt" % r)) for r in range(world)]
     cfg = get_config("tiny")
