@@ -12,7 +12,11 @@ One hop of a rank's batch (sampling step k, layer L-1-k):
                                 <-  all-to-all(v) rows of f picks  <-
     dedup + relabel + block CSR
 
-and after the last hop one more round trip for the feature rows.  The per-rank phases live in
+and after the last hop one more round trip for the feature rows (or one kernel that pulls them from the
+owners' memory).  The exchanges come in two forms: packed groups whose sizes the host reads back for the
+all-to-all (one host sync per hop), or segments of a fixed capacity per pair of ranks whose sizes travel
+as a device array (:meth:`ShardRank.set_capacities`: no host read inside a batch; owners then merge the
+requesters' lists and sample every distinct node once).  The per-rank phases live in
 :class:`ShardRank`; two drivers run them: :func:`sample_batch` (one process per GPU, the
 exchange is ``torch.distributed.all_to_all_single`` over NCCL / NVLink) and
 :func:`sample_batch_local` (all ranks in one process, the exchange is a copy; used to check a
@@ -239,8 +243,12 @@ class ShardRank:
             distinct, num = self.merge_distinct[:D], self.merge_num[self.L - 1 - layer]
             rows = self.merge_rows[: D * f].view(D, f)
             self.ops.gs_shard_merge(recv, recv_counts, self.world, self.first_row, self.merge_index, distinct, num)
-            self.ops.gs_shard_sample_rows(self.cache, distinct, layer, mode, rate, step, self.ws_owner, picks=rows, count=num[0:1])
-            self.ops.gs_shard_fan_out(recv, recv_counts, self.world, self.first_row, self.merge_index, distinct, num, rows, out)
+            try:
+                self.ops.gs_shard_sample_rows(self.cache, distinct, layer, mode, rate, step, self.ws_owner, picks=rows,
+                                              count=num[0:1])
+            finally:    # the fan-out also clears the index: it must run even when the sampling call was refused
+                self.ops.gs_shard_fan_out(recv, recv_counts, self.world, self.first_row, self.merge_index, distinct, num,
+                                          rows, out)
             return out
         for r in range(self.world):
             self.ops.gs_shard_sample_rows(self.cache, recv[r * C:(r + 1) * C], layer, mode, rate, step, self.ws_owner,
@@ -342,15 +350,15 @@ def _sample_batch_local_fixed(ranks, mode, rate, step, features):
 
     def round_trip(k, req, serve):
         C = ranks[0].caps[k]
-        replies = [r.fx[k]["reply"] for r in ranks]
-        for o, owner in enumerate(ranks):
+        for o, owner in enumerate(ranks):                        # what the ranks send to owner o, one copy per owner
             b = owner.fx[k]
-            for r in range(R):                                   # what rank r sends to owner o
-                b["recv"][r * C:(r + 1) * C].copy_(req[r][0][o * C:(o + 1) * C])
-                b["recv_counts"][r:r + 1].copy_(req[r][1][o:o + 1])
+            torch.stack([req[r][0].view(R, C)[o] for r in range(R)], out=b["recv"].view(R, C))
+            torch.stack([req[r][1][o] for r in range(R)], out=b["recv_counts"])
             serve(owner, b["recv"], b["recv_counts"], b["out"])
-            for r in range(R):                                   # and what comes back
-                replies[r][o * C:(o + 1) * C].copy_(b["out"][r * C:(r + 1) * C])
+        replies = [r.fx[k]["reply"] for r in ranks]
+        for r in range(R):                                       # and what comes back, one copy per requester
+            width = replies[r].shape[1]
+            torch.stack([ranks[o].fx[k]["out"].view(R, C, width)[r] for o in range(R)], out=replies[r].view(R, C, width))
         return replies
 
     for k in range(L):
