@@ -55,7 +55,7 @@ def test_large_split_cache_whole_batch_then_whole_cache_refresh():
     assert (gs.gs_cache_read_rows(C, 0, torch.from_numpy(sparse).cuda()).cpu().numpy() == -1).all()
 
 
-def test_large_two_shards_one_step():
+def test_large_two_shards_two_steps():
     """Node-sharded sampling at full size: two ranks run phase by phase on this GPU; each rank's whole
     batch must equal what one sampler (theta = 32) gives when it takes the two batches in turn."""
     import paper_2406_17918_b200 as gs
@@ -74,18 +74,26 @@ def test_large_two_shards_one_step():
                                        cfg["cache_width"], seed, False, theta, max_seeds=B, max_requests=B * 6 * 11))
     O = oracle.Sampler(g.indptr.numpy(), g.indices.numpy(), cfg["fanouts"], cfg["cache_width"], seed, False)
     O.set_theta(theta)
-    seeds = [batch_seeds(perm, 1, B, r, world) for r in range(world)]
-    res = sharded.sample_batch_local(ranks, [s.cuda() for s in seeds], gs.GS_MODE_OTF, 0.2, 1)
-    for r in range(world):
-        blocks, frontier, n, m, feats = res[r]
-        fr_o, n_o, blocks_o = O.sample_batch(seeds[r].numpy(), oracle.MODE_OTF, 0.2, 1)
-        assert n == n_o
-        assert np.array_equal(frontier[: n[L]].cpu().numpy(), fr_o)
-        for layer in range(L):
-            k = L - 1 - layer
-            assert np.array_equal(blocks[layer].indptr(n[k]).cpu().numpy(), blocks_o[layer].indptr)
-            assert np.array_equal(blocks[layer].indices(m[layer]).cpu().numpy(), blocks_o[layer].indices)
-        assert torch.equal(feats[:, 0].cpu(), torch.from_numpy(fr_o.astype(np.float32)))
+    for step in (1, 2):
+        if step == 2:
+            # the second step with fixed-capacity exchanges sized from the first one, the owners merging the two
+            # requesters' lists, and rank 1 finding first occurrences with the hash table
+            seen = np.max([r.seen for r in ranks], axis=0)
+            for r in ranks:
+                r.set_capacities([int(c * 1.3) + 64 for c in seen], merge=True)
+            gs.gs_cache_set_dedup(ranks[1].cache, gs.GS_DEDUP_HASH)
+        seeds = [batch_seeds(perm, step, B, r, world) for r in range(world)]
+        res = sharded.sample_batch_local(ranks, [s.cuda() for s in seeds], gs.GS_MODE_OTF, 0.2, step)
+        for r in range(world):
+            blocks, frontier, n, m, feats = res[r]
+            fr_o, n_o, blocks_o = O.sample_batch(seeds[r].numpy(), oracle.MODE_OTF, 0.2, step)
+            assert n == n_o
+            assert np.array_equal(frontier[: n[L]].cpu().numpy(), fr_o)
+            for layer in range(L):
+                k = L - 1 - layer
+                assert np.array_equal(blocks[layer].indptr(n[k]).cpu().numpy(), blocks_o[layer].indptr)
+                assert np.array_equal(blocks[layer].indices(m[layer]).cpu().numpy(), blocks_o[layer].indices)
+            assert torch.equal(feats[:, 0].cpu(), torch.from_numpy(fr_o.astype(np.float32)))
 
 
 def _is_neighbour(indptr, indices, dst, src):

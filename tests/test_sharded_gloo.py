@@ -134,6 +134,43 @@ def test_a_group_that_outgrows_its_segment_ends_the_batch_on_every_rank(tmp_path
         assert open(os.path.join(tmp_path, "f%d.txt" % r)).read() == "raised 1"
 
 
+@pytest.mark.parametrize("capacity,merge", [(None, None), (920, True), (920, False)])
+def test_all_ranks_in_one_process_equal_one_sampler(capacity, merge):
+    """The phase-by-phase driver (sharded.sample_batch_local, what a one-GPU check of a multi-rank run uses) with the
+    oracle's primitives standing in for the kernels: exact-size and fixed-capacity exchanges, owners serving list by
+    list and merged."""
+    import fake_shard_ops as ops
+    from paper_2406_17918_b200 import sharded
+
+    cfg = get_config("tiny")
+    g = build_graph(cfg)
+    perm = seed_permutation(cfg)
+    X = _features(cfg["num_nodes"])
+    world, L = 3, len(cfg["fanouts"])
+    ranks = []
+    for r in range(world):
+        ip, idx = sharded.shard_csr(g.indptr, g.indices, r, world)
+        lo, hi = sharded.shard_range(cfg["num_nodes"], r, world)
+        ranks.append(sharded.ShardRank(ops, r, world, ip, idx, X[lo:hi].contiguous(), cfg["fanouts"], cfg["cache_width"], SEED,
+                                       cfg["shared"], THETA, max_seeds=cfg["batch"], max_requests=cfg["num_nodes"]))
+        if capacity:
+            ranks[-1].set_capacities([capacity] * (L + 1), merge=merge)
+    O = oracle.Sampler(g.indptr.numpy(), g.indices.numpy(), cfg["fanouts"], cfg["cache_width"], SEED, cfg["shared"])
+    O.set_theta(THETA)
+    for t, (gm, om, rate) in enumerate([(ops.GS_MODE_OTF, oracle.MODE_OTF, 0.25), (ops.GS_MODE_FCR, oracle.MODE_FCR, 0.0),
+                                        (ops.GS_MODE_OTF_FETCH, oracle.MODE_OTF_FETCH, 0.5)], start=1):
+        seeds = [batch_seeds(perm, t, cfg["batch"], r, world) for r in range(world)]
+        res = sharded.sample_batch_local(ranks, seeds, gm, rate, t)
+        for r in range(world):
+            blocks, frontier, n, m, feats = res[r]
+            fr, n_o, blocks_o = O.sample_batch(seeds[r].numpy(), om, rate, t)
+            assert n == n_o and np.array_equal(frontier[: n[L]].numpy(), fr)
+            for l in range(L):
+                assert np.array_equal(blocks[l].indptr(n[L - 1 - l]).numpy(), blocks_o[l].indptr)
+                assert np.array_equal(blocks[l].indices(m[l]).numpy(), blocks_o[l].indices)
+            assert torch.equal(feats, X[torch.from_numpy(fr.astype(np.int64))])
+
+
 def test_refreshing_a_row_twice_in_one_step_equals_once():
     """Two ranks may ask an owner for the same node in the same step."""
     cfg = get_config("tiny")
