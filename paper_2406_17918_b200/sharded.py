@@ -162,6 +162,7 @@ class ShardRank:
         more than one rank (with one there is nothing to merge, only the cost of doing it)."""
         if merge is None:
             merge = self.world > 1
+        self.caps_agreed = False                   # checked against the other ranks by the first batch
         caps = [int(c) for c in caps] + [0] * (self.L + 1 - len(caps))
         if len(caps) != self.L + 1 or min(caps[: self.L]) < 1:
             raise ValueError("one positive capacity per hop (and optionally one for the features) expected")
@@ -485,6 +486,15 @@ def _sample_batch_fixed(me, mode, rate, step, features, group, feature_bases, st
     rank always takes part in every exchange, whatever it has met; errors (host- or device-detected, a group that
     outgrew its segment included) are reduced once, after the last exchange."""
     L, dev = me.L, me.features.device
+    if not me.caps_agreed:
+        # equal-split exchanges need the same segment sizes everywhere: compare once, and fail on every rank if not
+        lo = torch.tensor(me.caps, dtype=torch.int64, device=dev)
+        hi = lo.clone()
+        dist.all_reduce(lo, op=dist.ReduceOp.MIN, group=group)
+        dist.all_reduce(hi, op=dist.ReduceOp.MAX, group=group)
+        if not torch.equal(lo, hi):
+            raise ShardedBatchError(1, "the ranks were given different capacities: %s here" % me.caps)
+        me.caps_agreed = True
 
     def round_trip(k, serve):
         b = me.fx[k]

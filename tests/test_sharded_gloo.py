@@ -103,8 +103,8 @@ def _failing_worker(rank, world, port, out_dir, capacity=None):
     cap = 3 if rank == world - 1 and not capacity else cfg["num_nodes"]
     me = sharded.ShardRank(ops, rank, world, ip, idx, X[lo:hi].contiguous(), cfg["fanouts"], cfg["cache_width"], SEED,
                            cfg["shared"], THETA, max_seeds=cfg["batch"], max_requests=cap)
-    if capacity:
-        me.set_capacities([capacity] * (len(cfg["fanouts"]) + 1))
+    if capacity:            # negative: the last rank is given other segment sizes than the rest
+        me.set_capacities([abs(capacity) + (7 if capacity < 0 and rank == world - 1 else 0)] * (len(cfg["fanouts"]) + 1))
     seeds = batch_seeds(perm, 1, cfg["batch"], rank, world)
     outcome = "returned"
     try:
@@ -131,6 +131,13 @@ def test_a_group_that_outgrows_its_segment_ends_the_batch_on_every_rank(tmp_path
     exchange of the batch still takes place, and all ranks raise (a requester-side error: code 1)."""
     mp.spawn(_failing_worker, args=(world, _free_port(), str(tmp_path), 40), nprocs=world, join=True)
     for r in range(world):
+        assert open(os.path.join(tmp_path, "f%d.txt" % r)).read() == "raised 1"
+
+
+def test_ranks_with_different_capacities_are_told_before_any_exchange(tmp_path):
+    """Equal-split exchanges of unequal buffers would hang or corrupt: the first batch compares the capacities."""
+    mp.spawn(_failing_worker, args=(3, _free_port(), str(tmp_path), -920), nprocs=3, join=True)
+    for r in range(3):
         assert open(os.path.join(tmp_path, "f%d.txt" % r)).read() == "raised 1"
 
 
