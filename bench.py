@@ -771,10 +771,7 @@ def sharded_arm(args, cfg, mode, gamma, rank, local_rank, world, device):
 
     def largest_groups(seen):
         for r in mine:
-            got = list(r.seen)
-            if len(got) == L:                      # no feature request was bucketed (rows are pulled): size the output instead
-                got.append((r.n[L] + vworld - 1) // vworld)
-            seen = [max(a, b) for a, b in zip(seen, got)]
+            seen = [max(a, b) for a, b in zip(seen, r.largest_groups())]
         return seen
 
     # Warm-up with exact-size exchanges (the host reads the group sizes of every exchange): the largest group

@@ -203,6 +203,15 @@ class ShardRank:
             self.fx.append(b)
         self.fx_slot = None
 
+    def largest_groups(self):
+        """After an exact-size batch: the largest group of each of its exchanges (L hops, then the feature request;
+        when the rows were pulled instead, the share of the input nodes a rank would get).  The maximum of this over
+        some batches and all ranks, plus a margin, is what set_capacities needs."""
+        got = list(self.seen)
+        if len(got) == self.L:
+            got.append((self.n[self.L] + self.world - 1) // self.world)
+        return got
+
     def _product_bound(self, k):
         bound = self.n[0]
         for j in range(k):

@@ -78,7 +78,7 @@ def test_large_two_shards_two_steps():
         if step == 2:
             # the second step with fixed-capacity exchanges sized from the first one, the owners merging the two
             # requesters' lists, and rank 1 finding first occurrences with the hash table
-            seen = np.max([r.seen for r in ranks], axis=0)
+            seen = np.max([r.largest_groups() for r in ranks], axis=0)
             for r in ranks:
                 r.set_capacities([int(c * 1.3) + 64 for c in seen], merge=True)
             gs.gs_cache_set_dedup(ranks[1].cache, gs.GS_DEDUP_HASH)

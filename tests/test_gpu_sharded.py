@@ -108,7 +108,7 @@ def test_sharded_mid_fixed_capacity_exchanges():
     """Segments sized from an exact-size batch (the largest group seen, plus a margin), as a deployment would do."""
     s = Setup("mid", 3, theta=24, B=512)
     s.step("otf", 0.3, 1)
-    seen = np.max([r.seen for r in s.ranks], axis=0)                  # one entry per exchange: L hops + features
+    seen = np.max([r.largest_groups() for r in s.ranks], axis=0)      # one entry per exchange: L hops + features
     caps = [int(c * 1.3) + 8 for c in seen]
     for r in s.ranks:
         r.set_capacities(caps)
