@@ -579,7 +579,7 @@ static gs_status sample_impl(gs_cache* c, const int32_t* d_seeds, int32_t num_se
         C.d_refresh_from = (c->shared && k > 0 && mode != GS_MODE_OTF_FETCH && !fbl) ? hdr + HDR_N + (k - 1) : nullptr;   // k = 0 for a single hop
         C.tile_sums2 = (int32_t*)(ws + w.tiles_a2);
         C.item_start = (int32_t*)(ws + w.item_start);
-        C.items = (int32_t*)(ws + w.items);
+        C.items = (int4*)(ws + w.items);
         C.cand_count = (int32_t*)(ws + w.cand_count);
         C.scan_item_cap = w.scan_item_cap;
         GS_CUDA(launch_row_counts(C, b.nb[k], s));
@@ -908,7 +908,7 @@ static gs_status shard_extend_impl(gs_cache* c, int32_t k, const int32_t* d_seed
     C.r = 0;
     C.tile_sums2 = (int32_t*)(ws + w.tiles_a2);
     C.item_start = (int32_t*)(ws + w.item_start);
-    C.items = (int32_t*)(ws + w.items);
+    C.items = (int4*)(ws + w.items);
     C.cand_count = (int32_t*)(ws + w.cand_count);
     C.scan_item_cap = w.scan_item_cap;
     C.reply = d_reply;

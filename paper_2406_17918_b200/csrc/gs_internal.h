@@ -122,7 +122,7 @@ inline WorkspaceLayout make_layout(const Bounds& b, int64_t num_edges) {
     w.tiles_a2 = take(((size_t)max_n / SCAN_A_TILE + 2) * 4);
     w.item_start = take(((size_t)max_n + 1) * 4);
     w.scan_item_cap = max_n + num_edges / (4 * (int64_t)HUB_CHUNK_QUADS) + 1;
-    w.items = take((size_t)w.scan_item_cap * 4);
+    w.items = take((size_t)w.scan_item_cap * sizeof(int4));
     w.cand_count = take((size_t)max_n * 4);
     w.cand = take((size_t)max_n * SPLIT_CAND_CAP * 8);
     w.dedup = w.cand;   // free once the step's picks are written: scratch of the alternative dedup methods
@@ -179,7 +179,7 @@ struct StepParams {
     // split OTF path: scan work items (one per 4096-offset chunk of a refreshed node) and the
     // per-node candidate lists they produce
     const int32_t* item_start;       // [n+1] first item of each frontier position
-    const int32_t* items;            // item -> frontier position
+    const int4* items;               // item -> (frontier position, node, degree, chunk of the node's row)
     const int32_t* d_items_total;
     int32_t* cand_count;             // [n]
     unsigned long long* cand;        // [n][SPLIT_CAND_CAP]
@@ -209,7 +209,7 @@ struct CountParams {
     const int32_t* d_refresh_from;
     int32_t* tile_sums2;
     int32_t* item_start;
-    int32_t* items;
+    int4* items;
     int32_t* cand_count;
     int64_t scan_item_cap;
     // sharded sampling

@@ -684,21 +684,13 @@ __global__ void __launch_bounds__(RP_THREADS, GS_SCAN_MIN_BLOCKS) k_scan(const _
         int next_base = 0;
         if (lane == 0) next_base = atomicAdd(P.work_counter_scan, batch) + total_warps * batch;
         const int cnt = (base + batch < total ? base + batch : total) - base;
-        int p_l = 0, chunk_l = 0;
-        int32_t v_l = 0;
-        long long lo_l = 0, hi_l = 0;
-        if (lane < cnt) {
-            p_l = __ldg(P.items + base + lane);
-            chunk_l = base + lane - __ldg(P.item_start + p_l);
-            v_l = __ldg(P.frontier + p_l);
-            lo_l = __ldg(P.g.indptr + v_l);
-            hi_l = __ldg(P.g.indptr + v_l + 1);
-        }
+        int4 d_l = make_int4(0, 0, 0, 0);
+        if (lane < cnt) d_l = __ldg(P.items + base + lane);
         for (int i = 0; i < cnt; ++i) {
-            const int p = __shfl_sync(FULL, p_l, i);
-            const int chunk = __shfl_sync(FULL, chunk_l, i);
-            const int32_t v = __shfl_sync(FULL, v_l, i);
-            const uint32_t deg = (uint32_t)(__shfl_sync(FULL, hi_l, i) - __shfl_sync(FULL, lo_l, i));
+            const int p = __shfl_sync(FULL, d_l.x, i);
+            const int32_t v = __shfl_sync(FULL, d_l.y, i);
+            const uint32_t deg = (uint32_t)__shfl_sync(FULL, d_l.z, i);
+            const int chunk = __shfl_sync(FULL, d_l.w, i);
             const uint32_t nq = (deg + 3u) >> 2;
             const bool single = nq <= (uint32_t)HUB_CHUNK_QUADS;
             const uint32_t qa = (uint32_t)chunk * HUB_CHUNK_QUADS;

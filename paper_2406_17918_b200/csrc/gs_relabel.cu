@@ -124,12 +124,29 @@ __global__ void __launch_bounds__(1024) k_row_offsets(CountParams P) {
         else next = P.item_start[p + 1] + P.tile_sums2[tile];
     }
     __syncthreads();   // tile-local values are all read before any is overwritten below
+    // one descriptor per chunk of the node's row: the scan needs nothing else to start on it.  A thread writes the
+    // few chunks of an ordinary row itself; the hundreds of a hub are written by its whole warp.
+    int v = 0, deg = 0;
+    if ((int64_t)next > P.scan_item_cap) next = (int)P.scan_item_cap;
     if (p < n) {
         P.item_start[p] = first;
         P.cand_count[p] = 0;
-        for (int w = first; w < next && (int64_t)w < P.scan_item_cap; ++w) P.items[w] = p;
+        if (first < next) {
+            v = P.frontier[p];
+            deg = (int)(P.g.indptr[v + 1] - P.g.indptr[v]);
+            if (next - first <= 4)
+                for (int w = first; w < next; ++w) P.items[w] = make_int4(p, v, deg, w - first);
+        }
     } else if (p == n) {
         P.item_start[n] = __ldcg(P.hdr + HDR_ITEMS + P.k);
+    }
+    unsigned wide = __ballot_sync(FULL, next - first > 4);
+    while (wide) {
+        const int src = __ffs(wide) - 1;
+        wide &= wide - 1;
+        const int hp = __shfl_sync(FULL, p, src), hv = __shfl_sync(FULL, v, src), hd = __shfl_sync(FULL, deg, src);
+        const int hf = __shfl_sync(FULL, first, src), hn = __shfl_sync(FULL, next, src);
+        for (int w = hf + (int)(threadIdx.x & 31); w < hn; w += 32) P.items[w] = make_int4(hp, hv, hd, w - hf);
     }
     }
 }
