@@ -409,34 +409,52 @@ def main():
         torch.cuda.synchronize()
 
         pinned_counts = torch.zeros((K, 128), dtype=torch.int32).pin_memory()
-        events = [torch.cuda.Event(enable_timing=True) for _ in range(3 * K + 1)]
+        events = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
         clocks = ClockSampler(local_rank) if rank == 0 else None
         time.sleep(0.3)
         replicas.barrier()
         torch.cuda.synchronize()
         launches0 = gs.gs_kernel_launches()
-        gs.gs_cache_profile_begin(C, K)     # CUDA events around the batch's kernel groups, on the launching stream
         wall0 = time.time()
         for i in range(K):
             b = Wm + i
-            events[3 * i].record()
+            events[i].record()                                  # nothing but the batch boundaries is timed here
             blocks, input_nodes, cnt = one_step(b, b + 1, ws)
-            events[3 * i + 1].record()
             pinned_counts[i].copy_(hdr, non_blocking=True)      # the batch's counts, read after the run
-            events[3 * i + 2].record()
             gs.gs_gather_features(G, input_nodes, cnt, out_rows)
-        events[3 * K].record()
+        events[K].record()
         torch.cuda.synchronize()
         replicas.barrier()
         wall1 = time.time()
         launches = gs.gs_kernel_launches() - launches0
-        total_ms = events[0].elapsed_time(events[3 * K])
+        total_ms = events[0].elapsed_time(events[K])
+        gs.gs_sync_status(C)
+
+        # ---- leg 1b: where a batch's time goes.  The same loop with CUDA events around the kernel groups (inside the
+        # library, on the launching stream) and around sample_batch / gather_features; the events sit between kernels
+        # that otherwise follow each other without a gap, so this leg is a little slower than the headline and only
+        # its shares and per-kernel rates are used.
+        Kb = min(K, 200)
+        pinned_b = torch.zeros((Kb, 128), dtype=torch.int32).pin_memory()
+        ev_b = [torch.cuda.Event(enable_timing=True) for _ in range(3 * Kb + 1)]
+        gs.gs_cache_profile_begin(C, Kb)
+        for i in range(Kb):
+            b = Wm + i
+            ev_b[3 * i].record()
+            blocks, input_nodes, cnt = one_step(b, Wm + K + 1 + i, ws)
+            ev_b[3 * i + 1].record()
+            pinned_b[i].copy_(hdr, non_blocking=True)
+            ev_b[3 * i + 2].record()
+            gs.gs_gather_features(G, input_nodes, cnt, out_rows)
+        ev_b[3 * Kb].record()
+        torch.cuda.synchronize()
         group_ms, _ = gs.gs_cache_profile_end(C)
         gs.gs_sync_status(C)
-    batch_ms = sorted(events[3 * i].elapsed_time(events[3 * i + 3]) for i in range(K))
+    batch_ms = sorted(events[i].elapsed_time(events[i + 1]) for i in range(K))
     median_ms = batch_ms[K // 2]
-    sample_ms = sum(events[3 * i].elapsed_time(events[3 * i + 1]) for i in range(K))
-    gather_ms = sum(events[3 * i + 2].elapsed_time(events[3 * i + 3]) for i in range(K))
+    sample_ms = sum(ev_b[3 * i].elapsed_time(ev_b[3 * i + 1]) for i in range(Kb))
+    gather_ms = sum(ev_b[3 * i + 2].elapsed_time(ev_b[3 * i + 3]) for i in range(Kb))
+    breakdown_total_ms = ev_b[0].elapsed_time(ev_b[3 * Kb])
 
     # word positions of the counts inside the cache's state header, by sampling step
     n_words = [blocks[L - 1 - k].count_words()[0] for k in range(L)] + [blocks[0].count_words()[1]]
@@ -457,6 +475,7 @@ def main():
         listed_frac.append(float(listed[lo:n_last[k]].sum().item()) / max(1, n_last[k]) if r > 0 else 0.0)
     alg_total, alg_feat = 0, 0
     philox_blocks = sum(int(counts[i][stat0 + 3]) & 0xFFFFFFFF for i in range(K))
+    philox_blocks_b = sum(int(pinned_b[i][stat0 + 3]) & 0xFFFFFFFF for i in range(Kb))   # of the breakdown leg's batches
     slow_refills = sum(int(counts[i][stat0]) for i in range(K))
     for i in range(K):
         n = [int(counts[i][w]) for w in n_words]
@@ -537,15 +556,19 @@ def main():
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e_edges = 0
+        seeds_dev = torch.empty(B, dtype=torch.int32, device=device)
         with torch.cuda.stream(s_main):
             e0.record()
             for i in range(K):
                 step = step0 + i
                 if args.period and step % args.period == 0:
                     gs.gs_cache_refresh_all(C, refresh_mode, refresh_gamma, step)
-                # returns once the batch's counts are on the host (synchronises the sampling stream)
-                blocks, input_nodes, n, m = gs.gs_sample_batch_host(C, host_seeds[i], gm, gamma, step, ws)
-                gs.gs_gather_features(G, input_nodes, None, out_rows[: n[L]])
+                # seeds from pinned host memory, sampling and gather queued behind the copy, then the batch's counts
+                # read back (synchronises the stream): the host never holds the GPU up between the two calls
+                seeds_dev.copy_(host_seeds[i], non_blocking=True)
+                blocks, input_nodes, cnt = gs.gs_sample_batch(C, seeds_dev, gm, gamma, step, ws)
+                gs.gs_gather_features(G, input_nodes, cnt, out_rows)
+                n, m = gs.gs_batch_counts(C)
                 e_edges += sum(m)
             e1.record()
         torch.cuda.synchronize()
@@ -575,7 +598,7 @@ def main():
     clk = clocks.summary(wall0, wall1) if clocks else None
     sm_hz = (clk["sm_mhz"] or 1965.0) * 1e6 if clk else 1965.0e6
     gather_bytes_per_launch = alg_feat / K
-    gather_ms_per_launch = gather_ms / K
+    gather_ms_per_launch = gather_ms / Kb
     achieved = gather_bytes_per_launch / (gather_ms_per_launch * 1e-3) / 1e9
     last_rows = int(counts[K - 1][n_words[L]])
     alone_gbs = last_rows * (4 + 2 * cfg["feat_dim"] * esize) / (gather_alone_ms * 1e-3) / 1e9
@@ -592,10 +615,10 @@ def main():
                                    "256-byte rows, written bytes algorithmic" if gather_traffic else
                                    "no capture with this row size scales by rows"}
     # the threshold scan (k_scan, one launch per sampling step) is bound by integer ALU work: Philox blocks
-    scan_launches = K * L
+    scan_launches = Kb * L
     roof_scan = None
-    if group_ms["scan"] > 0 and philox_blocks > 0:
-        a_scan = philox_blocks / (group_ms["scan"] * 1e-3) / 1e9
+    if group_ms["scan"] > 0 and philox_blocks_b > 0:
+        a_scan = philox_blocks_b / (group_ms["scan"] * 1e-3) / 1e9
         # derived peak: a Philox4x32-10 block is 20 wide multiplies and 20 three-input logic operations; the multiply
         # pipe is the slower one.  Its width is taken from the measured multiply rate at the sampled clock
         # (rounded to a power of two lanes per SM and clock), the rest is unit counts and clocks.
@@ -611,7 +634,7 @@ def main():
                      "frac_of_measured": a_scan / (ceil["philox_blocks_per_s"] / 1e9),
                      "peak_measured_kind": "a kernel of nothing but Philox blocks and the threshold test, same run",
                      "ms_per_launch": group_ms["scan"] / scan_launches,
-                     "traffic": NCU_SCAN_BYTES_PER_BLOCK * philox_blocks / scan_launches,
+                     "traffic": NCU_SCAN_BYTES_PER_BLOCK * philox_blocks_b / scan_launches,
                      "traffic_note": "DRAM bytes per launch, scaled by Philox blocks from an ncu capture of the same kernel "
                                      "on the large workload (an upper estimate: the traffic follows work items, and larger "
                                      "rows have fewer items per block); the scan reads no CSR bytes"}
@@ -649,8 +672,11 @@ def main():
                    "parallelism": "replicas x%d" % world, "l2": "inputs_larger_than_L2",
                    "streams": "one: sample_batch then gather_features, batch after batch",
                    "sampled_edges_per_batch": edges / K, "input_nodes_per_batch": feat_rows / K},
-        "breakdown_ms_per_step": {"sample_batch": sample_ms / K, "gather_features": gather_ms / K,
-                                  "kernel_groups": {k: v / K for k, v in groups.items()}, "dominant": dominant},
+        "breakdown_ms_per_step": {"sample_batch": sample_ms / Kb, "gather_features": gather_ms / Kb,
+                                  "kernel_groups": {k: v / Kb for k, v in groups.items()}, "dominant": dominant,
+                                  "ms_per_step_with_these_events": breakdown_total_ms / Kb, "steps": Kb,
+                                  "what": "a second pass over the same batches with CUDA events around the kernel "
+                                          "groups; the headline pass above records batch boundaries only"},
         "frontier_shares_last_batch": {"refreshed": refreshed_frac, "refill_from_scan_list": listed_frac,
                                        "n_by_step": n_last},
         "pipelined": pipelined,
