@@ -420,8 +420,8 @@ def main():
             b = Wm + i
             events[i].record()                                  # nothing but the batch boundaries is timed here
             blocks, input_nodes, cnt = one_step(b, b + 1, ws)
-            pinned_counts[i].copy_(hdr, non_blocking=True)      # the batch's counts, read after the run
             gs.gs_gather_features(G, input_nodes, cnt, out_rows)
+            pinned_counts[i].copy_(hdr, non_blocking=True)      # the batch's counts, read after the run
         events[K].record()
         torch.cuda.synchronize()
         replicas.barrier()
