@@ -43,11 +43,12 @@ SAMPLER_SEED = 0x6A09E667F3BCC908
 #     blocks in 45 K work items.  The traffic is the items' descriptors, so it follows the number of items; larger
 #     rows mean fewer items per block, which makes the per-block scaling an upper estimate for the scale workload.
 #   k_gather with 256-byte bf16 rows, all 736,389 rows of workload shared once each in random order (--gather-only):
-#     191,470,592 B read (260 B per row: the row and its id, no over-fetch); 137 MB of the 188.5 MB written reached
+#     191,698,944 B read by the bulk-copy kernel (260 B per row: the row and its id, no over-fetch; the load/store
+#     kernel: 191,470,592 B); 141 MB of the 188.5 MB written reached
 #     DRAM inside the launch, the rest was still in L2 when it ended, so the written bytes are counted as the
 #     algorithmic 256 B per row.
 NCU_SCAN_BYTES_PER_BLOCK = (5612800 + 12544) / 16380004
-NCU_GATHER_READ_BYTES_PER_256B_ROW = 191470592 / 736389
+NCU_GATHER_READ_BYTES_PER_256B_ROW = 191698944 / 736389
 
 
 def measured_peak():
@@ -276,6 +277,9 @@ def main():
     ap.add_argument("--no-overlap", action="store_true",
                     help="skip the second, pipelined leg (gather of a batch on a second stream, overlapping the "
                          "first, latency-bound hops of the next batch)")
+    ap.add_argument("--gather-kernel", default="bulk", choices=["bulk", "loads"],
+                    help="the gather on the one stream: rows staged through shared memory by bulk copies (default), or the "
+                         "load/store kernel with 16 blocks per SM")
     ap.add_argument("--gather-grid", type=int, default=None,
                     help="blocks per SM in the gather's grid during the pipelined leg (default 1024 short blocks; "
                          "the one-stream leg always uses 16 long-lived ones)")
@@ -383,7 +387,8 @@ def main():
         raise SystemExit("--verify checks a batch with its own refresh; it does not combine with --period")
     if args.verify and rank == 0:
         verified = verify_first_batch(gs, cfg, g, G, C, X, seeds_all[0], gm, mode, gamma, ws, args.theta)
-    gs.gs_graph_set_gather_grid(G, 16)     # a few long-lived blocks per SM: the fastest shape when the gather runs alone
+    alone_grid = 16 if args.gather_kernel == "loads" else -1
+    gs.gs_graph_set_gather_grid(G, alone_grid)     # the gather with the GPU to itself: bulk copies where the rows allow it (-1), or loads/stores with a few long-lived blocks (16)
     s_main = torch.cuda.Stream(device=device, priority=-1)
     out_rows = None
     refresh_events = []
@@ -541,7 +546,7 @@ def main():
         pipelined = {"ms_per_step": p_ms / K, "what": "gather of batch t on a second stream beside the first hops of batch t+1; "
                      "same batches' worth of work, %d steps" % K,
                      "gather_grid_blocks_per_sm": args.gather_grid if args.gather_grid else 1024}
-        gs.gs_graph_set_gather_grid(G, 16)
+        gs.gs_graph_set_gather_grid(G, alone_grid)
         del ws_list, out_list
     if clocks:
         time.sleep(0.1)
@@ -577,6 +582,8 @@ def main():
         e2e = {"value": e_edges_all / (e_ms * 1e-3), "unit": "edges/s", "h2d_bytes_per_step": B * 4,
                "d2h_bytes_per_step": gs.COUNTS_READBACK_BYTES,
                "ms_per_step": e_ms / K}
+
+    gs.gs_gather_status()     # raises if a bulk-copy gather ever ran out of patience (it never should)
 
     # ---- measured integer-ALU ceilings (nothing but the arithmetic, same process, same clocks)
     ceil = None
@@ -671,6 +678,8 @@ def main():
                    "refresh": ({"mode": mode, "gamma": refresh_gamma} if args.period else "per batch, frontier rows"), "cache_bytes": C.storage.numel(),
                    "parallelism": "replicas x%d" % world, "l2": "inputs_larger_than_L2",
                    "streams": "one: sample_batch then gather_features, batch after batch",
+                   "gather_kernel": "bulk copies through shared memory where the rows allow it (128 - 512 bytes on 64-byte boundaries), else "
+                                    "loads / stores with 16 blocks per SM" if alone_grid < 0 else "loads / stores, 16 blocks per SM",
                    "sampled_edges_per_batch": edges / K, "input_nodes_per_batch": feat_rows / K},
         "breakdown_ms_per_step": {"sample_batch": sample_ms / Kb, "gather_features": gather_ms / Kb,
                                   "kernel_groups": {k: v / Kb for k, v in groups.items()}, "dominant": dominant,
@@ -722,7 +731,7 @@ def gather_arm(args, cfg, device):
     ids = torch.argsort(splitmix64(torch.arange(N, dtype=torch.int64, device=device) + 0x5EED))[:rows].to(torch.int32)
     indptr = torch.zeros(N + 1, dtype=torch.int64, device=device)
     G = gs.gs_graph_create(indptr, torch.zeros(1, dtype=torch.int32, device=device), X)
-    gs.gs_graph_set_gather_grid(G, 16)
+    gs.gs_graph_set_gather_grid(G, 16 if args.gather_kernel == "loads" else -1)
     out = torch.empty((rows, cfg["feat_dim"]), dtype=X.dtype, device=device)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
     times = []

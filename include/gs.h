@@ -70,11 +70,16 @@ gs_status gs_graph_create(int64_t num_nodes, int64_t num_edges, const int64_t* d
                           int32_t feat_dim, int64_t feat_ld, gs_graph** out);
 void gs_graph_destroy(gs_graph*);
 
-/* Launch shape of gs_gather_features for this graph: the grid has at most (SM count) * blocks_per_sm blocks
- * of 256 threads (8 are resident per SM; a block copies rows until the grid has covered them all).
- * 0 restores the default (256).  Few long-lived blocks (16) are fastest when the gather runs alone;
- * many short ones (256 - 1024) let kernels of a concurrent higher-priority stream start at once. */
+/* How gs_gather_features copies the rows of this graph.  0 (the default) and -1: rows of 128 to 512 bytes that
+ * are 64-byte aligned on both sides (base, pitch and row size) move as bulk copies staged through shared memory,
+ * a persistent grid of a few blocks per SM - the fastest when the gather has the GPU to itself; other rows take
+ * the load/store kernel (grid: 256 blocks per SM with 0; 16 with -1, which says that nothing runs beside the
+ * gather).  A positive value asks for the load/store kernel with a grid of at most
+ * (SM count) * blocks_per_sm blocks of 256 threads (8 are resident per SM): many short blocks (256 - 1024) let
+ * kernels of a concurrent higher-priority stream start at once.
+ * gs_gather_status synchronises `stream` and reports whether a bulk-copy gather ever gave up a (bounded) wait. */
 gs_status gs_graph_set_gather_grid(gs_graph*, int32_t blocks_per_sm);
+gs_status gs_gather_status(void* stream);
 
 /* Optional one-pass check of the graph contract on the device: row offsets start at 0, end at
  * num_edges and never decrease; every neighbour id lies in [0, num_nodes); each row is strictly

@@ -70,6 +70,7 @@ def _load():
         "gs_graph_create": [i64, i64, vp, vp, vp, ctypes.c_int, i32, i64, pvp],
         "gs_graph_validate": [vp, vp, ctypes.POINTER(i64)],
         "gs_graph_set_gather_grid": [vp, i32],
+        "gs_gather_status": [vp],
         "gs_cache_bytes": [vp, i32, i32, i32, psz],
         "gs_workspace_bytes": [vp, i32, vp, i32, psz],
         "gs_cache_init": [vp, i32, vp, i32, u64, i32, vp, sz, vp, pvp],
@@ -244,6 +245,11 @@ def gs_graph_create(indptr: torch.Tensor, indices: torch.Tensor, features, dtype
 
 def gs_graph_set_gather_grid(graph: Graph, blocks_per_sm: int):
     _check(_L.gs_graph_set_gather_grid(graph.handle, int(blocks_per_sm)))
+
+
+def gs_gather_status(stream=None):
+    """Synchronises; raises if a bulk-copy gather ever gave up waiting."""
+    _check(_L.gs_gather_status(_stream(stream)))
 
 
 def gs_graph_validate(graph: Graph, stream=None) -> int:

@@ -195,8 +195,15 @@ void gs_graph_destroy(gs_graph* g) { delete g; }
 
 gs_status gs_graph_set_gather_grid(gs_graph* g, int32_t blocks_per_sm) {
     if (!g) return fail(GS_ERR_ARG, "graph is NULL");
-    if (blocks_per_sm < 0 || blocks_per_sm > 4096) return fail(GS_ERR_ARG, "blocks_per_sm outside [0, 4096]");
+    if (blocks_per_sm < -1 || blocks_per_sm > 4096) return fail(GS_ERR_ARG, "blocks_per_sm outside [-1, 4096]");
     g->gather_blocks_per_sm = blocks_per_sm;
+    return GS_OK;
+}
+
+gs_status gs_gather_status(void* stream) {
+    int flag = 0;
+    GS_CUDA(gather_gave_up((cudaStream_t)stream, &flag));
+    if (flag) return fail(GS_ERR_CUDA, "a feature gather gave up waiting for a bulk copy");
     return GS_OK;
 }
 

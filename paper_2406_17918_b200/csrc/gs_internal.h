@@ -310,6 +310,7 @@ cudaError_t launch_gather(const void* src, int64_t src_ld_bytes, int64_t row_byt
                           const int32_t* d_count, int32_t count_bound, void* dst, int64_t dst_ld_bytes,
                           int32_t blocks_per_sm /* 0: the default */, int64_t id_lo, int64_t id_hi /* ids outside
                           [id_lo, id_hi) are skipped */, cudaStream_t s);
+cudaError_t gather_gave_up(cudaStream_t s, int* h_flag);
 cudaError_t launch_gather_sharded(const void* const* bases, int32_t world, int64_t num_rows, int64_t rows_per_shard,
                                   int64_t src_ld_bytes,
                                   int64_t row_bytes, const int32_t* ids, const int32_t* d_count, int32_t count_bound,

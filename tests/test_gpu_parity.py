@@ -432,6 +432,46 @@ def test_device_detected_errors(tiny):
     tiny.check_batch(C, ws, O, good, "otf", 0.25, 1)
 
 
+def test_gather_bulk_copy_variant():
+    """gs_graph_set_gather_grid(G, -1): the rows go through shared memory by bulk copies; same result, bit for bit."""
+    import paper_2406_17918_b200 as gs
+    from parity import bits
+    g = torch.Generator().manual_seed(4)
+    N = 5000
+    indptr = torch.zeros(N + 1, dtype=torch.int64, device="cuda")
+    indices = torch.zeros(1, dtype=torch.int32, device="cuda")
+    # eligible: rows of 128 .. 512 bytes on 64-byte boundaries (4 warps per block up to 384 bytes, 3 above); the others
+    # take the load/store kernel through the same call
+    for dtype, d, ld in ((torch.bfloat16, 128, 128), (torch.float32, 32, 48), (torch.bfloat16, 192, 192), (torch.float32, 112, 112),
+                         (torch.bfloat16, 256, 256), (torch.float32, 100, 100), (torch.bfloat16, 8, 8), (torch.float32, 36, 40),
+                         (torch.float32, 1433, 1433), (torch.bfloat16, 7, 7)):
+        base = torch.randn((N, ld), generator=g).to(dtype).cuda()
+        X = base[:, :d]
+        G = gs.gs_graph_create(indptr, indices, X)
+        gs.gs_graph_set_gather_grid(G, -1)
+        for n in (1, 31, 32, 33, 1000, 40001):
+            ids = torch.randint(0, N, (n,), generator=g).to(torch.int32).cuda()
+            out = torch.full((n + 5, d), 3, dtype=dtype, device="cuda")
+            cnt = torch.tensor(n, dtype=torch.int32, device="cuda")
+            gs.gs_gather_features(G, ids, cnt if n % 2 else None, out[:n])
+            assert np.array_equal(bits(out[:n]), oracle.gather(bits(X), ids.cpu().numpy())), (dtype, d, n)
+            assert bool((out[n:] == 3).all())
+        # a device count below the bound: the rows beyond it stay as they are
+        ids = torch.randint(0, N, (500,), generator=g).to(torch.int32).cuda()
+        out = torch.full((500, d), 3, dtype=dtype, device="cuda")
+        gs.gs_gather_features(G, ids, torch.tensor(77, dtype=torch.int32, device="cuda"), out)
+        assert np.array_equal(bits(out[:77]), oracle.gather(bits(X), ids[:77].cpu().numpy())) and bool((out[77:] == 3).all())
+    # rows of a shard addressed by global ids: ids outside the shard are skipped
+    Xs = torch.randn((300, 64), generator=g).to(torch.bfloat16).cuda()
+    ids = torch.randint(380, 720, (999,), generator=g).to(torch.int32).cuda()
+    out = torch.full((999, 64), 9, dtype=torch.bfloat16, device="cuda")
+    ref = out.clone()
+    gs.gs_gather_rows(Xs, ids, ref, first_row=400)
+    inside = (ids >= 400) & (ids < 700)
+    assert torch.equal(ref[inside], Xs[(ids[inside] - 400).long()]) and bool((ref[~inside] == 9).all())
+    gs.gs_gather_status()
+
+
 def test_gather_alignment_paths():
     import paper_2406_17918_b200 as gs
     from parity import bits
@@ -444,7 +484,8 @@ def test_gather_alignment_paths():
         base = torch.randn((100, ld), generator=g).to(dtype).cuda()
         X = base[:, :d]
         G = gs.gs_graph_create(indptr, indices, X)
-        for out_ld in (d, d + 3):
+        for out_ld, grid in ((d, 0), (d + 3, 0), (d, 16), (d + 3, 16)):     # default kernel choice, and the load/store kernel
+            gs.gs_graph_set_gather_grid(G, grid)
             outb = torch.zeros((257, out_ld), dtype=dtype, device="cuda")
             out = outb[:, :d]
             gs.gs_gather_features(G, ids, None, out)
