@@ -8,6 +8,8 @@
 // rows in flight per thread beats fewer, fatter threads (0.82 vs 0.70 of the copy rate on 256-byte rows).  It
 // serves every other row shape, and the many-short-blocks launch shape a gather beside another stream wants.
 // Loads and stores are marked streaming: no row is read twice (frontier ids are distinct).
+#include <atomic>
+
 #include "gs_device.cuh"
 #include "gs_internal.h"
 
@@ -248,11 +250,15 @@ static cudaError_t launch_bulk(const void* src, int64_t src_ld, int64_t row_byte
     int warps = (int)((96 << 10) / ((int64_t)BULK_STAGES * 32 * row_bytes));
     warps = warps < 1 ? 1 : (warps > BULK_WARPS ? BULK_WARPS : warps);
     const size_t smem = (size_t)warps * BULK_STAGES * 32 * (size_t)row_bytes;
-    static size_t configured = 0;
-    if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(k_gather_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    // the shared-memory limit of a kernel is a per-device setting: remember what each device has been told
+    static std::atomic<int> configured[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || (int)smem > configured[dev].load(std::memory_order_relaxed)) {
+        e = cudaFuncSetAttribute(k_gather_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        configured = smem;
+        if (dev >= 0 && dev < 64) configured[dev].store((int)smem, std::memory_order_relaxed);
     }
     int per_sm = (int)((200u << 10) / (smem + 1024));
     per_sm = per_sm < 1 ? 1 : (per_sm > 16 ? 16 : per_sm);
