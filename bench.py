@@ -626,20 +626,22 @@ def main():
     roof_scan = None
     if group_ms["scan"] > 0 and philox_blocks_b > 0:
         a_scan = philox_blocks_b / (group_ms["scan"] * 1e-3) / 1e9
-        # derived peak: a Philox4x32-10 block is 20 wide multiplies and 20 three-input logic operations; the multiply
-        # pipe is the slower one.  Its width is taken from the measured multiply rate at the sampled clock
-        # (rounded to a power of two lanes per SM and clock), the rest is unit counts and clocks.
-        mul_lanes = ceil["wide_multiplies_per_s"] / (sms * sm_hz)
-        lanes = 2 ** round(__import__("math").log2(max(mul_lanes, 1.0)))
-        p_scan = sms * lanes * sm_hz / 20.0 / 1e9
+        # derived peak: a Philox4x32-10 block is 20 wide multiplies and 20 three-input logic operations.  Integer
+        # multiplies and logic operations share one datapath (the profiler shows its two pipes' active cycles adding up
+        # to the elapsed ones, and a multiply + xor pair runs at half the rate of a lone logic operation), so the block
+        # costs 40 integer instructions at the measured integer rate (rounded to a power of two lanes per SM and clock).
+        int_lanes = ceil["logic_ops_per_s"] / (sms * sm_hz)
+        lanes = 2 ** round(__import__("math").log2(max(int_lanes, 1.0)))
+        p_scan = sms * lanes * sm_hz / 40.0 / 1e9
         roof_scan = {"kernel": "k_scan (Philox threshold scan), %d launches per step" % L, "bound": "alu",
                      "achieved": a_scan, "peak": p_scan,
-                     "peak_kind": "derived: %d SMs x %d wide-multiply lanes per SM and clock x %.0f MHz / 20 multiplies per "
-                                  "block (measured multiply rate: %.1f lanes per SM and clock)" % (sms, lanes, sm_hz / 1e6, mul_lanes),
+                     "peak_kind": "derived: %d SMs x %d integer lanes per SM and clock x %.0f MHz / 40 integer instructions per "
+                                  "block (measured: %.1f logic lanes, %.1f multiply + xor pairs per SM and clock)"
+                                  % (sms, lanes, sm_hz / 1e6, int_lanes, ceil["wide_multiplies_per_s"] / (sms * sm_hz)),
                      "unit": "G Philox4x32-10 blocks/s", "frac": a_scan / p_scan,
                      "peak_measured": ceil["philox_blocks_per_s"] / 1e9,
                      "frac_of_measured": a_scan / (ceil["philox_blocks_per_s"] / 1e9),
-                     "peak_measured_kind": "a kernel of nothing but Philox blocks and the threshold test, same run",
+                     "peak_measured_kind": "a kernel of nothing but the scan's Philox blocks and threshold test, same run",
                      "ms_per_launch": group_ms["scan"] / scan_launches,
                      "traffic": NCU_SCAN_BYTES_PER_BLOCK * philox_blocks_b / scan_launches,
                      "traffic_note": "DRAM bytes per launch, scaled by Philox blocks from an ncu capture of the same kernel "

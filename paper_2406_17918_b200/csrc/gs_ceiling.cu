@@ -13,18 +13,21 @@ constexpr int CEIL_THREADS = 256;
 
 // Philox blocks with the scan's threshold test: four independent blocks per thread and iteration,
 // counters that change every iteration, one warp vote per iteration - the inner loop of the scan
-// without any of its bookkeeping.  `tinc` is a run-time value no key ever meets, so nothing is stored.
+// without any of its bookkeeping, in the scan's form of the function (consecutive quads of one row:
+// 17 wide multiplies per block).  `tinc` is a run-time value no key ever meets, so nothing is stored.
 __global__ void __launch_bounds__(CEIL_THREADS) k_ceiling_philox(const __grid_constant__ StepParams P, int iters,
                                                                    uint32_t tinc) {
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t v = blockIdx.x * CEIL_THREADS + threadIdx.x;
     uint32_t found = 0;
-    for (int it = 0; it < iters; ++it) {
-        const uint32_t q = (uint32_t)it * 128u + lane;
-        const uint4 o0 = philox4x32_10_rk(q, v, P.step, P.word_fill, P.rk);
-        const uint4 o1 = philox4x32_10_rk(q + 32, v, P.step, P.word_fill, P.rk);
-        const uint4 o2 = philox4x32_10_rk(q + 64, v, P.step, P.word_fill, P.rk);
-        const uint4 o3 = philox4x32_10_rk(q + 96, v, P.step, P.word_fill, P.rk);
+    const RowKeys rkeys = philox_row_keys(v, P.step, P.word_fill, P.rk);
+    constexpr unsigned long long M0x32 = 32ull * PHILOX_M0;
+    unsigned long long p0 = (unsigned long long)PHILOX_M0 * lane;
+    for (int it = 0; it < iters; ++it, p0 = add64(p0, 4 * M0x32)) {
+        const uint4 o0 = philox_row_block(p0, rkeys, P.rk);
+        const uint4 o1 = philox_row_block(add64(p0, M0x32), rkeys, P.rk);
+        const uint4 o2 = philox_row_block(add64(p0, 2 * M0x32), rkeys, P.rk);
+        const uint4 o3 = philox_row_block(add64(p0, 3 * M0x32), rkeys, P.rk);
         const uint32_t m0 = min(min(o0.x, o0.y), min(o0.z, o0.w));
         const uint32_t m1 = min(min(o1.x, o1.y), min(o1.z, o1.w));
         const uint32_t m2 = min(min(o2.x, o2.y), min(o2.z, o2.w));

@@ -41,6 +41,54 @@ __device__ __forceinline__ uint4 philox4x32_10_rk(uint32_t c0, uint32_t c1, uint
     return make_uint4(c0, c1, c2, c3);
 }
 
+// The same function for the consecutive quads of one row, as the threshold scan evaluates it: counter
+// (q, node, step, word) with only q changing.  The first round's products are then M1 * step (one value per
+// launch) and M0 * q (which grows by a constant from quad to quad: a 64-bit add instead of a multiply), and
+// in the second round M0 multiplies a value that depends on the node alone (once per row).  What is left per
+// block are 17 wide multiplies instead of 20; the result is the same word for word.
+struct RowKeys {
+    uint32_t cw;    // word ^ rk[1]
+    uint32_t d;     // lo(M1 * step) ^ rk[2]
+    uint32_t b;     // hi(M0 * a) ^ rk[3], a = hi(M1 * step) ^ node ^ rk[0]
+    uint32_t lo_a;  // lo(M0 * a)
+};
+constexpr uint32_t PHILOX_M0 = 0xD2511F53u, PHILOX_M1 = 0xCD9E8D57u;
+
+__device__ __forceinline__ RowKeys philox_row_keys(uint32_t node, uint32_t step, uint32_t word, const uint32_t (&rk)[20]) {
+    const uint32_t a = __umulhi(PHILOX_M1, step) ^ node ^ rk[0];
+    RowKeys k;
+    k.cw = word ^ rk[1];
+    k.d = (PHILOX_M1 * step) ^ rk[2];
+    k.b = __umulhi(PHILOX_M0, a) ^ rk[3];
+    k.lo_a = PHILOX_M0 * a;
+    return k;
+}
+
+// a + b on the integer adder (add with carry), so that it does not compete with the multiplies for their pipe
+__device__ __forceinline__ unsigned long long add64(unsigned long long a, unsigned long long b) {
+    uint32_t lo, hi;
+    asm("add.cc.u32 %0, %2, %4;\n\taddc.u32 %1, %3, %5;"
+        : "=r"(lo), "=r"(hi)
+        : "r"((uint32_t)a), "r"((uint32_t)(a >> 32)), "r"((uint32_t)b), "r"((uint32_t)(b >> 32)));
+    return ((unsigned long long)hi << 32) | lo;
+}
+
+// p0 = M0 * q as a 64-bit product; the block of quad q + j is philox_row_block(p0 + j * M0, ...).
+__device__ __forceinline__ uint4 philox_row_block(unsigned long long p0, const RowKeys& k, const uint32_t (&rk)[20]) {
+    const uint32_t x = (uint32_t)(p0 >> 32) ^ k.cw;                 // third counter word after round one
+    uint32_t c0 = __umulhi(PHILOX_M1, x) ^ k.d, c1 = PHILOX_M1 * x;   // round two
+    uint32_t c2 = k.b ^ (uint32_t)p0, c3 = k.lo_a;
+#pragma unroll
+    for (int round = 2; round < 10; ++round) {
+        const uint32_t hi0 = __umulhi(PHILOX_M0, c0), lo0 = PHILOX_M0 * c0;
+        const uint32_t hi1 = __umulhi(PHILOX_M1, c2), lo1 = PHILOX_M1 * c2;
+        const uint32_t n0 = hi1 ^ c1 ^ rk[2 * round];
+        const uint32_t n2 = hi0 ^ c3 ^ rk[2 * round + 1];
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
 // Kernels of a batch are launched with programmatic stream serialization: a kernel may be set up on the GPU
 // while its predecessor in the stream is still draining, and must call this before it reads anything the
 // predecessor wrote (it returns once the predecessor has completed and its writes are visible).

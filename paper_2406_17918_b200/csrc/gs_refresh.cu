@@ -717,13 +717,17 @@ __global__ void __launch_bounds__(RP_THREADS, GS_SCAN_MIN_BLOCKS) k_scan(const _
             // Main loop: four independent Philox blocks per lane and iteration (512 offsets per warp
             // iteration), all quads in range, one vote per iteration.  The ragged end takes up to four
             // masked blocks at once as well.
+            // the row's quads share the first two Philox rounds' constants; M0 * q advances by adds
+            const RowKeys rkeys = philox_row_keys((uint32_t)v, P.step, P.word_fill, P.rk);
+            constexpr unsigned long long M0x32 = 32ull * PHILOX_M0;
+            unsigned long long p0 = (unsigned long long)PHILOX_M0 * (unsigned long long)(qa + (uint32_t)lane);
             uint32_t qb = qa;
-            for (; qb + 128 <= qe; qb += 128) {
+            for (; qb + 128 <= qe; qb += 128, p0 = add64(p0, 4 * M0x32)) {
                 const uint32_t q = qb + lane;
-                const uint4 o0 = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
-                const uint4 o1 = philox4x32_10_rk(q + 32, (uint32_t)v, P.step, P.word_fill, P.rk);
-                const uint4 o2 = philox4x32_10_rk(q + 64, (uint32_t)v, P.step, P.word_fill, P.rk);
-                const uint4 o3 = philox4x32_10_rk(q + 96, (uint32_t)v, P.step, P.word_fill, P.rk);
+                const uint4 o0 = philox_row_block(p0, rkeys, P.rk);
+                const uint4 o1 = philox_row_block(add64(p0, M0x32), rkeys, P.rk);
+                const uint4 o2 = philox_row_block(add64(p0, 2 * M0x32), rkeys, P.rk);
+                const uint4 o3 = philox_row_block(add64(p0, 3 * M0x32), rkeys, P.rk);
                 const uint32_t m0 = min(min(o0.x, o0.y), min(o0.z, o0.w));
                 const uint32_t m1 = min(min(o1.x, o1.y), min(o1.z, o1.w));
                 const uint32_t m2 = min(min(o2.x, o2.y), min(o2.z, o2.w));
@@ -738,21 +742,21 @@ __global__ void __launch_bounds__(RP_THREADS, GS_SCAN_MIN_BLOCKS) k_scan(const _
                 const uint32_t q = qb + lane;
                 const int groups = (int)((qe - qb + 31u) >> 5);   // 1..4 groups of 32 quads remain
                 if (groups > 2) {
-                    const uint4 o0 = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
-                    const uint4 o1 = philox4x32_10_rk(q + 32, (uint32_t)v, P.step, P.word_fill, P.rk);
-                    const uint4 o2 = philox4x32_10_rk(q + 64, (uint32_t)v, P.step, P.word_fill, P.rk);
+                    const uint4 o0 = philox_row_block(p0, rkeys, P.rk);
+                    const uint4 o1 = philox_row_block(add64(p0, M0x32), rkeys, P.rk);
+                    const uint4 o2 = philox_row_block(add64(p0, 2 * M0x32), rkeys, P.rk);
                     take_hits(q, o0, q < qe);
                     take_hits(q + 32, o1, q + 32 < qe);
                     take_hits(q + 64, o2, q + 64 < qe);
                     if (groups > 3) {
-                        const uint4 o3 = philox4x32_10_rk(q + 96, (uint32_t)v, P.step, P.word_fill, P.rk);
+                        const uint4 o3 = philox_row_block(add64(p0, 3 * M0x32), rkeys, P.rk);
                         take_hits(q + 96, o3, q + 96 < qe);
                     }
                 } else {
-                    const uint4 o0 = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
+                    const uint4 o0 = philox_row_block(p0, rkeys, P.rk);
                     take_hits(q, o0, q < qe);
                     if (groups > 1) {
-                        const uint4 o1 = philox4x32_10_rk(q + 32, (uint32_t)v, P.step, P.word_fill, P.rk);
+                        const uint4 o1 = philox_row_block(add64(p0, M0x32), rkeys, P.rk);
                         take_hits(q + 32, o1, q + 32 < qe);
                     }
                 }
