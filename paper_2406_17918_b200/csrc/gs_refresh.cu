@@ -728,11 +728,11 @@ __global__ void __launch_bounds__(RP_THREADS, GS_SCAN_MIN_BLOCKS) k_scan(const _
                 const uint4 o1 = philox_row_block(add64(p0, M0x32), rkeys, P.rk);
                 const uint4 o2 = philox_row_block(add64(p0, 2 * M0x32), rkeys, P.rk);
                 const uint4 o3 = philox_row_block(add64(p0, 3 * M0x32), rkeys, P.rk);
-                const uint32_t m0 = min(min(o0.x, o0.y), min(o0.z, o0.w));
-                const uint32_t m1 = min(min(o1.x, o1.y), min(o1.z, o1.w));
-                const uint32_t m2 = min(min(o2.x, o2.y), min(o2.z, o2.w));
-                const uint32_t m3 = min(min(o3.x, o3.y), min(o3.z, o3.w));
-                if (__ballot_sync(FULL, min(min(m0, m1), min(m2, m3)) <= tinc) == 0) continue;
+                // the smallest of the 16 keys with three-input minima: 8 instructions instead of 15
+                const uint32_t m0 = __vimin3_u32(o0.x, o0.y, o0.z), m1 = __vimin3_u32(o1.x, o1.y, o1.z);
+                const uint32_t m2 = __vimin3_u32(o2.x, o2.y, o2.z), m3 = __vimin3_u32(o3.x, o3.y, o3.z);
+                const uint32_t ma = __vimin3_u32(m0, o0.w, o1.w), mb = __vimin3_u32(m1, o2.w, o3.w);
+                if (__ballot_sync(FULL, min(__vimin3_u32(ma, mb, m2), m3) <= tinc) == 0) continue;
                 take_hits(q, o0, true);
                 take_hits(q + 32, o1, true);
                 take_hits(q + 64, o2, true);
