@@ -58,7 +58,7 @@ def _worker(rank, world, port, out_dir, capacity=None):
     dist.destroy_process_group()
 
 
-@pytest.mark.parametrize("world,capacity", [(2, None), (3, None), (2, 1500), (3, 920), (3, -920)])
+@pytest.mark.parametrize("world,capacity", [(2, None), (3, None), (2, 1500), (3, 920), (3, -920), (4, 680)])
 def test_ranks_equal_one_sampler_taking_the_batches_in_turn(tmp_path, world, capacity):
     """World size 3 gives uneven shards (2,708 nodes: 903 + 903 + 902).  With a capacity the exchanges have a
     fixed pitch (segments of that many ids per pair of ranks) and the driver reads no size inside a batch; the owners
