@@ -72,6 +72,9 @@ class ShardRank:
         self.blocks = [None] * self.L
         self.n = []
         self.caps = None                           # fixed-capacity exchanges: see set_capacities
+        self.merge_exact = world > 1               # exact-size exchanges: owners merge the requesters' lists too
+        self.exact_index = None                    # one word per owned row, -1 between hops (allocated on first use)
+        self.exact_merge_status = []
 
     # ---- requester side
     # The host learns the size of a frontier only from the group sizes it has to read back for the exchange
@@ -132,6 +135,9 @@ class ShardRank:
         n, m = self.ops.gs_batch_counts(self.cache)
         self.n, self.m = list(n), list(m)
         self.ops.gs_shard_status(self.cache)       # the lists this rank served
+        merged, self.exact_merge_status = self.exact_merge_status, []
+        if merged and any(int(w[1]) for w in merged):
+            raise ValueError("a requested node id is not a row of this shard")
 
     def feature_pull(self, shard_bases, bound=None):
         """The feature step as one kernel: every input node's row is read straight from its owner's
@@ -298,11 +304,36 @@ class ShardRank:
 
     # ---- owner side
     def hop_serve(self, layer, lists, mode, rate, step):
-        """One list of distinct nodes per requester -> one [len, f] tensor of picks each."""
+        """One list of distinct nodes per requester -> one [len, f] tensor of picks each.  With several requesters
+        the packed lists are merged like the fixed-pitch ones (one list with repeats, one requester): every
+        distinct node is sampled once and its row copied to every place that asked for it."""
+        sizes = [nodes.numel() for nodes in lists]
+        for n in sizes:
+            if n > self.max_requests:
+                raise ValueError("a request list of %d nodes exceeds max_requests %d" % (n, self.max_requests))
+        total = sum(sizes)
+        lo, hi = shard_range(self.num_nodes, self.rank, self.world)
+        # the distinct nodes must fit the owner's workspace like any single list
+        if len(lists) > 1 and total > 0 and hi > lo and self.merge_exact and min(total, hi - lo) <= self.max_requests:
+            dev, f = self.features.device, self.fanouts[layer]
+            i32 = dict(dtype=torch.int32, device=dev)
+            if self.exact_index is None:
+                self.exact_index = torch.full((hi - lo,), -1, **i32)
+            packed = torch.cat([nodes.contiguous() for nodes in lists])
+            count = torch.tensor([total], **i32)
+            D = min(total, hi - lo)
+            distinct, num = torch.empty(D, **i32), torch.zeros(2, **i32)
+            rows, out = torch.empty((distinct.numel(), f), **i32), torch.empty((total, f), **i32)
+            self.ops.gs_shard_merge(packed, count, 1, self.first_row, self.exact_index, distinct, num)
+            try:
+                self.ops.gs_shard_sample_rows(self.cache, distinct, layer, mode, rate, step, self.ws_owner, picks=rows,
+                                              count=num[0:1])
+            finally:    # the fan-out also clears the index
+                self.ops.gs_shard_fan_out(packed, count, 1, self.first_row, self.exact_index, distinct, num, rows, out)
+            self.exact_merge_status.append(num)
+            return list(torch.split(out, sizes))
         out = []
         for nodes in lists:
-            if nodes.numel() > self.max_requests:
-                raise ValueError("a request list of %d nodes exceeds max_requests %d" % (nodes.numel(), self.max_requests))
             out.append(self.ops.gs_shard_sample_rows(self.cache, nodes.contiguous(), layer, mode, rate, step, self.ws_owner))
         return out                                 # device-detected problems are read once, in finish_batch
 
