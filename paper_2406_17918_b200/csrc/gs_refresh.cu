@@ -65,12 +65,15 @@ __device__ __forceinline__ int warp_collect(const StepParams& P, int32_t v, uint
                                             uint32_t q_end, uint32_t tinc, unsigned long long* buf, int count,
                                             int lane) {
     const uint32_t lt = lanemask_lt();
-    for (uint32_t qb = q_begin; qb < q_end; qb += 32) {
+    // consecutive quads of one row: the row form of the key function (see philox_row_block)
+    const RowKeys rkeys = philox_row_keys((uint32_t)v, P.step, P.word_fill, P.rk);
+    unsigned long long p0 = (unsigned long long)PHILOX_M0 * (unsigned long long)(q_begin + (uint32_t)lane);
+    for (uint32_t qb = q_begin; qb < q_end; qb += 32, p0 = add64(p0, 32ull * PHILOX_M0)) {
         const uint32_t q = qb + lane;
-        const uint4 o = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
+        const uint4 o = philox_row_block(p0, rkeys, P.rk);
         const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
         const bool inq = q < q_end;
-        const bool any = inq && (min(min(kk[0], kk[1]), min(kk[2], kk[3])) <= tinc);
+        const bool any = inq && (__vimin3_u32(min(kk[0], kk[1]), kk[2], kk[3]) <= tinc);
         if (__ballot_sync(FULL, any) == 0) continue;   // the common case: nothing below the threshold
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
@@ -599,12 +602,14 @@ __global__ void __launch_bounds__(RP_THREADS, 4) k_refresh_pick_hub(const __grid
         const uint32_t tinc = threshold_for(lam, deg);
         unsigned long long* cand = P.hub_cand + (size_t)h * HUB_CAND_CAP;
         int* cand_count = &P.hub_state[h].x;
-        for (uint32_t qb = qa; qb < qe; qb += 32) {
+        const RowKeys rkeys = philox_row_keys((uint32_t)v, P.step, P.word_fill, P.rk);
+        unsigned long long p0 = (unsigned long long)PHILOX_M0 * (unsigned long long)(qa + (uint32_t)lane);
+        for (uint32_t qb = qa; qb < qe; qb += 32, p0 = add64(p0, 32ull * PHILOX_M0)) {
             const uint32_t q = qb + lane;
-            const uint4 o = philox4x32_10_rk(q, (uint32_t)v, P.step, P.word_fill, P.rk);
+            const uint4 o = philox_row_block(p0, rkeys, P.rk);
             const uint32_t kk[4] = {o.x, o.y, o.z, o.w};
             const bool inq = q < qe;
-            const bool any = inq && (min(min(kk[0], kk[1]), min(kk[2], kk[3])) <= tinc);
+            const bool any = inq && (__vimin3_u32(min(kk[0], kk[1]), kk[2], kk[3]) <= tinc);
             if (__ballot_sync(FULL, any) == 0) continue;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
